@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the bidirectional VDA forward pass (one "step" = one whole forward over one synthetic clip).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 768p] [--impl ours|reference]
+
+N > 1 (launched with torch.distributed.run, one rank per GPU) runs N independent replicas of the
+workload -- the layer needs no exchange between GPUs -- and reports the aggregate tokens/s over the
+slowest rank's time.  Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "vda_fwd_tokens_per_s"
+UNIT = "tokens/s"
+PAPER_CONTEXT = ("paper (context only, whole pipeline on 8xB200): 6.70 s DiT denoising for a 14.3 s 768p clip, "
+                 "14.5x over 50-step dense H3, attention >85% of dense denoiser runtime")
+
+
+# ------------------------------------------------------------------------------------------ helpers
+def algorithmic_bytes(w) -> dict:
+    """Bytes the method must move per forward: read q, k, v and beta once, write out once."""
+    es = 4 if w.dtype == "f32" else 2
+    tokh = w.B * w.T * w.F * w.H
+    return {
+        "gram": tokh * (2 * w.d * es + 4),          # k, v, beta
+        "readout": tokh * (2 * w.d * es),           # q in, out out
+        "total": tokh * (4 * w.d * es + 4),
+    }
+
+
+def algorithmic_flops(w) -> dict:
+    tokh = w.B * w.T * w.F * w.H
+    n = w.B * w.H * w.T
+    return {"tensor": 6 * tokh * w.d * w.d, "fp32": 6 * n * w.d ** 3}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            m = json.load(f)
+        return {"hbm_gbs": float(m["hbm_gbs"]), "bf16_tflops": float(m["bf16_tflops"]),
+                "bf16_tflops_sustained": float(m.get("bf16_tflops_sustained", m["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int, period_ms: int = 50):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+        self.period = period_ms
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", str(self.period)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        threading.Thread(target=self._read, daemon=True).start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                if int(parts[0]) != self.gpu:
+                    continue
+                self.rows.append((time.time(), float(parts[1]), float(parts[2]), parts[5:9]))
+            except ValueError:
+                continue
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float) -> dict:
+        rows = [r for r in self.rows if t0 <= r[0] <= t1 + self.period / 1000.0]
+        where = "timed region"
+        if not rows:
+            rows, where = self.rows, "whole run (timed region shorter than the sampling period)"
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "nvidia-smi unavailable"}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[i] for r in rows for i in range(4) if r[3][i].lower() == "active"})
+        return {"sm_mhz": statistics.median(r[1] for r in rows), "sm_max_mhz": max(r[2] for r in rows),
+                "reasons": reasons, "samples": len(rows), "window": where}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except (ValueError, IndexError):
+            return local
+    return local
+
+
+def aggregate_over_ranks(ms_local: float, units_local: int, world: int):
+    """Whole-job rate: all ranks' units over the slowest rank's time.  Returns (ms_max, units_total)."""
+    if world == 1:
+        return ms_local, units_local
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    u = torch.tensor([units_local], dtype=torch.int64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(u.item())
+
+
+# ------------------------------------------------------------------------------------------ CPU baseline
+def oracle_sample(w, heads: int, frames: int):
+    """A bounded sample of the workload for the CPU oracle: `heads` head slices of batch 0, the first
+    `frames` frames of each (every frame costs the same: F tokens, one d x d solve per direction)."""
+    from paper_2609_20744_b200 import inputs
+    ws = w.scaled(B=1, H=heads, T=frames)
+    x = inputs.generate(ws, "cpu")
+    return ws, [inputs.head_slice(x, 0, h) for h in range(heads)]
+
+
+def time_oracle(slices) -> float:
+    """Seconds for the oracle, as it stands, over the sampled head slices."""
+    from oracle import vda_oracle
+    t0 = time.perf_counter()
+    for (q, k, v, beta, gate) in slices:
+        vda_oracle.vda_slice(q, k, v, beta, gate, 1e-6)
+    return time.perf_counter() - t0
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def plan_sample(w, seconds_per_step: float):
+    """Choose (heads, frames) so that one oracle pass costs about `seconds_per_step` on this host."""
+    probe_T = min(w.T, 4)
+    _, sl = oracle_sample(w, 1, probe_T)
+    time_oracle(sl)                                       # page in numpy / BLAS
+    per_frame = time_oracle(sl) / probe_T                 # seconds per (head, frame)
+    per_head = per_frame * w.T
+    if per_head <= seconds_per_step:                      # at most 4 slices: drawing them on the CPU costs time too
+        return max(1, min(w.B * w.H, 4, int(seconds_per_step / per_head))), w.T
+    return 1, max(2, min(w.T, int(seconds_per_step / per_frame)))
+
+
+def sample_text(w, heads, frames):
+    return (f"{heads} of {w.B * w.H} (batch, head) slices x {frames} of {w.T} frames x {w.F} tokens per step; "
+            f"rate scaled by {w.B * w.H * w.T}/{heads * frames} (slices and frames are independent, equal-cost units)")
+
+
+def cpu_baseline(w, seconds: float = 15.0) -> dict:
+    heads, frames = plan_sample(w, seconds)
+    _, slices = oracle_sample(w, heads, frames)
+    sec = time_oracle(slices)
+    full = sec * (w.B * w.H * w.T) / (heads * frames)
+    return {"value": w.tokens / full, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": sample_text(w, heads, frames), "seconds_sample": sec}
+
+
+# ------------------------------------------------------------------------------------------ arms
+def run_reference(args, w, rank: int, world: int):
+    """The reference arm is the fp64 oracle on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    budget = 60.0                                         # seconds for the whole --steps/--warmup run
+    heads, frames = plan_sample(w, budget / max(1, args.steps + args.warmup))
+    _, slices = oracle_sample(w, heads, frames)
+    for _ in range(args.warmup):
+        time_oracle(slices)
+    sec = sum(time_oracle(slices) for _ in range(args.steps)) / max(1, args.steps)
+    full_ms = sec * (w.B * w.H * w.T) / (heads * frames) * 1e3
+    value = w.tokens / (full_ms / 1e3)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": full_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "T": w.T, "F": w.F, "H": w.H, "d": w.d, "io_dtype": w.dtype,
+                   "parallelism": "fp64 CPU oracle on rank 0's host cores"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": sample_text(w, heads, frames)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w, rank: int, local_rank: int, world: int):
+    import torch
+    from paper_2609_20744_b200 import binding, build, inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the VDA library has no CPU fallback")
+    if rank == 0:
+        build.build()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    x = inputs.generate(w, dev)
+    vda = binding.Vda(w.d, w.dtype, device=local_rank)
+    out = torch.empty_like(x["q"])
+    stream = torch.cuda.current_stream()
+
+    def step():
+        vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    vda.profile(True)                    # per-kernel CUDA events on the launch stream, sums cleared here
+
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    kt = {}
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms_local = ev0.elapsed_time(ev1) / args.steps
+    for name, ms, _n in vda.kernel_times():
+        kt[name] = ms                    # per-launch means over the timed region
+    vda.profile(False)
+    launches = vda.launch_count() * args.steps
+    if vda.status() != binding.VDN_OK:
+        raise SystemExit("bench.py: device-side status word reports an error")
+    clocks = sampler.summary(t_wall0, t_wall1) if rank == 0 else None
+
+    ms_max, tokens_total = aggregate_over_ranks(ms_local, w.tokens, world)
+    value = tokens_total / (ms_max / 1e3)
+
+    # ---- end to end through the host-buffer entry point (H2D + forward + D2H inside the timed region)
+    e2e = None
+    try:
+        xh = {n: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for n, t in x.items()}
+        outh = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
+        e_steps = max(1, min(args.steps, args.e2e_steps))
+        vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], outh)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ev0.record(stream)
+        for _ in range(e_steps):
+            vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], outh)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        e_ms, e_tok = aggregate_over_ranks(ev0.elapsed_time(ev1) / e_steps, w.tokens, world)
+        h2d = sum(xh[n].numel() * xh[n].element_size() for n in ("q", "k", "v", "beta", "gate"))
+        e2e = {"value": e_tok / (e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": outh.numel() * outh.element_size(), "ms_per_step": e_ms, "steps": e_steps,
+               "api": "vdn_vda_forward_host (pinned host buffers)"}
+        same = bool(torch.equal(outh, out.cpu()))
+        e2e["matches_device_entry_point"] = same
+        del xh, outh
+    except Exception as exc:  # host memory may be too small for the pinned copies
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+               "error": f"{type(exc).__name__}: {exc}"}
+
+    if rank != 0:
+        return
+    sampler.stop()
+
+    peaks = measured_peaks()
+    ab = algorithmic_bytes(w)
+    fl = algorithmic_flops(w)
+    # dominant kernel by time; its algorithmic bytes
+    roof = None
+    if kt:
+        dom = max(kt, key=kt.get)
+        kind = "gram" if "gram" in dom else ("readout" if "readout" in dom else None)
+        traffic = None
+        tp = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(tp):
+            with open(tp) as f:
+                tj = json.load(f)
+            per_token_head = tj.get(dom, {}).get("dram_bytes_per_token_head")
+            if per_token_head:
+                traffic = per_token_head * w.B * w.T * w.F * w.H
+        if kind is not None:
+            achieved = ab[kind] / (kt[dom] / 1e3) / 1e9
+            roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": traffic, "peak_source": f"of {peaks['source']}",
+                    "kernel_ms": kt[dom], "algorithmic_bytes_per_launch": ab[kind]}
+        else:
+            # fp32 ALU-bound stage (resolve / scan): peak = SMs x 128 lanes x 2 flop x max SM clock
+            import torch as _t
+            prop = _t.cuda.get_device_properties(local_rank)
+            peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+            work = (2 if "resolve" in dom else 4) * w.B * w.H * w.T * w.d ** 3
+            achieved = work / (kt[dom] / 1e3) / 1e12
+            roof = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "traffic": None, "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                    "kernel_ms": kt[dom]}
+    t_roof_ms = max(ab["total"] / (peaks["hbm_gbs"] * 1e9), fl["tensor"] / (peaks["bf16_tflops_sustained"] * 1e12)) * 1e3
+    t_roof_nominal_ms = max(ab["total"] / 8e12, fl["tensor"] / 2.25e15) * 1e3
+
+    base = cpu_baseline(w) if world == 1 else None
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 in / f32 accumulate, f32 state" if w.dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "T": w.T, "F": w.F, "H": w.H, "d": w.d, "io_dtype": w.dtype,
+                   "seed": w.seed, "parallelism": "single GPU" if world == 1 else f"{world} independent replicas",
+                   "l2": "inputs+outputs far larger than the 126 MB L2; no flush" if ab["total"] > 1e9
+                         else "inputs smaller than L2: numbers are L2-warm",
+                   "path": "tensor-core" if vda.launch_count() and any("tc" in n for n in kt) else "plain-fp32"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+        "roofline": roof,
+        "layer_roofline": {"t_roof_ms_measured_peaks": t_roof_ms, "frac_of_measured": t_roof_ms / (ms_max / 1.0),
+                           "t_roof_ms_nominal": t_roof_nominal_ms, "frac_of_nominal": t_roof_nominal_ms / ms_max,
+                           "algorithmic_bytes": ab["total"], "tensor_flops": fl["tensor"], "fp32_flops": fl["fp32"]},
+        "kernel_ms": kt,
+        "cpu_baseline": base,
+        "context": PAPER_CONTEXT,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="768p")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    args = ap.parse_args()
+
+    from paper_2609_20744_b200 import inputs
+    w = inputs.WORKLOADS[args.workload]
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, w, rank, world)
+        return
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    try:
+        run_ours(args, w, rank, local_rank, world)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,147 @@
+/*
+ * vdn_vda.h -- C ABI of the bidirectional Video Delta Attention (VDA) forward pass for NVIDIA B200.
+ *
+ * The layer (Video DeltaNet, Sec. 2.2, Sec. 3 and Algorithm 1 steps 3-7), per (batch, head):
+ *
+ *   frame statistics (Eq. 3b)        A_t = K_t^T Diag(beta_t) K_t,   B_t = V_t^T Diag(beta_t) K_t
+ *   joint frame update (Eq. 5, A.1)  S_t = (S_{t-1} + B_t)(I + A_t)^{-1}            (decay alpha_t = 1)
+ *   two scans (Sec. 2.2)             P_t: frames 0..t in order,  R_t: frames T-1..t in reverse order,
+ *                                    both started from the zero state (no text state at this boundary)
+ *   gather (Eq. A.4, Eq. 1a)         the queries of frame t read  P_{t-1} + R_{t+1}  (P_{-1} = R_T = 0):
+ *                                    the local window is the query frame itself, so no frame is counted
+ *                                    twice and a frame never reads its own write
+ *   read-out, norm, gate (Eq. 1c)    o = S q;  out = gate_h * o / sqrt(mean_j o_j^2 + rms_eps)
+ *
+ * No patch order inside a frame, no 1/sqrt(F) key scaling (Sec. 3.3).  The statistics are contracted on
+ * the tensor cores (bf16 operands, fp32 accumulation) in bf16 mode and in plain fp32 in f32 mode; the
+ * inverse, the scans and the norm are always fp32.
+ *
+ * Naming: T = latent frames, F = spatial tokens per frame, H = heads, d = d_k = d_v (the paper's F, U).
+ *
+ * Tensors.  All `const void*` / `void*` tensor arguments of vdn_vda_forward are DEVICE pointers, dense,
+ * row-major, last index fastest, 16-byte aligned:
+ *      q, k, v, out : [B, T, F, H, d]   elements of cfg.io_dtype
+ *      beta         : [B, T, F, H]      float, already through the sigmoid, must be >= 0 (Proposition 1)
+ *      gate         : [H]               float, already through the sigmoid
+ * q and k are *prepared* features (feature map and L2 normalisation already applied, Sec. 2.3); the
+ * library applies no normalisation of its own and does not assume unit norm.
+ *
+ * Ownership.  The caller owns every buffer, the workspace included; the library never allocates device
+ * memory on the forward path.  The handle owns host-side state and one pinned status word.  `out` must not
+ * alias an input.  Inputs are only read.
+ *
+ * Asynchrony.  vdn_vda_forward validates its arguments on the host, enqueues its kernels on `cuda_stream`
+ * (a cudaStream_t passed as void*, NULL = the legacy default stream) and returns without synchronising.
+ * One handle (one workspace) must not be used from two streams at the same time.
+ *
+ * Errors.  Every call returns a vdn_status; nothing throws, aborts or traps.  Problems the host can see
+ * (null or misaligned pointers, non-positive sizes, d != cfg.d, workspace too small, 32-bit index overflow,
+ * wrong device architecture) are reported synchronously and nothing is enqueued.  Every wait inside a
+ * kernel is bounded; a wait that runs out records VDN_ERR_TIMEOUT in the handle's status word, which
+ * vdn_vda_status returns once the caller has synchronised the stream.
+ *
+ * Determinism.  No atomics on the result path: the same inputs give bit-identical outputs run to run.
+ */
+#ifndef VDN_VDA_H_
+#define VDN_VDA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct vdn_vda_s* vdn_vda_t;
+
+typedef enum {
+  VDN_OK = 0,
+  VDN_ERR_INVALID_ARG = 1,  /* null / misaligned pointer, bad size, struct_size mismatch            */
+  VDN_ERR_UNSUPPORTED = 2,  /* shape or dtype this build has no kernel for                            */
+  VDN_ERR_WORKSPACE = 3,    /* workspace missing or smaller than vdn_vda_workspace_bytes              */
+  VDN_ERR_CUDA = 4,         /* a CUDA runtime / driver call failed; see vdn_vda_last_error            */
+  VDN_ERR_ARCH = 5,         /* the device is not compute capability 10.x                              */
+  VDN_ERR_TIMEOUT = 6       /* a bounded device-side wait expired (reported by vdn_vda_status)        */
+} vdn_status;
+
+typedef enum { VDN_F32 = 0, VDN_BF16 = 1 } vdn_dtype;
+
+/* cfg.flags */
+#define VDN_FLAG_FORCE_SIMT 1u /* bf16 I/O through the plain-fp32 kernels (a second opinion for tests) */
+
+typedef struct {
+  uint32_t struct_size; /* sizeof(vdn_vda_config), checked                                            */
+  int32_t io_dtype;     /* vdn_dtype of q, k, v, out                                                  */
+  int32_t d;            /* head dimension: 64 or 128 (bf16 tensor-core kernels: 128)                  */
+  float rms_eps;        /* epsilon inside the RMSNorm of Eq. 1c; <= 0 selects 1e-6                    */
+  uint32_t flags;
+  int32_t device;       /* CUDA device ordinal the handle is bound to                                 */
+} vdn_vda_config;
+
+/* Names of workspace regions for vdn_vda_workspace_view (stage-wise checks in the tests). */
+typedef enum {
+  VDN_VIEW_STATS = 0, /* float [B,H,T,d,2d]: row i = [ A_t[i,:] | B_t^T[i,:] ]            (Eq. 3b)    */
+  VDN_VIEW_INV = 1,   /* float [B,H,T,d,d]:  C_t = (I + A_t)^{-1}                         (Eq. 5)     */
+  VDN_VIEW_FWD = 2,   /* float [B,H,T,d_k,d_v]: transpose of P_t, the forward-scan state    (Eq. A.1)  */
+  VDN_VIEW_READ = 3   /* transpose of the state frame t's queries read, P_{t-1}+R_{t+1}    (Eq. A.4): */
+                      /*   plain-fp32 kernels: float [B,H,T,d_k,d_v]; tensor-core kernels: bf16       */
+                      /*   [B,H,T,d_v,d_k] (i.e. the paper's orientation)                              */
+} vdn_view;
+
+/* Sec. 3 (the layer as a whole).  Creates a handle bound to cfg->device.  Allocates host memory only
+ * (one pinned, device-mapped status word).  Returns VDN_ERR_ARCH when the device is not sm_100. */
+vdn_status vdn_vda_create(const vdn_vda_config* cfg, vdn_vda_t* out_handle);
+
+/* Bytes of device workspace a forward call of this shape needs (per-frame statistics of Eq. 3b, the
+ * inverses of Eq. 5 and the scanned states of Eq. A.1 live there).  Pure function; 0 on invalid shape. */
+size_t vdn_vda_workspace_bytes(vdn_vda_t h, int B, int T, int F, int H, int d);
+
+/* Hands the library a caller-owned device buffer (256-byte aligned).  It must stay valid until replaced
+ * or until the handle is destroyed, and must not be shared between handles that run concurrently. */
+vdn_status vdn_vda_set_workspace(vdn_vda_t h, void* dev_ptr, size_t bytes);
+
+/* Algorithm 1 steps 3-7 with the readings stated at the top of this file.  All tensor pointers are
+ * device pointers (layout above).  Enqueues on cuda_stream and returns; does not synchronise. */
+vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                           const float* gate, void* out, int B, int T, int F, int H, int d,
+                           void* cuda_stream);
+
+/* The same layer for callers whose tensors live in HOST memory (pinned memory recommended): copies
+ * q, k, v, beta, gate to the staging buffer, runs vdn_vda_forward, copies `out` back, all on
+ * cuda_stream, and returns without synchronising.  All six tensor pointers are HOST pointers.  The
+ * staging buffer is a caller-owned DEVICE buffer of at least vdn_vda_staging_bytes, set beforehand. */
+size_t vdn_vda_staging_bytes(vdn_vda_t h, int B, int T, int F, int H, int d);
+vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes);
+vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const void* v,
+                                const float* beta, const float* gate, void* out, int B, int T, int F,
+                                int H, int d, void* cuda_stream);
+
+/* Offset and size, inside the workspace, of an intermediate of the last forward call of this shape
+ * (see vdn_view).  For stage-wise parity checks; the contents are valid after the stream is synchronised. */
+vdn_status vdn_vda_workspace_view(vdn_vda_t h, int which, int B, int T, int F, int H, int d,
+                                  size_t* offset_bytes, size_t* size_bytes);
+
+/* Number of kernels the last vdn_vda_forward call on this handle launched (0 before the first call). */
+int vdn_vda_last_launch_count(vdn_vda_t h);
+
+/* Per-kernel timing for benchmarks (no counterpart in the paper).  vdn_vda_profile(h, 1) makes every
+ * later forward call record CUDA events between its kernels on the caller's stream and clears the running
+ * sums; vdn_vda_profile(h, 0) stops that.  vdn_vda_kernel_times waits for the recorded events, then fills
+ * up to max_kernels entries (kernel name, mean milliseconds per launch, launches seen since the sums were
+ * cleared) and returns how many it filled.  `names` receives pointers to static strings. */
+vdn_status vdn_vda_profile(vdn_vda_t h, int enable);
+int vdn_vda_kernel_times(vdn_vda_t h, int max_kernels, const char** names, float* mean_ms, int* launches);
+
+/* Last device-side status recorded by this handle's kernels (VDN_OK or VDN_ERR_TIMEOUT).  Does not
+ * synchronise: call it after synchronising the stream.  Reading it clears nothing. */
+vdn_status vdn_vda_status(vdn_vda_t h);
+
+/* Human-readable description of the last error returned on this handle (never NULL). */
+const char* vdn_vda_last_error(vdn_vda_t h);
+
+vdn_status vdn_vda_destroy(vdn_vda_t h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VDN_VDA_H_ */

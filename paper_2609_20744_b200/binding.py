@@ -1,0 +1,216 @@
+"""Thin ctypes binding over the C ABI declared in include/vdn_vda.h.
+
+Argument marshalling only: every step of the layer runs inside the CUDA library.  torch is used
+for device memory and streams.  There is no CPU fallback: if the shared library is missing or a
+call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvdn_vda.so")
+
+VDN_OK = 0
+STATUS_NAMES = {0: "VDN_OK", 1: "VDN_ERR_INVALID_ARG", 2: "VDN_ERR_UNSUPPORTED", 3: "VDN_ERR_WORKSPACE",
+                4: "VDN_ERR_CUDA", 5: "VDN_ERR_ARCH", 6: "VDN_ERR_TIMEOUT"}
+VDN_F32, VDN_BF16 = 0, 1
+VDN_FLAG_FORCE_SIMT = 1
+VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ = 0, 1, 2, 3
+
+EXPORTS = (
+    "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward",
+    "vdn_vda_staging_bytes", "vdn_vda_set_staging", "vdn_vda_forward_host", "vdn_vda_workspace_view",
+    "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_status", "vdn_vda_last_error", "vdn_vda_destroy",
+)
+
+
+class VdnConfig(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("io_dtype", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("rms_eps", ctypes.c_float), ("flags", ctypes.c_uint32), ("device", ctypes.c_int32)]
+
+
+class VdnError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {msg}")
+        self.status = status
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """dlopen the CUDA library and declare its signatures.  Raises if it has not been built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise FileNotFoundError(
+            f"{p} not found: build it with `python -m paper_2609_20744_b200.build` (there is no CPU fallback)")
+    lib = ctypes.CDLL(p)
+    vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    shape = [ci, ci, ci, ci, ci]
+    lib.vdn_vda_create.argtypes = [ctypes.POINTER(VdnConfig), ctypes.POINTER(vp)]
+    lib.vdn_vda_create.restype = ci
+    lib.vdn_vda_workspace_bytes.argtypes = [vp, *shape]
+    lib.vdn_vda_workspace_bytes.restype = sz
+    lib.vdn_vda_set_workspace.argtypes = [vp, vp, sz]
+    lib.vdn_vda_set_workspace.restype = ci
+    lib.vdn_vda_staging_bytes.argtypes = [vp, *shape]
+    lib.vdn_vda_staging_bytes.restype = sz
+    lib.vdn_vda_set_staging.argtypes = [vp, vp, sz]
+    lib.vdn_vda_set_staging.restype = ci
+    fwd_args = [vp, vp, vp, vp, vp, vp, vp, *shape, vp]
+    lib.vdn_vda_forward.argtypes = fwd_args
+    lib.vdn_vda_forward.restype = ci
+    lib.vdn_vda_forward_host.argtypes = fwd_args
+    lib.vdn_vda_forward_host.restype = ci
+    lib.vdn_vda_workspace_view.argtypes = [vp, ci, *shape, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+    lib.vdn_vda_workspace_view.restype = ci
+    lib.vdn_vda_last_launch_count.argtypes = [vp]
+    lib.vdn_vda_last_launch_count.restype = ci
+    lib.vdn_vda_profile.argtypes = [vp, ci]
+    lib.vdn_vda_profile.restype = ci
+    lib.vdn_vda_kernel_times.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float),
+                                         ctypes.POINTER(ci)]
+    lib.vdn_vda_kernel_times.restype = ci
+    lib.vdn_vda_status.argtypes = [vp]
+    lib.vdn_vda_status.restype = ci
+    lib.vdn_vda_last_error.argtypes = [vp]
+    lib.vdn_vda_last_error.restype = ctypes.c_char_p
+    lib.vdn_vda_destroy.argtypes = [vp]
+    lib.vdn_vda_destroy.restype = ci
+    if path is None:
+        _lib = lib
+    return lib
+
+
+class Vda:
+    """One handle of the library (vdn_vda_create .. vdn_vda_destroy) plus its torch-owned workspace."""
+
+    def __init__(self, d: int, dtype: str = "bf16", rms_eps: float = 1e-6, flags: int = 0, device: int = 0):
+        import torch
+        self._torch = torch
+        self.lib = load_library()
+        self.d = d
+        self.dtype = dtype
+        self.device = device
+        cfg = VdnConfig(ctypes.sizeof(VdnConfig), VDN_F32 if dtype == "f32" else VDN_BF16, d, rms_eps, flags, device)
+        self.h = ctypes.c_void_p()
+        st = self.lib.vdn_vda_create(ctypes.byref(cfg), ctypes.byref(self.h))
+        if st != VDN_OK:
+            self.h = None
+            raise VdnError(st, "vdn_vda_create failed")
+        self._ws = None
+        self._staging = None
+
+    # -- helpers ------------------------------------------------------------------------------
+    def _check(self, st: int):
+        if st != VDN_OK:
+            raise VdnError(st, self.lib.vdn_vda_last_error(self.h).decode())
+
+    def _stream(self, stream):
+        torch = self._torch
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        return ctypes.c_void_p(s.cuda_stream)
+
+    def workspace_bytes(self, B, T, F, H) -> int:
+        return int(self.lib.vdn_vda_workspace_bytes(self.h, B, T, F, H, self.d))
+
+    def ensure_workspace(self, B, T, F, H):
+        torch = self._torch
+        need = self.workspace_bytes(B, T, F, H)
+        if need == 0:
+            raise VdnError(1, "invalid shape")
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}")
+            self._check(self.lib.vdn_vda_set_workspace(self.h, ctypes.c_void_p(self._ws.data_ptr()), need))
+        return self._ws
+
+    def ensure_staging(self, B, T, F, H):
+        torch = self._torch
+        need = int(self.lib.vdn_vda_staging_bytes(self.h, B, T, F, H, self.d))
+        if need == 0:
+            raise VdnError(1, "invalid shape")
+        if self._staging is None or self._staging.numel() < need:
+            self._staging = torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}")
+            self._check(self.lib.vdn_vda_set_staging(self.h, ctypes.c_void_p(self._staging.data_ptr()), need))
+        return self._staging
+
+    # -- the two entry points -----------------------------------------------------------------
+    def forward(self, q, k, v, beta, gate, out=None, stream=None):
+        """vdn_vda_forward on device tensors q,k,v [B,T,F,H,d], beta [B,T,F,H], gate [H]."""
+        torch = self._torch
+        B, T, F, H, d = q.shape
+        for x in (q, k, v, beta, gate):
+            if not (x.is_cuda and x.is_contiguous()):
+                raise ValueError("vdn_vda_forward needs contiguous CUDA tensors")
+        if out is None:
+            out = torch.empty_like(q)
+        self.ensure_workspace(B, T, F, H)
+        p = lambda x: ctypes.c_void_p(x.data_ptr())
+        self._check(self.lib.vdn_vda_forward(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
+                                             B, T, F, H, d, self._stream(stream)))
+        return out
+
+    def forward_host(self, q, k, v, beta, gate, out, stream=None):
+        """vdn_vda_forward_host on HOST tensors (pinned recommended); `out` is a host tensor too."""
+        B, T, F, H, d = q.shape
+        for x in (q, k, v, beta, gate, out):
+            if x.is_cuda or not x.is_contiguous():
+                raise ValueError("vdn_vda_forward_host needs contiguous host tensors")
+        self.ensure_workspace(B, T, F, H)
+        self.ensure_staging(B, T, F, H)
+        p = lambda x: ctypes.c_void_p(x.data_ptr())
+        self._check(self.lib.vdn_vda_forward_host(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
+                                                  B, T, F, H, d, self._stream(stream)))
+        return out
+
+    # -- inspection ---------------------------------------------------------------------------
+    def view(self, which: int, B, T, F, H):
+        """A torch view of a workspace intermediate (valid after synchronising the stream)."""
+        torch = self._torch
+        off, size = ctypes.c_size_t(), ctypes.c_size_t()
+        self._check(self.lib.vdn_vda_workspace_view(self.h, which, B, T, F, H, self.d,
+                                                    ctypes.byref(off), ctypes.byref(size)))
+        raw = self._ws[off.value: off.value + size.value]
+        d = self.d
+        n = B * H * T
+        if which == VIEW_STATS:
+            return raw.view(torch.float32).view(B, H, T, d, 2 * d)
+        if size.value == n * d * d * 4:
+            return raw.view(torch.float32).view(B, H, T, d, d)
+        return raw.view(torch.bfloat16).view(B, H, T, d, d)
+
+    def profile(self, enable: bool = True):
+        """Start (and reset) or stop per-kernel CUDA-event timing of forward calls."""
+        self._check(self.lib.vdn_vda_profile(self.h, 1 if enable else 0))
+
+    def kernel_times(self):
+        """[(kernel name, mean ms per launch, launches)] since profile(True); waits for the events."""
+        n = 8
+        names = (ctypes.c_char_p * n)()
+        ms = (ctypes.c_float * n)()
+        cnt = (ctypes.c_int * n)()
+        got = self.lib.vdn_vda_kernel_times(self.h, n, names, ms, cnt)
+        return [(names[i].decode(), float(ms[i]), int(cnt[i])) for i in range(got)]
+
+    def launch_count(self) -> int:
+        return int(self.lib.vdn_vda_last_launch_count(self.h))
+
+    def status(self) -> int:
+        return int(self.lib.vdn_vda_status(self.h))
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.vdn_vda_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,149 @@
+// Bidirectional frame scan + gather (Alg. 1 steps 5-6; Eq. A.1, Eq. A.4, Eq. 1a), fp32.
+//
+// With Z = S^T (d_k x d_v) and alpha = 1 the frame update  S_t = (S_{t-1} + B_t)(I + A_t)^{-1}
+// reads  Z_t = C_t (Z_{t-1} + B_t^T).  The transition acts on the key index only, so the d_v columns
+// of Z evolve independently: one CTA owns W columns of one (batch, head) chain, keeps them in
+// registers for the whole clip and needs no communication with the CTAs that own the other columns.
+//
+// Pass 1 (t = 0..T-1) stores P_t^T.  Pass 2 (t = T-1..0) carries R_{t+1}^T, first emits the state the
+// queries of frame t read,  P_{t-1}^T + R_{t+1}^T  (zero where a side is missing: the scans start
+// from the zero state), then folds frame t in.  Both passes are written back by the very thread that
+// computed them, so the second pass needs no inter-CTA ordering.
+//
+// C_t is symmetric; the kernel reads it as C_t[j][i] so that each thread's row group is contiguous.
+#pragma once
+#include "common.cuh"
+
+namespace vdn {
+
+template <int D, int W>
+struct ScanSmem {
+  float C[D][D];
+  float X[2][D][W];
+};
+
+// READ_BF16_T = false: read state as float [d_k][d_v] (row i, column c)       -- plain-fp32 read-out
+// READ_BF16_T = true : read state as bf16  [d_v][d_k] (row c, column i)       -- tensor-core read-out
+template <int D, int W, bool READ_BF16_T>
+__global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ stats,
+                                                       const float* __restrict__ inv,
+                                                       float* __restrict__ fwd, void* __restrict__ read,
+                                                       int T) {
+  constexpr int TI = D / 32;          // rows per thread
+  constexpr int NCG = W / 4;          // column groups of 4
+  static_assert(256 / NCG * TI == D, "thread tiling must cover D rows");
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  ScanSmem<D, W>& sm = *reinterpret_cast<ScanSmem<D, W>*>(smem_raw);
+
+  const int bh = blockIdx.x;
+  const int c0 = blockIdx.y * W;
+  const int tid = threadIdx.x;
+  const int cg = tid % NCG, ig = tid / NCG;
+  const int i0 = ig * TI, cc0 = cg * 4;
+
+  float z[TI][4];
+#pragma unroll
+  for (int r = 0; r < TI; ++r)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) z[r][c] = 0.f;
+
+  int buf = 0;
+  for (int step = 0; step < 2 * T; ++step) {
+    const bool forward = step < T;
+    const int t = forward ? step : (2 * T - 1 - step);
+    const size_t n = (size_t)bh * T + t;
+
+    // C_t -> shared memory (asynchronously, 16 bytes per request)
+    {
+      const float* src = inv + n * D * D;
+      float* dst = &sm.C[0][0];
+      for (int e = tid * 4; e < D * D; e += 256 * 4) cp_async16(dst + e, src + e);
+      cp_async_commit();
+    }
+
+    if (!forward) {
+      // gather: the state read by frame t's queries
+      float p[TI][4];
+#pragma unroll
+      for (int r = 0; r < TI; ++r) {
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t > 0) x = load4(fwd + (n - 1) * D * D + (size_t)(i0 + r) * D + c0 + cc0);
+        p[r][0] = x.x + z[r][0]; p[r][1] = x.y + z[r][1]; p[r][2] = x.z + z[r][2]; p[r][3] = x.w + z[r][3];
+      }
+      if constexpr (READ_BF16_T) {
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(read) + n * D * D;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          __nv_bfloat16* row = dst + (size_t)(c0 + cc0 + c) * D + i0;
+          if constexpr (TI == 4) {
+            store4(row, make_float4(p[0][c], p[1][c], p[2][c], p[3][c]));
+          } else {
+#pragma unroll
+            for (int r = 0; r < TI; ++r) row[r] = __float2bfloat16_rn(p[r][c]);
+          }
+        }
+      } else {
+        float* dst = reinterpret_cast<float*>(read) + n * D * D;
+#pragma unroll
+        for (int r = 0; r < TI; ++r)
+          store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(p[r][0], p[r][1], p[r][2], p[r][3]));
+      }
+    }
+
+    // X = Z + B_t^T (this CTA's columns)
+    {
+      const float* bt = stats + n * D * 2 * D + D + c0 + cc0;
+#pragma unroll
+      for (int r = 0; r < TI; ++r) {
+        float4 x = load4(bt + (size_t)(i0 + r) * 2 * D);
+        x.x += z[r][0]; x.y += z[r][1]; x.z += z[r][2]; x.w += z[r][3];
+        store4(&sm.X[buf][i0 + r][cc0], x);
+      }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+
+    // Z = C_t X
+#pragma unroll
+    for (int r = 0; r < TI; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) z[r][c] = 0.f;
+#pragma unroll 8
+    for (int j = 0; j < D; ++j) {
+      float a[TI];
+      if constexpr (TI == 4) {
+        float4 v = load4(&sm.C[j][i0]);
+        a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w;
+      } else {
+        float2 v = *reinterpret_cast<const float2*>(&sm.C[j][i0]);
+        a[0] = v.x; a[1] = v.y;
+      }
+      float4 x = load4(&sm.X[buf][j][cc0]);
+#pragma unroll
+      for (int r = 0; r < TI; ++r) {
+        z[r][0] = fmaf(a[r], x.x, z[r][0]);
+        z[r][1] = fmaf(a[r], x.y, z[r][1]);
+        z[r][2] = fmaf(a[r], x.z, z[r][2]);
+        z[r][3] = fmaf(a[r], x.w, z[r][3]);
+      }
+    }
+    __syncthreads();   // everyone is done with C before the next step overwrites it
+    buf ^= 1;
+
+    if (forward) {
+      float* dst = fwd + n * D * D;
+#pragma unroll
+      for (int r = 0; r < TI; ++r)
+        store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(z[r][0], z[r][1], z[r][2], z[r][3]));
+    }
+    if (step == T - 1) {
+      // the reverse scan starts from the zero state
+#pragma unroll
+      for (int r = 0; r < TI; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) z[r][c] = 0.f;
+    }
+  }
+}
+
+}  // namespace vdn

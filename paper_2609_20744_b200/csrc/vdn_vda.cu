@@ -1,0 +1,409 @@
+// Host side of the VDA forward library: handle, argument checks, workspace layout, kernel dispatch.
+// The exported functions are documented in include/vdn_vda.h.
+#include "../../include/vdn_vda.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "common.cuh"
+#include "gram_simt.cuh"
+#include "readout_simt.cuh"
+#include "resolve.cuh"
+#include "scan.cuh"
+
+namespace {
+
+using vdn::Shape;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Offsets of the workspace regions (bytes).  One layout for every path; only the element size of the
+// read state differs.
+struct Layout {
+  size_t stats, inv, fwd, read, total;
+};
+
+struct StagingLayout {
+  size_t q, k, v, out, beta, gate, total;
+};
+
+}  // namespace
+
+// Optional per-kernel timing: a ring of CUDA-event sets recorded on the caller's stream, one set per
+// forward call, folded into running sums when read (or when the ring wraps).
+struct Profiler {
+  static constexpr int kMaxKernels = 8;
+  static constexpr int kSets = 128;
+  bool on = false;
+  cudaEvent_t ev[kSets][kMaxKernels + 1];
+  int marks[kSets];          // events recorded in each pending set
+  int head = 0, pending = 0; // ring state
+  const char* names[kMaxKernels] = {};
+  double sum_ms[kMaxKernels] = {};
+  int count[kMaxKernels] = {};
+  int cur = -1;
+};
+
+struct vdn_vda_s {
+  vdn_vda_config cfg;
+  Profiler prof;
+  int sm_count = 0;
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  void* staging = nullptr;
+  size_t staging_bytes = 0;
+  int* status_host = nullptr;  // pinned, device-mapped
+  int* status_dev = nullptr;
+  int launches = 0;
+  bool attrs_set = false;
+  std::string err = "no error";
+};
+
+namespace {
+
+vdn_status fail(vdn_vda_t h, vdn_status st, const std::string& msg) {
+  if (h) h->err = msg;
+  return st;
+}
+
+bool use_tensor_cores(const vdn_vda_s* h, int d) {
+  (void)h; (void)d;
+  return false;
+}
+
+size_t elem_size(const vdn_vda_s* h) { return h->cfg.io_dtype == VDN_BF16 ? 2 : 4; }
+
+bool shape_ok(const vdn_vda_s* h, int B, int T, int F, int H, int d, std::string* why) {
+  if (B <= 0 || T <= 0 || F <= 0 || H <= 0) { *why = "B, T, F, H must be positive"; return false; }
+  if (d != h->cfg.d) { *why = "d differs from the handle's configured head dimension"; return false; }
+  const long long tok = (long long)B * T * F;
+  if (tok > 0x7fffffffLL / 2) { *why = "B*T*F exceeds the 32-bit token index range"; return false; }
+  if ((long long)B * H * T > 0x7fffffffLL / 4) { *why = "B*H*T exceeds the grid range"; return false; }
+  if ((long long)B * H > 65535LL * 1024) { *why = "B*H too large"; return false; }
+  return true;
+}
+
+Layout make_layout(const vdn_vda_s* h, int B, int T, int H, int d) {
+  const size_t n = (size_t)B * H * T;
+  const size_t dd = (size_t)d * d;
+  Layout L;
+  size_t off = kAlign;  // a reserved header line
+  L.stats = off; off += align_up(n * dd * 2 * sizeof(float));
+  L.inv = off;   off += align_up(n * dd * sizeof(float));
+  L.fwd = off;   off += align_up(n * dd * sizeof(float));
+  L.read = off;  off += align_up(n * dd * (use_tensor_cores(h, d) ? 2 : sizeof(float)));
+  L.total = off;
+  return L;
+}
+
+StagingLayout make_staging(const vdn_vda_s* h, int B, int T, int F, int H, int d) {
+  const size_t tokh = (size_t)B * T * F * H;
+  const size_t big = align_up(tokh * d * elem_size(h));
+  StagingLayout S;
+  size_t off = 0;
+  S.q = off; off += big;
+  S.k = off; off += big;
+  S.v = off; off += big;
+  S.out = off; off += big;
+  S.beta = off; off += align_up(tokh * sizeof(float));
+  S.gate = off; off += align_up((size_t)H * sizeof(float));
+  S.total = off;
+  return S;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+#define VDN_CUDA(h, call)                                                                      \
+  do {                                                                                         \
+    cudaError_t e_ = (call);                                                                   \
+    if (e_ != cudaSuccess)                                                                     \
+      return fail((h), VDN_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_));      \
+  } while (0)
+
+void prof_fold_oldest(Profiler& p) {
+  const int set = (p.head - p.pending + Profiler::kSets) % Profiler::kSets;
+  const int m = p.marks[set];
+  if (m > 0 && cudaEventSynchronize(p.ev[set][m]) == cudaSuccess) {
+    for (int i = 0; i < m; ++i) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, p.ev[set][i], p.ev[set][i + 1]) == cudaSuccess) {
+        p.sum_ms[i] += ms;
+        p.count[i] += 1;
+      }
+    }
+  }
+  cudaGetLastError();
+  p.pending -= 1;
+}
+
+// Opens a new event set for this forward call and records its first event.
+void prof_begin(vdn_vda_t h, cudaStream_t st) {
+  Profiler& p = h->prof;
+  if (!p.on) return;
+  if (p.pending == Profiler::kSets) prof_fold_oldest(p);
+  p.cur = p.head;
+  p.head = (p.head + 1) % Profiler::kSets;
+  p.pending += 1;
+  p.marks[p.cur] = 0;
+  cudaEventRecord(p.ev[p.cur][0], st);
+}
+
+// Records the event that closes kernel number `idx` of this forward call.
+void prof_mark(vdn_vda_t h, cudaStream_t st, int idx, const char* name) {
+  Profiler& p = h->prof;
+  if (!p.on || p.cur < 0 || idx >= Profiler::kMaxKernels) return;
+  p.names[idx] = name;
+  cudaEventRecord(p.ev[p.cur][idx + 1], st);
+  p.marks[p.cur] = idx + 1;
+}
+
+template <typename Tio, int D>
+vdn_status set_attrs_simt(vdn_vda_t h) {
+  VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_kernel<D, 32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)sizeof(vdn::ScanSmem<D, 32>)));
+  VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_simt_kernel<Tio, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)sizeof(vdn::ReadoutSimtSmem<D>)));
+  return VDN_OK;
+}
+
+// The plain-fp32 path: four launches.
+template <typename Tio, int D>
+vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                        const float* gate, void* out, const Shape& s, const Layout& L, cudaStream_t st) {
+  if (!h->attrs_set) {
+    vdn_status r = set_attrs_simt<Tio, D>(h);
+    if (r != VDN_OK) return r;
+    h->attrs_set = true;
+  }
+  char* ws = static_cast<char*>(h->workspace);
+  float* stats = reinterpret_cast<float*>(ws + L.stats);
+  float* inv = reinterpret_cast<float*>(ws + L.inv);
+  float* fwd = reinterpret_cast<float*>(ws + L.fwd);
+  float* read = reinterpret_cast<float*>(ws + L.read);
+  const long long n = s.frames();
+
+  prof_begin(h, st);
+  vdn::gram_simt_kernel<Tio, D><<<dim3((unsigned)n, 2 * D / 64), 256, 0, st>>>(
+      static_cast<const Tio*>(k), static_cast<const Tio*>(v), beta, stats, s);
+  prof_mark(h, st, 0, "gram_simt");
+  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, n);
+  prof_mark(h, st, 1, "resolve");
+  vdn::scan_kernel<D, 32, false><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
+      stats, inv, fwd, read, s.T);
+  prof_mark(h, st, 2, "scan");
+  vdn::readout_simt_kernel<Tio, D><<<dim3((unsigned)n, (s.F + 63) / 64), 256, sizeof(vdn::ReadoutSimtSmem<D>), st>>>(
+      static_cast<const Tio*>(q), read, gate, static_cast<Tio*>(out), s, h->cfg.rms_eps);
+  prof_mark(h, st, 3, "readout_simt");
+  h->launches = 4;
+  VDN_CUDA(h, cudaGetLastError());
+  return VDN_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+vdn_status vdn_vda_create(const vdn_vda_config* cfg, vdn_vda_t* out_handle) {
+  if (!cfg || !out_handle) return VDN_ERR_INVALID_ARG;
+  *out_handle = nullptr;
+  if (cfg->struct_size != sizeof(vdn_vda_config)) return VDN_ERR_INVALID_ARG;
+  if (cfg->io_dtype != VDN_F32 && cfg->io_dtype != VDN_BF16) return VDN_ERR_INVALID_ARG;
+  if (cfg->d != 64 && cfg->d != 128) return VDN_ERR_UNSUPPORTED;
+  if (cfg->device < 0) return VDN_ERR_INVALID_ARG;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess) { cudaGetLastError(); return VDN_ERR_CUDA; }
+  if (cfg->device >= count) return VDN_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) { cudaGetLastError(); return VDN_ERR_CUDA; }
+  if (prop.major != 10) return VDN_ERR_ARCH;
+
+  vdn_vda_s* h = new (std::nothrow) vdn_vda_s();
+  if (!h) return VDN_ERR_CUDA;
+  h->cfg = *cfg;
+  if (!(h->cfg.rms_eps > 0.f)) h->cfg.rms_eps = 1e-6f;
+  h->sm_count = prop.multiProcessorCount;
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok || cudaHostAlloc(reinterpret_cast<void**>(&h->status_host), 64, cudaHostAllocMapped) != cudaSuccess ||
+      cudaHostGetDevicePointer(reinterpret_cast<void**>(&h->status_dev), h->status_host, 0) != cudaSuccess) {
+    cudaGetLastError();
+    if (h->status_host) cudaFreeHost(h->status_host);
+    delete h;
+    return VDN_ERR_CUDA;
+  }
+  std::memset(h->status_host, 0, 64);
+  *out_handle = h;
+  return VDN_OK;
+}
+
+size_t vdn_vda_workspace_bytes(vdn_vda_t h, int B, int T, int F, int H, int d) {
+  std::string why;
+  if (!h || !shape_ok(h, B, T, F, H, d, &why)) return 0;
+  return make_layout(h, B, T, H, d).total;
+}
+
+vdn_status vdn_vda_set_workspace(vdn_vda_t h, void* dev_ptr, size_t bytes) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) != 0)
+    return fail(h, VDN_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+  h->workspace = dev_ptr;
+  h->workspace_bytes = dev_ptr ? bytes : 0;
+  return VDN_OK;
+}
+
+size_t vdn_vda_staging_bytes(vdn_vda_t h, int B, int T, int F, int H, int d) {
+  std::string why;
+  if (!h || !shape_ok(h, B, T, F, H, d, &why)) return 0;
+  return make_staging(h, B, T, F, H, d).total;
+}
+
+vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) != 0)
+    return fail(h, VDN_ERR_INVALID_ARG, "staging buffer must be 256-byte aligned");
+  h->staging = dev_ptr;
+  h->staging_bytes = dev_ptr ? bytes : 0;
+  return VDN_OK;
+}
+
+vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                           const float* gate, void* out, int B, int T, int F, int H, int d,
+                           void* cuda_stream) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  if (!q || !k || !v || !beta || !gate || !out) return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(beta))
+    return fail(h, VDN_ERR_INVALID_ARG, "q, k, v, beta, out must be 16-byte aligned");
+  if (out == q || out == k || out == v) return fail(h, VDN_ERR_INVALID_ARG, "out must not alias an input");
+  std::string why;
+  if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
+  const Layout L = make_layout(h, B, T, H, d);
+  if (!h->workspace || h->workspace_bytes < L.total)
+    return fail(h, VDN_ERR_WORKSPACE, "workspace not set or smaller than vdn_vda_workspace_bytes");
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Shape s{B, T, F, H, d};
+  if (h->cfg.io_dtype == VDN_F32) {
+    return d == 64 ? forward_simt<float, 64>(h, q, k, v, beta, gate, out, s, L, st)
+                   : forward_simt<float, 128>(h, q, k, v, beta, gate, out, s, L, st);
+  }
+  return d == 64 ? forward_simt<__nv_bfloat16, 64>(h, q, k, v, beta, gate, out, s, L, st)
+                 : forward_simt<__nv_bfloat16, 128>(h, q, k, v, beta, gate, out, s, L, st);
+}
+
+vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const void* v,
+                                const float* beta, const float* gate, void* out, int B, int T, int F,
+                                int H, int d, void* cuda_stream) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  if (!q || !k || !v || !beta || !gate || !out) return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
+  std::string why;
+  if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
+  const StagingLayout S = make_staging(h, B, T, F, H, d);
+  if (!h->staging || h->staging_bytes < S.total)
+    return fail(h, VDN_ERR_WORKSPACE, "staging buffer not set or smaller than vdn_vda_staging_bytes");
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* sg = static_cast<char*>(h->staging);
+  const size_t tokh = (size_t)B * T * F * H;
+  const size_t big = tokh * d * elem_size(h);
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.k, k, big, cudaMemcpyHostToDevice, st));
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.v, v, big, cudaMemcpyHostToDevice, st));
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.beta, beta, tokh * sizeof(float), cudaMemcpyHostToDevice, st));
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.q, q, big, cudaMemcpyHostToDevice, st));
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.gate, gate, (size_t)H * sizeof(float), cudaMemcpyHostToDevice, st));
+  vdn_status r = vdn_vda_forward(h, sg + S.q, sg + S.k, sg + S.v, reinterpret_cast<const float*>(sg + S.beta),
+                                 reinterpret_cast<const float*>(sg + S.gate), sg + S.out, B, T, F, H, d,
+                                 cuda_stream);
+  if (r != VDN_OK) return r;
+  VDN_CUDA(h, cudaMemcpyAsync(out, sg + S.out, big, cudaMemcpyDeviceToHost, st));
+  return VDN_OK;
+}
+
+vdn_status vdn_vda_workspace_view(vdn_vda_t h, int which, int B, int T, int F, int H, int d,
+                                  size_t* offset_bytes, size_t* size_bytes) {
+  if (!h || !offset_bytes || !size_bytes) return VDN_ERR_INVALID_ARG;
+  std::string why;
+  if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
+  const Layout L = make_layout(h, B, T, H, d);
+  const size_t n = (size_t)B * H * T, dd = (size_t)d * d;
+  switch (which) {
+    case VDN_VIEW_STATS: *offset_bytes = L.stats; *size_bytes = n * dd * 2 * sizeof(float); break;
+    case VDN_VIEW_INV:   *offset_bytes = L.inv;   *size_bytes = n * dd * sizeof(float); break;
+    case VDN_VIEW_FWD:   *offset_bytes = L.fwd;   *size_bytes = n * dd * sizeof(float); break;
+    case VDN_VIEW_READ:  *offset_bytes = L.read;  *size_bytes = n * dd * (use_tensor_cores(h, d) ? 2 : sizeof(float)); break;
+    default: return fail(h, VDN_ERR_INVALID_ARG, "unknown view");
+  }
+  return VDN_OK;
+}
+
+int vdn_vda_last_launch_count(vdn_vda_t h) { return h ? h->launches : 0; }
+
+vdn_status vdn_vda_profile(vdn_vda_t h, int enable) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  Profiler& p = h->prof;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
+  if (enable && !p.on) {
+    for (int s = 0; s < Profiler::kSets; ++s)
+      for (int i = 0; i <= Profiler::kMaxKernels; ++i) VDN_CUDA(h, cudaEventCreate(&p.ev[s][i]));
+    p.on = true;
+  } else if (!enable && p.on) {
+    for (int s = 0; s < Profiler::kSets; ++s)
+      for (int i = 0; i <= Profiler::kMaxKernels; ++i) cudaEventDestroy(p.ev[s][i]);
+    p.on = false;
+  }
+  p.head = p.pending = 0;
+  p.cur = -1;
+  for (int i = 0; i < Profiler::kMaxKernels; ++i) { p.sum_ms[i] = 0.0; p.count[i] = 0; p.names[i] = nullptr; }
+  return VDN_OK;
+}
+
+int vdn_vda_kernel_times(vdn_vda_t h, int max_kernels, const char** names, float* mean_ms, int* launches) {
+  if (!h || !names || !mean_ms || !launches || max_kernels <= 0) return 0;
+  Profiler& p = h->prof;
+  if (!p.on) return 0;
+  DeviceGuard guard(h->cfg.device);
+  while (p.pending > 0) prof_fold_oldest(p);
+  int n = 0;
+  for (int i = 0; i < Profiler::kMaxKernels && n < max_kernels; ++i) {
+    if (!p.names[i] || p.count[i] == 0) continue;
+    names[n] = p.names[i];
+    mean_ms[n] = (float)(p.sum_ms[i] / p.count[i]);
+    launches[n] = p.count[i];
+    ++n;
+  }
+  return n;
+}
+
+vdn_status vdn_vda_status(vdn_vda_t h) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  const int v = *const_cast<volatile int*>(h->status_host);
+  return v == 0 ? VDN_OK : VDN_ERR_TIMEOUT;
+}
+
+const char* vdn_vda_last_error(vdn_vda_t h) { return h ? h->err.c_str() : "null handle"; }
+
+vdn_status vdn_vda_destroy(vdn_vda_t h) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  if (h->prof.on) vdn_vda_profile(h, 0);
+  if (h->status_host) cudaFreeHost(h->status_host);
+  delete h;
+  return VDN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,201 @@
+"""Parity of the CUDA library (through the C ABI) against the fp64 checker, element by element.
+
+Tolerances (the metric is oracle.slice_error: max |gpu - ref| over one (batch, head) slice divided
+by that slice's max |ref|):  1e-4 for f32 I/O,  2e-2 for bf16 I/O.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import vda_oracle as orc
+from paper_2609_20744_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    binding.load_library()
+
+
+def run_gpu(w, x, flags=0):
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    assert vda.launch_count() > 0
+    return vda, out
+
+
+def check_heads(w, x, out, pairs, tol):
+    worst = 0.0
+    for (b, h) in pairs:
+        q, k, v, beta, gate = inputs.head_slice(x, b, h)
+        ref = orc.vda_slice(q, k, v, beta, gate, 1e-6)["out"]
+        got = out[b, :, :, h, :].double().cpu().numpy()
+        assert np.isfinite(got).all()
+        e = orc.slice_error(got, ref)
+        worst = max(worst, e)
+        assert e <= tol, f"slice (b={b}, h={h}) error {e:.3e} > {tol}"
+    return worst
+
+
+def all_pairs(w):
+    return [(b, h) for b in range(w.B) for h in range(w.H)]
+
+
+# ------------------------------------------------------------------------------ whole layer
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", {}),                                              # the f32 benchmark config
+    ("tiny", dict(d=128, F=100, T=5, H=3)),                    # d=128, ragged token tail
+    ("tiny", dict(T=1)),                                       # single frame -> all zeros
+    ("tiny", dict(T=2, F=1)),                                  # one token per frame
+    ("tiny", dict(B=2, H=1, T=3, F=257)),                      # several tiles + tail, two batches
+    ("tiny", dict(dtype="bf16", d=128, T=6, F=300, H=2)),      # bf16 I/O
+    ("tiny", dict(dtype="bf16", d=64, T=3, F=70, H=2)),
+])
+def test_forward_matches_oracle_small(name, kw):
+    w = inputs.WORKLOADS[name].scaled(**kw)
+    x = inputs.generate(w, "cuda")
+    _, out = run_gpu(w, x)
+    if w.T == 1:
+        assert torch.count_nonzero(out) == 0
+    check_heads(w, x, out, all_pairs(w), TOL[w.dtype])
+
+
+def test_bf16_through_plain_fp32_kernels():
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=4, F=200, H=2)
+    x = inputs.generate(w, "cuda")
+    _, out = run_gpu(w, x, flags=binding.VDN_FLAG_FORCE_SIMT)
+    check_heads(w, x, out, all_pairs(w), TOL["bf16"])
+
+
+def test_480p_config_all_heads():
+    w = inputs.CLIP_480P
+    x = inputs.generate(w, "cuda")
+    _, out = run_gpu(w, x)
+    check_heads(w, x, out, all_pairs(w), TOL[w.dtype])
+
+
+# ------------------------------------------------------------------------------ stage-wise
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("f32", 128), ("bf16", 128)])
+def test_stagewise_intermediates(dtype, d):
+    w = inputs.TINY.scaled(dtype=dtype, d=d, T=5, F=150, H=2)
+    x = inputs.generate(w, "cuda")
+    vda, out = run_gpu(w, x)
+    B, T, F, H = w.B, w.T, w.F, w.H
+    stats = vda.view(binding.VIEW_STATS, B, T, F, H).double().cpu().numpy()
+    inv = vda.view(binding.VIEW_INV, B, T, F, H).double().cpu().numpy()
+    fwd = vda.view(binding.VIEW_FWD, B, T, F, H).double().cpu().numpy()
+    read = vda.view(binding.VIEW_READ, B, T, F, H)
+    read_is_bf16 = read.dtype == torch.bfloat16
+    read = read.double().cpu().numpy()
+    rel = lambda g, r: np.max(np.abs(g - r)) / max(np.max(np.abs(r)), 1e-30)
+    # bf16 products are exact in fp32; only the beta-scaled operand is rounded once to bf16
+    tol_stats = 1e-5 if dtype == "f32" else 4e-3
+    tol_state = 1e-4 if dtype == "f32" else 1e-2
+    for h in range(H):
+        q, k, v, beta, gate = inputs.head_slice(x, 0, h)
+        ref = orc.vda_slice(q, k, v, beta, gate, 1e-6, want=("A", "B", "C", "P", "R"))
+        for t in range(T):
+            assert rel(stats[0, h, t, :, :d], ref["A"][t]) < tol_stats
+            assert rel(stats[0, h, t, :, d:], ref["B"][t].T) < tol_stats
+            assert rel(inv[0, h, t], ref["C"][t]) < tol_state
+            assert rel(fwd[0, h, t], ref["P"][t].T) < tol_state
+            want = np.zeros((d, d))
+            if t > 0:
+                want = want + ref["P"][t - 1]
+            if t + 1 < T:
+                want = want + ref["R"][t + 1]
+            got = read[0, h, t] if read_is_bf16 else read[0, h, t].T     # -> paper orientation [d_v][d_k]
+            assert rel(got, want) < (tol_state if not read_is_bf16 else 1e-2)
+
+
+# ------------------------------------------------------------------------------ properties
+def test_run_to_run_bitwise_determinism_and_canaries():
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=4, F=333, H=3)
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    n = x["q"].numel()
+    pad = 4096
+    buf = torch.full((n + 2 * pad,), 7.0, dtype=x["q"].dtype, device="cuda")
+    out = buf[pad: pad + n].view_as(x["q"])
+    vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out)
+    torch.cuda.synchronize()
+    first = out.clone()
+    vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out)
+    torch.cuda.synchronize()
+    assert torch.equal(first, out)
+    assert torch.all(buf[:pad] == 7.0) and torch.all(buf[pad + n:] == 7.0)
+
+
+def test_token_permutation_within_frames_permutes_rows_only():
+    w = inputs.TINY.scaled(d=128, T=3, F=96, H=2)
+    x = inputs.generate(w, "cuda")
+    _, out = run_gpu(w, x)
+    perm = torch.randperm(w.F, generator=torch.Generator().manual_seed(5)).cuda()
+    xp = {n: (t[:, :, perm] if t.dim() >= 4 else t).contiguous() for n, t in x.items()}
+    _, outp = run_gpu(w, xp)
+    assert torch.allclose(outp, out[:, :, perm], atol=2e-5)
+
+
+def test_frame_reversal_reverses_output():
+    w = inputs.TINY.scaled(d=64, T=5, F=64, H=2)
+    x = inputs.generate(w, "cuda")
+    _, out = run_gpu(w, x)
+    xr = {n: (t.flip(1) if t.dim() >= 4 else t).contiguous() for n, t in x.items()}
+    _, outr = run_gpu(w, xr)
+    assert torch.allclose(outr.flip(1), out, atol=2e-5)
+
+
+def test_output_rows_have_gate_sized_rms():
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=4, F=130, H=3)
+    x = inputs.generate(w, "cuda")
+    _, out = run_gpu(w, x)
+    ms = out.float().pow(2).mean(dim=-1)                      # [B,T,F,H]
+    want = x["gate"].pow(2)[None, None, None, :].expand_as(ms)
+    assert torch.allclose(ms, want, rtol=3e-2)
+
+
+# ------------------------------------------------------------------------------ host-buffer entry point
+def test_forward_host_matches_device_entry_point():
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=3, F=200, H=2)
+    xh = inputs.generate(w, "cpu", pin=True)
+    xd = {n: t.cuda() for n, t in xh.items()}
+    vda, out_d = run_gpu(w, xd)
+    out_h = torch.empty_like(xh["q"]).pin_memory()
+    vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], out_h)
+    torch.cuda.synchronize()
+    assert torch.equal(out_h, out_d.cpu())
+
+
+# ------------------------------------------------------------------------------ argument errors (host side)
+def test_argument_errors_enqueue_nothing():
+    w = inputs.TINY
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    with pytest.raises(binding.VdnError) as e:
+        vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=x["q"])      # aliasing
+    assert e.value.status == 1
+    vda2 = binding.Vda(128, "f32")
+    with pytest.raises(binding.VdnError):
+        vda2.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])                 # d mismatch
+    import ctypes
+    vda3 = binding.Vda(w.d, w.dtype)
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    vda3.lib.vdn_vda_set_workspace(vda3.h, ctypes.c_void_p(small.data_ptr()), 1024)
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    out = torch.empty_like(x["q"])
+    st = vda3.lib.vdn_vda_forward(vda3.h, p(x["q"]), p(x["k"]), p(x["v"]), p(x["beta"]), p(x["gate"]), p(out),
+                                  w.B, w.T, w.F, w.H, w.d, None)
+    assert st == 3                                                                  # workspace too small
+    st = vda3.lib.vdn_vda_forward(vda3.h, None, p(x["k"]), p(x["v"]), p(x["beta"]), p(x["gate"]), p(out),
+                                  w.B, w.T, w.F, w.H, w.d, None)
+    assert st == 1
+    st = vda3.lib.vdn_vda_forward(vda3.h, ctypes.c_void_p(x["q"].data_ptr() + 4), p(x["k"]), p(x["v"]),
+                                  p(x["beta"]), p(x["gate"]), p(out), w.B, w.T, w.F, w.H, w.d, None)
+    assert st == 1                                                                  # misaligned
+    torch.cuda.synchronize()
