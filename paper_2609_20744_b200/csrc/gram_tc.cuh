@@ -1,0 +1,222 @@
+// Frame statistics (Eq. 3b) on the tcgen05 tensor cores, bf16 operands, fp32 accumulation in TMEM.
+//
+//   [ A_t | B_t^T ] = (Diag(beta_t) K_t)^T [ K_t | V_t ]          128 x 256 per frame (d = 128)
+//
+// The contraction index is the token, so both operands are "MN-major": a token's 128 channels are
+// contiguous in memory, and TMA drops each 128-token tile into shared memory as 64-channel boxes with
+// the 128-byte swizzle, exactly the canonical MN-major layout the MMA reads.
+//
+// Persistent CTAs, one per SM, loop over frames (b,h,t).  Warp roles:
+//   warp 0      TMA producer: K and V tiles (4 boxes of 16 KB) into a 3-stage ring
+//   warp 1      MMA issuer (one thread) and TMEM owner
+//   warps 2-5   weighting: K' = beta * K, rounded once to bf16, written to a second buffer in two halves of
+//               64 tokens so the MMA of one half overlaps the weighting of the other
+//   warps 6-9   epilogue: TMEM -> registers -> global fp32 [d][2d]; two accumulators, so the drain of
+//               frame i overlaps the main loop of frame i+1
+// Rows past the end of a frame are zero-filled by TMA (the map has F as its own dimension) and their
+// beta is forced to zero.  Every mbarrier wait is bounded.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace vdn {
+
+struct GramTc {
+  static constexpr int D = 128;
+  static constexpr int TILE = 128;                 // tokens per tile
+  static constexpr int STAGES = 3;
+  static constexpr int BOX_BYTES = TILE * 128;     // one 64-channel box: 128 tokens x 128 B
+  static constexpr int STAGE_BYTES = 4 * BOX_BYTES;       // K lo, K hi, V lo, V hi
+  static constexpr int KP_HALF_BYTES = 2 * 64 * 128;      // 2 boxes x 64 tokens x 128 B
+  static constexpr int OFF_KP = STAGES * STAGE_BYTES;
+  static constexpr int OFF_BAR = OFF_KP + 2 * KP_HALF_BYTES;
+  static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // barriers + alignment slack
+  static constexpr int THREADS = 320;
+};
+
+__global__ void __launch_bounds__(GramTc::THREADS, 1)
+gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+               const float* __restrict__ beta, float* __restrict__ stats, Shape s, int* status) {
+  using namespace tc;
+  using G = GramTc;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+
+  // barrier block
+  const uint32_t bar0 = base + G::OFF_BAR;
+  auto FULL = [&](int i) { return bar0 + 8u * i; };            // 3
+  auto EMPTY = [&](int i) { return bar0 + 8u * (3 + i); };     // 3
+  auto SCALED = [&](int i) { return bar0 + 8u * (6 + i); };    // 2
+  auto KPFREE = [&](int i) { return bar0 + 8u * (8 + i); };    // 2
+  auto ACCFULL = [&](int i) { return bar0 + 8u * (10 + i); };  // 2
+  auto ACCEMPTY = [&](int i) { return bar0 + 8u * (12 + i); }; // 2
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + G::OFF_BAR + 8 * 14);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + G::OFF_BAR + 8 * 14 + 8);
+  const WaitCtx wc{abort_flag, status};
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ntiles = (s.F + G::TILE - 1) / G::TILE;
+  const long long nitems = s.frames();
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 3; ++i) { mbar_init(FULL(i), 1); mbar_init(EMPTY(i), 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(SCALED(i), 128); mbar_init(KPFREE(i), 1);
+      mbar_init(ACCFULL(i), 1);  mbar_init(ACCEMPTY(i), 128);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmK);
+    tma_prefetch_desc(&tmV);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
+        int b, h, t;
+        split_frame(s, item, b, h, t);
+        for (int tile = 0; tile < ntiles; ++tile, ++it) {
+          const int st = it % G::STAGES;
+          if (!mbar_wait(EMPTY(st), ((it / G::STAGES) & 1) ^ 1, wc)) { ok = false; break; }
+          mbar_arrive_expect_tx(FULL(st), G::STAGE_BYTES);
+          const uint32_t dst = base + st * G::STAGE_BYTES;
+          const int u0 = tile * G::TILE;
+          tma_load_5d(dst + 0 * G::BOX_BYTES, &tmK, FULL(st), 0, h, u0, t, b);
+          tma_load_5d(dst + 1 * G::BOX_BYTES, &tmK, FULL(st), 64, h, u0, t, b);
+          tma_load_5d(dst + 2 * G::BOX_BYTES, &tmV, FULL(st), 0, h, u0, t, b);
+          tma_load_5d(dst + 3 * G::BOX_BYTES, &tmV, FULL(st), 64, h, u0, t, b);
+        }
+      }
+      if (!ok) {
+        // give copies that are already in flight a bounded chance to land before the CTA retires
+        for (int st = 0; st < G::STAGES; ++st)
+          for (int spin = 0; spin < 4096 && !mbar_try_wait(FULL(st), 0) && !mbar_try_wait(FULL(st), 1); ++spin) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(128, 256, true, true);
+      uint32_t it = 0, ai = 0;
+      bool ok = true;
+      for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++ai) {
+        const int a = ai & 1;
+        if (!mbar_wait(ACCEMPTY(a), ((ai >> 1) & 1) ^ 1, wc)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t acc = tmem_base + a * 256;
+        for (int tile = 0; tile < ntiles && ok; ++tile, ++it) {
+          const int st = it % G::STAGES;
+          if (!mbar_wait(FULL(st), (it / G::STAGES) & 1, wc)) { ok = false; break; }
+          for (int half = 0; half < 2; ++half) {
+            if (!mbar_wait(SCALED(half), it & 1, wc)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t a_base = base + G::OFF_KP + half * G::KP_HALF_BYTES;
+            const uint32_t b_base = base + st * G::STAGE_BYTES + half * 64 * 128;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint64_t adesc = make_smem_desc(a_base + j * 2048, 64 * 128, 1024);
+              const uint64_t bdesc = make_smem_desc(b_base + j * 2048, G::BOX_BYTES, 1024);
+              mma_bf16_ss(acc, adesc, bdesc, idesc, (tile | half | j) != 0 ? 1u : 0u);
+            }
+            mma_commit(KPFREE(half));
+          }
+          if (!ok) break;
+          mma_commit(EMPTY(st));
+        }
+        if (ok) mma_commit(ACCFULL(a));
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ weighting warps: K' = beta * K
+    const int ts = threadIdx.x - 64;          // 0..127
+    const int r = ts >> 1, c = ts & 1;        // row within the half, 64-channel box
+    uint32_t it = 0;
+    bool ok = true;
+    for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
+      int b, h, t;
+      split_frame(s, item, b, h, t);
+      const float* brow = beta + ((size_t)b * s.T + t) * s.F * s.H + h;
+      for (int tile = 0; tile < ntiles && ok; ++tile, ++it) {
+        const int st = it % G::STAGES;
+        float bu[2];
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int u = tile * G::TILE + half * 64 + r;
+          bu[half] = (u < s.F) ? __ldg(brow + (size_t)u * s.H) : 0.f;
+        }
+        if (!mbar_wait(FULL(st), (it / G::STAGES) & 1, wc)) { ok = false; break; }
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          if (!mbar_wait(KPFREE(half), (it & 1) ^ 1, wc)) { ok = false; break; }
+          const unsigned char* src = base_ptr + st * G::STAGE_BYTES + c * G::BOX_BYTES + (half * 64 + r) * 128;
+          unsigned char* dst = base_ptr + G::OFF_KP + half * G::KP_HALF_BYTES + c * (64 * 128) + r * 128;
+          const float w = bu[half];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int pj = (j ^ (r & 7)) * 16;   // stagger the 16-byte chunks across rows: conflict-free
+            uint4 raw = *reinterpret_cast<const uint4*>(src + pj);
+            uint32_t* x = reinterpret_cast<uint32_t*>(&raw);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float lo = __uint_as_float(x[e] << 16) * w;
+              const float hi = __uint_as_float(x[e] & 0xFFFF0000u) * w;
+              __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+              x[e] = *reinterpret_cast<uint32_t*>(&p);
+            }
+            *reinterpret_cast<uint4*>(dst + pj) = raw;
+          }
+          fence_proxy_async_smem();
+          mbar_arrive(SCALED(half));
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps: TMEM -> global
+    const int qd = warp & 3;                   // TMEM lane quarter this warp may read
+    const int row = qd * 32 + lane;
+    uint32_t ai = 0;
+    bool ok = true;
+    for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++ai) {
+      const int a = ai & 1;
+      if (!mbar_wait(ACCFULL(a), (ai >> 1) & 1, wc)) { ok = false; break; }
+      tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 256;
+      float* dst = stats + (size_t)item * (G::D * 2 * G::D) + (size_t)row * (2 * G::D);
+#pragma unroll 1
+      for (int cc = 0; cc < 8; ++cc) {
+        float v[32];
+        tmem_ld32(taddr + cc * 32, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) store4(dst + cc * 32 + e, make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]));
+      }
+      tc_fence_before_sync();
+      mbar_arrive(ACCEMPTY(a));
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace vdn

@@ -1,0 +1,215 @@
+// Read-out (Eq. 1a), RMSNorm and gate (Eq. 1c) on the tcgen05 tensor cores, d = 128, bf16 I/O.
+//
+//   O_t = Q_t (P_{t-1} + R_{t+1})^T      128-token tile x 128 channels, fp32 in TMEM
+//   out = gate_h * O / sqrt(mean_c O^2 + eps)   -> bf16
+//
+// The state each frame reads arrives already summed over the two directions, as bf16 [d_v][d_k]
+// (K-major for the MMA's B operand); Q tiles are K-major as they sit in memory.  Persistent CTAs loop
+// over frames (b,h,t).  Warp roles:
+//   warp 0      TMA producer: the frame's state (2 boxes, double-buffered across frames) and Q tiles
+//               (2 boxes of 16 KB, 3-stage ring)
+//   warp 1      MMA issuer (one thread), 4 accumulators of 128 TMEM columns
+//   warps 2-5   epilogue: tcgen05.ld gives every thread one whole token row, so the sum of squares is
+//               thread-local; the scaled row is packed to bf16, written to a swizzled staging tile and
+//               sent out with a TMA store whose map has F as its own dimension (the tail is clipped)
+// Every mbarrier wait is bounded.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace vdn {
+
+struct ReadoutTc {
+  static constexpr int D = 128;
+  static constexpr int TILE = 128;
+  static constexpr int QSTAGES = 3;
+  static constexpr int BOX_BYTES = 128 * 128;          // 128 rows x 128 B
+  static constexpr int TILE_BYTES = 2 * BOX_BYTES;     // 32 KB: state, Q tile or output tile
+  static constexpr int OFF_STATE = 0;
+  static constexpr int OFF_Q = 2 * TILE_BYTES;
+  static constexpr int OFF_OUT = OFF_Q + QSTAGES * TILE_BYTES;
+  static constexpr int OFF_BAR = OFF_OUT + 2 * TILE_BYTES;
+  static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
+  static constexpr int THREADS = 192;
+};
+
+__global__ void __launch_bounds__(ReadoutTc::THREADS, 1)
+readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmS,
+                  const __grid_constant__ CUtensorMap tmO, const float* __restrict__ gate, Shape s, float eps,
+                  int* status) {
+  using namespace tc;
+  using R = ReadoutTc;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+
+  const uint32_t bar0 = base + R::OFF_BAR;
+  auto QFULL = [&](int i) { return bar0 + 8u * i; };             // 3
+  auto QEMPTY = [&](int i) { return bar0 + 8u * (3 + i); };      // 3
+  auto STFULL = [&](int i) { return bar0 + 8u * (6 + i); };      // 2
+  auto STEMPTY = [&](int i) { return bar0 + 8u * (8 + i); };     // 2
+  auto ACCFULL = [&](int i) { return bar0 + 8u * (10 + i); };    // 4
+  auto ACCEMPTY = [&](int i) { return bar0 + 8u * (14 + i); };   // 4
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 8 * 18);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 8 * 18 + 8);
+  const WaitCtx wc{abort_flag, status};
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ntiles = (s.F + R::TILE - 1) / R::TILE;
+  const long long nitems = s.frames();
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 3; ++i) { mbar_init(QFULL(i), 1); mbar_init(QEMPTY(i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(STFULL(i), 1); mbar_init(STEMPTY(i), 1); }
+    for (int i = 0; i < 4; ++i) { mbar_init(ACCFULL(i), 1); mbar_init(ACCEMPTY(i), 128); }
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmQ);
+    tma_prefetch_desc(&tmS);
+    tma_prefetch_desc(&tmO);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t qi = 0, si = 0;
+      bool ok = true;
+      for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
+        int b, h, t;
+        split_frame(s, item, b, h, t);
+        const int sb = si & 1;
+        if (!mbar_wait(STEMPTY(sb), ((si >> 1) & 1) ^ 1, wc)) { ok = false; break; }
+        mbar_arrive_expect_tx(STFULL(sb), R::TILE_BYTES);
+        const uint32_t sdst = base + R::OFF_STATE + sb * R::TILE_BYTES;
+        tma_load_2d(sdst, &tmS, STFULL(sb), 0, (int)(item * R::D));
+        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(sb), 64, (int)(item * R::D));
+        for (int tile = 0; tile < ntiles; ++tile, ++qi) {
+          const int st = qi % R::QSTAGES;
+          if (!mbar_wait(QEMPTY(st), ((qi / R::QSTAGES) & 1) ^ 1, wc)) { ok = false; break; }
+          mbar_arrive_expect_tx(QFULL(st), R::TILE_BYTES);
+          const uint32_t dst = base + R::OFF_Q + st * R::TILE_BYTES;
+          tma_load_5d(dst, &tmQ, QFULL(st), 0, h, tile * R::TILE, t, b);
+          tma_load_5d(dst + R::BOX_BYTES, &tmQ, QFULL(st), 64, h, tile * R::TILE, t, b);
+        }
+      }
+      if (!ok) {
+        for (int st = 0; st < R::QSTAGES; ++st)
+          for (int spin = 0; spin < 4096 && !mbar_try_wait(QFULL(st), 0) && !mbar_try_wait(QFULL(st), 1); ++spin) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
+      uint32_t qi = 0, si = 0;
+      bool ok = true;
+      for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
+        const int sb = si & 1;
+        if (!mbar_wait(STFULL(sb), (si >> 1) & 1, wc)) { ok = false; break; }
+        const uint32_t sbase = base + R::OFF_STATE + sb * R::TILE_BYTES;
+        for (int tile = 0; tile < ntiles; ++tile, ++qi) {
+          const int st = qi % R::QSTAGES;
+          const int a = qi & 3;
+          if (!mbar_wait(QFULL(st), (qi / R::QSTAGES) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait(ACCEMPTY(a), ((qi >> 2) & 1) ^ 1, wc)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t qbase = base + R::OFF_Q + st * R::TILE_BYTES;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t off = (j >> 2) * R::BOX_BYTES + (j & 3) * 32;   // 16 channels = 32 B inside the swizzled row
+            const uint64_t adesc = make_smem_desc(qbase + off, 16, 1024);
+            const uint64_t bdesc = make_smem_desc(sbase + off, 16, 1024);
+            mma_bf16_ss(tmem_base + a * 128, adesc, bdesc, idesc, j != 0 ? 1u : 0u);
+          }
+          mma_commit(QEMPTY(st));
+          mma_commit(ACCFULL(a));
+        }
+        if (ok) mma_commit(STEMPTY(sb));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int qd = warp & 3;
+    const int row = qd * 32 + lane;             // token row inside the tile
+    const int et = threadIdx.x - 64;            // 0..127
+    uint32_t qi = 0;
+    bool ok = true;
+    for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
+      int b, h, t;
+      split_frame(s, item, b, h, t);
+      const float g = __ldg(gate + h);
+      for (int tile = 0; tile < ntiles; ++tile, ++qi) {
+        const int a = qi & 3;
+        if (!mbar_wait(ACCFULL(a), (qi >> 2) & 1, wc)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 128;
+        float v[4][32];
+        tmem_ld32(taddr + 0, v[0]);
+        tmem_ld32(taddr + 32, v[1]);
+        tmem_ld32(taddr + 64, v[2]);
+        tmem_ld32(taddr + 96, v[3]);
+        tmem_wait_ld();
+        tc_fence_before_sync();
+        mbar_arrive(ACCEMPTY(a));
+
+        float ss = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int e = 0; e < 32; ++e) ss = fmaf(v[c][e], v[c][e], ss);
+        const float scale = g * rsqrtf(ss * (1.0f / R::D) + eps);
+
+        const int ob = qi & 1;
+        if (et == 0) tma_store_wait_read<1>();   // the store that last used this staging tile has read it
+        named_barrier_sync(1, 128);
+        unsigned char* orow = base_ptr + R::OFF_OUT + ob * R::TILE_BYTES + row * 128;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint4 pk;
+            uint32_t* x = reinterpret_cast<uint32_t*>(&pk);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              __nv_bfloat162 p = __floats2bfloat162_rn(v[c][j * 8 + 2 * e] * scale, v[c][j * 8 + 2 * e + 1] * scale);
+              x[e] = *reinterpret_cast<uint32_t*>(&p);
+            }
+            const int chunk = (c & 1) * 4 + j;          // 16-byte chunk inside the 64-channel box
+            const int boxi = c >> 1;                    // channels 0-63 / 64-127
+            *reinterpret_cast<uint4*>(orow + boxi * R::BOX_BYTES + ((chunk ^ (row & 7)) * 16)) = pk;
+          }
+        }
+        fence_proxy_async_smem();
+        named_barrier_sync(2, 128);
+        if (et == 0) {
+          const uint32_t src = base + R::OFF_OUT + ob * R::TILE_BYTES;
+          tma_store_5d(&tmO, src, 0, h, tile * R::TILE, t, b);
+          tma_store_5d(&tmO, src + R::BOX_BYTES, 64, h, tile * R::TILE, t, b);
+          tma_store_commit();
+        }
+      }
+    }
+    if (et == 0) tma_store_wait_all<0>();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace vdn

@@ -2,6 +2,8 @@
 // The exported functions are documented in include/vdn_vda.h.
 #include "../../include/vdn_vda.h"
 
+#include <cuda.h>
+#include <cudaTypedefs.h>
 #include <cuda_runtime.h>
 
 #include <cstdio>
@@ -11,7 +13,9 @@
 
 #include "common.cuh"
 #include "gram_simt.cuh"
+#include "gram_tc.cuh"
 #include "readout_simt.cuh"
+#include "readout_tc.cuh"
 #include "resolve.cuh"
 #include "scan.cuh"
 
@@ -61,6 +65,8 @@ struct vdn_vda_s {
   int* status_dev = nullptr;
   int launches = 0;
   bool attrs_set = false;
+  bool tc_attrs_set = false;
+  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;  // driver entry point, resolved at create
   std::string err = "no error";
 };
 
@@ -71,9 +77,9 @@ vdn_status fail(vdn_vda_t h, vdn_status st, const std::string& msg) {
   return st;
 }
 
+// bf16 I/O with d = 128 runs on the tcgen05 kernels unless the handle asks for the plain-fp32 ones.
 bool use_tensor_cores(const vdn_vda_s* h, int d) {
-  (void)h; (void)d;
-  return false;
+  return h->cfg.io_dtype == VDN_BF16 && d == 128 && !(h->cfg.flags & VDN_FLAG_FORCE_SIMT);
 }
 
 size_t elem_size(const vdn_vda_s* h) { return h->cfg.io_dtype == VDN_BF16 ? 2 : 4; }
@@ -212,6 +218,85 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
   return VDN_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Tensor-core path (bf16, d = 128): TMA tensor maps + four launches.
+
+// [B,T,F,H,d] bf16 tensor as a 5-D map (d, H, F, T, B) with a (64, 1, 128, 1, 1) box and the 128-byte
+// swizzle: one box is 128 tokens x 64 channels of one head.  F is its own dimension so that a tile
+// hanging over the end of a frame is zero-filled on load and clipped on store.
+vdn_status make_token_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, const Shape& s) {
+  const cuuint64_t dims[5] = {(cuuint64_t)s.d, (cuuint64_t)s.H, (cuuint64_t)s.F, (cuuint64_t)s.T, (cuuint64_t)s.B};
+  const cuuint64_t es = 2;
+  const cuuint64_t strides[4] = {s.d * es, (cuuint64_t)s.H * s.d * es, (cuuint64_t)s.F * s.H * s.d * es,
+                                 (cuuint64_t)s.T * s.F * s.H * s.d * es};
+  const cuuint32_t box[5] = {64, 1, 128, 1, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = h->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled (token tensor) failed: " + std::to_string((int)r));
+  return VDN_OK;
+}
+
+// Read states, bf16 [frames*128][128] as a 2-D map with a (64, 128) box.
+vdn_status make_state_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, long long nframes) {
+  const cuuint64_t dims[2] = {128, (cuuint64_t)nframes * 128};
+  const cuuint64_t strides[1] = {256};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = h->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled (state tensor) failed: " + std::to_string((int)r));
+  return VDN_OK;
+}
+
+vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                      const float* gate, void* out, const Shape& s, const Layout& L, cudaStream_t st) {
+  constexpr int D = 128;
+  if (!h->encode) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  if (!h->tc_attrs_set) {
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::GramTc::SMEM_BYTES));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::ReadoutTc::SMEM_BYTES));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_kernel<D, 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(vdn::ScanSmem<D, 32>)));
+    h->tc_attrs_set = true;
+  }
+  char* ws = static_cast<char*>(h->workspace);
+  float* stats = reinterpret_cast<float*>(ws + L.stats);
+  float* inv = reinterpret_cast<float*>(ws + L.inv);
+  float* fwd = reinterpret_cast<float*>(ws + L.fwd);
+  void* read = ws + L.read;
+  const long long n = s.frames();
+
+  CUtensorMap tmQ, tmK, tmV, tmO, tmS;
+  vdn_status r;
+  if ((r = make_token_map(h, &tmK, k, s)) != VDN_OK) return r;
+  if ((r = make_token_map(h, &tmV, v, s)) != VDN_OK) return r;
+  if ((r = make_token_map(h, &tmQ, q, s)) != VDN_OK) return r;
+  if ((r = make_token_map(h, &tmO, out, s)) != VDN_OK) return r;
+  if ((r = make_state_map(h, &tmS, read, n)) != VDN_OK) return r;
+
+  const unsigned persistent = (unsigned)(n < h->sm_count ? n : h->sm_count);
+  prof_begin(h, st);
+  vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
+                                                                                       h->status_dev);
+  prof_mark(h, st, 0, "gram_tc");
+  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, n);
+  prof_mark(h, st, 1, "resolve");
+  vdn::scan_kernel<D, 32, true><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
+      stats, inv, fwd, read, s.T);
+  prof_mark(h, st, 2, "scan");
+  vdn::readout_tc_kernel<<<persistent, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
+      tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev);
+  prof_mark(h, st, 3, "readout_tc");
+  h->launches = 4;
+  VDN_CUDA(h, cudaGetLastError());
+  return VDN_OK;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
@@ -246,6 +331,15 @@ vdn_status vdn_vda_create(const vdn_vda_config* cfg, vdn_vda_t* out_handle) {
     return VDN_ERR_CUDA;
   }
   std::memset(h->status_host, 0, 64);
+  {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      h->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+    else
+      cudaGetLastError();
+  }
   *out_handle = h;
   return VDN_OK;
 }
@@ -297,6 +391,7 @@ vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void
   if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const Shape s{B, T, F, H, d};
+  if (use_tensor_cores(h, d)) return forward_tc(h, q, k, v, beta, gate, out, s, L, st);
   if (h->cfg.io_dtype == VDN_F32) {
     return d == 64 ? forward_simt<float, 64>(h, q, k, v, beta, gate, out, s, L, st)
                    : forward_simt<float, 128>(h, q, k, v, beta, gate, out, s, L, st);
