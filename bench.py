@@ -277,6 +277,8 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     # ---- end to end through the host-buffer entry point (H2D + forward + D2H inside the timed region)
     e2e = None
     try:
+        if args.skip_e2e:
+            raise RuntimeError("skipped (--skip-e2e)")
         xh = {n: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for n, t in x.items()}
         outh = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
         e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -339,7 +341,7 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     t_roof_ms = max(ab["total"] / (peaks["hbm_gbs"] * 1e9), fl["tensor"] / (peaks["bf16_tflops_sustained"] * 1e12)) * 1e3
     t_roof_nominal_ms = max(ab["total"] / 8e12, fl["tensor"] / 2.25e15) * 1e3
 
-    base = cpu_baseline(w) if world == 1 else None
+    base = cpu_baseline(w) if (world == 1 and not args.skip_cpu) else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
@@ -370,10 +372,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="768p")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--heads", type=int, default=0, help="override H (smaller cases for profiler captures)")
+    ap.add_argument("--frames", type=int, default=0, help="override T (smaller cases for profiler captures)")
+    ap.add_argument("--skip-e2e", action="store_true", help="no host-buffer pass (profiler captures)")
+    ap.add_argument("--skip-cpu", action="store_true", help="no CPU-oracle timing (profiler captures)")
     args = ap.parse_args()
 
     from paper_2609_20744_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
+    if args.heads > 0:
+        w = w.scaled(H=args.heads, name=f"{w.name}_H{args.heads}")
+    if args.frames > 0:
+        w = w.scaled(T=args.frames, name=f"{w.name}_T{args.frames}")
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

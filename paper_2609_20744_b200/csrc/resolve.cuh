@@ -2,20 +2,32 @@
 //
 // I + A_t is symmetric positive definite with every eigenvalue >= 1 (A_t is a Gram matrix weighted
 // by beta >= 0), so in-place Gauss-Jordan elimination needs no pivot search.  The matrix lives in
-// registers, an R x R tile per thread on a 16 x 16 thread grid; for every pivot the owning threads
-// publish the pivot row and column through (double-buffered) shared memory and everybody applies
-// the rank-1 update: one barrier per pivot.
+// registers: thread (ty,tx) of a 16 x 16 grid owns rows ty+16r and columns tx+16c (cyclic), so the
+// owner of pivot p = 16q+o is known from o alone and the register index q is a compile-time constant.
+//
+// Per pivot the owners publish the pivot row and column through double-buffered shared memory and
+// then zero them in their registers; with the published column entry of the pivot row set to -1 and
+// the published row entry of the pivot column set to 1/pivot, the uniform update
+//        m[i][j] -= col[i] * row[j] / pivot
+// also produces the pivot row (row/pivot), the pivot column (-col/pivot) and the pivot (1/pivot):
+// one FMA per element, no predication, one barrier per pivot.
+//
+// When `split` is non-null the inverse is also written as three bf16 matrices C1 + C2 + C3 (each the
+// bf16 rounding of what the previous ones leave over, 24 mantissa bits in all) for the tensor-core scan.
 #pragma once
+#include <cuda_bf16.h>
+
 #include "common.cuh"
 
 namespace vdn {
 
 template <int D>
-__global__ void __launch_bounds__(256) resolve_kernel(const float* __restrict__ stats,
-                                                       float* __restrict__ inv, long long nframes) {
+__global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict__ stats,
+                                                          float* __restrict__ inv,
+                                                          __nv_bfloat16* __restrict__ split, long long nframes) {
   constexpr int R = D / 16;
-  __shared__ __align__(16) float rowbuf[2][D];
-  __shared__ __align__(16) float colbuf[2][D];
+  __shared__ __align__(16) float rowbuf[2][D];   // indexed [owner tx][c]
+  __shared__ __align__(16) float colbuf[2][D];   // indexed [owner ty][r]
 
   const long long n = blockIdx.x;
   if (n >= nframes) return;
@@ -24,72 +36,78 @@ __global__ void __launch_bounds__(256) resolve_kernel(const float* __restrict__ 
 
   float m[R][R];
 #pragma unroll
-  for (int r = 0; r < R; ++r) {
-    const int i = ty * R + r;
-#pragma unroll
-    for (int c = 0; c < R; c += 4) {
-      float4 x = load4(A + (size_t)i * 2 * D + tx * R + c);
-      m[r][c] = x.x; m[r][c + 1] = x.y; m[r][c + 2] = x.z; m[r][c + 3] = x.w;
-    }
-#pragma unroll
-    for (int c = 0; c < R; ++c)
-      if (i == tx * R + c) m[r][c] += 1.0f;
-  }
-
-  for (int p = 0; p < D; ++p) {
-    const int par = p & 1;
-    const int pb = p / R, pr = p % R;
-    if (ty == pb) {
-#pragma unroll
-      for (int r = 0; r < R; ++r)
-        if (r == pr) {
-#pragma unroll
-          for (int c = 0; c < R; ++c) rowbuf[par][tx * R + c] = m[r][c];
-        }
-    }
-    if (tx == pb) {
-#pragma unroll
-      for (int c = 0; c < R; ++c)
-        if (c == pr) {
-#pragma unroll
-          for (int r = 0; r < R; ++r) colbuf[par][ty * R + r] = m[r][c];
-        }
-    }
-    __syncthreads();
-    const float ipiv = 1.0f / rowbuf[par][p];
-    float rowv[R], colv[R];
-#pragma unroll
-    for (int c = 0; c < R; c += 4) {
-      float4 x = load4(&rowbuf[par][tx * R + c]);
-      rowv[c] = x.x; rowv[c + 1] = x.y; rowv[c + 2] = x.z; rowv[c + 3] = x.w;
-    }
-#pragma unroll
-    for (int r = 0; r < R; r += 4) {
-      float4 x = load4(&colbuf[par][ty * R + r]);
-      colv[r] = x.x; colv[r + 1] = x.y; colv[r + 2] = x.z; colv[r + 3] = x.w;
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const bool prow = (ty * R + r == p);
-      const float f = colv[r] * ipiv;
-#pragma unroll
-      for (int c = 0; c < R; ++c) {
-        const bool pcol = (tx * R + c == p);
-        float upd = fmaf(-f, rowv[c], m[r][c]);       // ordinary entry
-        if (prow) upd = rowv[c] * ipiv;               // pivot row
-        if (pcol) upd = -f;                           // pivot column
-        if (prow && pcol) upd = ipiv;                 // pivot itself
-        m[r][c] = upd;
-      }
-    }
-  }
-
-  float* C = inv + (size_t)n * D * D;
-#pragma unroll
   for (int r = 0; r < R; ++r)
 #pragma unroll
-    for (int c = 0; c < R; c += 4)
-      store4(C + (size_t)(ty * R + r) * D + tx * R + c, make_float4(m[r][c], m[r][c + 1], m[r][c + 2], m[r][c + 3]));
+    for (int c = 0; c < R; ++c) {
+      const int i = ty + 16 * r, j = tx + 16 * c;
+      m[r][c] = __ldg(A + (size_t)i * 2 * D + j) + (i == j ? 1.0f : 0.0f);
+    }
+
+#pragma unroll
+  for (int q = 0; q < R; ++q) {
+#pragma unroll 2
+    for (int o = 0; o < 16; ++o) {
+      const int par = o & 1;
+      if (ty == o) {                      // owners of the pivot row: publish it, then clear it
+#pragma unroll
+        for (int c = 0; c < R; c += 4) {
+          store4(&rowbuf[par][tx * R + c], make_float4(m[q][c], m[q][c + 1], m[q][c + 2], m[q][c + 3]));
+          m[q][c] = 0.f; m[q][c + 1] = 0.f; m[q][c + 2] = 0.f; m[q][c + 3] = 0.f;
+        }
+      }
+      if (tx == o) {                      // owners of the pivot column
+        float cv[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) { cv[r] = m[r][q]; m[r][q] = 0.f; }
+        if (ty == o) cv[q] = -1.0f;       // (the pivot itself was already published with the row)
+#pragma unroll
+        for (int r = 0; r < R; r += 4) store4(&colbuf[par][ty * R + r], make_float4(cv[r], cv[r + 1], cv[r + 2], cv[r + 3]));
+      }
+      __syncthreads();
+      const float ipiv = __frcp_rn(rowbuf[par][o * R + q]);
+      float rv[R], cv[R];
+#pragma unroll
+      for (int c = 0; c < R; c += 4) {
+        float4 x = load4(&rowbuf[par][tx * R + c]);
+        rv[c] = x.x * ipiv; rv[c + 1] = x.y * ipiv; rv[c + 2] = x.z * ipiv; rv[c + 3] = x.w * ipiv;
+      }
+      if (tx == o) rv[q] = ipiv;
+#pragma unroll
+      for (int r = 0; r < R; r += 4) {
+        float4 x = load4(&colbuf[par][ty * R + r]);
+        cv[r] = x.x; cv[r + 1] = x.y; cv[r + 2] = x.z; cv[r + 3] = x.w;
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int c = 0; c < R; ++c) m[r][c] = fmaf(-cv[r], rv[c], m[r][c]);
+    }
+  }
+
+  if (inv != nullptr) {
+    float* C = inv + (size_t)n * D * D;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int c = 0; c < R; ++c) C[(size_t)(ty + 16 * r) * D + tx + 16 * c] = m[r][c];
+  }
+  if (split != nullptr) {
+    __nv_bfloat16* S = split + (size_t)n * 3 * D * D;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int c = 0; c < R; ++c) {
+        const size_t e = (size_t)(ty + 16 * r) * D + tx + 16 * c;
+        const float x = m[r][c];
+        const __nv_bfloat16 p1 = __float2bfloat16_rn(x);
+        const float r1 = x - __bfloat162float(p1);
+        const __nv_bfloat16 p2 = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 p3 = __float2bfloat16_rn(r1 - __bfloat162float(p2));
+        S[e] = p1;
+        S[(size_t)D * D + e] = p2;
+        S[(size_t)2 * D * D + e] = p3;
+      }
+  }
 }
 
 }  // namespace vdn

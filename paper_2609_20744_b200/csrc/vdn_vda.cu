@@ -205,7 +205,7 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
   vdn::gram_simt_kernel<Tio, D><<<dim3((unsigned)n, 2 * D / 64), 256, 0, st>>>(
       static_cast<const Tio*>(k), static_cast<const Tio*>(v), beta, stats, s);
   prof_mark(h, st, 0, "gram_simt");
-  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, n);
+  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n);
   prof_mark(h, st, 1, "resolve");
   vdn::scan_kernel<D, 32, false><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
       stats, inv, fwd, read, s.T);
@@ -284,7 +284,7 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
                                                                                        h->status_dev);
   prof_mark(h, st, 0, "gram_tc");
-  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, n);
+  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n);
   prof_mark(h, st, 1, "resolve");
   vdn::scan_kernel<D, 32, true><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
       stats, inv, fwd, read, s.T);
