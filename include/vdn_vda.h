@@ -14,7 +14,9 @@
  *
  * No patch order inside a frame, no 1/sqrt(F) key scaling (Sec. 3.3).  The statistics are contracted on
  * the tensor cores (bf16 operands, fp32 accumulation) in bf16 mode and in plain fp32 in f32 mode; the
- * inverse, the scans and the norm are always fp32.
+ * inverse and the norm are always plain fp32, and the scan carries its state at fp32 accuracy (plain fp32
+ * FMA in f32 mode; in bf16 mode fp32 factors split three-way into bf16 parts, multiplied on the tensor
+ * cores and accumulated in fp32).
  *
  * Naming: T = latent frames, F = spatial tokens per frame, H = heads, d = d_k = d_v (the paper's F, U).
  *
@@ -78,14 +80,18 @@ typedef struct {
   int32_t device;       /* CUDA device ordinal the handle is bound to                                 */
 } vdn_vda_config;
 
-/* Names of workspace regions for vdn_vda_workspace_view (stage-wise checks in the tests). */
+/* Names of workspace regions for vdn_vda_workspace_view (stage-wise checks in the tests).  Which views
+ * exist depends on the kernels the handle runs; asking for one of the others returns VDN_ERR_UNSUPPORTED. */
 typedef enum {
-  VDN_VIEW_STATS = 0, /* float [B,H,T,d,2d]: row i = [ A_t[i,:] | B_t^T[i,:] ]            (Eq. 3b)    */
-  VDN_VIEW_INV = 1,   /* float [B,H,T,d,d]:  C_t = (I + A_t)^{-1}                         (Eq. 5)     */
-  VDN_VIEW_FWD = 2,   /* float [B,H,T,d_k,d_v]: transpose of P_t, the forward-scan state    (Eq. A.1)  */
-  VDN_VIEW_READ = 3   /* transpose of the state frame t's queries read, P_{t-1}+R_{t+1}    (Eq. A.4): */
-                      /*   plain-fp32 kernels: float [B,H,T,d_k,d_v]; tensor-core kernels: bf16       */
-                      /*   [B,H,T,d_v,d_k] (i.e. the paper's orientation)                              */
+  VDN_VIEW_STATS = 0,     /* float [B,H,T,2d,d]: rows 0..d-1 = A_t, rows d..2d-1 = B_t (d_v x d_k)  (Eq. 3b) */
+  /* plain-fp32 kernels (f32 I/O, or VDN_FLAG_FORCE_SIMT, or d = 64) */
+  VDN_VIEW_INV = 1,       /* float [B,H,T,d,d]: C_t = (I + A_t)^{-1}                                (Eq. 5)  */
+  VDN_VIEW_FWD = 2,       /* float [B,H,T,d_k,d_v]: transpose of P_t, the forward-scan state      (Eq. A.1)  */
+  VDN_VIEW_READ = 3,      /* float [B,H,T,d_k,d_v]: transpose of P_{t-1} + R_{t+1}, what frame t reads (A.4) */
+  /* tensor-core kernels (bf16 I/O, d = 128) */
+  VDN_VIEW_INV_SPLIT = 4, /* bf16 [B,H,T,3,d,d]: C_t as C1 + C2 + C3 (bf16 parts of the fp32 inverse)         */
+  VDN_VIEW_READ_FWD = 5,  /* bf16 [B,H,T,d_k,d_v]: slot t = transpose of P_{t-1} (zero for t = 0)     (A.4)  */
+  VDN_VIEW_READ_BWD = 6   /* bf16 [B,H,T,d_k,d_v]: slot t = transpose of R_{t+1} (zero for t = T-1)   (A.4)  */
 } vdn_view;
 
 /* Sec. 3 (the layer as a whole).  Creates a handle bound to cfg->device.  Allocates host memory only

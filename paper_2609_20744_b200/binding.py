@@ -18,7 +18,7 @@ STATUS_NAMES = {0: "VDN_OK", 1: "VDN_ERR_INVALID_ARG", 2: "VDN_ERR_UNSUPPORTED",
                 4: "VDN_ERR_CUDA", 5: "VDN_ERR_ARCH", 6: "VDN_ERR_TIMEOUT"}
 VDN_F32, VDN_BF16 = 0, 1
 VDN_FLAG_FORCE_SIMT = 1
-VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ = 0, 1, 2, 3
+VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_READ_BWD = range(7)
 
 EXPORTS = (
     "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward",
@@ -178,12 +178,19 @@ class Vda:
                                                     ctypes.byref(off), ctypes.byref(size)))
         raw = self._ws[off.value: off.value + size.value]
         d = self.d
-        n = B * H * T
         if which == VIEW_STATS:
-            return raw.view(torch.float32).view(B, H, T, d, 2 * d)
-        if size.value == n * d * d * 4:
-            return raw.view(torch.float32).view(B, H, T, d, d)
-        return raw.view(torch.bfloat16).view(B, H, T, d, d)
+            return raw.view(torch.float32).view(B, H, T, 2 * d, d)
+        if which == VIEW_INV_SPLIT:
+            return raw.view(torch.bfloat16).view(B, H, T, 3, d, d)
+        if which in (VIEW_READ_FWD, VIEW_READ_BWD):
+            return raw.view(torch.bfloat16).view(B, H, T, d, d)
+        return raw.view(torch.float32).view(B, H, T, d, d)
+
+    def uses_tensor_cores(self) -> bool:
+        """True when this handle runs the tcgen05 kernels (bf16 I/O, d = 128, plain-fp32 path not forced)."""
+        off, size = ctypes.c_size_t(), ctypes.c_size_t()
+        return self.lib.vdn_vda_workspace_view(self.h, VIEW_INV_SPLIT, 1, 1, 1, 1, self.d,
+                                               ctypes.byref(off), ctypes.byref(size)) == VDN_OK
 
     def profile(self, enable: bool = True):
         """Start (and reset) or stop per-kernel CUDA-event timing of forward calls."""

@@ -1,6 +1,6 @@
 // Frame statistics (Eq. 3b) in plain fp32:  for frame n = (b,h,t)
-//     stats[n][i][0:d)   = A_t[i][:]    = sum_u beta_u k_u[i] k_u[:]
-//     stats[n][i][d:2d)  = B_t^T[i][:]  = sum_u beta_u k_u[i] v_u[:]
+//     stats[n][j][i]      = A_t[j][i] = sum_u beta_u k_u[j] k_u[i]      rows 0..d-1
+//     stats[n][d + c][i]  = B_t[c][i] = sum_u beta_u v_u[c] k_u[i]      rows d..2d-1  (B_t is d_v x d_k)
 // One CTA per (frame, 64-wide column block of [K | V]); tokens are streamed in tiles of TU and
 // summed in token order, so the result is deterministic.  Used by f32 mode and as a second opinion
 // for the tensor-core kernel.
@@ -74,11 +74,12 @@ __global__ void __launch_bounds__(256) gram_simt_kernel(const Tio* __restrict__ 
     }
     __syncthreads();
   }
-  float* dst = stats + (size_t)n * D * 2 * D;
+  float* dst = stats + (size_t)n * 2 * D * D;
 #pragma unroll
-  for (int r = 0; r < TI; ++r) {
-    int i = ig * TI + r;
-    store4(dst + (size_t)i * 2 * D + cb * CB + cg * 4, make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]));
+  for (int c = 0; c < 4; ++c) {
+    float* row = dst + (size_t)(cb * CB + cg * 4 + c) * D + ig * TI;
+#pragma unroll
+    for (int r = 0; r < TI; r += 4) store4(row + r, make_float4(acc[r][c], acc[r + 1][c], acc[r + 2][c], acc[r + 3][c]));
   }
 }
 

@@ -1,6 +1,7 @@
 // Frame statistics (Eq. 3b) on the tcgen05 tensor cores, bf16 operands, fp32 accumulation in TMEM.
 //
 //   [ A_t | B_t^T ] = (Diag(beta_t) K_t)^T [ K_t | V_t ]          128 x 256 per frame (d = 128)
+// (stored transposed: A_t is symmetric, and the second block becomes B_t itself, d_v x d_k)
 //
 // The contraction index is the token, so both operands are "MN-major": a token's 128 channels are
 // contiguous in memory, and TMA drops each 128-token tile into shared memory as 64-channel boxes with
@@ -11,7 +12,7 @@
 //   warp 1      MMA issuer (one thread) and TMEM owner
 //   warps 2-5   weighting: K' = beta * K, rounded once to bf16, written to a second buffer in two halves of
 //               64 tokens so the MMA of one half overlaps the weighting of the other
-//   warps 6-9   epilogue: TMEM -> registers -> global fp32 [d][2d]; two accumulators, so the drain of
+//   warps 6-9   epilogue: TMEM -> registers -> global fp32 [2d][d] (A_t, then B_t); two accumulators, so the drain of
 //               frame i overlaps the main loop of frame i+1
 // Rows past the end of a frame are zero-filled by TMA (the map has F as its own dimension) and their
 // beta is forced to zero.  Every mbarrier wait is bounded.
@@ -195,14 +196,16 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       if (!mbar_wait(ACCFULL(a), (ai >> 1) & 1, wc)) { ok = false; break; }
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 256;
-      float* dst = stats + (size_t)item * (G::D * 2 * G::D) + (size_t)row * (2 * G::D);
+      // accumulator lane = key channel i, column = column of [K|V]; stored transposed, [2d][d], so that
+      // the 32 lanes of a warp write 32 consecutive floats
+      float* dst = stats + (size_t)item * (2 * G::D * G::D) + row;
 #pragma unroll 1
       for (int cc = 0; cc < 8; ++cc) {
         float v[32];
         tmem_ld32(taddr + cc * 32, v);
         tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; e += 4) store4(dst + cc * 32 + e, make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]));
+        for (int e = 0; e < 32; ++e) dst[(size_t)(cc * 32 + e) * G::D] = v[e];
       }
       tc_fence_before_sync();
       mbar_arrive(ACCEMPTY(a));

@@ -3,11 +3,11 @@
 //   O_t = Q_t (P_{t-1} + R_{t+1})^T      128-token tile x 128 channels, fp32 in TMEM
 //   out = gate_h * O / sqrt(mean_c O^2 + eps)   -> bf16
 //
-// The state each frame reads arrives already summed over the two directions, as bf16 [d_v][d_k]
-// (K-major for the MMA's B operand); Q tiles are K-major as they sit in memory.  Persistent CTAs loop
-// over frames (b,h,t).  Warp roles:
-//   warp 0      TMA producer: the frame's state (2 boxes, double-buffered across frames) and Q tiles
-//               (2 boxes of 16 KB, 3-stage ring)
+// The two states a frame reads (forward state of the frames before it, reverse state of the frames after
+// it) arrive as bf16 [d_k][d_v], i.e. MN-major B operands; both products go into the same accumulator,
+// which is the sum of Eq. 1a.  Q tiles are K-major as they sit in memory.  Persistent CTAs loop over
+// frames (b,h,t).  Warp roles:
+//   warp 0      TMA producer: the frame's two states (4 boxes of 16 KB) and Q tiles (2 boxes, 3-stage ring)
 //   warp 1      MMA issuer (one thread), 4 accumulators of 128 TMEM columns
 //   warps 2-5   epilogue: tcgen05.ld gives every thread one whole token row, so the sum of squares is
 //               thread-local; the scaled row is packed to bf16, written to a swizzled staging tile and
@@ -87,12 +87,14 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
         int b, h, t;
         split_frame(s, item, b, h, t);
-        const int sb = si & 1;
-        if (!mbar_wait(STEMPTY(sb), ((si >> 1) & 1) ^ 1, wc)) { ok = false; break; }
-        mbar_arrive_expect_tx(STFULL(sb), R::TILE_BYTES);
-        const uint32_t sdst = base + R::OFF_STATE + sb * R::TILE_BYTES;
-        tma_load_2d(sdst, &tmS, STFULL(sb), 0, (int)(item * R::D));
-        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(sb), 64, (int)(item * R::D));
+        if (!mbar_wait(STEMPTY(0), (si & 1) ^ 1, wc)) { ok = false; break; }
+        mbar_arrive_expect_tx(STFULL(0), 2 * R::TILE_BYTES);
+        const uint32_t sdst = base + R::OFF_STATE;
+        // rows [item*128, +128) hold the forward state, rows [(nitems+item)*128, +128) the reverse state
+        tma_load_2d(sdst, &tmS, STFULL(0), 0, (int)(item * R::D));
+        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(item * R::D));
+        tma_load_2d(sdst + 2 * R::BOX_BYTES, &tmS, STFULL(0), 0, (int)((nitems + item) * R::D));
+        tma_load_2d(sdst + 3 * R::BOX_BYTES, &tmS, STFULL(0), 64, (int)((nitems + item) * R::D));
         for (int tile = 0; tile < ntiles; ++tile, ++qi) {
           const int st = qi % R::QSTAGES;
           if (!mbar_wait(QEMPTY(st), ((qi / R::QSTAGES) & 1) ^ 1, wc)) { ok = false; break; }
@@ -110,13 +112,12 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
+      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
       uint32_t qi = 0, si = 0;
       bool ok = true;
       for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
-        const int sb = si & 1;
-        if (!mbar_wait(STFULL(sb), (si >> 1) & 1, wc)) { ok = false; break; }
-        const uint32_t sbase = base + R::OFF_STATE + sb * R::TILE_BYTES;
+        if (!mbar_wait(STFULL(0), si & 1, wc)) { ok = false; break; }
+        const uint32_t sbase = base + R::OFF_STATE;
         for (int tile = 0; tile < ntiles; ++tile, ++qi) {
           const int st = qi % R::QSTAGES;
           const int a = qi & 3;
@@ -125,16 +126,19 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           tc_fence_after_sync();
           const uint32_t qbase = base + R::OFF_Q + st * R::TILE_BYTES;
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint32_t off = (j >> 2) * R::BOX_BYTES + (j & 3) * 32;   // 16 channels = 32 B inside the swizzled row
-            const uint64_t adesc = make_smem_desc(qbase + off, 16, 1024);
-            const uint64_t bdesc = make_smem_desc(sbase + off, 16, 1024);
-            mma_bf16_ss(tmem_base + a * 128, adesc, bdesc, idesc, j != 0 ? 1u : 0u);
+          for (int dirn = 0; dirn < 2; ++dirn) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              // A: 16 key channels = 32 B inside the swizzled Q row; B: 16 key rows of the state = 2 KB
+              const uint64_t adesc = make_smem_desc(qbase + (j >> 2) * R::BOX_BYTES + (j & 3) * 32, 16, 1024);
+              const uint64_t bdesc = make_smem_desc(sbase + dirn * R::TILE_BYTES + j * 2048, R::BOX_BYTES, 1024);
+              mma_bf16_ss(tmem_base + a * 128, adesc, bdesc, idesc, (dirn | j) != 0 ? 1u : 0u);
+            }
           }
           mma_commit(QEMPTY(st));
           mma_commit(ACCFULL(a));
         }
-        if (ok) mma_commit(STEMPTY(sb));
+        if (ok) mma_commit(STEMPTY(0));
       }
     }
   } else {

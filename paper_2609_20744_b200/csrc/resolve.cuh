@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict
   const long long n = blockIdx.x;
   if (n >= nframes) return;
   const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
-  const float* A = stats + (size_t)n * D * 2 * D;   // row stride 2D: [A | B^T]
+  const float* A = stats + (size_t)n * 2 * D * D;   // first d rows of the frame's [2d][d] block
 
   float m[R][R];
 #pragma unroll
@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict
 #pragma unroll
     for (int c = 0; c < R; ++c) {
       const int i = ty + 16 * r, j = tx + 16 * c;
-      m[r][c] = __ldg(A + (size_t)i * 2 * D + j) + (i == j ? 1.0f : 0.0f);
+      m[r][c] = __ldg(A + (size_t)i * D + j) + (i == j ? 1.0f : 0.0f);
     }
 
 #pragma unroll

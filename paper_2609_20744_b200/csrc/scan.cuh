@@ -1,4 +1,4 @@
-// Bidirectional frame scan + gather (Alg. 1 steps 5-6; Eq. A.1, Eq. A.4, Eq. 1a), fp32.
+// Bidirectional frame scan + gather (Alg. 1 steps 5-6; Eq. A.1, Eq. A.4, Eq. 1a), plain fp32 FMA.
 //
 // With Z = S^T (d_k x d_v) and alpha = 1 the frame update  S_t = (S_{t-1} + B_t)(I + A_t)^{-1}
 // reads  Z_t = C_t (Z_{t-1} + B_t^T).  The transition acts on the key index only, so the d_v columns
@@ -22,12 +22,11 @@ struct ScanSmem {
   float X[2][D][W];
 };
 
-// READ_BF16_T = false: read state as float [d_k][d_v] (row i, column c)       -- plain-fp32 read-out
-// READ_BF16_T = true : read state as bf16  [d_v][d_k] (row c, column i)       -- tensor-core read-out
-template <int D, int W, bool READ_BF16_T>
+// The read state is written as float [d_k][d_v] (row i, column c).
+template <int D, int W>
 __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ stats,
                                                        const float* __restrict__ inv,
-                                                       float* __restrict__ fwd, void* __restrict__ read,
+                                                       float* __restrict__ fwd, float* __restrict__ read,
                                                        int T) {
   constexpr int TI = D / 32;          // rows per thread
   constexpr int NCG = W / 4;          // column groups of 4
@@ -70,35 +69,30 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
         if (t > 0) x = load4(fwd + (n - 1) * D * D + (size_t)(i0 + r) * D + c0 + cc0);
         p[r][0] = x.x + z[r][0]; p[r][1] = x.y + z[r][1]; p[r][2] = x.z + z[r][2]; p[r][3] = x.w + z[r][3];
       }
-      if constexpr (READ_BF16_T) {
-        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(read) + n * D * D;
+      float* dst = read + n * D * D;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          __nv_bfloat16* row = dst + (size_t)(c0 + cc0 + c) * D + i0;
-          if constexpr (TI == 4) {
-            store4(row, make_float4(p[0][c], p[1][c], p[2][c], p[3][c]));
-          } else {
-#pragma unroll
-            for (int r = 0; r < TI; ++r) row[r] = __float2bfloat16_rn(p[r][c]);
-          }
-        }
-      } else {
-        float* dst = reinterpret_cast<float*>(read) + n * D * D;
-#pragma unroll
-        for (int r = 0; r < TI; ++r)
-          store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(p[r][0], p[r][1], p[r][2], p[r][3]));
-      }
+      for (int r = 0; r < TI; ++r)
+        store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(p[r][0], p[r][1], p[r][2], p[r][3]));
     }
 
     // X = Z + B_t^T (this CTA's columns)
     {
-      const float* bt = stats + n * D * 2 * D + D + c0 + cc0;
+      // B_t is stored [d_v][d_k]: element (c, i) is B_t^T[i][c]
+      const float* bsrc = stats + n * 2 * D * D + (size_t)(D + c0 + cc0) * D + i0;
+      float bt[TI][4];
 #pragma unroll
-      for (int r = 0; r < TI; ++r) {
-        float4 x = load4(bt + (size_t)(i0 + r) * 2 * D);
-        x.x += z[r][0]; x.y += z[r][1]; x.z += z[r][2]; x.w += z[r][3];
-        store4(&sm.X[buf][i0 + r][cc0], x);
+      for (int c = 0; c < 4; ++c) {
+        if constexpr (TI == 4) {
+          float4 x = load4(bsrc + (size_t)c * D);
+          bt[0][c] = x.x; bt[1][c] = x.y; bt[2][c] = x.z; bt[3][c] = x.w;
+        } else {
+          float2 x = *reinterpret_cast<const float2*>(bsrc + (size_t)c * D);
+          bt[0][c] = x.x; bt[1][c] = x.y;
+        }
       }
+#pragma unroll
+      for (int r = 0; r < TI; ++r)
+        store4(&sm.X[buf][i0 + r][cc0], make_float4(bt[r][0] + z[r][0], bt[r][1] + z[r][1], bt[r][2] + z[r][2], bt[r][3] + z[r][3]));
     }
     cp_async_wait<0>();
     __syncthreads();

@@ -1,0 +1,216 @@
+// Frame scan (Alg. 1 step 5; Eq. A.1) with the d x d products on the tcgen05 tensor cores at fp32
+// accuracy, d = 128.  One CTA per (batch, head, direction) chain; the state never leaves the SM.
+//
+// With Z = S^T and alpha = 1 the frame update reads  Z_t = C_t (Z_{t-1} + B_t^T),  C_t = (I+A_t)^{-1}.
+// Both factors are fp32.  Each is written as a sum of three bf16 numbers (x = x1 + x2 + x3, every part the
+// bf16 rounding of what the earlier parts leave over: 24 mantissa bits, i.e. all of fp32), and the product
+// is accumulated in fp32 (TMEM) from the six partial products whose weight is above 2^-24:
+//        C1 X1 + C1 X2 + C2 X1 + C2 X2 + C1 X3 + C3 X1.
+// The dropped terms are below 2^-24 relative to |C||X|, the rounding level of an fp32 dot product, so the
+// state is carried at fp32 accuracy while the 2 d^3 flops per step run on the tensor pipe.
+//
+// C_t arrives already split (the resolve kernel writes the three parts), by TMA, K-major.  The state
+// parts are produced on chip: after each step the 8 epilogue warps read Z_t from TMEM (a thread owns one
+// key row and 64 value columns), store it as bf16 for the read-out of the next frame in scan order, add
+// the next frame's B^T, split the sum and write the three parts to shared memory as the next MN-major B
+// operand.  The next frame's B^T row is fetched into registers while the MMAs run.
+//
+// Gather (Eq. A.4 with the window shrunk to the query frame): the forward chain stores P_t in slot t+1 of
+// `pf`, the reverse chain stores R_t in slot t-1 of `pb`; slot 0 of pf and slot T-1 of pb are zeroed here
+// (the scans start from the zero state).  The read-out kernel adds the two in its accumulator (Eq. 1a).
+#pragma once
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace vdn {
+
+struct ScanTc {
+  static constexpr int D = 128;
+  static constexpr int BOX_BYTES = 128 * 128;        // 128 rows x 64 bf16
+  static constexpr int PART_BYTES = 2 * BOX_BYTES;   // one 128 x 128 bf16 matrix
+  static constexpr int OFF_C = 0;                    // C1, C2, C3
+  static constexpr int OFF_X = 3 * PART_BYTES;       // X1, X2, X3
+  static constexpr int OFF_BAR = 6 * PART_BYTES;
+  static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
+  static constexpr int THREADS = 320;
+};
+
+// x -> three bf16 parts for two neighbouring elements at once (packed as bf16x2 words).
+__device__ __forceinline__ void split3_pair(float x0, float x1, uint32_t& p1, uint32_t& p2, uint32_t& p3) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(x0, x1);
+  p1 = *reinterpret_cast<uint32_t*>(&a);
+  x0 -= __uint_as_float(p1 << 16);
+  x1 -= __uint_as_float(p1 & 0xFFFF0000u);
+  __nv_bfloat162 b = __floats2bfloat162_rn(x0, x1);
+  p2 = *reinterpret_cast<uint32_t*>(&b);
+  x0 -= __uint_as_float(p2 << 16);
+  x1 -= __uint_as_float(p2 & 0xFFFF0000u);
+  __nv_bfloat162 c = __floats2bfloat162_rn(x0, x1);
+  p3 = *reinterpret_cast<uint32_t*>(&c);
+}
+
+__global__ void __launch_bounds__(ScanTc::THREADS, 1)
+scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict__ stats,
+               __nv_bfloat16* __restrict__ pf, __nv_bfloat16* __restrict__ pb, int T, int* status) {
+  using namespace tc;
+  using S = ScanTc;
+  constexpr int D = S::D;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+
+  const uint32_t bar0 = base + S::OFF_BAR;
+  const uint32_t CFULL = bar0, CFREE = bar0 + 8, XREADY = bar0 + 16, ACCFULL = bar0 + 24;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + S::OFF_BAR + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + S::OFF_BAR + 40);
+  const WaitCtx wc{abort_flag, status};
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.x >> 1, dir = blockIdx.x & 1;
+  auto frame_of = [&](int s) { return dir == 0 ? s : T - 1 - s; };   // frame folded in at scan step s
+
+  if (threadIdx.x == 0) {
+    mbar_init(CFULL, 1);
+    mbar_init(CFREE, 1);
+    mbar_init(XREADY, 256);
+    mbar_init(ACCFULL, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmC);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), 128);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer: C_t parts
+    if (lane == 0) {
+      for (int s = 0; s + 1 < T; ++s) {     // the last frame of a chain is never folded in: nobody reads it
+        if (!mbar_wait(CFREE, (s & 1) ^ 1, wc)) break;
+        mbar_arrive_expect_tx(CFULL, 3 * S::PART_BYTES);
+        const long long n = (long long)bh * T + frame_of(s);
+#pragma unroll
+        for (int p = 0; p < 3; ++p) {
+          const uint32_t dst = base + S::OFF_C + p * S::PART_BYTES;
+          const int row = (int)((n * 3 + p) * D);
+          tma_load_2d(dst, &tmC, CFULL, 0, row);
+          tma_load_2d(dst + S::BOX_BYTES, &tmC, CFULL, 64, row);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
+      // (C part, X part), smallest contributions first
+      constexpr int PA[6] = {0, 2, 1, 0, 1, 0};
+      constexpr int PX[6] = {2, 0, 1, 1, 0, 0};
+      for (int s = 0; s + 1 < T; ++s) {
+        if (!mbar_wait(CFULL, s & 1, wc)) break;
+        if (!mbar_wait(XREADY, s & 1, wc)) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int pr = 0; pr < 6; ++pr) {
+          const uint32_t cb = base + S::OFF_C + PA[pr] * S::PART_BYTES;
+          const uint32_t xb = base + S::OFF_X + PX[pr] * S::PART_BYTES;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint64_t adesc = make_smem_desc(cb + (k >> 2) * S::BOX_BYTES + (k & 3) * 32, 16, 1024);
+            const uint64_t bdesc = make_smem_desc(xb + k * 2048, S::BOX_BYTES, 1024);
+            mma_bf16_ss(tmem_base, adesc, bdesc, idesc, (pr | k) != 0 ? 1u : 0u);
+          }
+        }
+        mma_commit(CFREE);
+        mma_commit(ACCFULL);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ state warps
+    const int qd = warp & 3;                 // TMEM lane quarter
+    const int row = qd * 32 + lane;          // key channel (row of Z, row of X)
+    const int half = (warp - 2) >> 2;        // value columns [64*half, 64*half + 64)
+    const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + half * 64;
+    unsigned char* xrow = base_ptr + S::OFF_X + half * S::BOX_BYTES + row * 128;
+    const int sw = row & 7;
+
+    auto load_bt = [&](int frame, float (&bt)[64]) {
+      // B_t is stored [d_v][d_k]; lanes read consecutive key channels
+      const float* src = stats + ((size_t)bh * T + frame) * (2 * D * D) + (size_t)(D + half * 64) * D + row;
+#pragma unroll
+      for (int e = 0; e < 64; ++e) bt[e] = __ldg(src + (size_t)e * D);
+    };
+    auto publish_x = [&](const float (&x)[64]) {
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        uint4 w1, w2, w3;
+        uint32_t* a1 = reinterpret_cast<uint32_t*>(&w1);
+        uint32_t* a2 = reinterpret_cast<uint32_t*>(&w2);
+        uint32_t* a3 = reinterpret_cast<uint32_t*>(&w3);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) split3_pair(x[ch * 8 + 2 * e], x[ch * 8 + 2 * e + 1], a1[e], a2[e], a3[e]);
+        const int off = (ch ^ sw) * 16;
+        *reinterpret_cast<uint4*>(xrow + off) = w1;
+        *reinterpret_cast<uint4*>(xrow + S::PART_BYTES + off) = w2;
+        *reinterpret_cast<uint4*>(xrow + 2 * S::PART_BYTES + off) = w3;
+      }
+      fence_proxy_async_smem();
+      tc_fence_before_sync();
+      mbar_arrive(XREADY);
+    };
+
+    float bt[64];
+    load_bt(frame_of(0), bt);
+    publish_x(bt);                           // Z_{-1} = 0
+    {
+      // the chain's first read slot holds the zero state
+      __nv_bfloat16* z0 = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(0)) * (D * D) + (size_t)row * D + half * 64;
+#pragma unroll
+      for (int e = 0; e < 64; e += 8) *reinterpret_cast<uint4*>(z0 + e) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    for (int s = 0; s + 1 < T; ++s) {
+      load_bt(frame_of(s + 1), bt);          // lands while the MMAs of step s run
+      if (!mbar_wait(ACCFULL, s & 1, wc)) break;
+      tc_fence_after_sync();
+      float z[64];
+      tmem_ld32(taddr, *reinterpret_cast<float(*)[32]>(&z[0]));
+      tmem_ld32(taddr + 32, *reinterpret_cast<float(*)[32]>(&z[32]));
+      tmem_wait_ld();
+      // the state after step s is what the next frame in scan order reads
+      __nv_bfloat16* dst = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(s + 1)) * (D * D) + (size_t)row * D + half * 64;
+#pragma unroll
+      for (int e = 0; e < 64; e += 8) {
+        uint4 w;
+        uint32_t* a = reinterpret_cast<uint32_t*>(&w);
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+          __nv_bfloat162 v2 = __floats2bfloat162_rn(z[e + 2 * p], z[e + 2 * p + 1]);
+          a[p] = *reinterpret_cast<uint32_t*>(&v2);
+        }
+        *reinterpret_cast<uint4*>(dst + e) = w;
+      }
+      if (s + 2 < T) {                       // another step follows: build its B operand
+#pragma unroll
+        for (int e = 0; e < 64; ++e) z[e] += bt[e];
+        publish_x(z);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 128);
+  }
+}
+
+}  // namespace vdn

@@ -18,6 +18,7 @@
 #include "readout_tc.cuh"
 #include "resolve.cuh"
 #include "scan.cuh"
+#include "scan_tc.cuh"
 
 namespace {
 
@@ -26,10 +27,13 @@ using vdn::Shape;
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-// Offsets of the workspace regions (bytes).  One layout for every path; only the element size of the
-// read state differs.
+// Offsets of the workspace regions (bytes).
+//   plain-fp32 path : stats f32 [n][2d][d] | inv f32 [n][d][d] | fwd f32 [n][d][d] | read f32 [n][d][d]
+//   tensor-core path: stats f32 [n][2d][d] | inv bf16 [n][3][d][d] (C1,C2,C3) | fwd bf16 [n][d][d] (P_{t-1}^T)
+//                     | read bf16 [n][d][d] (R_{t+1}^T), the last two contiguous
 struct Layout {
   size_t stats, inv, fwd, read, total;
+  size_t inv_bytes, state_bytes;
 };
 
 struct StagingLayout {
@@ -89,7 +93,7 @@ bool shape_ok(const vdn_vda_s* h, int B, int T, int F, int H, int d, std::string
   if (d != h->cfg.d) { *why = "d differs from the handle's configured head dimension"; return false; }
   const long long tok = (long long)B * T * F;
   if (tok > 0x7fffffffLL / 2) { *why = "B*T*F exceeds the 32-bit token index range"; return false; }
-  if ((long long)B * H * T > 0x7fffffffLL / 4) { *why = "B*H*T exceeds the grid range"; return false; }
+  if ((long long)B * H * T > (1LL << 22)) { *why = "B*H*T exceeds 2^22 frames"; return false; }
   if ((long long)B * H > 65535LL * 1024) { *why = "B*H too large"; return false; }
   return true;
 }
@@ -99,10 +103,13 @@ Layout make_layout(const vdn_vda_s* h, int B, int T, int H, int d) {
   const size_t dd = (size_t)d * d;
   Layout L;
   size_t off = kAlign;  // a reserved header line
+  const bool tcp = use_tensor_cores(h, d);
+  L.inv_bytes = tcp ? n * dd * 3 * 2 : n * dd * sizeof(float);
+  L.state_bytes = tcp ? n * dd * 2 : n * dd * sizeof(float);
   L.stats = off; off += align_up(n * dd * 2 * sizeof(float));
-  L.inv = off;   off += align_up(n * dd * sizeof(float));
-  L.fwd = off;   off += align_up(n * dd * sizeof(float));
-  L.read = off;  off += align_up(n * dd * (use_tensor_cores(h, d) ? 2 : sizeof(float)));
+  L.inv = off;   off += align_up(L.inv_bytes);
+  L.fwd = off;   off += L.state_bytes;             // fwd and read stay contiguous (n*d*d*es is 256-aligned)
+  L.read = off;  off += align_up(L.state_bytes);
   L.total = off;
   return L;
 }
@@ -178,7 +185,7 @@ void prof_mark(vdn_vda_t h, cudaStream_t st, int idx, const char* name) {
 
 template <typename Tio, int D>
 vdn_status set_attrs_simt(vdn_vda_t h) {
-  VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_kernel<D, 32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_kernel<D, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)sizeof(vdn::ScanSmem<D, 32>)));
   VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_simt_kernel<Tio, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)sizeof(vdn::ReadoutSimtSmem<D>)));
@@ -207,7 +214,7 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
   prof_mark(h, st, 0, "gram_simt");
   vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n);
   prof_mark(h, st, 1, "resolve");
-  vdn::scan_kernel<D, 32, false><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
+  vdn::scan_kernel<D, 32><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
       stats, inv, fwd, read, s.T);
   prof_mark(h, st, 2, "scan");
   vdn::readout_simt_kernel<Tio, D><<<dim3((unsigned)n, (s.F + 63) / 64), 256, sizeof(vdn::ReadoutSimtSmem<D>), st>>>(
@@ -238,16 +245,16 @@ vdn_status make_token_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, const Sh
   return VDN_OK;
 }
 
-// Read states, bf16 [frames*128][128] as a 2-D map with a (64, 128) box.
-vdn_status make_state_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, long long nframes) {
-  const cuuint64_t dims[2] = {128, (cuuint64_t)nframes * 128};
+// A stack of 128 x 128 bf16 matrices, [rows][128], as a 2-D map with a (64, 128) box.
+vdn_status make_matrix_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, long long rows) {
+  const cuuint64_t dims[2] = {128, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {256};
   const cuuint32_t box[2] = {64, 128};
   const cuuint32_t estr[2] = {1, 1};
   CUresult r = h->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled (state tensor) failed: " + std::to_string((int)r));
+  if (r != CUDA_SUCCESS) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled (matrix stack) failed: " + std::to_string((int)r));
   return VDN_OK;
 }
 
@@ -260,35 +267,36 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
                                      vdn::GramTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ReadoutTc::SMEM_BYTES));
-    VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_kernel<D, 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)sizeof(vdn::ScanSmem<D, 32>)));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::ScanTc::SMEM_BYTES));
     h->tc_attrs_set = true;
   }
   char* ws = static_cast<char*>(h->workspace);
   float* stats = reinterpret_cast<float*>(ws + L.stats);
-  float* inv = reinterpret_cast<float*>(ws + L.inv);
-  float* fwd = reinterpret_cast<float*>(ws + L.fwd);
-  void* read = ws + L.read;
+  __nv_bfloat16* csplit = reinterpret_cast<__nv_bfloat16*>(ws + L.inv);
+  __nv_bfloat16* pf = reinterpret_cast<__nv_bfloat16*>(ws + L.fwd);
+  __nv_bfloat16* pb = reinterpret_cast<__nv_bfloat16*>(ws + L.read);
   const long long n = s.frames();
 
-  CUtensorMap tmQ, tmK, tmV, tmO, tmS;
+  CUtensorMap tmQ, tmK, tmV, tmO, tmS, tmC;
   vdn_status r;
   if ((r = make_token_map(h, &tmK, k, s)) != VDN_OK) return r;
   if ((r = make_token_map(h, &tmV, v, s)) != VDN_OK) return r;
   if ((r = make_token_map(h, &tmQ, q, s)) != VDN_OK) return r;
   if ((r = make_token_map(h, &tmO, out, s)) != VDN_OK) return r;
-  if ((r = make_state_map(h, &tmS, read, n)) != VDN_OK) return r;
+  if ((r = make_matrix_map(h, &tmS, pf, 2 * n * D)) != VDN_OK) return r;      // pf then pb
+  if ((r = make_matrix_map(h, &tmC, csplit, 3 * n * D)) != VDN_OK) return r;
 
   const unsigned persistent = (unsigned)(n < h->sm_count ? n : h->sm_count);
   prof_begin(h, st);
   vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
                                                                                        h->status_dev);
   prof_mark(h, st, 0, "gram_tc");
-  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n);
+  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n);
   prof_mark(h, st, 1, "resolve");
-  vdn::scan_kernel<D, 32, true><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
-      stats, inv, fwd, read, s.T);
-  prof_mark(h, st, 2, "scan");
+  vdn::scan_tc_kernel<<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS, vdn::ScanTc::SMEM_BYTES, st>>>(
+      tmC, stats, pf, pb, s.T, h->status_dev);
+  prof_mark(h, st, 2, "scan_tc");
   vdn::readout_tc_kernel<<<persistent, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
       tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev);
   prof_mark(h, st, 3, "readout_tc");
@@ -435,12 +443,25 @@ vdn_status vdn_vda_workspace_view(vdn_vda_t h, int which, int B, int T, int F, i
   std::string why;
   if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
   const Layout L = make_layout(h, B, T, H, d);
+  (void)F;
   const size_t n = (size_t)B * H * T, dd = (size_t)d * d;
+  const bool tcp = use_tensor_cores(h, d);
   switch (which) {
     case VDN_VIEW_STATS: *offset_bytes = L.stats; *size_bytes = n * dd * 2 * sizeof(float); break;
-    case VDN_VIEW_INV:   *offset_bytes = L.inv;   *size_bytes = n * dd * sizeof(float); break;
-    case VDN_VIEW_FWD:   *offset_bytes = L.fwd;   *size_bytes = n * dd * sizeof(float); break;
-    case VDN_VIEW_READ:  *offset_bytes = L.read;  *size_bytes = n * dd * (use_tensor_cores(h, d) ? 2 : sizeof(float)); break;
+    case VDN_VIEW_INV:
+      if (tcp) return fail(h, VDN_ERR_UNSUPPORTED, "this handle keeps the inverse as three bf16 parts (VDN_VIEW_INV_SPLIT)");
+      *offset_bytes = L.inv; *size_bytes = L.inv_bytes; break;
+    case VDN_VIEW_FWD:
+    case VDN_VIEW_READ:
+      if (tcp) return fail(h, VDN_ERR_UNSUPPORTED, "this handle keeps the two read states apart (VDN_VIEW_READ_FWD / _BWD)");
+      *offset_bytes = which == VDN_VIEW_FWD ? L.fwd : L.read; *size_bytes = L.state_bytes; break;
+    case VDN_VIEW_INV_SPLIT:
+      if (!tcp) return fail(h, VDN_ERR_UNSUPPORTED, "only the tensor-core kernels split the inverse");
+      *offset_bytes = L.inv; *size_bytes = L.inv_bytes; break;
+    case VDN_VIEW_READ_FWD:
+    case VDN_VIEW_READ_BWD:
+      if (!tcp) return fail(h, VDN_ERR_UNSUPPORTED, "the plain-fp32 kernels store the summed read state (VDN_VIEW_READ)");
+      *offset_bytes = which == VDN_VIEW_READ_FWD ? L.fwd : L.read; *size_bytes = L.state_bytes; break;
     default: return fail(h, VDN_ERR_INVALID_ARG, "unknown view");
   }
   return VDN_OK;
