@@ -28,6 +28,12 @@ PAPER_CONTEXT = ("paper (context only, whole pipeline on 8xB200): 6.70 s DiT den
                  "14.5x over 50-step dense H3, attention >85% of dense denoiser runtime")
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per token-head from the ncu captures summarised
+# under profiles/ (an 8-head case of the 768p recipe; traffic grows in proportion to the token-heads a launch
+# processes, so it is scaled to the benchmarked workload by that count).
+DRAM_BYTES_PER_TOKEN_HEAD = {"gram_tc": 561.1, "readout_tc": 511.5}
+
+
 # ------------------------------------------------------------------------------------------ helpers
 def algorithmic_bytes(w) -> dict:
     """Bytes the method must move per forward: read q, k, v and beta once, write out once."""
@@ -315,14 +321,8 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     if kt:
         dom = max(kt, key=kt.get)
         kind = "gram" if "gram" in dom else ("readout" if "readout" in dom else None)
-        traffic = None
-        tp = os.path.join(ROOT, "profiles", "traffic.json")
-        if os.path.exists(tp):
-            with open(tp) as f:
-                tj = json.load(f)
-            per_token_head = tj.get(dom, {}).get("dram_bytes_per_token_head")
-            if per_token_head:
-                traffic = per_token_head * w.B * w.T * w.F * w.H
+        per_th = DRAM_BYTES_PER_TOKEN_HEAD.get(dom)
+        traffic = per_th * w.B * w.T * w.F * w.H if per_th else None
         if kind is not None:
             achieved = ab[kind] / (kt[dom] / 1e3) / 1e9
             roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
