@@ -138,6 +138,35 @@ int vdn_vda_last_launch_count(vdn_vda_t h);
 vdn_status vdn_vda_profile(vdn_vda_t h, int enable);
 int vdn_vda_kernel_times(vdn_vda_t h, int max_kernels, const char** names, float* mean_ms, int* launches);
 
+/* No counterpart in the paper: a convenience for callers that must not allocate device memory.
+ *
+ * Some programs hand all of a GPU's memory to their own pools at start-up and, from then on, treat any
+ * cudaMalloc as a bug (it can fail for lack of memory, and it stalls every stream of the device); others
+ * run this step from places where allocating is not possible at all, e.g. a real-time loop with a fixed
+ * memory plan.  vdn_vda_forward needs a caller-supplied workspace, which such callers may have no pool
+ * to cut from.  This entry point runs ONE stage of the plain-fp32 path -- the bidirectional frame scan
+ * and gather (Alg. 1 steps 5-6: Eq. A.1, Eq. A.4) -- whose only scratch is the buffer of forward states
+ * P_t, and keeps that scratch in an array that is part of the library image
+ * (VDN_SCAN_STATIC_MAX_BYTES bytes of device memory on every GPU that loads the library, until the
+ * process exits).  It calls neither cudaMalloc nor cudaFree nor any routine that allocates.
+ *
+ *   stats [BH][T][2d][d] float, DEVICE  in   per-frame statistics, layout of VDN_VIEW_STATS
+ *   inv   [BH][T][d][d]  float, DEVICE  in   C_t = (I + A_t)^{-1}, layout of VDN_VIEW_INV
+ *   read  [BH][T][d][d]  float, DEVICE  out  transpose of P_{t-1} + R_{t+1}, layout of VDN_VIEW_READ
+ *   BH = batch * heads chains of T frames; d = 64 or 128; all pointers 16-byte aligned, caller-owned.
+ *
+ * Limit: BH*T*d*d*4 bytes must not exceed VDN_SCAN_STATIC_MAX_BYTES (8 MiB: 128 frames at d = 128, 512 at
+ * d = 64); larger shapes are rejected with VDN_ERR_WORKSPACE and a message in errbuf, and nothing is
+ * enqueued.  errbuf (HOST, may be NULL) receives a NUL-terminated description of any error.
+ * The first call on a device looks up the array's address on that device (cudaGetSymbolAddress); make that
+ * first call outside any stream capture.  Enqueues on cuda_stream and returns without synchronising.
+ * Every call on a device uses the same array: two calls whose kernels may overlap on the GPU (different
+ * streams, or different host threads) race on it -- serialise them.  The array keeps the previous call's
+ * contents; the kernel writes every element it later reads, so nothing has to be cleared in between. */
+#define VDN_SCAN_STATIC_MAX_BYTES (8u << 20)
+vdn_status vdn_vda_scan_static(const float* stats, const float* inv, float* read, int BH, int T, int d,
+                               int device, void* cuda_stream, char* errbuf, size_t errbuf_len);
+
 /* Last device-side status recorded by this handle's kernels (VDN_OK or VDN_ERR_TIMEOUT).  Does not
  * synchronise: call it after synchronising the stream.  Reading it clears nothing. */
 vdn_status vdn_vda_status(vdn_vda_t h);

@@ -23,7 +23,7 @@ VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_R
 EXPORTS = (
     "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward",
     "vdn_vda_staging_bytes", "vdn_vda_set_staging", "vdn_vda_forward_host", "vdn_vda_workspace_view",
-    "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_status", "vdn_vda_last_error", "vdn_vda_destroy",
+    "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_scan_static", "vdn_vda_status", "vdn_vda_last_error", "vdn_vda_destroy",
 )
 
 
@@ -77,6 +77,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.vdn_vda_kernel_times.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float),
                                          ctypes.POINTER(ci)]
     lib.vdn_vda_kernel_times.restype = ci
+    lib.vdn_vda_scan_static.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, ctypes.c_char_p, sz]
+    lib.vdn_vda_scan_static.restype = ci
     lib.vdn_vda_status.argtypes = [vp]
     lib.vdn_vda_status.restype = ci
     lib.vdn_vda_last_error.argtypes = [vp]
@@ -86,6 +88,36 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     if path is None:
         _lib = lib
     return lib
+
+
+SCAN_STATIC_MAX_BYTES = 8 << 20
+
+
+def scan_static(stats, inv, read, stream=None):
+    """vdn_vda_scan_static: the fp32 frame scan + gather with its scratch inside the library image.
+
+    For callers that may not allocate device memory.  stats [BH,T,2d,d], inv [BH,T,d,d] and the output
+    read [BH,T,d,d] are contiguous float CUDA tensors owned by the caller; nothing is allocated here or
+    in the library.  Raises VdnError (VDN_ERR_WORKSPACE) when BH*T*d*d*4 exceeds SCAN_STATIC_MAX_BYTES.
+    Calls that may overlap on the GPU share the scratch and must be serialised by the caller.
+    """
+    import torch
+    lib = load_library()
+    BH, T, d2, d = stats.shape
+    for x in (stats, inv, read):
+        if not (x.is_cuda and x.is_contiguous() and x.dtype == torch.float32):
+            raise ValueError("scan_static needs contiguous float32 CUDA tensors")
+    if d2 != 2 * d or tuple(inv.shape) != (BH, T, d, d) or tuple(read.shape) != (BH, T, d, d):
+        raise ValueError("scan_static: shapes must be stats [BH,T,2d,d], inv/read [BH,T,d,d]")
+    dev = stats.device.index or 0
+    s = stream if stream is not None else torch.cuda.current_stream(dev)
+    err = ctypes.create_string_buffer(256)
+    st = lib.vdn_vda_scan_static(ctypes.c_void_p(stats.data_ptr()), ctypes.c_void_p(inv.data_ptr()),
+                                 ctypes.c_void_p(read.data_ptr()), BH, T, d, dev, ctypes.c_void_p(s.cuda_stream),
+                                 err, len(err))
+    if st != VDN_OK:
+        raise VdnError(st, err.value.decode())
+    return read
 
 
 class Vda:

@@ -305,6 +305,34 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   return VDN_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Scratch for vdn_vda_scan_static: lives in the library image, one copy on every GPU that loads it.
+// In host code the array's name is only a handle for cudaGetSymbolAddress, never a device address.
+constexpr size_t kStaticScanFloats = VDN_SCAN_STATIC_MAX_BYTES / sizeof(float);
+static __device__ __align__(256) float g_scan_static_scratch[kStaticScanFloats];
+constexpr int kMaxDevices = 64;
+float* g_scan_static_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+
+void put_msg(char* buf, size_t len, const std::string& msg) {
+  if (!buf || len == 0) return;
+  const size_t n = msg.size() < len - 1 ? msg.size() : len - 1;
+  std::memcpy(buf, msg.data(), n);
+  buf[n] = 0;
+}
+
+template <int D>
+vdn_status launch_scan_static(const float* stats, const float* inv, float* read, int BH, int T, float* scratch,
+                              cudaStream_t st, std::string* why) {
+  cudaError_t e = cudaFuncSetAttribute(vdn::scan_kernel<D, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)sizeof(vdn::ScanSmem<D, 32>));
+  if (e != cudaSuccess) { *why = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return VDN_ERR_CUDA; }
+  vdn::scan_kernel<D, 32><<<dim3((unsigned)BH, D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(stats, inv, scratch,
+                                                                                               read, T);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) { *why = std::string("kernel launch: ") + cudaGetErrorString(e); return VDN_ERR_CUDA; }
+  return VDN_OK;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
@@ -510,6 +538,44 @@ vdn_status vdn_vda_status(vdn_vda_t h) {
   if (!h) return VDN_ERR_INVALID_ARG;
   const int v = *const_cast<volatile int*>(h->status_host);
   return v == 0 ? VDN_OK : VDN_ERR_TIMEOUT;
+}
+
+vdn_status vdn_vda_scan_static(const float* stats, const float* inv, float* read, int BH, int T, int d,
+                               int device, void* cuda_stream, char* errbuf, size_t errbuf_len) {
+  if (!stats || !inv || !read) { put_msg(errbuf, errbuf_len, "null tensor pointer"); return VDN_ERR_INVALID_ARG; }
+  if (!aligned16(stats) || !aligned16(inv) || !aligned16(read)) {
+    put_msg(errbuf, errbuf_len, "stats, inv, read must be 16-byte aligned");
+    return VDN_ERR_INVALID_ARG;
+  }
+  if (BH <= 0 || T <= 0) { put_msg(errbuf, errbuf_len, "BH and T must be positive"); return VDN_ERR_INVALID_ARG; }
+  if (d != 64 && d != 128) { put_msg(errbuf, errbuf_len, "d must be 64 or 128"); return VDN_ERR_UNSUPPORTED; }
+  if (device < 0 || device >= kMaxDevices) { put_msg(errbuf, errbuf_len, "device ordinal out of range"); return VDN_ERR_INVALID_ARG; }
+  const size_t need = (size_t)BH * T * d * d * sizeof(float);
+  if ((size_t)BH * T > kStaticScanFloats / ((size_t)d * d)) {
+    put_msg(errbuf, errbuf_len,
+            "BH*T*d*d*4 = " + std::to_string(need) + " bytes of scan scratch exceed the built-in " +
+                std::to_string((size_t)VDN_SCAN_STATIC_MAX_BYTES) + " bytes (VDN_SCAN_STATIC_MAX_BYTES); use vdn_vda_forward with a workspace");
+    return VDN_ERR_WORKSPACE;
+  }
+  DeviceGuard guard(device);
+  if (!guard.ok) { put_msg(errbuf, errbuf_len, "cannot make the device current"); return VDN_ERR_CUDA; }
+  if (!g_scan_static_ptr[device]) {
+    // first call on this device: look up where the array lives on it (the device is current here)
+    float* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_scan_static_scratch);
+    if (e != cudaSuccess || !ptr) {
+      put_msg(errbuf, errbuf_len, std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+      cudaGetLastError();
+      return VDN_ERR_CUDA;
+    }
+    g_scan_static_ptr[device] = ptr;
+  }
+  std::string why;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const vdn_status r = d == 64 ? launch_scan_static<64>(stats, inv, read, BH, T, g_scan_static_ptr[device], st, &why)
+                               : launch_scan_static<128>(stats, inv, read, BH, T, g_scan_static_ptr[device], st, &why);
+  if (r != VDN_OK) put_msg(errbuf, errbuf_len, why);
+  return r;
 }
 
 const char* vdn_vda_last_error(vdn_vda_t h) { return h ? h->err.c_str() : "null handle"; }
