@@ -25,6 +25,18 @@ __device__ __forceinline__ void split_frame(const Shape& s, long long n, int& b,
   b = (int)(bh / s.H);
 }
 
+// Work order of the persistent tensor-core kernels: work item w -> (b, t, h) with the head fastest, so
+// that CTAs running side by side stream the same token rows (a token's H heads are contiguous in memory:
+// neighbouring 256-byte pieces of one DRAM page, and shared 32-byte sectors of beta).  Returns the frame
+// index n = (b*H + h)*T + t that addresses the workspace.
+__device__ __forceinline__ long long split_work(const Shape& s, long long w, int& b, int& h, int& t) {
+  h = (int)(w % s.H);
+  long long bt = w / s.H;
+  t = (int)(bt % s.T);
+  b = (int)(bt / s.T);
+  return ((long long)b * s.H + h) * s.T + t;
+}
+
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 

@@ -89,7 +89,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       bool ok = true;
       for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
         int b, h, t;
-        split_frame(s, item, b, h, t);
+        split_work(s, item, b, h, t);
         for (int tile = 0; tile < ntiles; ++tile, ++it) {
           const int st = it % G::STAGES;
           if (!mbar_wait(EMPTY(st), ((it / G::STAGES) & 1) ^ 1, wc)) { ok = false; break; }
@@ -149,7 +149,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     bool ok = true;
     for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
       int b, h, t;
-      split_frame(s, item, b, h, t);
+      split_work(s, item, b, h, t);
       const float* brow = beta + ((size_t)b * s.T + t) * s.F * s.H + h;
       for (int tile = 0; tile < ntiles && ok; ++tile, ++it) {
         const int st = it % G::STAGES;
@@ -198,7 +198,9 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 256;
       // accumulator lane = key channel i, column = column of [K|V]; stored transposed, [2d][d], so that
       // the 32 lanes of a warp write 32 consecutive floats
-      float* dst = stats + (size_t)item * (2 * G::D * G::D) + row;
+      int b, h, t;
+      const long long n = split_work(s, item, b, h, t);
+      float* dst = stats + (size_t)n * (2 * G::D * G::D) + row;
 #pragma unroll 1
       for (int cc = 0; cc < 8; ++cc) {
         float v[32];

@@ -86,15 +86,15 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       bool ok = true;
       for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
         int b, h, t;
-        split_frame(s, item, b, h, t);
+        const long long n = split_work(s, item, b, h, t);
         if (!mbar_wait(STEMPTY(0), (si & 1) ^ 1, wc)) { ok = false; break; }
         mbar_arrive_expect_tx(STFULL(0), 2 * R::TILE_BYTES);
         const uint32_t sdst = base + R::OFF_STATE;
-        // rows [item*128, +128) hold the forward state, rows [(nitems+item)*128, +128) the reverse state
-        tma_load_2d(sdst, &tmS, STFULL(0), 0, (int)(item * R::D));
-        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(item * R::D));
-        tma_load_2d(sdst + 2 * R::BOX_BYTES, &tmS, STFULL(0), 0, (int)((nitems + item) * R::D));
-        tma_load_2d(sdst + 3 * R::BOX_BYTES, &tmS, STFULL(0), 64, (int)((nitems + item) * R::D));
+        // rows [n*128, +128) hold the forward state, rows [(nitems+n)*128, +128) the reverse state
+        tma_load_2d(sdst, &tmS, STFULL(0), 0, (int)(n * R::D));
+        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(n * R::D));
+        tma_load_2d(sdst + 2 * R::BOX_BYTES, &tmS, STFULL(0), 0, (int)((nitems + n) * R::D));
+        tma_load_2d(sdst + 3 * R::BOX_BYTES, &tmS, STFULL(0), 64, (int)((nitems + n) * R::D));
         for (int tile = 0; tile < ntiles; ++tile, ++qi) {
           const int st = qi % R::QSTAGES;
           if (!mbar_wait(QEMPTY(st), ((qi / R::QSTAGES) & 1) ^ 1, wc)) { ok = false; break; }
@@ -150,7 +150,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     bool ok = true;
     for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
       int b, h, t;
-      split_frame(s, item, b, h, t);
+      split_work(s, item, b, h, t);
       const float g = __ldg(gate + h);
       for (int tile = 0; tile < ntiles; ++tile, ++qi) {
         const int a = qi & 3;
