@@ -21,13 +21,82 @@
 
 namespace vdn {
 
+// In-place inverse of the D x D matrix held as R x R cyclic tiles by a 16 x 16 thread grid.
+// rowbuf / colbuf: 2 x D floats each in shared memory; sync(): a barrier over the 256 threads.
+template <int D, typename Sync>
+__device__ __forceinline__ void gauss_jordan_tiles(float (&m)[D / 16][D / 16], float* rowbuf, float* colbuf,
+                                                   int tx, int ty, Sync sync) {
+  constexpr int R = D / 16;
+#pragma unroll
+  for (int q = 0; q < R; ++q) {
+#pragma unroll 2
+    for (int o = 0; o < 16; ++o) {
+      float* rb = rowbuf + (o & 1) * D;      // indexed [owner tx][c]
+      float* cb = colbuf + (o & 1) * D;      // indexed [owner ty][r]
+      if (ty == o) {                      // owners of the pivot row: publish it, then clear it
+#pragma unroll
+        for (int c = 0; c < R; c += 4) {
+          store4(rb + tx * R + c, make_float4(m[q][c], m[q][c + 1], m[q][c + 2], m[q][c + 3]));
+          m[q][c] = 0.f; m[q][c + 1] = 0.f; m[q][c + 2] = 0.f; m[q][c + 3] = 0.f;
+        }
+      }
+      if (tx == o) {                      // owners of the pivot column
+        float cv[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) { cv[r] = m[r][q]; m[r][q] = 0.f; }
+        if (ty == o) cv[q] = -1.0f;       // (the pivot itself was already published with the row)
+#pragma unroll
+        for (int r = 0; r < R; r += 4) store4(cb + ty * R + r, make_float4(cv[r], cv[r + 1], cv[r + 2], cv[r + 3]));
+      }
+      sync();
+      const float ipiv = __frcp_rn(rb[o * R + q]);
+      float rv[R], cv[R];
+#pragma unroll
+      for (int c = 0; c < R; c += 4) {
+        float4 x = load4(rb + tx * R + c);
+        rv[c] = x.x * ipiv; rv[c + 1] = x.y * ipiv; rv[c + 2] = x.z * ipiv; rv[c + 3] = x.w * ipiv;
+      }
+      if (tx == o) rv[q] = ipiv;
+#pragma unroll
+      for (int r = 0; r < R; r += 4) {
+        float4 x = load4(cb + ty * R + r);
+        cv[r] = x.x; cv[r + 1] = x.y; cv[r + 2] = x.z; cv[r + 3] = x.w;
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int c = 0; c < R; ++c) m[r][c] = fmaf(-cv[r], rv[c], m[r][c]);
+    }
+  }
+}
+
+// The tiles as three bf16 matrices S[0] + S[1] + S[2] (each D x D, row-major).
+template <int D>
+__device__ __forceinline__ void store_split_tiles(const float (&m)[D / 16][D / 16], __nv_bfloat16* S, int tx, int ty) {
+  constexpr int R = D / 16;
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+      const size_t e = (size_t)(ty + 16 * r) * D + tx + 16 * c;
+      const float x = m[r][c];
+      const __nv_bfloat16 p1 = __float2bfloat16_rn(x);
+      const float r1 = x - __bfloat162float(p1);
+      const __nv_bfloat16 p2 = __float2bfloat16_rn(r1);
+      const __nv_bfloat16 p3 = __float2bfloat16_rn(r1 - __bfloat162float(p2));
+      S[e] = p1;
+      S[(size_t)D * D + e] = p2;
+      S[(size_t)2 * D * D + e] = p3;
+    }
+}
+
 template <int D>
 __global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict__ stats,
                                                           float* __restrict__ inv,
                                                           __nv_bfloat16* __restrict__ split, long long nframes) {
   constexpr int R = D / 16;
-  __shared__ __align__(16) float rowbuf[2][D];   // indexed [owner tx][c]
-  __shared__ __align__(16) float colbuf[2][D];   // indexed [owner ty][r]
+  __shared__ __align__(16) float rowbuf[2 * D];
+  __shared__ __align__(16) float colbuf[2 * D];
 
   const long long n = blockIdx.x;
   if (n >= nframes) return;
@@ -43,46 +112,7 @@ __global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict
       m[r][c] = __ldg(A + (size_t)i * D + j) + (i == j ? 1.0f : 0.0f);
     }
 
-#pragma unroll
-  for (int q = 0; q < R; ++q) {
-#pragma unroll 2
-    for (int o = 0; o < 16; ++o) {
-      const int par = o & 1;
-      if (ty == o) {                      // owners of the pivot row: publish it, then clear it
-#pragma unroll
-        for (int c = 0; c < R; c += 4) {
-          store4(&rowbuf[par][tx * R + c], make_float4(m[q][c], m[q][c + 1], m[q][c + 2], m[q][c + 3]));
-          m[q][c] = 0.f; m[q][c + 1] = 0.f; m[q][c + 2] = 0.f; m[q][c + 3] = 0.f;
-        }
-      }
-      if (tx == o) {                      // owners of the pivot column
-        float cv[R];
-#pragma unroll
-        for (int r = 0; r < R; ++r) { cv[r] = m[r][q]; m[r][q] = 0.f; }
-        if (ty == o) cv[q] = -1.0f;       // (the pivot itself was already published with the row)
-#pragma unroll
-        for (int r = 0; r < R; r += 4) store4(&colbuf[par][ty * R + r], make_float4(cv[r], cv[r + 1], cv[r + 2], cv[r + 3]));
-      }
-      __syncthreads();
-      const float ipiv = __frcp_rn(rowbuf[par][o * R + q]);
-      float rv[R], cv[R];
-#pragma unroll
-      for (int c = 0; c < R; c += 4) {
-        float4 x = load4(&rowbuf[par][tx * R + c]);
-        rv[c] = x.x * ipiv; rv[c + 1] = x.y * ipiv; rv[c + 2] = x.z * ipiv; rv[c + 3] = x.w * ipiv;
-      }
-      if (tx == o) rv[q] = ipiv;
-#pragma unroll
-      for (int r = 0; r < R; r += 4) {
-        float4 x = load4(&colbuf[par][ty * R + r]);
-        cv[r] = x.x; cv[r + 1] = x.y; cv[r + 2] = x.z; cv[r + 3] = x.w;
-      }
-#pragma unroll
-      for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int c = 0; c < R; ++c) m[r][c] = fmaf(-cv[r], rv[c], m[r][c]);
-    }
-  }
+  gauss_jordan_tiles<D>(m, rowbuf, colbuf, tx, ty, [] { __syncthreads(); });
 
   if (inv != nullptr) {
     float* C = inv + (size_t)n * D * D;
@@ -91,23 +121,7 @@ __global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict
 #pragma unroll
       for (int c = 0; c < R; ++c) C[(size_t)(ty + 16 * r) * D + tx + 16 * c] = m[r][c];
   }
-  if (split != nullptr) {
-    __nv_bfloat16* S = split + (size_t)n * 3 * D * D;
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-      for (int c = 0; c < R; ++c) {
-        const size_t e = (size_t)(ty + 16 * r) * D + tx + 16 * c;
-        const float x = m[r][c];
-        const __nv_bfloat16 p1 = __float2bfloat16_rn(x);
-        const float r1 = x - __bfloat162float(p1);
-        const __nv_bfloat16 p2 = __float2bfloat16_rn(r1);
-        const __nv_bfloat16 p3 = __float2bfloat16_rn(r1 - __bfloat162float(p2));
-        S[e] = p1;
-        S[(size_t)D * D + e] = p2;
-        S[(size_t)2 * D * D + e] = p3;
-      }
-  }
+  if (split != nullptr) store_split_tiles<D>(m, split + (size_t)n * 3 * D * D, tx, ty);
 }
 
 }  // namespace vdn

@@ -1,0 +1,255 @@
+// Resolve (Eq. 5, Alg. 1 step 4):  C_t = (I + A_t)^{-1}, d = 128, with the O(d^3) part of the elimination on
+// the tcgen05 tensor cores at fp32 accuracy.  One CTA per frame; the matrix lives in TMEM.
+//
+// Blocked Gauss-Jordan, 16 pivots per step (8 steps), no pivot search (I + A_t is SPD, eigenvalues >= 1).
+// With P the pivot indices of a step, G = M[P][P] and Gi = G^{-1}, the in-place inverse update is
+//     rows outside P :  M[i][:] += c_i M[P][:],   c_i = -M[i][P] Gi,          then  M[i][P] = c_i
+//     rows inside  P :  M[a][:] += (Gi[a] - e_a) M[P][:]   (= Gi[a] M[P][:]), then  M[a][P] = Gi[a]
+// i.e. one rank-16 update  M += Cm * M[P][:]  of the whole matrix plus a 128 x 16 column fix.  The rank-16
+// update is a 128 x 128 x 16 MMA accumulating into the TMEM-resident matrix.  Both factors are fp32 values
+// split three-way into bf16 parts (24 mantissa bits); the six partial products of weight >= 2^-24 are
+// accumulated in fp32, so the update carries fp32 accuracy.  Everything else is plain fp32:
+//   * the 16 x 16 pivot block is inverted inside the warp that owns those rows, one row per lane, the pivot
+//     rows travelling by shuffle;
+//   * every thread owns one matrix row (its TMEM lane) and forms its 16 coefficients from Gi.
+// The inverse is written as three bf16 parts C1 + C2 + C3 for the tensor-core scan.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace vdn {
+
+struct ResolveTc {
+  static constexpr int D = 128;
+  static constexpr int NB = 16;                       // pivots per step
+  static constexpr int CM_PART = 128 * 128;           // coefficient part: 128 rows x 128 B (32 B used), K-major
+  static constexpr int PR_PART = 2 * NB * 128;        // pivot-row part: 2 boxes x 16 rows x 128 B, MN-major
+  static constexpr int OFF_CM = 0;
+  static constexpr int OFF_PR = 3 * CM_PART;
+  static constexpr int OFF_GI = OFF_PR + 3 * PR_PART; // Gi, 16 x 16 floats
+  static constexpr int OFF_BAR = OFF_GI + 1024;
+  static constexpr int SMEM_BYTES = OFF_BAR + 64 + 1024;
+  static constexpr int THREADS = 160;                 // 4 row warps + 1 MMA warp
+};
+
+__global__ void __launch_bounds__(ResolveTc::THREADS)
+resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ csplit, long long nframes,
+                  int* status) {
+  using namespace tc;
+  using R = ResolveTc;
+  constexpr int D = R::D;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t OPREADY = base + R::OFF_BAR, MMADONE = base + R::OFF_BAR + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 20);
+  float* gi = reinterpret_cast<float*>(base_ptr + R::OFF_GI);
+  const WaitCtx wc{abort_flag, status};
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long n = blockIdx.x;
+  if (n >= nframes) return;
+
+  if (threadIdx.x == 0) {
+    mbar_init(OPREADY, 128);
+    mbar_init(MMADONE, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(smem_u32(tmem_slot), 128);
+    tmem_relinquish();
+  }
+  // the unused 96 bytes of every coefficient row are never read by the MMA (K = 16 = 32 bytes)
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
+      constexpr int PA[6] = {0, 2, 1, 0, 1, 0};   // (coefficient part, pivot-row part), smallest first
+      constexpr int PB[6] = {2, 0, 1, 1, 0, 0};
+      for (int blk = 0; blk < D / R::NB; ++blk) {
+        if (!mbar_wait(OPREADY, blk & 1, wc)) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int pr = 0; pr < 6; ++pr) {
+          const uint64_t adesc = make_smem_desc(base + R::OFF_CM + PA[pr] * R::CM_PART, 16, 1024);
+          const uint64_t bdesc = make_smem_desc(base + R::OFF_PR + PB[pr] * R::PR_PART, R::NB * 128, 1024);
+          mma_bf16_ss(tmem_base, adesc, bdesc, idesc, 1u);
+        }
+        mma_commit(MMADONE);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ row threads
+    const int row = warp * 32 + lane;
+    const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
+    // M = I + A_t into TMEM, 32 columns at a time
+    {
+      const float* src = stats + (size_t)n * (2 * D * D) + (size_t)row * D;
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        float v[32];
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 x = __ldg(reinterpret_cast<const float4*>(src + cc * 32 + e));
+          v[e] = x.x; v[e + 1] = x.y; v[e + 2] = x.z; v[e + 3] = x.w;
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (cc * 32 + e == row) v[e] += 1.0f;
+        tmem_st32(trow + cc * 32, v);
+      }
+      tmem_wait_st();
+    }
+
+    bool ok = true;
+#pragma unroll 1
+    for (int blk = 0; blk < D / R::NB && ok; ++blk) {
+      const int p0 = blk * R::NB;
+      const bool owner = (row >> 4) == blk;               // rows p0 .. p0+15: 16 lanes of warp blk/2
+      float x[16];
+      tmem_ld16(trow + p0, x);
+      tmem_wait_ld();
+
+      if (warp == (blk >> 1)) {
+        // ---- invert the 16 x 16 pivot block: lane (l0 + a) holds row a; pivot rows travel by shuffle
+        const int l0 = (blk & 1) * 16;
+        float g[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) g[j] = x[j];
+#pragma unroll
+        for (int p = 0; p < 16; ++p) {
+          float rp[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) rp[j] = __shfl_sync(0xffffffffu, g[j], l0 + p);
+          const float ip = __frcp_rn(rp[p]);
+          const bool prow = lane == l0 + p;
+          const float f = prow ? -1.0f : g[p];              // coefficient on the scaled pivot row
+          const uint32_t keep = prow ? 0u : 0xFFFFFFFFu;    // the pivot row itself restarts from zero
+          const float fi = f * ip;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) g[j] = fmaf(-fi, rp[j], __uint_as_float(__float_as_uint(g[j]) & keep));
+          g[p] = prow ? ip : -fi;
+        }
+        if (owner) {
+          float* dst = gi + (row & 15) * 16;
+#pragma unroll
+          for (int j = 0; j < 16; j += 4) store4(dst + j, make_float4(g[j], g[j + 1], g[j + 2], g[j + 3]));
+        }
+      }
+      named_barrier_sync(1, 128);
+
+      // ---- coefficients: c = -xx Gi  with xx = M[i][P] (other rows) or -e_a (pivot row a, giving Gi[a])
+      float c[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) c[k] = 0.f;
+#pragma unroll
+      for (int l = 0; l < 16; ++l) {
+        const float xl = owner ? ((row & 15) == l ? 1.0f : 0.0f) : -x[l];
+#pragma unroll
+        for (int k = 0; k < 16; k += 4) {
+          const float4 gq = load4(gi + l * 16 + k);
+          c[k] = fmaf(xl, gq.x, c[k]);
+          c[k + 1] = fmaf(xl, gq.y, c[k + 1]);
+          c[k + 2] = fmaf(xl, gq.z, c[k + 2]);
+          c[k + 3] = fmaf(xl, gq.w, c[k + 3]);
+        }
+      }
+      // ---- A operand: this row's 16 update coefficients (pivot rows: Gi[a] - e_a), three bf16 parts
+      {
+        uint4 w[3][2];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          float u0 = c[2 * q], u1 = c[2 * q + 1];
+          if (owner && (row & 15) == 2 * q) u0 -= 1.0f;
+          if (owner && (row & 15) == 2 * q + 1) u1 -= 1.0f;
+          uint32_t a1, a2, a3;
+          split3_pair(u0, u1, a1, a2, a3);
+          reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
+          reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
+          reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
+        }
+        unsigned char* crow = base_ptr + R::OFF_CM + row * 128;
+#pragma unroll
+        for (int part = 0; part < 3; ++part) {
+          *reinterpret_cast<uint4*>(crow + part * R::CM_PART + ((0 ^ (row & 7)) * 16)) = w[part][0];
+          *reinterpret_cast<uint4*>(crow + part * R::CM_PART + ((1 ^ (row & 7)) * 16)) = w[part][1];
+        }
+      }
+      // ---- B operand: the 16 pivot rows as they stand, three bf16 parts, MN-major
+      if (warp == (blk >> 1)) {
+        const int kr = row & 15;
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          float v[32];
+          tmem_ld32(trow + cc * 32, v);
+          tmem_wait_ld();
+          if (owner) {
+            unsigned char* prow = base_ptr + R::OFF_PR + (cc >> 1) * (R::NB * 128) + kr * 128;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+              uint4 w1, w2, w3;
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                split3_pair(v[ch * 8 + 2 * q], v[ch * 8 + 2 * q + 1], reinterpret_cast<uint32_t*>(&w1)[q],
+                            reinterpret_cast<uint32_t*>(&w2)[q], reinterpret_cast<uint32_t*>(&w3)[q]);
+              const int off = ((((cc & 1) * 4 + ch) ^ (kr & 7)) * 16);
+              *reinterpret_cast<uint4*>(prow + off) = w1;
+              *reinterpret_cast<uint4*>(prow + R::PR_PART + off) = w2;
+              *reinterpret_cast<uint4*>(prow + 2 * R::PR_PART + off) = w3;
+            }
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      tc_fence_before_sync();
+      mbar_arrive(OPREADY);
+      if (!mbar_wait(MMADONE, blk & 1, wc)) { ok = false; break; }
+      tc_fence_after_sync();
+      // ---- column fix: M[i][P] = c (for a pivot row: Gi[a])
+      tmem_st16(trow + p0, c);
+      tmem_wait_st();
+    }
+
+    if (ok) {
+      // ---- the inverse, row by row, as three bf16 parts
+      __nv_bfloat16* c1 = csplit + (size_t)n * (3 * D * D) + (size_t)row * D;
+#pragma unroll 1
+      for (int cc = 0; cc < 4; ++cc) {
+        float v[32];
+        tmem_ld32(trow + cc * 32, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint4 w1, w2, w3;
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            split3_pair(v[ch * 8 + 2 * q], v[ch * 8 + 2 * q + 1], reinterpret_cast<uint32_t*>(&w1)[q],
+                        reinterpret_cast<uint32_t*>(&w2)[q], reinterpret_cast<uint32_t*>(&w3)[q]);
+          const int e = cc * 32 + ch * 8;
+          *reinterpret_cast<uint4*>(c1 + e) = w1;
+          *reinterpret_cast<uint4*>(c1 + D * D + e) = w2;
+          *reinterpret_cast<uint4*>(c1 + 2 * D * D + e) = w3;
+        }
+      }
+    }
+  }
+
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 128);
+  }
+}
+
+}  // namespace vdn

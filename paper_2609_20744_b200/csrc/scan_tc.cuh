@@ -37,20 +37,6 @@ struct ScanTc {
   static constexpr int THREADS = 320;
 };
 
-// x -> three bf16 parts for two neighbouring elements at once (packed as bf16x2 words).
-__device__ __forceinline__ void split3_pair(float x0, float x1, uint32_t& p1, uint32_t& p2, uint32_t& p3) {
-  __nv_bfloat162 a = __floats2bfloat162_rn(x0, x1);
-  p1 = *reinterpret_cast<uint32_t*>(&a);
-  x0 -= __uint_as_float(p1 << 16);
-  x1 -= __uint_as_float(p1 & 0xFFFF0000u);
-  __nv_bfloat162 b = __floats2bfloat162_rn(x0, x1);
-  p2 = *reinterpret_cast<uint32_t*>(&b);
-  x0 -= __uint_as_float(p2 << 16);
-  x1 -= __uint_as_float(p2 & 0xFFFF0000u);
-  __nv_bfloat162 c = __floats2bfloat162_rn(x0, x1);
-  p3 = *reinterpret_cast<uint32_t*>(&c);
-}
-
 __global__ void __launch_bounds__(ScanTc::THREADS, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict__ stats,
                __nv_bfloat16* __restrict__ pf, __nv_bfloat16* __restrict__ pb, int T, int* status) {

@@ -17,6 +17,7 @@
 #include "readout_simt.cuh"
 #include "readout_tc.cuh"
 #include "resolve.cuh"
+#include "resolve_tc.cuh"
 #include "scan.cuh"
 #include "scan_tc.cuh"
 
@@ -269,6 +270,8 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
                                      vdn::ReadoutTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::resolve_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::ResolveTc::SMEM_BYTES));
     h->tc_attrs_set = true;
   }
   char* ws = static_cast<char*>(h->workspace);
@@ -289,18 +292,27 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
 
   const unsigned persistent = (unsigned)(n < h->sm_count ? n : h->sm_count);
   prof_begin(h, st);
-  vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
-                                                                                       h->status_dev);
-  prof_mark(h, st, 0, "gram_tc");
-  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n);
-  prof_mark(h, st, 1, "resolve");
+  int nk = 0;
+  if (h->cfg.flags & VDN_FLAG_RESOLVE_IN_GRAM) {
+    // statistics + resolve in one kernel: spare warps invert I + A_t (plain fp32) while the next frame streams in
+    vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(
+        tmK, tmV, beta, stats, csplit, s, h->status_dev);
+    prof_mark(h, st, nk++, "gram_tc");
+  } else {
+    vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(
+        tmK, tmV, beta, stats, nullptr, s, h->status_dev);
+    prof_mark(h, st, nk++, "gram_tc");
+    vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
+        stats, csplit, n, h->status_dev);
+    prof_mark(h, st, nk++, "resolve_tc");
+  }
   vdn::scan_tc_kernel<<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS, vdn::ScanTc::SMEM_BYTES, st>>>(
       tmC, stats, pf, pb, s.T, h->status_dev);
-  prof_mark(h, st, 2, "scan_tc");
+  prof_mark(h, st, nk++, "scan_tc");
   vdn::readout_tc_kernel<<<persistent, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
       tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev);
-  prof_mark(h, st, 3, "readout_tc");
-  h->launches = 4;
+  prof_mark(h, st, nk++, "readout_tc");
+  h->launches = nk;
   VDN_CUDA(h, cudaGetLastError());
   return VDN_OK;
 }

@@ -134,6 +134,8 @@ def test_stagewise_intermediates_tensor_core_kernels():
             # bf16 products are exact in fp32; only the beta-weighted key operand is rounded (2^-9 relative)
             assert rel(stats[0, h, t, :d, :], ref["A"][t]) < 4e-3
             assert rel(stats[0, h, t, d:, :], ref["B"][t]) < 4e-3
+            # (the stored A block is K^T (beta K) with only one factor rounded to bf16, hence symmetric up to
+            # that rounding only; the resolve inverts I + the stored block as it stands)
             inv_g = np.linalg.inv(np.eye(d) + stats[0, h, t, :d, :])
             assert rel(split[0, h, t].sum(axis=0), inv_g) < 1e-5            # three parts carry fp32 accuracy
             assert rel(split[0, h, t, 0], inv_g) < 5e-3                     # the leading part alone is bf16
