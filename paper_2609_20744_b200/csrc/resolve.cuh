@@ -13,7 +13,7 @@
 // one FMA per element, no predication, one barrier per pivot.
 //
 // When `split` is non-null the inverse is also written as three bf16 matrices C1 + C2 + C3 (each the
-// bf16 rounding of what the previous ones leave over, 24 mantissa bits in all) for the tensor-core scan.
+// truncation to bf16 of what the previous ones leave over, 24 mantissa bits in all) for the tensor-core scan.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -79,14 +79,15 @@ __device__ __forceinline__ void store_split_tiles(const float (&m)[D / 16][D / 1
 #pragma unroll
     for (int c = 0; c < R; ++c) {
       const size_t e = (size_t)(ty + 16 * r) * D + tx + 16 * c;
+      // truncating three-way split: x = p1 + p2 + p3 exactly
       const float x = m[r][c];
-      const __nv_bfloat16 p1 = __float2bfloat16_rn(x);
-      const float r1 = x - __bfloat162float(p1);
-      const __nv_bfloat16 p2 = __float2bfloat16_rn(r1);
-      const __nv_bfloat16 p3 = __float2bfloat16_rn(r1 - __bfloat162float(p2));
-      S[e] = p1;
-      S[(size_t)D * D + e] = p2;
-      S[(size_t)2 * D * D + e] = p3;
+      const uint32_t u1 = __float_as_uint(x) & 0xFFFF0000u;
+      const float r1 = x - __uint_as_float(u1);
+      const uint32_t u2 = __float_as_uint(r1) & 0xFFFF0000u;
+      const uint32_t u3 = __float_as_uint(r1 - __uint_as_float(u2)) & 0xFFFF0000u;
+      S[e] = __ushort_as_bfloat16((unsigned short)(u1 >> 16));
+      S[(size_t)D * D + e] = __ushort_as_bfloat16((unsigned short)(u2 >> 16));
+      S[(size_t)2 * D * D + e] = __ushort_as_bfloat16((unsigned short)(u3 >> 16));
     }
 }
 

@@ -21,6 +21,14 @@
 
 namespace vdn {
 
+// 1/x for x >= 1 (a pivot of an SPD matrix with eigenvalues >= 1): hardware approximation plus one Newton
+// step, good to about 1 ulp, on a much shorter dependency chain than the correctly rounded reciprocal.
+__device__ __forceinline__ float fast_rcp(float x) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return fmaf(r, fmaf(-x, r, 1.0f), r);
+}
+
 struct ResolveTc {
   static constexpr int D = 128;
   static constexpr int NB = 16;                       // pivots per step
@@ -34,7 +42,7 @@ struct ResolveTc {
   static constexpr int THREADS = 160;                 // 4 row warps + 1 MMA warp
 };
 
-__global__ void __launch_bounds__(ResolveTc::THREADS)
+__global__ void __launch_bounds__(ResolveTc::THREADS, 3)
 resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ csplit, long long nframes,
                   int* status) {
   using namespace tc;
@@ -95,17 +103,24 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
     {
       const float* src = stats + (size_t)n * (2 * D * D) + (size_t)row * D;
 #pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        float v[32];
+      for (int hf = 0; hf < 2; ++hf) {
+        float4 raw[16];                                   // half a row in flight before any use
 #pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-          const float4 x = __ldg(reinterpret_cast<const float4*>(src + cc * 32 + e));
-          v[e] = x.x; v[e + 1] = x.y; v[e + 2] = x.z; v[e + 3] = x.w;
+        for (int e = 0; e < 16; ++e) raw[e] = __ldg(reinterpret_cast<const float4*>(src) + hf * 16 + e);
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+          const int cc = hf * 2 + c2;
+          float v[32];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            v[4 * e] = raw[c2 * 8 + e].x; v[4 * e + 1] = raw[c2 * 8 + e].y;
+            v[4 * e + 2] = raw[c2 * 8 + e].z; v[4 * e + 3] = raw[c2 * 8 + e].w;
+          }
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (cc * 32 + e == row) v[e] += 1.0f;
+          tmem_st32(trow + cc * 32, v);
         }
-#pragma unroll
-        for (int e = 0; e < 32; ++e)
-          if (cc * 32 + e == row) v[e] += 1.0f;
-        tmem_st32(trow + cc * 32, v);
       }
       tmem_wait_st();
     }
@@ -130,7 +145,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           float rp[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) rp[j] = __shfl_sync(0xffffffffu, g[j], l0 + p);
-          const float ip = __frcp_rn(rp[p]);
+          const float ip = fast_rcp(rp[p]);
           const bool prow = lane == l0 + p;
           const float f = prow ? -1.0f : g[p];              // coefficient on the scaled pivot row
           const uint32_t keep = prow ? 0u : 0xFFFFFFFFu;    // the pivot row itself restarts from zero

@@ -48,9 +48,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
 
   const uint32_t bar0 = base + S::OFF_BAR;
-  const uint32_t CFULL = bar0, CFREE = bar0 + 8, XREADY = bar0 + 16, ACCFULL = bar0 + 24;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + S::OFF_BAR + 32);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + S::OFF_BAR + 40);
+  auto CFULL = [&](int p) { return bar0 + 8u * p; };          // one per part of C_t
+  auto CFREE = [&](int p) { return bar0 + 8u * (3 + p); };
+  const uint32_t XREADY = bar0 + 48, ACCFULL = bar0 + 56;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + S::OFF_BAR + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + S::OFF_BAR + 72);
   const WaitCtx wc{abort_flag, status};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -58,8 +60,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
   auto frame_of = [&](int s) { return dir == 0 ? s : T - 1 - s; };   // frame folded in at scan step s
 
   if (threadIdx.x == 0) {
-    mbar_init(CFULL, 1);
-    mbar_init(CFREE, 1);
+    for (int p = 0; p < 3; ++p) { mbar_init(CFULL(p), 1); mbar_init(CFREE(p), 1); }
     mbar_init(XREADY, 256);
     mbar_init(ACCFULL, 1);
     *abort_flag = 0;
@@ -77,17 +78,21 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer: C_t parts
+    // Each part has its own pair of barriers and is re-loaded as soon as the MMAs that read it have retired:
+    // the smallest part (C3) is used first and freed first, so every part's copy for the next step has most
+    // of this step's MMA time plus the state warps' turn to arrive.
     if (lane == 0) {
-      for (int s = 0; s + 1 < T; ++s) {     // the last frame of a chain is never folded in: nobody reads it
-        if (!mbar_wait(CFREE, (s & 1) ^ 1, wc)) break;
-        mbar_arrive_expect_tx(CFULL, 3 * S::PART_BYTES);
+      bool ok = true;
+      for (int s = 0; s + 1 < T && ok; ++s) {     // the last frame of a chain is never folded in: nobody reads it
         const long long n = (long long)bh * T + frame_of(s);
 #pragma unroll
-        for (int p = 0; p < 3; ++p) {
+        for (int p = 2; p >= 0; --p) {
+          if (!mbar_wait(CFREE(p), (s & 1) ^ 1, wc)) { ok = false; break; }
+          mbar_arrive_expect_tx(CFULL(p), S::PART_BYTES);
           const uint32_t dst = base + S::OFF_C + p * S::PART_BYTES;
           const int row = (int)((n * 3 + p) * D);
-          tma_load_2d(dst, &tmC, CFULL, 0, row);
-          tma_load_2d(dst + S::BOX_BYTES, &tmC, CFULL, 64, row);
+          tma_load_2d(dst, &tmC, CFULL(p), 0, row);
+          tma_load_2d(dst + S::BOX_BYTES, &tmC, CFULL(p), 64, row);
         }
       }
     }
@@ -95,26 +100,28 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
-      // (C part, X part), smallest contributions first
-      constexpr int PA[6] = {0, 2, 1, 0, 1, 0};
-      constexpr int PX[6] = {2, 0, 1, 1, 0, 0};
-      for (int s = 0; s + 1 < T; ++s) {
-        if (!mbar_wait(CFULL, s & 1, wc)) break;
+      bool ok = true;
+      for (int s = 0; s + 1 < T && ok; ++s) {
         if (!mbar_wait(XREADY, s & 1, wc)) break;
         tc_fence_after_sync();
+        // C3 X1, then C2 (X2, X1), then C1 (X3, X2, X1): smallest contributions first
 #pragma unroll
-        for (int pr = 0; pr < 6; ++pr) {
-          const uint32_t cb = base + S::OFF_C + PA[pr] * S::PART_BYTES;
-          const uint32_t xb = base + S::OFF_X + PX[pr] * S::PART_BYTES;
+        for (int pc = 2; pc >= 0; --pc) {
+          if (!mbar_wait(CFULL(pc), s & 1, wc)) { ok = false; break; }
+          const uint32_t cb = base + S::OFF_C + pc * S::PART_BYTES;
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint64_t adesc = make_smem_desc(cb + (k >> 2) * S::BOX_BYTES + (k & 3) * 32, 16, 1024);
-            const uint64_t bdesc = make_smem_desc(xb + k * 2048, S::BOX_BYTES, 1024);
-            mma_bf16_ss(tmem_base, adesc, bdesc, idesc, (pr | k) != 0 ? 1u : 0u);
+          for (int px = 2 - pc; px >= 0; --px) {
+            const uint32_t xb = base + S::OFF_X + px * S::PART_BYTES;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const uint64_t adesc = make_smem_desc(cb + (k >> 2) * S::BOX_BYTES + (k & 3) * 32, 16, 1024);
+              const uint64_t bdesc = make_smem_desc(xb + k * 2048, S::BOX_BYTES, 1024);
+              mma_bf16_ss(tmem_base, adesc, bdesc, idesc, (pc == 2 && k == 0) ? 0u : 1u);
+            }
           }
+          mma_commit(CFREE(pc));
         }
-        mma_commit(CFREE);
-        mma_commit(ACCFULL);
+        if (ok) mma_commit(ACCFULL);
       }
     }
   } else {

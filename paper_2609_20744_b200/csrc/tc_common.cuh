@@ -215,18 +215,21 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// x -> three bf16 parts for two neighbouring elements at once (packed as bf16x2 words).
+// x -> three bf16 parts with x = x1 + x2 + x3 exactly, for two neighbouring elements at once (packed as
+// bf16x2 words, element 0 in the low half).  Each part is the remainder truncated to its top 8 mantissa bits
+// (a mask on the fp32 bit pattern), so three parts hold all 24 bits and the remainders are formed without
+// rounding error.  Only integer/FMA-pipe instructions: the float->bf16 conversion instruction is an order of
+// magnitude slower per warp on this GPU and sat on the critical path of the scan and the resolve.
 __device__ __forceinline__ void split3_pair(float x0, float x1, uint32_t& p1, uint32_t& p2, uint32_t& p3) {
-  __nv_bfloat162 a = __floats2bfloat162_rn(x0, x1);
-  p1 = *reinterpret_cast<uint32_t*>(&a);
-  x0 -= __uint_as_float(p1 << 16);
-  x1 -= __uint_as_float(p1 & 0xFFFF0000u);
-  __nv_bfloat162 b = __floats2bfloat162_rn(x0, x1);
-  p2 = *reinterpret_cast<uint32_t*>(&b);
-  x0 -= __uint_as_float(p2 << 16);
-  x1 -= __uint_as_float(p2 & 0xFFFF0000u);
-  __nv_bfloat162 c = __floats2bfloat162_rn(x0, x1);
-  p3 = *reinterpret_cast<uint32_t*>(&c);
+  uint32_t u0 = __float_as_uint(x0), u1 = __float_as_uint(x1);
+  p1 = __byte_perm(u0, u1, 0x7632);                       // {hi16(x1), hi16(x0)}
+  x0 -= __uint_as_float(u0 & 0xFFFF0000u);
+  x1 -= __uint_as_float(u1 & 0xFFFF0000u);
+  u0 = __float_as_uint(x0); u1 = __float_as_uint(x1);
+  p2 = __byte_perm(u0, u1, 0x7632);
+  x0 -= __uint_as_float(u0 & 0xFFFF0000u);
+  x1 -= __uint_as_float(u1 & 0xFFFF0000u);
+  p3 = __byte_perm(__float_as_uint(x0), __float_as_uint(x1), 0x7632);
 }
 
 __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {

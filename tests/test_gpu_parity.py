@@ -138,7 +138,7 @@ def test_stagewise_intermediates_tensor_core_kernels():
             # that rounding only; the resolve inverts I + the stored block as it stands)
             inv_g = np.linalg.inv(np.eye(d) + stats[0, h, t, :d, :])
             assert rel(split[0, h, t].sum(axis=0), inv_g) < 1e-5            # three parts carry fp32 accuracy
-            assert rel(split[0, h, t, 0], inv_g) < 5e-3                     # the leading part alone is bf16
+            assert rel(split[0, h, t, 0], inv_g) < 8e-3                     # the leading part alone: bf16, truncated (2^-7)
             want_f = ref["P"][t - 1].T if t > 0 else np.zeros((d, d))
             want_b = ref["R"][t + 1].T if t + 1 < T else np.zeros((d, d))
             assert rel(pf[0, h, t], want_f) < 1e-2 or not want_f.any()
