@@ -92,8 +92,8 @@ typedef enum {
   VDN_VIEW_READ = 3,      /* float [B,H,T,d_k,d_v]: transpose of P_{t-1} + R_{t+1}, what frame t reads (A.4) */
   /* tensor-core kernels (bf16 I/O, d = 128) */
   VDN_VIEW_INV_SPLIT = 4, /* bf16 [B,H,T,3,d,d]: C_t as C1 + C2 + C3 (bf16 parts of the fp32 inverse)         */
-  VDN_VIEW_READ_FWD = 5,  /* bf16 [B,H,T,d_k,d_v]: slot t = transpose of P_{t-1} (zero for t = 0)     (A.4)  */
-  VDN_VIEW_READ_BWD = 6   /* bf16 [B,H,T,d_k,d_v]: slot t = transpose of R_{t+1} (zero for t = T-1)   (A.4)  */
+  VDN_VIEW_READ_FWD = 5,  /* bf16 [B,H,T,d_v,d_k]: slot t = P_{t-1} (zero for t = 0)                  (A.4)  */
+  VDN_VIEW_READ_BWD = 6   /* bf16 [B,H,T,d_v,d_k]: slot t = R_{t+1} (zero for t = T-1)                (A.4)  */
 } vdn_view;
 
 /* Sec. 3 (the layer as a whole).  Creates a handle bound to cfg->device.  Allocates host memory only

@@ -4,7 +4,7 @@
 //   out = gate_h * O / sqrt(mean_c O^2 + eps)   -> bf16
 //
 // The two states a frame reads (forward state of the frames before it, reverse state of the frames after
-// it) arrive as bf16 [d_k][d_v], i.e. MN-major B operands; both products go into the same accumulator,
+// it) arrive as bf16 [d_v][d_k], i.e. K-major B operands; both products go into the same accumulator,
 // which is the sum of Eq. 1a.  Q tiles are K-major as they sit in memory.  Persistent CTAs loop over
 // frames (b,h,t).  Warp roles:
 //   warp 0      TMA producer: the frame's two states (4 boxes of 16 KB) and Q tiles (2 boxes, 3-stage ring)
@@ -112,7 +112,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
+      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
       uint32_t qi = 0, si = 0;
       bool ok = true;
       for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
@@ -129,9 +129,10 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           for (int dirn = 0; dirn < 2; ++dirn) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              // A: 16 key channels = 32 B inside the swizzled Q row; B: 16 key rows of the state = 2 KB
-              const uint64_t adesc = make_smem_desc(qbase + (j >> 2) * R::BOX_BYTES + (j & 3) * 32, 16, 1024);
-              const uint64_t bdesc = make_smem_desc(sbase + dirn * R::TILE_BYTES + j * 2048, R::BOX_BYTES, 1024);
+              // both operands K-major: 16 key channels = 32 B inside a swizzled row of Q / of the state
+              const uint32_t off = (j >> 2) * R::BOX_BYTES + (j & 3) * 32;
+              const uint64_t adesc = make_smem_desc(qbase + off, 16, 1024);
+              const uint64_t bdesc = make_smem_desc(sbase + dirn * R::TILE_BYTES + off, 16, 1024);
               mma_bf16_ss(tmem_base + a * 128, adesc, bdesc, idesc, (dirn | j) != 0 ? 1u : 0u);
             }
           }

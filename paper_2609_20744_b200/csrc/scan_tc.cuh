@@ -11,7 +11,7 @@
 //
 // C_t arrives already split (the resolve kernel writes the three parts), by TMA, K-major.  The state
 // parts are produced on chip: after each step the 8 epilogue warps read Z_t from TMEM (a thread owns one
-// key row and 64 value columns), store it as bf16 for the read-out of the next frame in scan order, add
+// key row and 64 value columns), add
 // the next frame's B^T, split the sum and write the three parts to shared memory as the next MN-major B
 // operand.  The next frame's B^T row is fetched into registers while the MMAs run.
 //
@@ -134,7 +134,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     const int sw = row & 7;
 
     auto load_bt = [&](int frame, float (&bt)[64]) {
-      // B_t is stored [d_v][d_k]; lanes read consecutive key channels
+      // B_t is stored [d_v][d_k]; lanes read consecutive key channels (scalar but coalesced: measured
+      // faster than 16-byte loads of a thread-contiguous layout, whose lanes sit 512 bytes apart)
       const float* src = stats + ((size_t)bh * T + frame) * (2 * D * D) + (size_t)(D + half * 64) * D + row;
 #pragma unroll
       for (int e = 0; e < 64; ++e) bt[e] = __ldg(src + (size_t)e * D);
@@ -163,36 +164,36 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     publish_x(bt);                           // Z_{-1} = 0
     {
       // the chain's first read slot holds the zero state
-      __nv_bfloat16* z0 = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(0)) * (D * D) + (size_t)row * D + half * 64;
+      __nv_bfloat16* z0 = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(0)) * (D * D) + (size_t)(half * 64) * D + row;
 #pragma unroll
-      for (int e = 0; e < 64; e += 8) *reinterpret_cast<uint4*>(z0 + e) = make_uint4(0u, 0u, 0u, 0u);
+      for (int e = 0; e < 64; ++e) z0[(size_t)e * D] = __float2bfloat16_rn(0.f);
     }
+    if (T > 1) load_bt(frame_of(1), bt);
     for (int s = 0; s + 1 < T; ++s) {
-      load_bt(frame_of(s + 1), bt);          // lands while the MMAs of step s run
       if (!mbar_wait(ACCFULL, s & 1, wc)) break;
       tc_fence_after_sync();
       float z[64];
       tmem_ld32(taddr, *reinterpret_cast<float(*)[32]>(&z[0]));
       tmem_ld32(taddr + 32, *reinterpret_cast<float(*)[32]>(&z[32]));
       tmem_wait_ld();
-      // the state after step s is what the next frame in scan order reads
-      __nv_bfloat16* dst = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(s + 1)) * (D * D) + (size_t)row * D + half * 64;
+      // first what the next MMAs are waiting for: X = Z + B^T of the next frame, split, into shared memory
+      if (s + 2 < T) {
+        float x[64];
 #pragma unroll
-      for (int e = 0; e < 64; e += 8) {
-        uint4 w;
-        uint32_t* a = reinterpret_cast<uint32_t*>(&w);
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-          __nv_bfloat162 v2 = __floats2bfloat162_rn(z[e + 2 * p], z[e + 2 * p + 1]);
-          a[p] = *reinterpret_cast<uint32_t*>(&v2);
-        }
-        *reinterpret_cast<uint4*>(dst + e) = w;
+        for (int e = 0; e < 64; ++e) x[e] = z[e] + bt[e];
+        publish_x(x);
       }
-      if (s + 2 < T) {                       // another step follows: build its B operand
+      // then, under the next step's MMAs: the state after step s is what the next frame in scan order reads.
+      // Stored as bf16 [d_v][d_k] (the paper's orientation), so the 32 lanes of a warp (consecutive key
+      // channels) write 64 contiguous bytes per value column.
+      __nv_bfloat16* dst = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(s + 1)) * (D * D) + (size_t)(half * 64) * D + row;
 #pragma unroll
-        for (int e = 0; e < 64; ++e) z[e] += bt[e];
-        publish_x(z);
+      for (int e = 0; e < 64; e += 2) {
+        const __nv_bfloat162 v2 = __floats2bfloat162_rn(z[e], z[e + 1]);
+        dst[(size_t)e * D] = v2.x;
+        dst[(size_t)(e + 1) * D] = v2.y;
       }
+      if (s + 2 < T) load_bt(frame_of(s + 2), bt);   // B^T of the frame after next, also under the MMAs
     }
   }
 

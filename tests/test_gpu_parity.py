@@ -139,8 +139,8 @@ def test_stagewise_intermediates_tensor_core_kernels():
             inv_g = np.linalg.inv(np.eye(d) + stats[0, h, t, :d, :])
             assert rel(split[0, h, t].sum(axis=0), inv_g) < 1e-5            # three parts carry fp32 accuracy
             assert rel(split[0, h, t, 0], inv_g) < 8e-3                     # the leading part alone: bf16, truncated (2^-7)
-            want_f = ref["P"][t - 1].T if t > 0 else np.zeros((d, d))
-            want_b = ref["R"][t + 1].T if t + 1 < T else np.zeros((d, d))
+            want_f = ref["P"][t - 1] if t > 0 else np.zeros((d, d))
+            want_b = ref["R"][t + 1] if t + 1 < T else np.zeros((d, d))
             assert rel(pf[0, h, t], want_f) < 1e-2 or not want_f.any()
             assert rel(pb[0, h, t], want_b) < 1e-2 or not want_b.any()
             if t == 0:
@@ -150,9 +150,9 @@ def test_stagewise_intermediates_tensor_core_kernels():
             # against the checker fed with the GPU's statistics the stored states differ by their own bf16
             # rounding only (2^-9 relative per element): the scan itself runs at fp32 accuracy
             if t > 0:
-                assert np.max(np.abs(pf[0, h, t] - Pg[t - 1].T) / (np.abs(Pg[t - 1].T) + 1e-3 * np.abs(Pg[t - 1]).max())) < 2.0 ** -8
+                assert np.max(np.abs(pf[0, h, t] - Pg[t - 1]) / (np.abs(Pg[t - 1]) + 1e-3 * np.abs(Pg[t - 1]).max())) < 2.0 ** -8
             if t + 1 < T:
-                assert np.max(np.abs(pb[0, h, t] - Rg[t + 1].T) / (np.abs(Rg[t + 1].T) + 1e-3 * np.abs(Rg[t + 1]).max())) < 2.0 ** -8
+                assert np.max(np.abs(pb[0, h, t] - Rg[t + 1]) / (np.abs(Rg[t + 1]) + 1e-3 * np.abs(Rg[t + 1]).max())) < 2.0 ** -8
 
 
 # ------------------------------------------------------------------------------ properties
