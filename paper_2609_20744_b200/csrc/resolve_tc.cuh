@@ -99,28 +99,20 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
     // ------------------------------------------------------------------ row threads
     const int row = warp * 32 + lane;
     const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
-    // M = I + A_t into TMEM, 32 columns at a time
+    // M = (I + A_t)^T into TMEM: thread `row` reads column `row` of the stored block, so that the 32 lanes of
+    // a warp read 32 consecutive floats.  Inverting the transpose gives the transpose of the inverse; the final
+    // store transposes back (again with consecutive lanes on consecutive addresses).
     {
-      const float* src = stats + (size_t)n * (2 * D * D) + (size_t)row * D;
+      const float* src = stats + (size_t)n * (2 * D * D) + row;
 #pragma unroll 1
-      for (int hf = 0; hf < 2; ++hf) {
-        float4 raw[16];                                   // half a row in flight before any use
+      for (int cc = 0; cc < 4; ++cc) {
+        float v[32];
 #pragma unroll
-        for (int e = 0; e < 16; ++e) raw[e] = __ldg(reinterpret_cast<const float4*>(src) + hf * 16 + e);
+        for (int e = 0; e < 32; ++e) v[e] = __ldg(src + (size_t)(cc * 32 + e) * D);
 #pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) {
-          const int cc = hf * 2 + c2;
-          float v[32];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            v[4 * e] = raw[c2 * 8 + e].x; v[4 * e + 1] = raw[c2 * 8 + e].y;
-            v[4 * e + 2] = raw[c2 * 8 + e].z; v[4 * e + 3] = raw[c2 * 8 + e].w;
-          }
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (cc * 32 + e == row) v[e] += 1.0f;
-          tmem_st32(trow + cc * 32, v);
-        }
+        for (int e = 0; e < 32; ++e)
+          if (cc * 32 + e == row) v[e] += 1.0f;
+        tmem_st32(trow + cc * 32, v);
       }
       tmem_wait_st();
     }
@@ -235,24 +227,24 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
     }
 
     if (ok) {
-      // ---- the inverse, row by row, as three bf16 parts
-      __nv_bfloat16* c1 = csplit + (size_t)n * (3 * D * D) + (size_t)row * D;
+      // ---- the inverse as three bf16 parts; this thread holds column `row` of it
+      __nv_bfloat16* c1 = csplit + (size_t)n * (3 * D * D) + row;
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
         float v[32];
         tmem_ld32(trow + cc * 32, v);
         tmem_wait_ld();
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint4 w1, w2, w3;
-#pragma unroll
-          for (int q = 0; q < 4; ++q)
-            split3_pair(v[ch * 8 + 2 * q], v[ch * 8 + 2 * q + 1], reinterpret_cast<uint32_t*>(&w1)[q],
-                        reinterpret_cast<uint32_t*>(&w2)[q], reinterpret_cast<uint32_t*>(&w3)[q]);
-          const int e = cc * 32 + ch * 8;
-          *reinterpret_cast<uint4*>(c1 + e) = w1;
-          *reinterpret_cast<uint4*>(c1 + D * D + e) = w2;
-          *reinterpret_cast<uint4*>(c1 + 2 * D * D + e) = w3;
+        for (int e = 0; e < 32; e += 2) {
+          uint32_t w1, w2, w3;
+          split3_pair(v[e], v[e + 1], w1, w2, w3);
+          unsigned short* o = reinterpret_cast<unsigned short*>(c1 + (size_t)(cc * 32 + e) * D);
+          o[0] = (unsigned short)(w1 & 0xFFFFu);
+          o[D] = (unsigned short)(w1 >> 16);
+          o[(size_t)D * D] = (unsigned short)(w2 & 0xFFFFu);
+          o[(size_t)D * D + D] = (unsigned short)(w2 >> 16);
+          o[(size_t)2 * D * D] = (unsigned short)(w3 & 0xFFFFu);
+          o[(size_t)2 * D * D + D] = (unsigned short)(w3 >> 16);
         }
       }
     }
