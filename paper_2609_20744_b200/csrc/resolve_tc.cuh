@@ -11,7 +11,11 @@
 // accumulated in fp32, so the update carries fp32 accuracy.  Everything else is plain fp32:
 //   * the 16 x 16 pivot block is inverted inside the warp that owns those rows, one row per lane, the pivot
 //     rows travelling by shuffle;
-//   * every thread owns one matrix row (its TMEM lane) and forms its 16 coefficients from Gi.
+//   * every thread owns one matrix row (its TMEM lane), forms its 16 coefficients from Gi, and -- the matrix
+//     being symmetric up to the sign pattern of in-place elimination -- also supplies its column of the 16
+//     pivot rows, so nobody has to read whole rows back.
+// The matrix that is inverted is I + (A_t + A_t^T)/2: the stored statistics are symmetric only up to the bf16
+// rounding of one factor, and the symmetric part is the natural reading of Eq. 3b (and keeps Proposition 1).
 // The inverse is written as three bf16 parts C1 + C2 + C3 for the tensor-core scan.
 #pragma once
 #include <cuda_bf16.h>
@@ -83,8 +87,8 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
       constexpr int PA[6] = {0, 2, 1, 0, 1, 0};   // (coefficient part, pivot-row part), smallest first
       constexpr int PB[6] = {2, 0, 1, 1, 0, 0};
-      for (int blk = 0; blk < D / R::NB; ++blk) {
-        if (!mbar_wait(OPREADY, blk & 1, wc)) break;
+      for (int step = 0; step < D / R::NB; ++step) {
+        if (!mbar_wait(OPREADY, step & 1, wc)) break;
         tc_fence_after_sync();
 #pragma unroll
         for (int pr = 0; pr < 6; ++pr) {
@@ -99,16 +103,26 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
     // ------------------------------------------------------------------ row threads
     const int row = warp * 32 + lane;
     const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
-    // M = (I + A_t)^T into TMEM: thread `row` reads column `row` of the stored block, so that the 32 lanes of
-    // a warp read 32 consecutive floats.  Inverting the transpose gives the transpose of the inverse; the final
-    // store transposes back (again with consecutive lanes on consecutive addresses).
+    // M = I + (A_t + A_t^T)/2 into TMEM.  The stored block is K^T (beta K) with one factor rounded to bf16,
+    // symmetric only up to that rounding; its symmetric part is what gets inverted, and exact symmetry is
+    // what lets every thread supply its share of the pivot rows below.  Column `row` is read with
+    // consecutive lanes on consecutive addresses, row `row` as 16-byte pieces (mostly L1/L2 hits).
     {
-      const float* src = stats + (size_t)n * (2 * D * D) + row;
+      const float* col = stats + (size_t)n * (2 * D * D) + row;
+      const float4* rw = reinterpret_cast<const float4*>(stats + (size_t)n * (2 * D * D) + (size_t)row * D);
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
         float v[32];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = __ldg(src + (size_t)(cc * 32 + e) * D);
+        for (int e = 0; e < 32; ++e) v[e] = __ldg(col + (size_t)(cc * 32 + e) * D);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float4 x = __ldg(rw + cc * 8 + e);
+          v[4 * e] = 0.5f * (v[4 * e] + x.x);
+          v[4 * e + 1] = 0.5f * (v[4 * e + 1] + x.y);
+          v[4 * e + 2] = 0.5f * (v[4 * e + 2] + x.z);
+          v[4 * e + 3] = 0.5f * (v[4 * e + 3] + x.w);
+        }
 #pragma unroll
         for (int e = 0; e < 32; ++e)
           if (cc * 32 + e == row) v[e] += 1.0f;
@@ -117,9 +131,15 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       tmem_wait_st();
     }
 
+    // Pivot blocks may be taken in any order (symmetric pivoting of an SPD matrix).  CTAs that share an SM start
+    // at different blocks, so that their serial sections (the 16 x 16 inverse, done by the warp that owns the
+    // pivot rows) fall on different warp schedulers instead of queueing on one.
+    const int blk0 = (int)((blockIdx.x & 3) * 2);
+    uint32_t done = 0;                                    // bit b set: pivot block b has been eliminated
     bool ok = true;
 #pragma unroll 1
-    for (int blk = 0; blk < D / R::NB && ok; ++blk) {
+    for (int step = 0; step < D / R::NB && ok; ++step) {
+      const int blk = (blk0 + step) & 7;
       const int p0 = blk * R::NB;
       const bool owner = (row >> 4) == blk;               // rows p0 .. p0+15: 16 lanes of warp blk/2
       float x[16];
@@ -191,39 +211,37 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           *reinterpret_cast<uint4*>(crow + part * R::CM_PART + ((1 ^ (row & 7)) * 16)) = w[part][1];
         }
       }
-      // ---- B operand: the 16 pivot rows as they stand, three bf16 parts, MN-major
-      if (warp == (blk >> 1)) {
-        const int kr = row & 15;
-#pragma unroll 1
-        for (int cc = 0; cc < 4; ++cc) {
-          float v[32];
-          tmem_ld32(trow + cc * 32, v);
-          tmem_wait_ld();
-          if (owner) {
-            unsigned char* prow = base_ptr + R::OFF_PR + (cc >> 1) * (R::NB * 128) + kr * 128;
+      // ---- B operand: the 16 pivot rows, three bf16 parts, MN-major.  M is symmetric up to the sign pattern
+      // of in-place elimination: M[P_k][j] = M[j][P_k] for rows j not yet eliminated and -M[j][P_k] for rows
+      // already eliminated (`done`).  So thread j owns column j of the pivot rows: its own x, signed.
+      {
+        const float sgn = ((done >> (row >> 4)) & 1u) ? -1.0f : 1.0f;
+        const int jj = row & 63;
+        unsigned char* pcol = base_ptr + R::OFF_PR + (row >> 6) * (R::NB * 128) + (jj & 7) * 2;
+        const int ch = jj >> 3;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              uint4 w1, w2, w3;
-#pragma unroll
-              for (int q = 0; q < 4; ++q)
-                split3_pair(v[ch * 8 + 2 * q], v[ch * 8 + 2 * q + 1], reinterpret_cast<uint32_t*>(&w1)[q],
-                            reinterpret_cast<uint32_t*>(&w2)[q], reinterpret_cast<uint32_t*>(&w3)[q]);
-              const int off = ((((cc & 1) * 4 + ch) ^ (kr & 7)) * 16);
-              *reinterpret_cast<uint4*>(prow + off) = w1;
-              *reinterpret_cast<uint4*>(prow + R::PR_PART + off) = w2;
-              *reinterpret_cast<uint4*>(prow + 2 * R::PR_PART + off) = w3;
-            }
-          }
+        for (int k = 0; k < 16; k += 2) {
+          uint32_t w1, w2, w3;
+          split3_pair(sgn * x[k], sgn * x[k + 1], w1, w2, w3);
+          unsigned char* r0 = pcol + k * 128 + ((ch ^ (k & 7)) * 16);
+          unsigned char* r1 = pcol + (k + 1) * 128 + ((ch ^ ((k + 1) & 7)) * 16);
+          *reinterpret_cast<unsigned short*>(r0) = (unsigned short)(w1 & 0xFFFFu);
+          *reinterpret_cast<unsigned short*>(r1) = (unsigned short)(w1 >> 16);
+          *reinterpret_cast<unsigned short*>(r0 + R::PR_PART) = (unsigned short)(w2 & 0xFFFFu);
+          *reinterpret_cast<unsigned short*>(r1 + R::PR_PART) = (unsigned short)(w2 >> 16);
+          *reinterpret_cast<unsigned short*>(r0 + 2 * R::PR_PART) = (unsigned short)(w3 & 0xFFFFu);
+          *reinterpret_cast<unsigned short*>(r1 + 2 * R::PR_PART) = (unsigned short)(w3 >> 16);
         }
       }
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(OPREADY);
-      if (!mbar_wait(MMADONE, blk & 1, wc)) { ok = false; break; }
+      if (!mbar_wait(MMADONE, step & 1, wc)) { ok = false; break; }
       tc_fence_after_sync();
       // ---- column fix: M[i][P] = c (for a pivot row: Gi[a])
       tmem_st16(trow + p0, c);
       tmem_wait_st();
+      done |= 1u << blk;
     }
 
     if (ok) {

@@ -128,15 +128,16 @@ def test_stagewise_intermediates_tensor_core_kernels():
         ref = orc.vda_slice(q, k, v, beta, gate, 1e-6, want=("A", "B", "C", "P", "R"))
         # the checker's states from the GPU's own statistics isolate the scan's arithmetic from the
         # bf16 rounding of the weighted keys in the Gram stage
-        Pg, Rg = orc.scan_states([stats[0, h, t, :d, :] for t in range(T)], [stats[0, h, t, d:, :] for t in range(T)],
+        Pg, Rg = orc.scan_states([0.5 * (stats[0, h, t, :d, :] + stats[0, h, t, :d, :].T) for t in range(T)], [stats[0, h, t, d:, :] for t in range(T)],
                                  np.ones((T, d)), np.zeros((d, d)))
         for t in range(T):
             # bf16 products are exact in fp32; only the beta-weighted key operand is rounded (2^-9 relative)
             assert rel(stats[0, h, t, :d, :], ref["A"][t]) < 4e-3
             assert rel(stats[0, h, t, d:, :], ref["B"][t]) < 4e-3
             # (the stored A block is K^T (beta K) with only one factor rounded to bf16, hence symmetric up to
-            # that rounding only; the resolve inverts I + the stored block as it stands)
-            inv_g = np.linalg.inv(np.eye(d) + stats[0, h, t, :d, :])
+            # that rounding only; the resolve inverts I + its symmetric part)
+            a_sym = 0.5 * (stats[0, h, t, :d, :] + stats[0, h, t, :d, :].T)
+            inv_g = np.linalg.inv(np.eye(d) + a_sym)
             assert rel(split[0, h, t].sum(axis=0), inv_g) < 1e-5            # three parts carry fp32 accuracy
             assert rel(split[0, h, t, 0], inv_g) < 8e-3                     # the leading part alone: bf16, truncated (2^-7)
             want_f = ref["P"][t - 1] if t > 0 else np.zeros((d, d))
