@@ -199,19 +199,30 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       return true;
     };
 
-    long long prev_item = -1;
-    for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
+    // beta of (frame, tile), one value per half for this thread's row; zero past the end of the frame.
+    // Fetched one tile ahead: the loads are scattered 4-byte reads (one head out of H) whose L2 latency would
+    // otherwise sit between a tile's arrival and its weighting.
+    auto load_beta = [&](long long witem, int tile, float (&bw)[2]) {
+      if (witem >= nitems) { bw[0] = bw[1] = 0.f; return; }
       int b, h, t;
-      split_work(s, item, b, h, t);
+      split_work(s, witem, b, h, t);
       const float* brow = beta + ((size_t)b * s.T + t) * s.F * s.H + h;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const int u = tile * G::TILE + half * 64 + r;
+        bw[half] = (u < s.F) ? __ldg(brow + (size_t)u * s.H) : 0.f;
+      }
+    };
+
+    long long prev_item = -1;
+    float bnext[2];
+    load_beta(blockIdx.x, 0, bnext);
+    for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
       for (int tile = 0; tile < ntiles && ok; ++tile, ++it) {
         const int st = it % G::STAGES;
-        float bu[2];
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const int u = tile * G::TILE + half * 64 + r;
-          bu[half] = (u < s.F) ? __ldg(brow + (size_t)u * s.H) : 0.f;
-        }
+        const float bu[2] = {bnext[0], bnext[1]};
+        if (tile + 1 < ntiles) load_beta(item, tile + 1, bnext);
+        else load_beta(item + gridDim.x, 0, bnext);
         if (!mbar_wait(FULL(st), (it / G::STAGES) & 1, wc)) { ok = false; break; }
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
