@@ -10,7 +10,7 @@
 // Persistent CTAs, one per SM, loop over frames (b,h,t).  Warp roles:
 //   warp 0      TMA producer: K and V tiles (4 boxes of 16 KB) into a 3-stage ring
 //   warp 1      MMA issuer (one thread) and TMEM owner
-//   warps 2-5   weighting: K' = beta * K, rounded once to bf16, written to a second buffer in two halves of
+//   warps 2-5   weighting: K' = bf16(beta) * K in packed bf16 arithmetic, written to a second buffer in two halves of
 //               64 tokens so the MMA of one half overlaps the weighting of the other.  Once per frame (after the
 //               first tile of the next frame is with the MMA) the same warps drain the finished accumulator:
 //               TMEM -> registers -> global fp32 [2d][d] (A_t, then B_t); there are two accumulators
@@ -229,19 +229,16 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           if (!mbar_wait(KPFREE(half), (it & 1) ^ 1, wc)) { ok = false; break; }
           const unsigned char* src = base_ptr + st * G::STAGE_BYTES + c * G::BOX_BYTES + (half * 64 + r) * 128;
           unsigned char* dst = base_ptr + G::OFF_KP + half * G::KP_HALF_BYTES + c * (64 * 128) + r * 128;
-          const float w = bu[half];
+          // beta rounded to bf16, then one packed bf16 multiply per channel pair (round to nearest): the
+          // float->bf16 conversion instruction is slow on this GPU and kept this loop from hiding under HBM
+          const __nv_bfloat162 w2 = __float2bfloat162_rn(bu[half]);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const int pj = (j ^ (r & 7)) * 16;   // stagger the 16-byte chunks across rows: conflict-free
             uint4 raw = *reinterpret_cast<const uint4*>(src + pj);
-            uint32_t* x = reinterpret_cast<uint32_t*>(&raw);
+            __nv_bfloat162* x = reinterpret_cast<__nv_bfloat162*>(&raw);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float lo = __uint_as_float(x[e] << 16) * w;
-              const float hi = __uint_as_float(x[e] & 0xFFFF0000u) * w;
-              __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
-              x[e] = *reinterpret_cast<uint32_t*>(&p);
-            }
+            for (int e = 0; e < 4; ++e) x[e] = __hmul2(x[e], w2);
             *reinterpret_cast<uint4*>(dst + pj) = raw;
           }
           fence_proxy_async_smem();
