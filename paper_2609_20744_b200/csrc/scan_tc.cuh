@@ -10,8 +10,8 @@
 // state is carried at fp32 accuracy while the 2 d^3 flops per step run on the tensor pipe.
 //
 // C_t arrives already split (the resolve kernel writes the three parts), by TMA, K-major.  The state
-// parts are produced on chip: after each step the 8 epilogue warps read Z_t from TMEM (a thread owns one
-// key row and 64 value columns), add
+// parts are produced on chip: after each step the 16 state warps read Z_t from TMEM (a thread owns one
+// key row and 32 value columns), add
 // the next frame's B^T, split the sum and write the three parts to shared memory as the next MN-major B
 // operand.  The next frame's B^T row is fetched into registers while the MMAs run.
 //
@@ -34,7 +34,8 @@ struct ScanTc {
   static constexpr int OFF_X = 3 * PART_BYTES;       // X1, X2, X3
   static constexpr int OFF_BAR = 6 * PART_BYTES;
   static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
-  static constexpr int THREADS = 320;
+  static constexpr int CW = 32;                      // value columns per state thread
+  static constexpr int THREADS = 64 + 4 * 32 * (D / CW);  // producer + MMA + state warps
 };
 
 __global__ void __launch_bounds__(ScanTc::THREADS, 1)
@@ -61,7 +62,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
 
   if (threadIdx.x == 0) {
     for (int p = 0; p < 3; ++p) { mbar_init(CFULL(p), 1); mbar_init(CFREE(p), 1); }
-    mbar_init(XREADY, 256);
+    mbar_init(XREADY, S::THREADS - 64);
     mbar_init(ACCFULL, 1);
     *abort_flag = 0;
     mbar_fence_init();
@@ -126,30 +127,34 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     }
   } else {
     // ------------------------------------------------------------------ state warps
+    // 16 warps: 4 per TMEM lane quarter, each thread owns one key row and CW = 32 value columns.
+    constexpr int CW = S::CW;
     const int qd = warp & 3;                 // TMEM lane quarter
     const int row = qd * 32 + lane;          // key channel (row of Z, row of X)
-    const int half = (warp - 2) >> 2;        // value columns [64*half, 64*half + 64)
-    const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + half * 64;
-    unsigned char* xrow = base_ptr + S::OFF_X + half * S::BOX_BYTES + row * 128;
+    const int slice = (warp - 2) >> 2;       // value columns [CW*slice, CW*slice + CW)
+    const int col0 = slice * CW;
+    const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + col0;
+    unsigned char* xrow = base_ptr + S::OFF_X + (col0 >> 6) * S::BOX_BYTES + row * 128;
+    const int ch0 = (col0 & 63) >> 3;        // first 16-byte chunk of this thread inside the 64-column box
     const int sw = row & 7;
 
-    auto load_bt = [&](int frame, float (&bt)[64]) {
+    auto load_bt = [&](int frame, float (&bt)[CW]) {
       // B_t is stored [d_v][d_k]; lanes read consecutive key channels (scalar but coalesced: measured
       // faster than 16-byte loads of a thread-contiguous layout, whose lanes sit 512 bytes apart)
-      const float* src = stats + ((size_t)bh * T + frame) * (2 * D * D) + (size_t)(D + half * 64) * D + row;
+      const float* src = stats + ((size_t)bh * T + frame) * (2 * D * D) + (size_t)(D + col0) * D + row;
 #pragma unroll
-      for (int e = 0; e < 64; ++e) bt[e] = __ldg(src + (size_t)e * D);
+      for (int e = 0; e < CW; ++e) bt[e] = __ldg(src + (size_t)e * D);
     };
-    auto publish_x = [&](const float (&x)[64]) {
+    auto publish_x = [&](const float (&x)[CW]) {
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
+      for (int ch = 0; ch < CW / 8; ++ch) {
         uint4 w1, w2, w3;
         uint32_t* a1 = reinterpret_cast<uint32_t*>(&w1);
         uint32_t* a2 = reinterpret_cast<uint32_t*>(&w2);
         uint32_t* a3 = reinterpret_cast<uint32_t*>(&w3);
 #pragma unroll
         for (int e = 0; e < 4; ++e) split3_pair(x[ch * 8 + 2 * e], x[ch * 8 + 2 * e + 1], a1[e], a2[e], a3[e]);
-        const int off = (ch ^ sw) * 16;
+        const int off = ((ch0 + ch) ^ sw) * 16;
         *reinterpret_cast<uint4*>(xrow + off) = w1;
         *reinterpret_cast<uint4*>(xrow + S::PART_BYTES + off) = w2;
         *reinterpret_cast<uint4*>(xrow + 2 * S::PART_BYTES + off) = w3;
@@ -159,36 +164,34 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
       mbar_arrive(XREADY);
     };
 
-    float bt[64];
+    float bt[CW];
     load_bt(frame_of(0), bt);
     publish_x(bt);                           // Z_{-1} = 0
     {
       // the chain's first read slot holds the zero state
-      __nv_bfloat16* z0 = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(0)) * (D * D) + (size_t)(half * 64) * D + row;
+      __nv_bfloat16* z0 = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(0)) * (D * D) + (size_t)col0 * D + row;
 #pragma unroll
-      for (int e = 0; e < 64; ++e) z0[(size_t)e * D] = __float2bfloat16_rn(0.f);
+      for (int e = 0; e < CW; ++e) z0[(size_t)e * D] = __float2bfloat16_rn(0.f);
     }
     if (T > 1) load_bt(frame_of(1), bt);
     for (int s = 0; s + 1 < T; ++s) {
       if (!mbar_wait(ACCFULL, s & 1, wc)) break;
       tc_fence_after_sync();
-      float z[64];
-      tmem_ld32(taddr, *reinterpret_cast<float(*)[32]>(&z[0]));
-      tmem_ld32(taddr + 32, *reinterpret_cast<float(*)[32]>(&z[32]));
+      float z[CW];
+      tmem_ld32(taddr, z);
       tmem_wait_ld();
       // first what the next MMAs are waiting for: X = Z + B^T of the next frame, split, into shared memory
       if (s + 2 < T) {
-        float x[64];
 #pragma unroll
-        for (int e = 0; e < 64; ++e) x[e] = z[e] + bt[e];
-        publish_x(x);
+        for (int e = 0; e < CW; ++e) bt[e] += z[e];
+        publish_x(bt);
       }
       // then, under the next step's MMAs: the state after step s is what the next frame in scan order reads.
       // Stored as bf16 [d_v][d_k] (the paper's orientation), so the 32 lanes of a warp (consecutive key
       // channels) write 64 contiguous bytes per value column.
-      __nv_bfloat16* dst = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(s + 1)) * (D * D) + (size_t)(half * 64) * D + row;
+      __nv_bfloat16* dst = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(s + 1)) * (D * D) + (size_t)col0 * D + row;
 #pragma unroll
-      for (int e = 0; e < 64; e += 2) {
+      for (int e = 0; e < CW; e += 2) {
         const __nv_bfloat162 v2 = __floats2bfloat162_rn(z[e], z[e + 1]);
         dst[(size_t)e * D] = v2.x;
         dst[(size_t)(e + 1) * D] = v2.y;
