@@ -69,9 +69,7 @@ typedef enum {
 typedef enum { VDN_F32 = 0, VDN_BF16 = 1 } vdn_dtype;
 
 /* cfg.flags */
-#define VDN_FLAG_FORCE_SIMT 1u      /* bf16 I/O through the plain-fp32 kernels (a second opinion for tests) */
-#define VDN_FLAG_RESOLVE_IN_GRAM 2u /* tensor-core path: invert I + A_t with plain fp32 FMA inside the         */
-                                    /* statistics kernel instead of the tensor-core resolve kernel            */
+#define VDN_FLAG_FORCE_SIMT 1u /* bf16 I/O through the plain-fp32 kernels (a second opinion for tests) */
 
 typedef struct {
   uint32_t struct_size; /* sizeof(vdn_vda_config), checked                                            */

@@ -14,18 +14,12 @@
 //               64 tokens so the MMA of one half overlaps the weighting of the other.  Once per frame (after the
 //               first tile of the next frame is with the MMA) the same warps drain the finished accumulator:
 //               TMEM -> registers -> global fp32 [2d][d] (A_t, then B_t); there are two accumulators
-//   warps 6-13  resolve (Eq. 5), when `csplit` is set: once A_t is stored these 256 threads read it back (from
-//               L2) as 8 x 8 cyclic register tiles, invert I + A_t by Gauss-Jordan in fp32 while the next
-//               frame's tiles stream in, and write the inverse as three bf16 parts for the tensor-core scan.
-//               (A TMEM row sits in one thread, the wrong shape for elimination: every thread would need every
-//               pivot row.  The 2-D tiling needs 8 + 8 broadcast values per pivot instead of 128.)
 // Rows past the end of a frame are zero-filled by TMA (the map has F as its own dimension) and their
 // beta is forced to zero.  Every mbarrier wait is bounded.
 #pragma once
 #include <cuda_bf16.h>
 
 #include "common.cuh"
-#include "resolve.cuh"
 #include "tc_common.cuh"
 
 namespace vdn {
@@ -39,17 +33,15 @@ struct GramTc {
   static constexpr int KP_HALF_BYTES = 2 * 64 * 128;      // 2 boxes x 64 tokens x 128 B
   static constexpr int OFF_KP = STAGES * STAGE_BYTES;
   static constexpr int OFF_BAR = OFF_KP + 2 * KP_HALF_BYTES;
-  static constexpr int OFF_ROWBUF = OFF_BAR + 144;         // pivot row / column exchange of the resolve warps (2 KB)
-  static constexpr int USED_BYTES = OFF_ROWBUF + 2048;
+  static constexpr int USED_BYTES = OFF_BAR + 128;
   static constexpr int SMEM_BYTES = 232448;                // everything an SM offers one CTA; the slack
-                                                           // (880 B) absorbs the 1024-byte alignment
-  static constexpr int THREADS = 448;
+                                                           // absorbs the 1024-byte alignment
+  static constexpr int THREADS = 192;
 };
 
 __global__ void __launch_bounds__(GramTc::THREADS, 1)
 gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-               const float* __restrict__ beta, float* __restrict__ stats, __nv_bfloat16* __restrict__ csplit,
-               Shape s, int* status) {
+               const float* __restrict__ beta, float* __restrict__ stats, Shape s, int* status) {
   using namespace tc;
   using G = GramTc;
   extern __shared__ unsigned char smem_dyn[];
@@ -64,10 +56,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   auto KPFREE = [&](int i) { return bar0 + 8u * (8 + i); };    // 2
   auto ACCFULL = [&](int i) { return bar0 + 8u * (10 + i); };  // 2
   auto ACCEMPTY = [&](int i) { return bar0 + 8u * (12 + i); }; // 2
-  const uint32_t AREADY = bar0 + 8u * 14;                      // epilogue -> resolve: A_t of a frame is in memory
-  const uint32_t ATAKEN = bar0 + 8u * 15;                      // resolve -> epilogue: that signal has been seen
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + G::OFF_BAR + 8 * 16);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + G::OFF_BAR + 8 * 16 + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + G::OFF_BAR + 8 * 14);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + G::OFF_BAR + 8 * 14 + 4);
   const WaitCtx wc{abort_flag, status};
 
   if ((base - smem_u32(smem_dyn)) + G::USED_BYTES > (uint32_t)G::SMEM_BYTES) {
@@ -85,8 +75,6 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       mbar_init(SCALED(i), 128); mbar_init(KPFREE(i), 1);
       mbar_init(ACCFULL(i), 1);  mbar_init(ACCEMPTY(i), 128);
     }
-    mbar_init(AREADY, 128);
-    mbar_init(ATAKEN, 256);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmK);
@@ -160,7 +148,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (ok) mma_commit(ACCFULL(a));
       }
     }
-  } else if (warp < 6) {
+  } else {
     // ------------------------------------------------------------------ weighting warps: K' = beta * K,
     // and, once per frame, the drain of the previous frame's accumulator
     const int ts = threadIdx.x - 64;          // 0..127
@@ -190,12 +178,6 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
       tc_fence_before_sync();
       mbar_arrive(ACCEMPTY(a));                 // the accumulator is free for the frame after next
-      if (csplit != nullptr) {
-        // one signal in flight at most: the resolve warps have seen the previous frame's before this one is sent
-        if (!mbar_wait(ATAKEN, (dai & 1) ^ 1, wc)) return false;
-        __threadfence_block();                  // A_t is visible to the resolve warps of this CTA
-        mbar_arrive(AREADY);
-      }
       return true;
     };
 
@@ -254,35 +236,6 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       ++ai;
     }
     if (ok && prev_item >= 0) drain(prev_item, ai - 1);
-  } else {
-    // ------------------------------------------------------------------ resolve warps (Eq. 5)
-    if (csplit != nullptr) {
-      const int gt = threadIdx.x - 192;         // 0..255
-      const int tx = gt & 15, ty = gt >> 4;
-      float* rowbuf = reinterpret_cast<float*>(base_ptr + G::OFF_ROWBUF);
-      float* colbuf = rowbuf + 2 * G::D;
-      uint32_t ai = 0;
-      for (long long item = blockIdx.x; item < nitems; item += gridDim.x, ++ai) {
-        int b, h, t;
-        const long long n = split_work(s, item, b, h, t);
-        if (!mbar_wait(AREADY, ai & 1, wc)) break;
-        mbar_arrive(ATAKEN);
-        // The stored block K^T (beta K) is symmetric up to the bf16 rounding of the weighted factor; it is
-        // inverted as it stands.  L2-only loads: the lines were written by this CTA moments ago and L1 is
-        // not coherent.
-        const float* A = stats + (size_t)n * (2 * G::D * G::D);
-        float m[8][8];
-#pragma unroll
-        for (int r = 0; r < 8; ++r)
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const int i = ty + 16 * r, j = tx + 16 * c;
-            m[r][c] = __ldcg(A + (size_t)i * G::D + j) + (i == j ? 1.0f : 0.0f);
-          }
-        gauss_jordan_tiles<G::D>(m, rowbuf, colbuf, tx, ty, [] { tc::named_barrier_sync(2, 256); });
-        store_split_tiles<G::D>(m, csplit + (size_t)n * (3 * G::D * G::D), tx, ty);
-      }
-    }
   }
 
   // ------------------------------------------------------------------ teardown

@@ -293,19 +293,12 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   const unsigned persistent = (unsigned)(n < h->sm_count ? n : h->sm_count);
   prof_begin(h, st);
   int nk = 0;
-  if (h->cfg.flags & VDN_FLAG_RESOLVE_IN_GRAM) {
-    // statistics + resolve in one kernel: spare warps invert I + A_t (plain fp32) while the next frame streams in
-    vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(
-        tmK, tmV, beta, stats, csplit, s, h->status_dev);
-    prof_mark(h, st, nk++, "gram_tc");
-  } else {
-    vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(
-        tmK, tmV, beta, stats, nullptr, s, h->status_dev);
-    prof_mark(h, st, nk++, "gram_tc");
-    vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
-        stats, csplit, n, h->status_dev);
-    prof_mark(h, st, nk++, "resolve_tc");
-  }
+  vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
+                                                                                       h->status_dev);
+  prof_mark(h, st, nk++, "gram_tc");
+  vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
+      stats, csplit, n, h->status_dev);
+  prof_mark(h, st, nk++, "resolve_tc");
   vdn::scan_tc_kernel<<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS, vdn::ScanTc::SMEM_BYTES, st>>>(
       tmC, stats, pf, pb, s.T, h->status_dev);
   prof_mark(h, st, nk++, "scan_tc");
