@@ -214,15 +214,21 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           // beta rounded to bf16, then one packed bf16 multiply per channel pair (round to nearest): the
           // float->bf16 conversion instruction is slow on this GPU and kept this loop from hiding under HBM
           const __nv_bfloat162 w2 = __float2bfloat162_rn(bu[half]);
+          // all eight loads first, then the stores: written as one load-store pair per chunk the compiler
+          // must keep them in order (the two shared-memory pointers might alias) and every chunk pays the
+          // full shared-memory latency
+          uint4 raw[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) raw[j] = *reinterpret_cast<const uint4*>(src + ((j ^ (r & 7)) * 16));
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            const int pj = (j ^ (r & 7)) * 16;   // stagger the 16-byte chunks across rows: conflict-free
-            uint4 raw = *reinterpret_cast<const uint4*>(src + pj);
-            __nv_bfloat162* x = reinterpret_cast<__nv_bfloat162*>(&raw);
+            __nv_bfloat162* x = reinterpret_cast<__nv_bfloat162*>(&raw[j]);
 #pragma unroll
             for (int e = 0; e < 4; ++e) x[e] = __hmul2(x[e], w2);
-            *reinterpret_cast<uint4*>(dst + pj) = raw;
           }
+#pragma unroll
+          for (int j = 0; j < 8; ++j)            // chunks staggered across rows: conflict-free
+            *reinterpret_cast<uint4*>(dst + ((j ^ (r & 7)) * 16)) = raw[j];
           fence_proxy_async_smem();
           mbar_arrive(SCALED(half));
         }
