@@ -66,6 +66,29 @@ def test_forward_matches_oracle_small(name, kw):
     check_heads(w, x, out, all_pairs(w), TOL[w.dtype])
 
 
+@pytest.mark.parametrize("B,H,T,F", [
+    (1, 1, 1, 5),        # one frame: nothing to read, all zeros
+    (1, 1, 2, 1),        # one token per frame
+    (2, 3, 3, 127),      # one short tile, several batches and heads
+    (1, 2, 4, 129),      # one full tile + one token
+    (3, 1, 2, 256),      # exact tiles, batch > heads
+    (1, 5, 7, 64),       # more chains than frames
+    (1, 2, 33, 40),      # a deeper scan than anything else in this file
+])
+def test_tensor_core_path_edge_shapes(B, H, T, F):
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=B, H=H, T=T, F=F, seed=B * 1000 + H * 100 + T * 10 + F)
+    x = inputs.generate(w, "cuda")
+    vda, out = run_gpu(w, x)
+    assert vda.uses_tensor_cores()
+    if T == 1:
+        assert torch.count_nonzero(out) == 0
+    check_heads(w, x, out, all_pairs(w), TOL["bf16"])
+    # the plain-fp32 kernels on the same bf16 inputs are a second GPU opinion
+    _, out2 = run_gpu(w, x, flags=binding.VDN_FLAG_FORCE_SIMT)
+    scale = out2.float().abs().amax().clamp_min(1e-30)
+    assert float((out.float() - out2.float()).abs().amax() / scale) < 2e-2
+
+
 def test_bf16_through_plain_fp32_kernels():
     w = inputs.TINY.scaled(dtype="bf16", d=128, T=4, F=200, H=2)
     x = inputs.generate(w, "cuda")
