@@ -4,9 +4,9 @@
  * The layer (Video DeltaNet, Sec. 2.2, Sec. 3 and Algorithm 1 steps 3-7), per (batch, head):
  *
  *   frame statistics (Eq. 3b)        A_t = K_t^T Diag(beta_t) K_t,   B_t = V_t^T Diag(beta_t) K_t
- *   joint frame update (Eq. 5, A.1)  S_t = (S_{t-1} + B_t)(I + A_t)^{-1}            (decay alpha_t = 1)
+ *   joint frame update (Eq. 5, A.1)  S_t = (S_{t-1} + B_t)(I + A_t)^{-1}   (decay alpha_t = 1; see forward_ex)
  *   two scans (Sec. 2.2)             P_t: frames 0..t in order,  R_t: frames T-1..t in reverse order,
- *                                    both started from the zero state (no text state at this boundary)
+ *                                    both started from the zero state (vdn_vda_forward_ex: from S_T / 2)
  *   gather (Eq. A.4, Eq. 1a)         the queries of frame t read  P_{t-1} + R_{t+1}  (P_{-1} = R_T = 0):
  *                                    the local window is the query frame itself, so no frame is counted
  *                                    twice and a frame never reads its own write
@@ -111,6 +111,19 @@ vdn_status vdn_vda_set_workspace(vdn_vda_t h, void* dev_ptr, size_t bytes);
 vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
                            const float* gate, void* out, int B, int T, int F, int H, int d,
                            void* cuda_stream);
+
+/* The same layer with the two inputs of the paper's recurrence that vdn_vda_forward fixes (first item of the
+ * "next" list; the local window is still the query frame itself, and there are no anchor frames):
+ *   alpha [B,T,H,d] float, DEVICE, in [0,1], or NULL (= 1): channel-wise decay gate of frame t (Eq. 2, Eq. A.1:
+ *         M_t = Diag(alpha_t)(I + A_t)^{-1}).  It decays the inherited state before frame t is folded in, in both
+ *         scans, and bridges the state that frame t's queries read (Eq. A.4 with l_t = h_t = t):
+ *         (P_{t-1} + R_{t+1}) Diag(alpha_t).
+ *   s0    [B,H,d_v,d_k] float, DEVICE, or NULL (= 0): the text state S_T; each scan starts from S_T / 2 (Eq. 1b),
+ *         and a missing side of the gather reads S_T / 2 (Eq. A.4).
+ * Everything else is as for vdn_vda_forward, which is this call with alpha = s0 = NULL. */
+vdn_status vdn_vda_forward_ex(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                              const float* gate, const float* alpha, const float* s0, void* out, int B, int T,
+                              int F, int H, int d, void* cuda_stream);
 
 /* The same layer for callers whose tensors live in HOST memory (pinned memory recommended): copies
  * q, k, v, beta, gate to the staging buffer, runs vdn_vda_forward, copies `out` back, all on

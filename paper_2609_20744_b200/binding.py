@@ -21,7 +21,7 @@ VDN_FLAG_FORCE_SIMT = 1
 VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_READ_BWD = range(7)
 
 EXPORTS = (
-    "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward",
+    "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward", "vdn_vda_forward_ex",
     "vdn_vda_staging_bytes", "vdn_vda_set_staging", "vdn_vda_forward_host", "vdn_vda_workspace_view",
     "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_scan_static", "vdn_vda_status", "vdn_vda_last_error", "vdn_vda_destroy",
 )
@@ -66,6 +66,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     fwd_args = [vp, vp, vp, vp, vp, vp, vp, *shape, vp]
     lib.vdn_vda_forward.argtypes = fwd_args
     lib.vdn_vda_forward.restype = ci
+    lib.vdn_vda_forward_ex.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, *shape, vp]
+    lib.vdn_vda_forward_ex.restype = ci
     lib.vdn_vda_forward_host.argtypes = fwd_args
     lib.vdn_vda_forward_host.restype = ci
     lib.vdn_vda_workspace_view.argtypes = [vp, ci, *shape, ctypes.POINTER(sz), ctypes.POINTER(sz)]
@@ -173,19 +175,35 @@ class Vda:
         return self._staging
 
     # -- the two entry points -----------------------------------------------------------------
-    def forward(self, q, k, v, beta, gate, out=None, stream=None):
-        """vdn_vda_forward on device tensors q,k,v [B,T,F,H,d], beta [B,T,F,H], gate [H]."""
+    def forward(self, q, k, v, beta, gate, out=None, stream=None, alpha=None, s0=None):
+        """vdn_vda_forward on device tensors q,k,v [B,T,F,H,d], beta [B,T,F,H], gate [H].
+
+        With alpha [B,T,H,d] (decay gates) and/or s0 [B,H,d,d] (text state) the call goes to vdn_vda_forward_ex.
+        """
         torch = self._torch
         B, T, F, H, d = q.shape
-        for x in (q, k, v, beta, gate):
+        extras = [x for x in (alpha, s0) if x is not None]
+        for x in (q, k, v, beta, gate, *extras):
             if not (x.is_cuda and x.is_contiguous()):
                 raise ValueError("vdn_vda_forward needs contiguous CUDA tensors")
+        for x in extras:
+            if x.dtype != torch.float32:
+                raise ValueError("alpha and s0 must be float32")
+        if alpha is not None and tuple(alpha.shape) != (B, T, H, d):
+            raise ValueError("alpha must be [B, T, H, d]")
+        if s0 is not None and tuple(s0.shape) != (B, H, d, d):
+            raise ValueError("s0 must be [B, H, d, d]")
         if out is None:
             out = torch.empty_like(q)
         self.ensure_workspace(B, T, F, H)
-        p = lambda x: ctypes.c_void_p(x.data_ptr())
-        self._check(self.lib.vdn_vda_forward(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
-                                             B, T, F, H, d, self._stream(stream)))
+        p = lambda x: ctypes.c_void_p(x.data_ptr()) if x is not None else None
+        if extras:
+            st = self.lib.vdn_vda_forward_ex(self.h, p(q), p(k), p(v), p(beta), p(gate), p(alpha), p(s0), p(out),
+                                             B, T, F, H, d, self._stream(stream))
+        else:
+            st = self.lib.vdn_vda_forward(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
+                                          B, T, F, H, d, self._stream(stream))
+        self._check(st)
         return out
 
     def forward_host(self, q, k, v, beta, gate, out, stream=None):

@@ -6,8 +6,8 @@
 // registers for the whole clip and needs no communication with the CTAs that own the other columns.
 //
 // Pass 1 (t = 0..T-1) stores P_t^T.  Pass 2 (t = T-1..0) carries R_{t+1}^T, first emits the state the
-// queries of frame t read,  P_{t-1}^T + R_{t+1}^T  (zero where a side is missing: the scans start
-// from the zero state), then folds frame t in.  Both passes are written back by the very thread that
+// queries of frame t read,  P_{t-1}^T + R_{t+1}^T  (the initial state where a side is missing), then folds
+// frame t in.  Both passes are written back by the very thread that
 // computed them, so the second pass needs no inter-CTA ordering.
 //
 // C_t is symmetric; the kernel reads it as C_t[j][i] so that each thread's row group is contiguous.
@@ -27,7 +27,8 @@ template <int D, int W>
 __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ stats,
                                                        const float* __restrict__ inv,
                                                        float* __restrict__ fwd, float* __restrict__ read,
-                                                       int T) {
+                                                       int T, const float* __restrict__ alpha = nullptr,
+                                                       const float* __restrict__ s0 = nullptr, int H = 1) {
   constexpr int TI = D / 32;          // rows per thread
   constexpr int NCG = W / 4;          // column groups of 4
   static_assert(256 / NCG * TI == D, "thread tiling must cover D rows");
@@ -40,11 +41,26 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
   const int cg = tid % NCG, ig = tid / NCG;
   const int i0 = ig * TI, cc0 = cg * 4;
 
+  // Optional extras (Eq. A.1, Eq. 1b, Eq. A.4): alpha [B,T,H,d] decays key channel i of the inherited state
+  // before frame t is folded in and bridges the state read by frame t; s0 [B,H,d_v,d_k] is the text state,
+  // each scan starting from half of it.
+  float zinit[TI][4];
+#pragma unroll
+  for (int r = 0; r < TI; ++r)
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      zinit[r][c] = s0 ? 0.5f * s0[((size_t)bh * D + c0 + cc0 + c) * D + i0 + r] : 0.f;
+  auto alpha_of = [&](int t, float (&a)[TI]) {
+#pragma unroll
+    for (int r = 0; r < TI; ++r)
+      a[r] = alpha ? alpha[(((size_t)(bh / H) * T + t) * H + (bh % H)) * D + i0 + r] : 1.0f;
+  };
+
   float z[TI][4];
 #pragma unroll
   for (int r = 0; r < TI; ++r)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) z[r][c] = 0.f;
+    for (int c = 0; c < 4; ++c) z[r][c] = zinit[r][c];
 
   int buf = 0;
   for (int step = 0; step < 2 * T; ++step) {
@@ -60,14 +76,17 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
       cp_async_commit();
     }
 
+    float al[TI];
+    alpha_of(t, al);
     if (!forward) {
-      // gather: the state read by frame t's queries
+      // gather: the state read by frame t's queries, bridged by frame t's decay
       float p[TI][4];
 #pragma unroll
       for (int r = 0; r < TI; ++r) {
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 x = make_float4(zinit[r][0], zinit[r][1], zinit[r][2], zinit[r][3]);
         if (t > 0) x = load4(fwd + (n - 1) * D * D + (size_t)(i0 + r) * D + c0 + cc0);
-        p[r][0] = x.x + z[r][0]; p[r][1] = x.y + z[r][1]; p[r][2] = x.z + z[r][2]; p[r][3] = x.w + z[r][3];
+        p[r][0] = al[r] * (x.x + z[r][0]); p[r][1] = al[r] * (x.y + z[r][1]);
+        p[r][2] = al[r] * (x.z + z[r][2]); p[r][3] = al[r] * (x.w + z[r][3]);
       }
       float* dst = read + n * D * D;
 #pragma unroll
@@ -75,7 +94,7 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
         store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(p[r][0], p[r][1], p[r][2], p[r][3]));
     }
 
-    // X = Z + B_t^T (this CTA's columns)
+    // X = alpha_t * Z + B_t^T (this CTA's columns)
     {
       // B_t is stored [d_v][d_k]: element (c, i) is B_t^T[i][c]
       const float* bsrc = stats + n * 2 * D * D + (size_t)(D + c0 + cc0) * D + i0;
@@ -92,7 +111,8 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
       }
 #pragma unroll
       for (int r = 0; r < TI; ++r)
-        store4(&sm.X[buf][i0 + r][cc0], make_float4(bt[r][0] + z[r][0], bt[r][1] + z[r][1], bt[r][2] + z[r][2], bt[r][3] + z[r][3]));
+        store4(&sm.X[buf][i0 + r][cc0], make_float4(fmaf(al[r], z[r][0], bt[r][0]), fmaf(al[r], z[r][1], bt[r][1]),
+                                                     fmaf(al[r], z[r][2], bt[r][2]), fmaf(al[r], z[r][3], bt[r][3])));
     }
     cp_async_wait<0>();
     __syncthreads();
@@ -131,11 +151,11 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
         store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(z[r][0], z[r][1], z[r][2], z[r][3]));
     }
     if (step == T - 1) {
-      // the reverse scan starts from the zero state
+      // the reverse scan starts from the initial state as well
 #pragma unroll
       for (int r = 0; r < TI; ++r)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) z[r][c] = 0.f;
+        for (int c = 0; c < 4; ++c) z[r][c] = zinit[r][c];
     }
   }
 }

@@ -1,7 +1,8 @@
 // Frame scan (Alg. 1 step 5; Eq. A.1) with the d x d products on the tcgen05 tensor cores at fp32
 // accuracy, d = 128.  One CTA per (batch, head, direction) chain; the state never leaves the SM.
 //
-// With Z = S^T and alpha = 1 the frame update reads  Z_t = C_t (Z_{t-1} + B_t^T),  C_t = (I+A_t)^{-1}.
+// With Z = S^T the frame update reads  Z_t = C_t (alpha_t * Z_{t-1} + B_t^T),  C_t = (I+A_t)^{-1}  (alpha_t acts on
+// the key rows of Z; it is 1 unless the caller passes a decay).
 // Both factors are fp32.  Each is written as a sum of three bf16 numbers (x = x1 + x2 + x3, every part the
 // bf16 rounding of what the earlier parts leave over: 24 mantissa bits, i.e. all of fp32), and the product
 // is accumulated in fp32 (TMEM) from the six partial products whose weight is above 2^-24:
@@ -16,8 +17,8 @@
 // operand.  The next frame's B^T row is fetched into registers while the MMAs run.
 //
 // Gather (Eq. A.4 with the window shrunk to the query frame): the forward chain stores P_t in slot t+1 of
-// `pf`, the reverse chain stores R_t in slot t-1 of `pb`; slot 0 of pf and slot T-1 of pb are zeroed here
-// (the scans start from the zero state).  The read-out kernel adds the two in its accumulator (Eq. 1a).
+// `pf`, the reverse chain stores R_t in slot t-1 of `pb`, each already bridged by the reading frame's decay; slot 0
+// of pf and slot T-1 of pb receive the initial state (zero unless a text state is passed).  The read-out kernel adds the two in its accumulator (Eq. 1a).
 #pragma once
 #include <cuda_bf16.h>
 
@@ -40,7 +41,8 @@ struct ScanTc {
 
 __global__ void __launch_bounds__(ScanTc::THREADS, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict__ stats,
-               __nv_bfloat16* __restrict__ pf, __nv_bfloat16* __restrict__ pb, int T, int* status) {
+               __nv_bfloat16* __restrict__ pf, __nv_bfloat16* __restrict__ pb, int T,
+               const float* __restrict__ alpha, const float* __restrict__ s0, int H, int* status) {
   using namespace tc;
   using S = ScanTc;
   constexpr int D = S::D;
@@ -164,16 +166,28 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
       mbar_arrive(XREADY);
     };
 
+    // Optional extras (Eq. A.1, Eq. 1b, Eq. A.4): alpha [B,T,H,d] decays key channel `row` of the inherited
+    // state before a frame is folded in, and bridges the state that frame reads; s0 [B,H,d_v,d_k] is the text
+    // state, each scan starting from half of it.  Both act on a thread's own row: one scalar per step.
+    auto alpha_of = [&](int frame) {
+      return alpha ? __ldg(alpha + (((size_t)(bh / H) * T + frame) * H + (bh % H)) * D + row) : 1.0f;
+    };
     float bt[CW];
     load_bt(frame_of(0), bt);
-    publish_x(bt);                           // Z_{-1} = 0
     {
-      // the chain's first read slot holds the zero state
+      // the chain's first read slot holds the (bridged) initial state, and X_0 = alpha_0 * Z_init + B_0^T
+      const float a0 = alpha_of(frame_of(0));
       __nv_bfloat16* z0 = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(0)) * (D * D) + (size_t)col0 * D + row;
 #pragma unroll
-      for (int e = 0; e < CW; ++e) z0[(size_t)e * D] = __float2bfloat16_rn(0.f);
+      for (int e = 0; e < CW; ++e) {
+        const float zi = s0 ? 0.5f * __ldg(s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
+        z0[(size_t)e * D] = __float2bfloat16_rn(a0 * zi);
+        bt[e] = fmaf(a0, zi, bt[e]);
+      }
     }
+    publish_x(bt);
     if (T > 1) load_bt(frame_of(1), bt);
+    float a_next = T > 1 ? alpha_of(frame_of(1)) : 1.0f;
     for (int s = 0; s + 1 < T; ++s) {
       if (!mbar_wait(ACCFULL, s & 1, wc)) break;
       tc_fence_after_sync();
@@ -183,7 +197,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
       // first what the next MMAs are waiting for: X = Z + B^T of the next frame, split, into shared memory
       if (s + 2 < T) {
 #pragma unroll
-        for (int e = 0; e < CW; ++e) bt[e] += z[e];
+        for (int e = 0; e < CW; ++e) bt[e] = fmaf(a_next, z[e], bt[e]);
         publish_x(bt);
       }
       // then, under the next step's MMAs: the state after step s is what the next frame in scan order reads.
@@ -192,11 +206,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
       __nv_bfloat16* dst = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(s + 1)) * (D * D) + (size_t)col0 * D + row;
 #pragma unroll
       for (int e = 0; e < CW; e += 2) {
-        const __nv_bfloat162 v2 = __floats2bfloat162_rn(z[e], z[e + 1]);
+        const __nv_bfloat162 v2 = __floats2bfloat162_rn(a_next * z[e], a_next * z[e + 1]);   // decay bridge of the reader
         dst[(size_t)e * D] = v2.x;
         dst[(size_t)(e + 1) * D] = v2.y;
       }
-      if (s + 2 < T) load_bt(frame_of(s + 2), bt);   // B^T of the frame after next, also under the MMAs
+      if (s + 2 < T) {                                 // B^T and decay of the frame after next, also under the MMAs
+        load_bt(frame_of(s + 2), bt);
+        a_next = alpha_of(frame_of(s + 2));
+      }
     }
   }
 

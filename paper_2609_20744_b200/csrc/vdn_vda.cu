@@ -196,7 +196,8 @@ vdn_status set_attrs_simt(vdn_vda_t h) {
 // The plain-fp32 path: four launches.
 template <typename Tio, int D>
 vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
-                        const float* gate, void* out, const Shape& s, const Layout& L, cudaStream_t st) {
+                        const float* gate, const float* alpha, const float* s0, void* out, const Shape& s,
+                        const Layout& L, cudaStream_t st) {
   if (!h->attrs_set) {
     vdn_status r = set_attrs_simt<Tio, D>(h);
     if (r != VDN_OK) return r;
@@ -216,7 +217,7 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
   vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n);
   prof_mark(h, st, 1, "resolve");
   vdn::scan_kernel<D, 32><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
-      stats, inv, fwd, read, s.T);
+      stats, inv, fwd, read, s.T, alpha, s0, s.H);
   prof_mark(h, st, 2, "scan");
   vdn::readout_simt_kernel<Tio, D><<<dim3((unsigned)n, (s.F + 63) / 64), 256, sizeof(vdn::ReadoutSimtSmem<D>), st>>>(
       static_cast<const Tio*>(q), read, gate, static_cast<Tio*>(out), s, h->cfg.rms_eps);
@@ -260,7 +261,8 @@ vdn_status make_matrix_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, long lo
 }
 
 vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
-                      const float* gate, void* out, const Shape& s, const Layout& L, cudaStream_t st) {
+                      const float* gate, const float* alpha, const float* s0, void* out, const Shape& s,
+                      const Layout& L, cudaStream_t st) {
   constexpr int D = 128;
   if (!h->encode) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   if (!h->tc_attrs_set) {
@@ -300,7 +302,7 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
       stats, csplit, n, h->status_dev);
   prof_mark(h, st, nk++, "resolve_tc");
   vdn::scan_tc_kernel<<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS, vdn::ScanTc::SMEM_BYTES, st>>>(
-      tmC, stats, pf, pb, s.T, h->status_dev);
+      tmC, stats, pf, pb, s.T, alpha, s0, s.H, h->status_dev);
   prof_mark(h, st, nk++, "scan_tc");
   // The read-out streams reads and writes in equal parts and is fastest on about five SMs out of six
   // (measured on three workloads: 124 CTAs beat 148 by 5 %; fewer interleaved read/write streams at the DRAM).
@@ -419,13 +421,14 @@ vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes) {
   return VDN_OK;
 }
 
-vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
-                           const float* gate, void* out, int B, int T, int F, int H, int d,
-                           void* cuda_stream) {
+vdn_status vdn_vda_forward_ex(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                              const float* gate, const float* alpha, const float* s0, void* out, int B, int T,
+                              int F, int H, int d, void* cuda_stream) {
   if (!h) return VDN_ERR_INVALID_ARG;
   if (!q || !k || !v || !beta || !gate || !out) return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(beta))
-    return fail(h, VDN_ERR_INVALID_ARG, "q, k, v, beta, out must be 16-byte aligned");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(beta) ||
+      !aligned16(alpha) || !aligned16(s0))
+    return fail(h, VDN_ERR_INVALID_ARG, "q, k, v, beta, alpha, s0, out must be 16-byte aligned");
   if (out == q || out == k || out == v) return fail(h, VDN_ERR_INVALID_ARG, "out must not alias an input");
   std::string why;
   if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
@@ -436,13 +439,19 @@ vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void
   if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const Shape s{B, T, F, H, d};
-  if (use_tensor_cores(h, d)) return forward_tc(h, q, k, v, beta, gate, out, s, L, st);
+  if (use_tensor_cores(h, d)) return forward_tc(h, q, k, v, beta, gate, alpha, s0, out, s, L, st);
   if (h->cfg.io_dtype == VDN_F32) {
-    return d == 64 ? forward_simt<float, 64>(h, q, k, v, beta, gate, out, s, L, st)
-                   : forward_simt<float, 128>(h, q, k, v, beta, gate, out, s, L, st);
+    return d == 64 ? forward_simt<float, 64>(h, q, k, v, beta, gate, alpha, s0, out, s, L, st)
+                   : forward_simt<float, 128>(h, q, k, v, beta, gate, alpha, s0, out, s, L, st);
   }
-  return d == 64 ? forward_simt<__nv_bfloat16, 64>(h, q, k, v, beta, gate, out, s, L, st)
-                 : forward_simt<__nv_bfloat16, 128>(h, q, k, v, beta, gate, out, s, L, st);
+  return d == 64 ? forward_simt<__nv_bfloat16, 64>(h, q, k, v, beta, gate, alpha, s0, out, s, L, st)
+                 : forward_simt<__nv_bfloat16, 128>(h, q, k, v, beta, gate, alpha, s0, out, s, L, st);
+}
+
+vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                           const float* gate, void* out, int B, int T, int F, int H, int d,
+                           void* cuda_stream) {
+  return vdn_vda_forward_ex(h, q, k, v, beta, gate, nullptr, nullptr, out, B, T, F, H, d, cuda_stream);
 }
 
 vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const void* v,

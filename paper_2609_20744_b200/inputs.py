@@ -121,6 +121,17 @@ def generate(w: VdaWorkload, device="cpu", pin: bool = False):
     return {"q": q, "k": k, "v": v, "beta": beta, "gate": gate}
 
 
+def generate_recurrence_extras(w: VdaWorkload, device="cpu"):
+    """Seeded decay gates alpha [B,T,H,d] = sigmoid(N(2,1)) (mostly close to 1, as decay gates are) and a text
+    state s0 [B,H,d,d] ~ N(0, 1/d), for the extended entry point.  float32."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(_seed(w.seed, 0xA1FA))
+    alpha = torch.sigmoid(2.0 + torch.randn((w.B, w.T, w.H, w.d), generator=g, device=dev))
+    s0 = torch.randn((w.B, w.H, w.d, w.d), generator=g, device=dev) / (w.d ** 0.5)
+    return alpha.contiguous(), s0.contiguous()
+
+
 def head_slice(x: dict, b: int, h: int):
     """Host float64 numpy copies of one (batch, head) slice: q,k,v [T,F,d], beta [T,F], gate scalar."""
     import numpy as np

@@ -89,6 +89,48 @@ def test_tensor_core_path_edge_shapes(B, H, T, F):
     assert float((out.float() - out2.float()).abs().amax() / scale) < 2e-2
 
 
+# ------------------------------------------------------------------------------ decay gates and text state
+@pytest.mark.parametrize("dtype,d,flags,use_alpha,use_s0", [
+    ("f32", 64, 0, True, True), ("f32", 128, 0, True, False), ("f32", 64, 0, False, True),
+    ("bf16", 128, 0, True, True), ("bf16", 128, 0, True, False), ("bf16", 128, 0, False, True),
+    ("bf16", 128, binding.VDN_FLAG_FORCE_SIMT, True, True),
+])
+def test_forward_ex_decay_and_text_state(dtype, d, flags, use_alpha, use_s0):
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=2, H=2, T=5, F=140, seed=77)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    alpha = alpha if use_alpha else None
+    s0 = s0 if use_s0 else None
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    for (b, h) in all_pairs(w):
+        q, k, v, beta, gate = inputs.head_slice(x, b, h)
+        a = None if alpha is None else alpha[b, :, h, :].double().cpu().numpy()
+        s = None if s0 is None else s0[b, h].double().cpu().numpy()
+        ref = orc.vda_slice(q, k, v, beta, gate, 1e-6, alpha=a, s0=s)["out"]
+        e = orc.slice_error(out[b, :, :, h, :].double().cpu().numpy(), ref)
+        assert e <= TOL[dtype], f"slice (b={b}, h={h}) error {e:.3e}"
+    # the extras matter: the plain call gives something else
+    plain = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
+    torch.cuda.synchronize()
+    assert not torch.allclose(plain.float(), out.float(), atol=1e-2)
+
+
+def test_forward_ex_single_frame_reads_the_text_state():
+    # T = 1: nothing but S_T is read (both halves), bridged by alpha_0 (Eq. 1b, Eq. A.4)
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=1, F=70, H=2)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0)
+    torch.cuda.synchronize()
+    o = torch.einsum("bhck,bfhk->bfhc", s0, (alpha[:, 0][:, None] * x["q"][:, 0].float()))
+    want = x["gate"][None, None, :, None] * o / torch.sqrt(o.pow(2).mean(-1, keepdim=True) + 1e-6)
+    assert torch.allclose(out[:, 0].float(), want, atol=3e-2, rtol=3e-2)
+
+
 def test_bf16_through_plain_fp32_kernels():
     w = inputs.TINY.scaled(dtype="bf16", d=128, T=4, F=200, H=2)
     x = inputs.generate(w, "cuda")
