@@ -280,6 +280,21 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     ms_max, tokens_total = aggregate_over_ranks(ms_local, w.tokens, world)
     value = tokens_total / (ms_max / 1e3)
 
+    # ---- parity of this very launch configuration against the fp64 oracle, on sampled (batch, head) slices
+    parity = None
+    if rank == 0 and not args.skip_cpu:
+        from oracle import vda_oracle
+        tol = 1e-4 if w.dtype == "f32" else 2e-2
+        pairs = [(0, 0), (w.B - 1, w.H - 1)]
+        errs = []
+        for (b, hh) in pairs:
+            qs, ks, vs, bs, gs = inputs.head_slice(x, b, hh)
+            ref = vda_oracle.vda_slice(qs, ks, vs, bs, gs, 1e-6)["out"]
+            errs.append(vda_oracle.slice_error(out[b, :, :, hh, :].double().cpu().numpy(), ref))
+            del qs, ks, vs, ref
+        parity = {"metric": "max over a (batch, head) slice of |gpu - oracle| / max |oracle|", "slices": pairs,
+                  "errors": errs, "tolerance": tol, "ok": bool(max(errs) <= tol)}
+
     # ---- end to end through the host-buffer entry point (H2D + forward + D2H inside the timed region)
     e2e = None
     try:
@@ -352,7 +367,7 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
                    "l2": "inputs+outputs far larger than the 126 MB L2; no flush" if ab["total"] > 1e9
                          else "inputs smaller than L2: numbers are L2-warm",
                    "path": "tensor-core" if vda.launch_count() and any("tc" in n for n in kt) else "plain-fp32"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "parity": parity,
         "roofline": roof,
         "layer_roofline": {"t_roof_ms_measured_peaks": t_roof_ms, "frac_of_measured": t_roof_ms / (ms_max / 1.0),
                            "t_roof_ms_nominal": t_roof_nominal_ms, "frac_of_nominal": t_roof_nominal_ms / ms_max,
