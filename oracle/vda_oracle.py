@@ -14,6 +14,9 @@ No blocking, fusion or re-ordering: one frame at a time, one equation per line.
 
 Pinning status (see tests/test_oracle_*.py):
   frame_statistics   pinned: literal per-token sums, permutation invariance
+  frame_update_additive
+                     pinned: literal token sum of Eq. 3a with keys scaled by 1/sqrt(U), Eq. 3c, the
+                     non-expansive bound of Sec. A.3 for unit keys, agreement with Eq. 5 as beta -> 0
   frame_update       pinned: least-squares brute force of Eq. 4, first-order
                      condition, token-space (Woodbury) form, Eq. 2 for U=1,
                      Eq. A.3 repeated keys, orthonormal keys, Eq. 3c as beta->0
@@ -70,7 +73,19 @@ def frame_update(S_prev, alpha, A, B):
     return np.linalg.solve(np.eye(d) + A, (S_bar + B).T).T
 
 
-def scan_states(A, B, alpha, S_init):
+def frame_update_additive(S_prev, alpha, A, B, U):
+    """The baseline VDA replaces (Eq. 3a/3c with the frame-size key scaling of Sec. 3.3): all token corrections
+    are evaluated at the same decayed state, keys scaled by 1/sqrt(U), i.e. A_t -> A_t/U, B_t -> B_t/sqrt(U):
+
+        S_bar = S_{t-1} Diag(alpha_t);   S_t = S_bar (I - A_t/U) + B_t/sqrt(U).
+    """
+    S_prev = np.asarray(S_prev, F64)
+    d = A.shape[0]
+    S_bar = S_prev * np.asarray(alpha, F64)[None, :]
+    return S_bar @ (np.eye(d) - np.asarray(A, F64) / U) + np.asarray(B, F64) / np.sqrt(U)
+
+
+def scan_states(A, B, alpha, S_init, rule="vda", U=None):
     """Sec. 2.2 / Alg. 1 step 5.  Both temporal scans of S <- S M_t + J_t.
 
     Returns P, R with P[t] = forward state through frame t (t = 0..T-1) and
@@ -80,13 +95,17 @@ def scan_states(A, B, alpha, S_init):
     T = len(A)
     P = [None] * T
     R = [None] * T
+    def step(S, t):
+        if rule == "additive":
+            return frame_update_additive(S, alpha[t], A[t], B[t], U)
+        return frame_update(S, alpha[t], A[t], B[t])
     S = np.asarray(S_init, F64)
     for t in range(T):
-        S = frame_update(S, alpha[t], A[t], B[t])
+        S = step(S, t)
         P[t] = S
     S = np.asarray(S_init, F64)
     for t in range(T - 1, -1, -1):
-        S = frame_update(S, alpha[t], A[t], B[t])
+        S = step(S, t)
         R[t] = S
     return P, R
 
@@ -112,8 +131,8 @@ def rmsnorm_gate(O, gate, eps):
     return gate * (O / np.sqrt(ms + eps))
 
 
-def vda_slice(q, k, v, beta, gate, eps=1e-6, alpha=None, s0=None, want=()):
-    """Whole layer for ONE (batch, head) slice.
+def vda_slice(q, k, v, beta, gate, eps=1e-6, alpha=None, s0=None, want=(), rule="vda"):
+    """Whole layer for ONE (batch, head) slice.  rule = "vda" (Eq. 5) or "additive" (Eq. 3c with 1/sqrt(U) keys).
 
     q, k : [T, U, d_k]   v : [T, U, d_v]   beta : [T, U]   gate : scalar
     alpha: [T, d_k] or None (ones)         s0   : [d_v, d_k] text state S_T or None (zero)
@@ -134,7 +153,7 @@ def vda_slice(q, k, v, beta, gate, eps=1e-6, alpha=None, s0=None, want=()):
     B = [None] * T
     for t in range(T):                                         # Alg. 1 step 3
         A[t], B[t] = frame_statistics(k[t], v[t], beta[t])
-    P, R = scan_states(A, B, alpha, S_init)                    # Alg. 1 steps 4-5
+    P, R = scan_states(A, B, alpha, S_init, rule, U)           # Alg. 1 steps 4-5
 
     o_fwd = np.zeros((T, U, dv))
     o_bwd = np.zeros((T, U, dv))

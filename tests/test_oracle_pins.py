@@ -152,6 +152,65 @@ def test_zero_write_gate_passes_decayed_state_through():
     assert np.array_equal(orc.frame_update(S_prev, alpha, A, B), S_prev * alpha[None, :])
 
 
+# ---------------------------------------------------------------- Eq. 3a / 3c: the additive baseline
+def test_additive_rule_is_the_literal_frozen_state_sum_with_scaled_keys():
+    r = rng(40)
+    U, dk, dv = 9, 5, 4
+    K, V, beta = random_frame(r, U, dk, dv)
+    S_prev = r.standard_normal((dv, dk))
+    alpha = r.uniform(0, 1, dk)
+    A, B = orc.frame_statistics(K, V, beta)
+    S = orc.frame_update_additive(S_prev, alpha, A, B, U)
+    S_bar = S_prev * alpha[None, :]
+    want = S_bar.copy()                                          # Eq. 3a with k -> k / sqrt(U)
+    for u in range(U):
+        ks = K[u] / np.sqrt(U)
+        want += beta[u] * np.outer(V[u] - S_bar @ ks, ks)
+    assert np.allclose(S, want, atol=1e-13)
+    # Eq. 3c written with the scaled statistics
+    assert np.allclose(S, S_bar @ (np.eye(dk) - A / U) + B / np.sqrt(U), atol=1e-13)
+
+
+def test_additive_rule_scaled_transition_is_non_expansive_for_unit_keys():
+    r = rng(41)
+    for U in (1, 7, 200):
+        K = unit(r.standard_normal((U, 8)))
+        if U > 1:
+            K[: U // 2] = unit(K[0] + 0.01 * r.standard_normal((U // 2, 8)))      # aligned keys: the worst case
+        beta = r.uniform(0, 1, U)
+        A, _ = orc.frame_statistics(K, np.zeros((U, 8)), beta)
+        assert np.linalg.norm(np.eye(8) - A / U, 2) <= 1.0 + 1e-12               # Sec. A.3
+    # without the scale the factor I - A does leave [-1, 1] for aligned keys
+    assert np.linalg.norm(np.eye(8) - A, 2) > 1.0
+
+
+def test_additive_whole_layer_matches_literal_loops():
+    r = rng(42)
+    T, U, d = 4, 6, 5
+    q, k, v, beta = random_slice(r, T, U, d, d)
+    alpha = r.uniform(0.3, 1, (T, d))
+    s0 = r.standard_normal((d, d))
+    res = orc.vda_slice(q, k, v, beta, 0.7, 1e-6, alpha, s0, want=("P", "R", "O"), rule="additive")
+    def fold(S, t):
+        Sb = S * alpha[t][None, :]
+        out = Sb.copy()
+        for u in range(U):
+            ks = k[t, u] / np.sqrt(U)
+            out += beta[t, u] * np.outer(v[t, u] - Sb @ ks, ks)
+        return out
+    S = 0.5 * s0
+    for t in range(T):
+        S = fold(S, t)
+        assert np.allclose(res["P"][t], S, atol=1e-12)
+    S = 0.5 * s0
+    for t in range(T - 1, -1, -1):
+        S = fold(S, t)
+        assert np.allclose(res["R"][t], S, atol=1e-12)
+    t = 2
+    want = (res["P"][t - 1] + res["R"][t + 1]) * alpha[t][None, :]
+    assert np.allclose(res["O"][t], q[t] @ want.T, atol=1e-12)
+
+
 # ---------------------------------------------------------------- golden worked examples
 def golden():
     with open(GOLDEN) as f:
