@@ -69,7 +69,10 @@ typedef enum {
 typedef enum { VDN_F32 = 0, VDN_BF16 = 1 } vdn_dtype;
 
 /* cfg.flags */
-#define VDN_FLAG_FORCE_SIMT 1u /* bf16 I/O through the plain-fp32 kernels (a second opinion for tests) */
+#define VDN_FLAG_FORCE_SIMT 1u    /* bf16 I/O through the plain-fp32 kernels (a second opinion for tests)      */
+#define VDN_FLAG_ADDITIVE_RULE 4u /* the baseline VDA replaces, for ablations: frozen-state additive frame      */
+                                  /* update with 1/sqrt(F) key scaling, S_t = S_bar (I - A_t/F) + B_t/sqrt(F)   */
+                                  /* (Eq. 3c, Sec. 3.3), no resolve; everything else unchanged                  */
 
 typedef struct {
   uint32_t struct_size; /* sizeof(vdn_vda_config), checked                                            */

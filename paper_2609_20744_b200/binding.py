@@ -18,6 +18,7 @@ STATUS_NAMES = {0: "VDN_OK", 1: "VDN_ERR_INVALID_ARG", 2: "VDN_ERR_UNSUPPORTED",
                 4: "VDN_ERR_CUDA", 5: "VDN_ERR_ARCH", 6: "VDN_ERR_TIMEOUT"}
 VDN_F32, VDN_BF16 = 0, 1
 VDN_FLAG_FORCE_SIMT = 1
+VDN_FLAG_ADDITIVE_RULE = 4
 VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_READ_BWD = range(7)
 
 EXPORTS = (

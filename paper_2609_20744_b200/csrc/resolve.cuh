@@ -91,6 +91,34 @@ __device__ __forceinline__ void store_split_tiles(const float (&m)[D / 16][D / 1
     }
 }
 
+// The transition of the additive baseline (Eq. 3c with the frame-size key scaling of Sec. 3.3): no inverse,
+//     C_t = I - sym(A_t) / F          (fp32, and/or its three-way bf16 split for the tensor-core scan)
+// taking the place of (I + A_t)^{-1} in the scan.  One CTA per frame.
+template <int D>
+__global__ void __launch_bounds__(256) additive_transition_kernel(const float* __restrict__ stats,
+                                                                  float* __restrict__ inv,
+                                                                  __nv_bfloat16* __restrict__ split,
+                                                                  long long nframes, float inv_f) {
+  const long long n = blockIdx.x;
+  if (n >= nframes) return;
+  const float* A = stats + (size_t)n * 2 * D * D;
+  for (int e = threadIdx.x; e < D * D; e += 256) {
+    const int i = e / D, j = e % D;
+    const float c = (i == j ? 1.0f : 0.0f) - 0.5f * (__ldg(A + e) + __ldg(A + (size_t)j * D + i)) * inv_f;
+    if (inv != nullptr) inv[(size_t)n * D * D + e] = c;
+    if (split != nullptr) {
+      __nv_bfloat16* S = split + (size_t)n * 3 * D * D;
+      const uint32_t u1 = __float_as_uint(c) & 0xFFFF0000u;
+      const float r1 = c - __uint_as_float(u1);
+      const uint32_t u2 = __float_as_uint(r1) & 0xFFFF0000u;
+      const uint32_t u3 = __float_as_uint(r1 - __uint_as_float(u2)) & 0xFFFF0000u;
+      S[e] = __ushort_as_bfloat16((unsigned short)(u1 >> 16));
+      S[(size_t)D * D + e] = __ushort_as_bfloat16((unsigned short)(u2 >> 16));
+      S[(size_t)2 * D * D + e] = __ushort_as_bfloat16((unsigned short)(u3 >> 16));
+    }
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict__ stats,
                                                           float* __restrict__ inv,

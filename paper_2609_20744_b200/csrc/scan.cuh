@@ -28,7 +28,8 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
                                                        const float* __restrict__ inv,
                                                        float* __restrict__ fwd, float* __restrict__ read,
                                                        int T, const float* __restrict__ alpha = nullptr,
-                                                       const float* __restrict__ s0 = nullptr, int H = 1) {
+                                                       const float* __restrict__ s0 = nullptr, int H = 1,
+                                                       float additive_bscale = 0.f) {
   constexpr int TI = D / 32;          // rows per thread
   constexpr int NCG = W / 4;          // column groups of 4
   static_assert(256 / NCG * TI == D, "thread tiling must cover D rows");
@@ -94,7 +95,10 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
         store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(p[r][0], p[r][1], p[r][2], p[r][3]));
     }
 
-    // X = alpha_t * Z + B_t^T (this CTA's columns)
+    // X = alpha_t * Z + B_t^T (this CTA's columns).  Additive baseline (additive_bscale > 0, Eq. 3c): the write is
+    // not resolved against the frame's keys, X = alpha_t * Z and Z_t = C_t X + B_t^T / sqrt(F), with C_t = I - A_t/F.
+    const bool additive = additive_bscale > 0.f;
+    float badd[TI][4];
     {
       // B_t is stored [d_v][d_k]: element (c, i) is B_t^T[i][c]
       const float* bsrc = stats + n * 2 * D * D + (size_t)(D + c0 + cc0) * D + i0;
@@ -111,17 +115,24 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
       }
 #pragma unroll
       for (int r = 0; r < TI; ++r)
+      {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          badd[r][c] = additive ? additive_bscale * bt[r][c] : 0.f;
+          if (additive) bt[r][c] = 0.f;
+        }
         store4(&sm.X[buf][i0 + r][cc0], make_float4(fmaf(al[r], z[r][0], bt[r][0]), fmaf(al[r], z[r][1], bt[r][1]),
                                                      fmaf(al[r], z[r][2], bt[r][2]), fmaf(al[r], z[r][3], bt[r][3])));
+      }
     }
     cp_async_wait<0>();
     __syncthreads();
 
-    // Z = C_t X
+    // Z = C_t X  (+ the unresolved write of the additive baseline)
 #pragma unroll
     for (int r = 0; r < TI; ++r)
 #pragma unroll
-      for (int c = 0; c < 4; ++c) z[r][c] = 0.f;
+      for (int c = 0; c < 4; ++c) z[r][c] = badd[r][c];
 #pragma unroll 8
     for (int j = 0; j < D; ++j) {
       float a[TI];

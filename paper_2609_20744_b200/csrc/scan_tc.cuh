@@ -42,7 +42,8 @@ struct ScanTc {
 __global__ void __launch_bounds__(ScanTc::THREADS, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict__ stats,
                __nv_bfloat16* __restrict__ pf, __nv_bfloat16* __restrict__ pb, int T,
-               const float* __restrict__ alpha, const float* __restrict__ s0, int H, int* status) {
+               const float* __restrict__ alpha, const float* __restrict__ s0, int H, float additive_bscale,
+               int* status) {
   using namespace tc;
   using S = ScanTc;
   constexpr int D = S::D;
@@ -172,21 +173,37 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     auto alpha_of = [&](int frame) {
       return alpha ? __ldg(alpha + (((size_t)(bh / H) * T + frame) * H + (bh % H)) * D + row) : 1.0f;
     };
+    // Additive baseline (additive_bscale = 1/sqrt(F) > 0; Eq. 3c with the key scaling of Sec. 3.3): the frame's
+    // write is not resolved against its keys,  Z_t = C_t (alpha_t * Z_{t-1}) + B_t^T / sqrt(F)  with
+    // C_t = I - A_t / F prepared by the host's choice of kernel; the same MMAs, the write added after them.
+    const bool additive = additive_bscale > 0.f;
+    const int lead = additive ? 0 : 1;       // bt holds B^T of frame_of(step + lead) when step's MMAs retire
     float bt[CW];
     load_bt(frame_of(0), bt);
     {
-      // the chain's first read slot holds the (bridged) initial state, and X_0 = alpha_0 * Z_init + B_0^T
+      // the chain's first read slot holds the (bridged) initial state, and X_0 = alpha_0 * Z_init (+ B_0^T)
       const float a0 = alpha_of(frame_of(0));
       __nv_bfloat16* z0 = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(0)) * (D * D) + (size_t)col0 * D + row;
+      if (additive) {
+        float x0[CW];
 #pragma unroll
-      for (int e = 0; e < CW; ++e) {
-        const float zi = s0 ? 0.5f * __ldg(s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
-        z0[(size_t)e * D] = __float2bfloat16_rn(a0 * zi);
-        bt[e] = fmaf(a0, zi, bt[e]);
+        for (int e = 0; e < CW; ++e) {
+          const float zi = s0 ? 0.5f * __ldg(s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
+          z0[(size_t)e * D] = __float2bfloat16_rn(a0 * zi);
+          x0[e] = a0 * zi;
+        }
+        publish_x(x0);
+      } else {
+#pragma unroll
+        for (int e = 0; e < CW; ++e) {
+          const float zi = s0 ? 0.5f * __ldg(s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
+          z0[(size_t)e * D] = __float2bfloat16_rn(a0 * zi);
+          bt[e] = fmaf(a0, zi, bt[e]);
+        }
+        publish_x(bt);
       }
     }
-    publish_x(bt);
-    if (T > 1) load_bt(frame_of(1), bt);
+    if (!additive && T > 1) load_bt(frame_of(1), bt);
     float a_next = T > 1 ? alpha_of(frame_of(1)) : 1.0f;
     for (int s = 0; s + 1 < T; ++s) {
       if (!mbar_wait(ACCFULL, s & 1, wc)) break;
@@ -194,10 +211,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
       float z[CW];
       tmem_ld32(taddr, z);
       tmem_wait_ld();
-      // first what the next MMAs are waiting for: X = Z + B^T of the next frame, split, into shared memory
-      if (s + 2 < T) {
+      if (additive) {
 #pragma unroll
-        for (int e = 0; e < CW; ++e) bt[e] = fmaf(a_next, z[e], bt[e]);
+        for (int e = 0; e < CW; ++e) z[e] = fmaf(additive_bscale, bt[e], z[e]);
+      }
+      // first what the next MMAs are waiting for: X = alpha * Z (+ B^T of the next frame), split, into shared memory
+      if (s + 2 < T) {                       // in place: bt is dead once it has been added
+#pragma unroll
+        for (int e = 0; e < CW; ++e) bt[e] = additive ? a_next * z[e] : fmaf(a_next, z[e], bt[e]);
         publish_x(bt);
       }
       // then, under the next step's MMAs: the state after step s is what the next frame in scan order reads.
@@ -210,8 +231,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
         dst[(size_t)e * D] = v2.x;
         dst[(size_t)(e + 1) * D] = v2.y;
       }
-      if (s + 2 < T) {                                 // B^T and decay of the frame after next, also under the MMAs
-        load_bt(frame_of(s + 2), bt);
+      if (s + 2 < T) {                                 // B^T and decay for the step after, also under the MMAs
+        load_bt(frame_of(s + 1 + lead), bt);
         a_next = alpha_of(frame_of(s + 2));
       }
     }

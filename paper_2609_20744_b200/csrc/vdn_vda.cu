@@ -6,6 +6,7 @@
 #include <cudaTypedefs.h>
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -214,10 +215,17 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
   vdn::gram_simt_kernel<Tio, D><<<dim3((unsigned)n, 2 * D / 64), 256, 0, st>>>(
       static_cast<const Tio*>(k), static_cast<const Tio*>(v), beta, stats, s);
   prof_mark(h, st, 0, "gram_simt");
-  vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n);
-  prof_mark(h, st, 1, "resolve");
+  const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
+  const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
+  if (additive) {
+    vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n, 1.0f / (float)s.F);
+    prof_mark(h, st, 1, "additive_transition");
+  } else {
+    vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n);
+    prof_mark(h, st, 1, "resolve");
+  }
   vdn::scan_kernel<D, 32><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
-      stats, inv, fwd, read, s.T, alpha, s0, s.H);
+      stats, inv, fwd, read, s.T, alpha, s0, s.H, bscale);
   prof_mark(h, st, 2, "scan");
   vdn::readout_simt_kernel<Tio, D><<<dim3((unsigned)n, (s.F + 63) / 64), 256, sizeof(vdn::ReadoutSimtSmem<D>), st>>>(
       static_cast<const Tio*>(q), read, gate, static_cast<Tio*>(out), s, h->cfg.rms_eps);
@@ -298,11 +306,18 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
                                                                                        h->status_dev);
   prof_mark(h, st, nk++, "gram_tc");
-  vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
-      stats, csplit, n, h->status_dev);
-  prof_mark(h, st, nk++, "resolve_tc");
+  const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
+  const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
+  if (additive) {
+    vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n, 1.0f / (float)s.F);
+    prof_mark(h, st, nk++, "additive_transition");
+  } else {
+    vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
+        stats, csplit, n, h->status_dev);
+    prof_mark(h, st, nk++, "resolve_tc");
+  }
   vdn::scan_tc_kernel<<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS, vdn::ScanTc::SMEM_BYTES, st>>>(
-      tmC, stats, pf, pb, s.T, alpha, s0, s.H, h->status_dev);
+      tmC, stats, pf, pb, s.T, alpha, s0, s.H, bscale, h->status_dev);
   prof_mark(h, st, nk++, "scan_tc");
   // The read-out streams reads and writes in equal parts and is fastest on about five SMs out of six
   // (measured on three workloads: 124 CTAs beat 148 by 5 %; fewer interleaved read/write streams at the DRAM).

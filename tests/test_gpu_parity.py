@@ -131,6 +131,33 @@ def test_forward_ex_single_frame_reads_the_text_state():
     assert torch.allclose(out[:, 0].float(), want, atol=3e-2, rtol=3e-2)
 
 
+# ------------------------------------------------------------------------------ the additive baseline (ablation)
+@pytest.mark.parametrize("dtype,d,flags,extras", [
+    ("f32", 64, 0, False), ("f32", 128, 0, True), ("bf16", 128, 0, False), ("bf16", 128, 0, True),
+    ("bf16", 128, binding.VDN_FLAG_FORCE_SIMT, True),
+])
+def test_additive_rule_matches_oracle(dtype, d, flags, extras):
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=1, H=2, T=6, F=200, seed=91)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda") if extras else (None, None)
+    vda = binding.Vda(w.d, w.dtype, flags=flags | binding.VDN_FLAG_ADDITIVE_RULE)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    for (b, h) in all_pairs(w):
+        q, k, v, beta, gate = inputs.head_slice(x, b, h)
+        a = None if alpha is None else alpha[b, :, h, :].double().cpu().numpy()
+        s = None if s0 is None else s0[b, h].double().cpu().numpy()
+        ref = orc.vda_slice(q, k, v, beta, gate, 1e-6, alpha=a, s0=s, rule="additive")["out"]
+        e = orc.slice_error(out[b, :, :, h, :].double().cpu().numpy(), ref)
+        assert e <= TOL[dtype], f"slice (b={b}, h={h}) error {e:.3e}"
+    # and it is not the joint solve
+    vda2 = binding.Vda(w.d, w.dtype, flags=flags)
+    out2 = vda2.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0)
+    torch.cuda.synchronize()
+    assert not torch.allclose(out.float(), out2.float(), atol=1e-2)
+
+
 def test_bf16_through_plain_fp32_kernels():
     w = inputs.TINY.scaled(dtype="bf16", d=128, T=4, F=200, H=2)
     x = inputs.generate(w, "cuda")
