@@ -60,3 +60,58 @@ def vda_bruteforce(q, k, v, beta, gate, eps, alpha=None, s0=None):
             ms = sum(x * x for x in o) / dv
             out[t, u] = gate * o / np.sqrt(ms + eps)
     return out, o_fwd, o_bwd
+
+
+def softmax_sees(t, j, T, chunk, radius, anchors):
+    """Sec. 2.1: is frame j visible to the Softmax branch of query frame t?  Frames are grouped into temporal
+    chunks of `chunk` frames from the start of the clip; a query chunk attends to itself and `radius` chunks on
+    either side; with boundary anchors every frame also attends to the first and the last frame and those two
+    attend to everything."""
+    if abs(t // chunk - j // chunk) <= radius:
+        return True
+    if anchors and (j in (0, T - 1) or t in (0, T - 1)):
+        return True
+    return False
+
+
+def vda_bruteforce_windowed(q, k, v, beta, gate, eps, alpha=None, s0=None, chunk=1, radius=0, anchors=False,
+                            norm_weight=None):
+    """The layer with chunk windows and boundary anchors, from the text of Sec. 2.1-2.2 and Sec. A.4.
+
+    For every query frame the two linear regions are whatever Softmax does not see, before and after the frame;
+    each is folded from the initial state in scan order, and the decay across the skipped local span is applied
+    by running the same frame update over that span with every write gate set to zero.  `gate` may be a scalar
+    or an array [T, U, dv]; `norm_weight` an optional [dv] vector.
+    """
+    T, U, dk = k.shape
+    dv = v.shape[2]
+    alpha = np.ones((T, dk)) if alpha is None else alpha
+    S_init = np.zeros((dv, dk)) if s0 is None else 0.5 * s0
+    gate = np.broadcast_to(np.asarray(gate, float), (T, U, dv))
+    w = np.ones(dv) if norm_weight is None else norm_weight
+    anchor_frames = (0, T - 1) if anchors else ()
+    interior = [j for j in range(T) if j not in anchor_frames]
+    out = np.zeros((T, U, dv))
+    o_fwd = np.zeros((T, U, dv))
+    o_bwd = np.zeros((T, U, dv))
+    no_write = np.zeros(U)
+    for t in interior:
+        far_before = [j for j in interior if j < t and not softmax_sees(t, j, T, chunk, radius, anchors)]
+        far_after = [j for j in interior if j > t and not softmax_sees(t, j, T, chunk, radius, anchors)]
+        near_before = [j for j in interior if j <= t and j not in far_before]       # skipped span, ends at t
+        near_after = [j for j in interior if j >= t and j not in far_after]         # skipped span, starts at t
+        S_f = state_after(far_before, k, v, beta, alpha, S_init)
+        for j in near_before:
+            S_f = lstsq_frame_update(S_f * alpha[j][None, :], k[j], v[j], no_write)
+        S_b = state_after(far_after[::-1], k, v, beta, alpha, S_init)
+        for j in near_after[::-1]:
+            S_b = lstsq_frame_update(S_b * alpha[j][None, :], k[j], v[j], no_write)
+        for u in range(U):
+            for c in range(dv):
+                o_fwd[t, u, c] = sum(S_f[c, j] * q[t, u, j] for j in range(dk))
+                o_bwd[t, u, c] = sum(S_b[c, j] * q[t, u, j] for j in range(dk))
+            o = o_fwd[t, u] + o_bwd[t, u]
+            ms = sum(x * x for x in o) / dv
+            for c in range(dv):
+                out[t, u, c] = gate[t, u, c] * w[c] * o[c] / np.sqrt(ms + eps)
+    return out, o_fwd, o_bwd

@@ -10,7 +10,7 @@ import numpy as np
 import pytest
 
 from oracle import vda_oracle as orc
-from tests.bruteforce import lstsq_frame_update, vda_bruteforce
+from tests.bruteforce import lstsq_frame_update, softmax_sees, vda_bruteforce, vda_bruteforce_windowed
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "worked_examples.json")
 
@@ -238,13 +238,15 @@ def test_repeated_key_closed_form_random():
     assert np.allclose(S @ k, want, atol=1e-13)
 
 
-@pytest.mark.parametrize("case", ["two_frames_whole_layer", "three_frames_decay_text"])
+@pytest.mark.parametrize("case", ["two_frames_whole_layer", "three_frames_decay_text",
+                                  "six_frames_chunk_window_anchors"])
 def test_golden_whole_layer(case):
     g = golden()[case]
     arr = lambda n: np.array(g[n], float)
     res = orc.vda_slice(arr("q"), arr("k"), arr("v"), arr("beta"), g["gate"], g["eps"],
                         alpha=arr("alpha") if "alpha" in g else None,
-                        s0=arr("s0") if "s0" in g else None, want=("P", "R", "O"))
+                        s0=arr("s0") if "s0" in g else None, want=("P", "R", "O"),
+                        chunk=g.get("chunk", 1), radius=g.get("radius", 0), anchors=g.get("anchors", False))
     assert np.allclose(res["P"], arr("P"), atol=1e-14)
     assert np.allclose(res["R"], arr("R"), atol=1e-14)
     if "O" in g:
@@ -372,6 +374,100 @@ def test_invariant_d_bruteforce_agreement(T, U, dk, dv, extras):
     assert np.allclose(res["o_fwd"], of, atol=1e-12)
     assert np.allclose(res["o_bwd"], ob, atol=1e-12)
     assert np.allclose(res["out"], out, atol=1e-11)
+
+
+# ---------------------------------------------------------------- chunk windows, anchors (Sec. 2.1, Sec. A.4)
+@pytest.mark.parametrize("T,chunk,radius,anchors", [
+    (6, 2, 0, True), (7, 2, 1, False), (11, 3, 1, True), (10, 5, 0, True), (9, 1, 1, False), (5, 1, 0, True),
+    (4, 5, 1, True), (3, 1, 0, True), (2, 1, 0, True), (12, 2, 2, True), (6, 1, 0, False)])
+def test_windowed_layer_matches_mask_driven_bruteforce(T, chunk, radius, anchors):
+    r = rng(2000 + 100 * T + 10 * chunk + radius)
+    U, dk, dv = 3, 4, 3
+    q, k, v, beta = random_slice(r, T, U, dk, dv)
+    alpha = r.uniform(0.2, 1, (T, dk))
+    s0 = r.standard_normal((dv, dk))
+    gate = r.uniform(0.1, 1, (T, U, dv))
+    w = r.uniform(0.5, 2, dv)
+    res = orc.vda_slice(q, k, v, beta, gate, 1e-6, alpha, s0, want=("o_fwd", "o_bwd"),
+                        chunk=chunk, radius=radius, anchors=anchors, norm_weight=w)
+    out, of, ob = vda_bruteforce_windowed(q, k, v, beta, gate, 1e-6, alpha, s0, chunk, radius, anchors, w)
+    assert np.allclose(res["o_fwd"], of, atol=1e-12)
+    assert np.allclose(res["o_bwd"], ob, atol=1e-12)
+    assert np.allclose(res["out"], out, atol=1e-11)
+    if anchors:
+        assert np.array_equal(res["out"][0], np.zeros((U, dv)))
+        assert np.array_equal(res["out"][T - 1], np.zeros((U, dv)))
+
+
+def test_window_bounds_are_the_clipped_chunk_neighbourhood():
+    for T, chunk, radius, anchors in [(12, 5, 1, True), (17, 5, 1, False), (9, 2, 0, True), (8, 3, 2, False)]:
+        first, last = orc.interior_range(T, anchors)
+        for t in range(first, last + 1):
+            lo, hi = orc.local_window(t, T, chunk, radius, anchors)
+            seen = [j for j in range(first, last + 1) if softmax_sees(t, j, T, chunk, radius, False)]
+            assert (lo, hi) == (seen[0], seen[-1]) and seen == list(range(lo, hi + 1))
+    # the 15-frame window of Sec. 2.1: chunk 5, radius 1, away from the ends of the clip
+    assert orc.local_window(52, 102, 5, 1, True) == (45, 59)
+    assert orc.local_window(3, 102, 5, 1, True) == (1, 9)
+    assert orc.local_window(99, 102, 5, 1, True) == (90, 100)
+
+
+def test_windowed_regions_are_disjoint_and_complete_by_linearity_in_values():
+    # Only frame j writes a value.  Queries of frame t see it through the forward state iff j lies before t's
+    # window, through the reverse state iff it lies after it, and not at all when Softmax sees it (inside the
+    # window, or an anchor): no frame is counted twice and none is lost (Sec. 2.2).
+    r = rng(2100)
+    T, U, d, chunk, radius = 11, 3, 4, 2, 1
+    q, k, v, beta = random_slice(r, T, U, d, d)
+    alpha = r.uniform(0.5, 1, (T, d))
+    for j in range(T):
+        v0 = np.zeros_like(v)
+        v0[j] = v[j]
+        res = orc.vda_slice(q, k, v0, beta, 1.0, 1e-6, alpha, want=("o_fwd", "o_bwd"),
+                            chunk=chunk, radius=radius, anchors=True)
+        for t in range(T):
+            f = np.abs(res["o_fwd"][t]).max() > 1e-9
+            b = np.abs(res["o_bwd"][t]).max() > 1e-9
+            linear = t not in (0, T - 1) and not softmax_sees(t, j, T, chunk, radius, True)
+            assert f == (linear and j < t)
+            assert b == (linear and j > t)
+
+
+def test_window_of_one_frame_without_anchors_is_the_default_layer():
+    r = rng(2200)
+    q, k, v, beta = random_slice(r, 5, 4, 4, 4)
+    alpha = r.uniform(0.2, 1, (5, 4))
+    a = orc.vda_slice(q, k, v, beta, 0.5, 1e-6, alpha)["out"]
+    b = orc.vda_slice(q, k, v, beta, 0.5, 1e-6, alpha, chunk=1, radius=0, anchors=False)["out"]
+    assert np.array_equal(a, b)
+
+
+def test_windowed_frame_reversal_swaps_directions():
+    # chunk grids line up under reversal when T is a multiple of the chunk length
+    r = rng(2300)
+    T, U, d = 8, 3, 4
+    q, k, v, beta = random_slice(r, T, U, d, d)
+    alpha = r.uniform(0.3, 1, (T, d))
+    s0 = r.standard_normal((d, d))
+    kw = dict(want=("o_fwd", "o_bwd"), chunk=2, radius=1, anchors=True)
+    a = orc.vda_slice(q, k, v, beta, 0.8, 1e-6, alpha, s0, **kw)
+    b = orc.vda_slice(q[::-1], k[::-1], v[::-1], beta[::-1], 0.8, 1e-6, alpha[::-1], s0, **kw)
+    assert np.allclose(a["o_fwd"], b["o_bwd"][::-1], atol=1e-13)
+    assert np.allclose(a["out"], b["out"][::-1], atol=1e-12)
+
+
+def test_elementwise_gate_and_norm_weight_literal():
+    # Eq. 1c with a content-dependent gate (one value per token and channel) and a per-channel norm scale
+    r = rng(2400)
+    O = r.standard_normal((2, 3, 5))
+    g = r.uniform(0, 1, (2, 3, 5))
+    w = r.uniform(0.5, 2, 5)
+    y = orc.rmsnorm_gate(O, g, 1e-3, w)
+    for t in range(2):
+        for u in range(3):
+            ms = sum(O[t, u, c] ** 2 for c in range(5)) / 5
+            for c in range(5):
+                assert abs(y[t, u, c] - g[t, u, c] * w[c] * O[t, u, c] / np.sqrt(ms + 1e-3)) < 1e-14
 
 
 def test_boundary_layout_wrapper_matches_slices():
