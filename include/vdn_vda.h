@@ -116,7 +116,8 @@ vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void
                            void* cuda_stream);
 
 /* The same layer with the two inputs of the paper's recurrence that vdn_vda_forward fixes (first item of the
- * "next" list; the local window is still the query frame itself, and there are no anchor frames):
+ * "next" list; the local window is still the query frame itself, and there are no anchor frames -- see
+ * vdn_vda_forward_opt for those):
  *   alpha [B,T,H,d] float, DEVICE, in [0,1], or NULL (= 1): channel-wise decay gate of frame t (Eq. 2, Eq. A.1:
  *         M_t = Diag(alpha_t)(I + A_t)^{-1}).  It decays the inherited state before frame t is folded in, in both
  *         scans, and bridges the state that frame t's queries read (Eq. A.4 with l_t = h_t = t):
@@ -127,6 +128,43 @@ vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void
 vdn_status vdn_vda_forward_ex(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
                               const float* gate, const float* alpha, const float* s0, void* out, int B, int T,
                               int F, int H, int d, void* cuda_stream);
+
+/* The layer with every optional input of the paper's linear branch (the "paper-faithful gather" and the
+ * content-dependent output gate).  `opt` may be NULL (= vdn_vda_forward).  Zero-initialise the struct, set
+ * struct_size, then the fields you need; all pointers are DEVICE pointers, 16-byte aligned, caller-owned.
+ *
+ *   alpha, s0    as for vdn_vda_forward_ex.
+ *   chunk, radius  the local Softmax window in temporal chunks (Sec. 2.1): latent frames are grouped into
+ *                chunks of `chunk` frames counted from frame 0 of the clip; a query frame's window [l_t, h_t]
+ *                is its own chunk and `radius` chunks on either side, clipped to the scanned frames.  Its
+ *                queries read (Eq. A.4)
+ *                    P_{l_t - 1} Diag(prod_{r=l_t..t} alpha_r)  +  R_{h_t + 1} Diag(prod_{r=t..h_t} alpha_r),
+ *                the forward state of the frames before the window and the reverse state of the frames after
+ *                it, each bridged by the decay of the skipped span; a side with no distant frame reads S_T / 2.
+ *                chunk <= 1 and radius = 0 give the window {t} of vdn_vda_forward.  The paper's release uses
+ *                chunk = 5, radius = 1 (a 15-frame window).
+ *   anchors      non-zero: frames 0 and T-1 are boundary anchors (Sec. 2.1): they belong to Softmax alone, are
+ *                excluded from both scans (Alg. 1 step 2), and their output rows are zero (Alg. 1 step 7).
+ *                A clip of at most two frames then has no linear output at all (Sec. A.4).
+ *   gate_elem    [B,T,F,H,d] of cfg.io_dtype or NULL: element-wise output gate G^L of Eq. 1c, already through the
+ *                sigmoid.  It multiplies the per-head `gate`, which may then be NULL (= 1).
+ *   norm_weight  [H,d] float or NULL (= 1): per-channel scale of the RMSNorm in Eq. 1c, applied after the
+ *                normalisation: out = gate_h * gate_elem * norm_weight * o / sqrt(mean_j o_j^2 + rms_eps).
+ * When a window covers every scanned frame both sides read S_T / 2 (Eq. A.4 as written); bypassing the linear
+ * branch for such clips (Sec. A.4) is the caller's decision. */
+typedef struct {
+  uint32_t struct_size;     /* sizeof(vdn_vda_options), checked */
+  int32_t chunk;            /* frames per temporal chunk; 0 is read as 1 */
+  int32_t radius;           /* chunks on either side of the query chunk inside the window, >= 0 */
+  int32_t anchors;          /* boolean */
+  const float* alpha;
+  const float* s0;
+  const void* gate_elem;
+  const float* norm_weight;
+} vdn_vda_options;
+vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                               const float* gate, void* out, int B, int T, int F, int H, int d,
+                               const vdn_vda_options* opt, void* cuda_stream);
 
 /* The same layer for callers whose tensors live in HOST memory (pinned memory recommended): copies
  * q, k, v, beta, gate to the staging buffer, runs vdn_vda_forward, copies `out` back, all on

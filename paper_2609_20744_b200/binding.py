@@ -23,6 +23,7 @@ VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_R
 
 EXPORTS = (
     "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward", "vdn_vda_forward_ex",
+    "vdn_vda_forward_opt",
     "vdn_vda_staging_bytes", "vdn_vda_set_staging", "vdn_vda_forward_host", "vdn_vda_workspace_view",
     "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_scan_static", "vdn_vda_status", "vdn_vda_last_error", "vdn_vda_destroy",
 )
@@ -31,6 +32,12 @@ EXPORTS = (
 class VdnConfig(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("io_dtype", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("rms_eps", ctypes.c_float), ("flags", ctypes.c_uint32), ("device", ctypes.c_int32)]
+
+
+class VdnOptions(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("chunk", ctypes.c_int32), ("radius", ctypes.c_int32),
+                ("anchors", ctypes.c_int32), ("alpha", ctypes.c_void_p), ("s0", ctypes.c_void_p),
+                ("gate_elem", ctypes.c_void_p), ("norm_weight", ctypes.c_void_p)]
 
 
 class VdnError(RuntimeError):
@@ -69,6 +76,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.vdn_vda_forward.restype = ci
     lib.vdn_vda_forward_ex.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, *shape, vp]
     lib.vdn_vda_forward_ex.restype = ci
+    lib.vdn_vda_forward_opt.argtypes = [vp, vp, vp, vp, vp, vp, vp, *shape, ctypes.POINTER(VdnOptions), vp]
+    lib.vdn_vda_forward_opt.restype = ci
     lib.vdn_vda_forward_host.argtypes = fwd_args
     lib.vdn_vda_forward_host.restype = ci
     lib.vdn_vda_workspace_view.argtypes = [vp, ci, *shape, ctypes.POINTER(sz), ctypes.POINTER(sz)]
@@ -176,29 +185,44 @@ class Vda:
         return self._staging
 
     # -- the two entry points -----------------------------------------------------------------
-    def forward(self, q, k, v, beta, gate, out=None, stream=None, alpha=None, s0=None):
+    def forward(self, q, k, v, beta, gate, out=None, stream=None, alpha=None, s0=None,
+                chunk=1, radius=0, anchors=False, gate_elem=None, norm_weight=None):
         """vdn_vda_forward on device tensors q,k,v [B,T,F,H,d], beta [B,T,F,H], gate [H].
 
-        With alpha [B,T,H,d] (decay gates) and/or s0 [B,H,d,d] (text state) the call goes to vdn_vda_forward_ex.
+        With alpha [B,T,H,d] (decay gates) and/or s0 [B,H,d,d] (text state) the call goes to vdn_vda_forward_ex;
+        with a chunk window (chunk, radius), boundary anchors, an element-wise gate gate_elem [B,T,F,H,d] (then
+        `gate` may be None) or a norm weight norm_weight [H,d] it goes to vdn_vda_forward_opt.
         """
         torch = self._torch
         B, T, F, H, d = q.shape
-        extras = [x for x in (alpha, s0) if x is not None]
-        for x in (q, k, v, beta, gate, *extras):
+        extras = [x for x in (alpha, s0, norm_weight) if x is not None]
+        for x in (q, k, v, beta, *([gate] if gate is not None else []), *([gate_elem] if gate_elem is not None else []),
+                  *extras):
             if not (x.is_cuda and x.is_contiguous()):
                 raise ValueError("vdn_vda_forward needs contiguous CUDA tensors")
         for x in extras:
             if x.dtype != torch.float32:
-                raise ValueError("alpha and s0 must be float32")
+                raise ValueError("alpha, s0 and norm_weight must be float32")
         if alpha is not None and tuple(alpha.shape) != (B, T, H, d):
             raise ValueError("alpha must be [B, T, H, d]")
         if s0 is not None and tuple(s0.shape) != (B, H, d, d):
             raise ValueError("s0 must be [B, H, d, d]")
+        if norm_weight is not None and tuple(norm_weight.shape) != (H, d):
+            raise ValueError("norm_weight must be [H, d]")
+        if gate_elem is not None and (tuple(gate_elem.shape) != (B, T, F, H, d) or gate_elem.dtype != q.dtype):
+            raise ValueError("gate_elem must be [B, T, F, H, d] of the I/O dtype")
         if out is None:
             out = torch.empty_like(q)
         self.ensure_workspace(B, T, F, H)
         p = lambda x: ctypes.c_void_p(x.data_ptr()) if x is not None else None
-        if extras:
+        a = lambda x: x.data_ptr() if x is not None else None
+        if (chunk, radius, bool(anchors)) != (1, 0, False) or gate_elem is not None or norm_weight is not None \
+                or gate is None:
+            opt = VdnOptions(ctypes.sizeof(VdnOptions), chunk, radius, 1 if anchors else 0, a(alpha), a(s0),
+                             a(gate_elem), a(norm_weight))
+            st = self.lib.vdn_vda_forward_opt(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
+                                              B, T, F, H, d, ctypes.byref(opt), self._stream(stream))
+        elif alpha is not None or s0 is not None:
             st = self.lib.vdn_vda_forward_ex(self.h, p(q), p(k), p(v), p(beta), p(gate), p(alpha), p(s0), p(out),
                                              B, T, F, H, d, self._stream(stream))
         else:

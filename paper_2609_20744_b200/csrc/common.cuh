@@ -7,9 +7,29 @@
 namespace vdn {
 
 // Problem shape in the library's naming: T latent frames of F tokens, H heads, d = d_k = d_v.
+// t0 / Tn: the frames the linear branch works on, t0 .. t0+Tn-1 (all T frames, or the interior frames when the
+// first and the last frame are boundary anchors, Sec. A.4).  Workspace indices always count all T frames.
 struct Shape {
   int B, T, F, H, d;
-  __host__ __device__ long long frames() const { return (long long)B * H * T; }  // (b,h,t) triples
+  int t0, Tn;
+  __host__ __device__ long long frames() const { return (long long)B * H * T; }       // (b,h,t) triples
+  __host__ __device__ long long work_items() const { return (long long)B * H * Tn; }  // ... that are worked on
+};
+
+// Local window of a query frame in temporal chunks (Sec. 2.1), clipped to the scanned frames first..last
+// (Sec. A.4): chunks of `chunk` frames counted from frame 0 of the clip, `radius` chunks on either side.
+// chunk = 1, radius = 0 is the window {t}.
+struct Window {
+  int chunk, radius, first, last;
+  __host__ __device__ int lo(int t) const {
+    const int x = (t / chunk - radius) * chunk;
+    return x > first ? x : first;
+  }
+  __host__ __device__ int hi(int t) const {
+    const int x = (t / chunk + radius + 1) * chunk - 1;
+    return x < last ? x : last;
+  }
+  __host__ __device__ int span() const { return (radius + 1) * chunk; }   // frames from a window end to its query chunk's far end
 };
 
 // Element offset of token (b,t,u), head h in a [B,T,F,H,d] tensor.
@@ -25,15 +45,15 @@ __device__ __forceinline__ void split_frame(const Shape& s, long long n, int& b,
   b = (int)(bh / s.H);
 }
 
-// Work order of the persistent tensor-core kernels: work item w -> (b, t, h) with the head fastest, so
+// Work order of the persistent tensor-core kernels: work item w (of s.work_items()) -> (b, t, h) with the head fastest, so
 // that CTAs running side by side stream the same token rows (a token's H heads are contiguous in memory:
 // neighbouring 256-byte pieces of one DRAM page, and shared 32-byte sectors of beta).  Returns the frame
 // index n = (b*H + h)*T + t that addresses the workspace.
 __device__ __forceinline__ long long split_work(const Shape& s, long long w, int& b, int& h, int& t) {
   h = (int)(w % s.H);
   long long bt = w / s.H;
-  t = (int)(bt % s.T);
-  b = (int)(bt / s.T);
+  t = s.t0 + (int)(bt % s.Tn);
+  b = (int)(bt / s.Tn);
   return ((long long)b * s.H + h) * s.T + t;
 }
 

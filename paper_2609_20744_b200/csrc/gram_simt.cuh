@@ -23,6 +23,7 @@ __global__ void __launch_bounds__(256) gram_simt_kernel(const Tio* __restrict__ 
   const int cb = blockIdx.y;                    // column block: cols [cb*64, cb*64+64) of [K|V]
   int b, h, t;
   split_frame(s, n, b, h, t);
+  if (t < s.t0 || t >= s.t0 + s.Tn) return;     // an anchor frame: not scanned
   const Tio* wsrc = (cb * CB < D) ? k : v;
   const int wcol0 = (cb * CB) % D;
 

@@ -67,7 +67,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ntiles = (s.F + G::TILE - 1) / G::TILE;
-  const long long nitems = s.frames();
+  const long long nitems = s.work_items();
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 3; ++i) { mbar_init(FULL(i), 1); mbar_init(EMPTY(i), 1); }

@@ -18,7 +18,9 @@ template <typename Tio, int D>
 __global__ void __launch_bounds__(256) readout_simt_kernel(const Tio* __restrict__ q,
                                                             const float* __restrict__ read,
                                                             const float* __restrict__ gate,
-                                                            Tio* __restrict__ out, Shape s, float eps) {
+                                                            Tio* __restrict__ out, Shape s, float eps,
+                                                            const Tio* __restrict__ gate_elem,
+                                                            const float* __restrict__ norm_weight) {
   constexpr int TU = 64;
   constexpr int DC = D / 16;   // output channels per thread
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -28,6 +30,7 @@ __global__ void __launch_bounds__(256) readout_simt_kernel(const Tio* __restrict
   const int u0 = blockIdx.y * TU;
   int b, h, t;
   split_frame(s, n, b, h, t);
+  if (t < s.t0 || t >= s.t0 + s.Tn) return;     // an anchor frame: its output rows are zeroed by the host
   const int tid = threadIdx.x;
 
   {
@@ -70,7 +73,11 @@ __global__ void __launch_bounds__(256) readout_simt_kernel(const Tio* __restrict
       for (int c = 0; c < DC; ++c) acc[r][c] = fmaf(qa[r], zc[c], acc[r][c]);
   }
 
-  const float g = gate[h];
+  // Eq. 1c: per-head gate (null = 1), optional element-wise gate [B,T,F,H,d] and per-channel norm scale [H,d]
+  const float g = gate ? gate[h] : 1.0f;
+  float wn[DC];
+#pragma unroll
+  for (int c = 0; c < DC; ++c) wn[c] = norm_weight ? norm_weight[(size_t)h * D + tc * DC + c] : 1.0f;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
     float ss = 0.f;
@@ -81,11 +88,15 @@ __global__ void __launch_bounds__(256) readout_simt_kernel(const Tio* __restrict
     const float scale = g * rsqrtf(ss * (1.0f / D) + eps);
     const int u = u0 + tu * 4 + r;
     if (u < s.F) {
-      Tio* dst = out + token_offset(s, b, t, u, h) + tc * DC;
+      const size_t off = token_offset(s, b, t, u, h) + tc * DC;
+      Tio* dst = out + off;
 #pragma unroll
-      for (int c = 0; c < DC; c += 4)
-        store4(dst + c, make_float4(acc[r][c] * scale, acc[r][c + 1] * scale, acc[r][c + 2] * scale,
-                                    acc[r][c + 3] * scale));
+      for (int c = 0; c < DC; c += 4) {
+        float4 ge = make_float4(1.f, 1.f, 1.f, 1.f);
+        if (gate_elem) ge = load4(gate_elem + off + c);
+        store4(dst + c, make_float4(acc[r][c] * scale * wn[c] * ge.x, acc[r][c + 1] * scale * wn[c + 1] * ge.y,
+                                    acc[r][c + 2] * scale * wn[c + 2] * ge.z, acc[r][c + 3] * scale * wn[c + 3] * ge.w));
+      }
     }
   }
 }

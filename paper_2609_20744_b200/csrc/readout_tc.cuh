@@ -35,10 +35,14 @@ struct ReadoutTc {
   static constexpr int THREADS = 192;
 };
 
+// EXTRAS = true adds the two optional factors of Eq. 1c to the epilogue: an element-wise (content-dependent) gate
+// gate_elem [B,T,F,H,d] bf16 and a per-channel norm scale norm_weight [H,d]; either may be null, and so may the
+// per-head gate (read as 1).  The plain instantiation carries none of that code.
+template <bool EXTRAS>
 __global__ void __launch_bounds__(ReadoutTc::THREADS, 1)
 readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmS,
                   const __grid_constant__ CUtensorMap tmO, const float* __restrict__ gate, Shape s, float eps,
-                  int* status) {
+                  int* status, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight) {
   using namespace tc;
   using R = ReadoutTc;
   extern __shared__ unsigned char smem_dyn[];
@@ -58,7 +62,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ntiles = (s.F + R::TILE - 1) / R::TILE;
-  const long long nitems = s.frames();
+  const long long nitems = s.work_items();
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 3; ++i) { mbar_init(QFULL(i), 1); mbar_init(QEMPTY(i), 1); }
@@ -90,11 +94,12 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!mbar_wait(STEMPTY(0), (si & 1) ^ 1, wc)) { ok = false; break; }
         mbar_arrive_expect_tx(STFULL(0), 2 * R::TILE_BYTES);
         const uint32_t sdst = base + R::OFF_STATE;
-        // rows [n*128, +128) hold the forward state, rows [(nitems+n)*128, +128) the reverse state
+        // rows [n*128, +128) hold the forward state, rows [(frames+n)*128, +128) the reverse state
+        const long long nrev = s.frames() + n;
         tma_load_2d(sdst, &tmS, STFULL(0), 0, (int)(n * R::D));
         tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(n * R::D));
-        tma_load_2d(sdst + 2 * R::BOX_BYTES, &tmS, STFULL(0), 0, (int)((nitems + n) * R::D));
-        tma_load_2d(sdst + 3 * R::BOX_BYTES, &tmS, STFULL(0), 64, (int)((nitems + n) * R::D));
+        tma_load_2d(sdst + 2 * R::BOX_BYTES, &tmS, STFULL(0), 0, (int)(nrev * R::D));
+        tma_load_2d(sdst + 3 * R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(nrev * R::D));
         for (int tile = 0; tile < ntiles; ++tile, ++qi) {
           const int st = qi % R::QSTAGES;
           if (!mbar_wait(QEMPTY(st), ((qi / R::QSTAGES) & 1) ^ 1, wc)) { ok = false; break; }
@@ -152,9 +157,21 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
       int b, h, t;
       split_work(s, item, b, h, t);
-      const float g = __ldg(gate + h);
+      const float g = (!EXTRAS || gate) ? __ldg(gate + h) : 1.0f;
       for (int tile = 0; tile < ntiles; ++tile, ++qi) {
         const int a = qi & 3;
+        // the token's 128 gate values (256 contiguous bytes), requested before the accumulator is waited for
+        uint4 graw[EXTRAS ? 16 : 1];
+        bool has_ge = false;
+        if constexpr (EXTRAS) {
+          const int u = tile * R::TILE + row;
+          has_ge = gate_elem != nullptr && u < s.F;
+          if (has_ge) {
+            const uint4* gp = reinterpret_cast<const uint4*>(gate_elem + token_offset(s, b, t, u, h));
+#pragma unroll
+            for (int j = 0; j < 16; ++j) graw[j] = __ldg(gp + j);
+          }
+        }
         if (!mbar_wait(ACCFULL(a), (qi >> 2) & 1, wc)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 128;
@@ -173,6 +190,33 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
           for (int e = 0; e < 32; ++e) ss = fmaf(v[c][e], v[c][e], ss);
         const float scale = g * rsqrtf(ss * (1.0f / R::D) + eps);
+        if constexpr (EXTRAS) {
+          // v <- v * norm_weight[c] * gate_elem[c]; the common factor `scale` is applied while packing
+          if (norm_weight != nullptr) {
+            const float4* wp = reinterpret_cast<const float4*>(norm_weight + (size_t)h * R::D);
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+              for (int e = 0; e < 32; e += 4) {
+                const float4 w4 = __ldg(wp + c * 8 + (e >> 2));
+                v[c][e] *= w4.x; v[c][e + 1] *= w4.y; v[c][e + 2] *= w4.z; v[c][e + 3] *= w4.w;
+              }
+          }
+          if (has_ge) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const __nv_bfloat162* gp2 = reinterpret_cast<const __nv_bfloat162*>(&graw[c * 4 + j]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float2 gf = __bfloat1622float2(gp2[e]);
+                  v[c][j * 8 + 2 * e] *= gf.x;
+                  v[c][j * 8 + 2 * e + 1] *= gf.y;
+                }
+              }
+          }
+        }
 
         const int ob = qi & 1;
         if (et == 0) tma_store_wait_read<1>();   // the store that last used this staging tile has read it

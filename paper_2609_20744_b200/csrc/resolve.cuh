@@ -98,9 +98,10 @@ template <int D>
 __global__ void __launch_bounds__(256) additive_transition_kernel(const float* __restrict__ stats,
                                                                   float* __restrict__ inv,
                                                                   __nv_bfloat16* __restrict__ split,
-                                                                  long long nframes, float inv_f) {
+                                                                  long long nframes, float inv_f, Shape shp) {
   const long long n = blockIdx.x;
   if (n >= nframes) return;
+  if ((int)(n % shp.T) < shp.t0 || (int)(n % shp.T) >= shp.t0 + shp.Tn) return;   // an anchor frame: not scanned
   const float* A = stats + (size_t)n * 2 * D * D;
   for (int e = threadIdx.x; e < D * D; e += 256) {
     const int i = e / D, j = e % D;
@@ -122,13 +123,15 @@ __global__ void __launch_bounds__(256) additive_transition_kernel(const float* _
 template <int D>
 __global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict__ stats,
                                                           float* __restrict__ inv,
-                                                          __nv_bfloat16* __restrict__ split, long long nframes) {
+                                                          __nv_bfloat16* __restrict__ split, long long nframes,
+                                                          Shape shp) {
   constexpr int R = D / 16;
   __shared__ __align__(16) float rowbuf[2 * D];
   __shared__ __align__(16) float colbuf[2 * D];
 
   const long long n = blockIdx.x;
   if (n >= nframes) return;
+  if ((int)(n % shp.T) < shp.t0 || (int)(n % shp.T) >= shp.t0 + shp.Tn) return;   // an anchor frame: not scanned
   const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
   const float* A = stats + (size_t)n * 2 * D * D;   // first d rows of the frame's [2d][d] block
 

@@ -48,7 +48,7 @@ struct ResolveTc {
 
 __global__ void __launch_bounds__(ResolveTc::THREADS, 3)
 resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ csplit, long long nframes,
-                  int* status) {
+                  int* status, Shape shp) {
   using namespace tc;
   using R = ResolveTc;
   constexpr int D = R::D;
@@ -64,6 +64,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long n = blockIdx.x;
   if (n >= nframes) return;
+  if ((int)(n % shp.T) < shp.t0 || (int)(n % shp.T) >= shp.t0 + shp.Tn) return;   // an anchor frame: not scanned
 
   if (threadIdx.x == 0) {
     mbar_init(OPREADY, 128);

@@ -5,10 +5,12 @@
 // of Z evolve independently: one CTA owns W columns of one (batch, head) chain, keeps them in
 // registers for the whole clip and needs no communication with the CTAs that own the other columns.
 //
-// Pass 1 (t = 0..T-1) stores P_t^T.  Pass 2 (t = T-1..0) carries R_{t+1}^T, first emits the state the
-// queries of frame t read,  P_{t-1}^T + R_{t+1}^T  (the initial state where a side is missing), then folds
-// frame t in.  Both passes are written back by the very thread that
-// computed them, so the second pass needs no inter-CTA ordering.
+// Pass 1 (the scanned frames first..last in order) stores P_t^T.  Pass 2 (last..first) carries R_{t+1}^T and, before
+// it folds frame t in, emits the state read by every query frame whose local window [l, h] ends at h = t (Eq. A.4):
+//     P_{l-1}^T bridged by prod_{r=l..q} alpha_r  +  R_{t+1}^T bridged by prod_{r=q..t} alpha_r
+// (the initial state where a side has no distant frame; with the default window {t} this is
+// alpha_t (P_{t-1} + R_{t+1})^T).  Both passes are written back by the very thread that computed them, so the
+// second pass needs no inter-CTA ordering.
 //
 // C_t is symmetric; the kernel reads it as C_t[j][i] so that each thread's row group is contiguous.
 #pragma once
@@ -27,9 +29,9 @@ template <int D, int W>
 __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ stats,
                                                        const float* __restrict__ inv,
                                                        float* __restrict__ fwd, float* __restrict__ read,
-                                                       int T, const float* __restrict__ alpha = nullptr,
-                                                       const float* __restrict__ s0 = nullptr, int H = 1,
-                                                       float additive_bscale = 0.f) {
+                                                       int T, const float* __restrict__ alpha,
+                                                       const float* __restrict__ s0, int H,
+                                                       float additive_bscale, Window win) {
   constexpr int TI = D / 32;          // rows per thread
   constexpr int NCG = W / 4;          // column groups of 4
   static_assert(256 / NCG * TI == D, "thread tiling must cover D rows");
@@ -64,9 +66,10 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
     for (int c = 0; c < 4; ++c) z[r][c] = zinit[r][c];
 
   int buf = 0;
-  for (int step = 0; step < 2 * T; ++step) {
-    const bool forward = step < T;
-    const int t = forward ? step : (2 * T - 1 - step);
+  const int Tn = win.last - win.first + 1;
+  for (int step = 0; step < 2 * Tn; ++step) {
+    const bool forward = step < Tn;
+    const int t = forward ? win.first + step : win.last - (step - Tn);
     const size_t n = (size_t)bh * T + t;
 
     // C_t -> shared memory (asynchronously, 16 bytes per request)
@@ -79,20 +82,32 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
 
     float al[TI];
     alpha_of(t, al);
-    if (!forward) {
-      // gather: the state read by frame t's queries, bridged by frame t's decay
-      float p[TI][4];
+    if (!forward && (t == win.last || (t + 1) % win.chunk == 0)) {
+      // gather: the query frames whose window ends at t read the reverse state carried here
+      for (int qf = max(win.first, t - win.span()); qf <= t; ++qf) {
+        if (win.hi(qf) != t) continue;
+        const int l = win.lo(qf);
+        float af[TI], ab[TI], ar[TI];
 #pragma unroll
-      for (int r = 0; r < TI; ++r) {
-        float4 x = make_float4(zinit[r][0], zinit[r][1], zinit[r][2], zinit[r][3]);
-        if (t > 0) x = load4(fwd + (n - 1) * D * D + (size_t)(i0 + r) * D + c0 + cc0);
-        p[r][0] = al[r] * (x.x + z[r][0]); p[r][1] = al[r] * (x.y + z[r][1]);
-        p[r][2] = al[r] * (x.z + z[r][2]); p[r][3] = al[r] * (x.w + z[r][3]);
+        for (int r = 0; r < TI; ++r) af[r] = ab[r] = 1.0f;
+        for (int fr = l; fr <= t; ++fr) {
+          alpha_of(fr, ar);
+#pragma unroll
+          for (int r = 0; r < TI; ++r) {
+            if (fr <= qf) af[r] *= ar[r];
+            if (fr >= qf) ab[r] *= ar[r];
+          }
+        }
+        float* dst = read + ((size_t)bh * T + qf) * D * D;
+#pragma unroll
+        for (int r = 0; r < TI; ++r) {
+          float4 x = make_float4(zinit[r][0], zinit[r][1], zinit[r][2], zinit[r][3]);
+          if (l > win.first) x = load4(fwd + ((size_t)bh * T + l - 1) * D * D + (size_t)(i0 + r) * D + c0 + cc0);
+          store4(dst + (size_t)(i0 + r) * D + c0 + cc0,
+                 make_float4(fmaf(af[r], x.x, ab[r] * z[r][0]), fmaf(af[r], x.y, ab[r] * z[r][1]),
+                             fmaf(af[r], x.z, ab[r] * z[r][2]), fmaf(af[r], x.w, ab[r] * z[r][3])));
+        }
       }
-      float* dst = read + n * D * D;
-#pragma unroll
-      for (int r = 0; r < TI; ++r)
-        store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(p[r][0], p[r][1], p[r][2], p[r][3]));
     }
 
     // X = alpha_t * Z + B_t^T (this CTA's columns).  Additive baseline (additive_bscale > 0, Eq. 3c): the write is
@@ -161,7 +176,7 @@ __global__ void __launch_bounds__(256, 2) scan_kernel(const float* __restrict__ 
       for (int r = 0; r < TI; ++r)
         store4(dst + (size_t)(i0 + r) * D + c0 + cc0, make_float4(z[r][0], z[r][1], z[r][2], z[r][3]));
     }
-    if (step == T - 1) {
+    if (step == Tn - 1) {
       // the reverse scan starts from the initial state as well
 #pragma unroll
       for (int r = 0; r < TI; ++r)

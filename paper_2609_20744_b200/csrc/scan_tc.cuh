@@ -16,9 +16,14 @@
 // the next frame's B^T, split the sum and write the three parts to shared memory as the next MN-major B
 // operand.  The next frame's B^T row is fetched into registers while the MMAs run.
 //
-// Gather (Eq. A.4 with the window shrunk to the query frame): the forward chain stores P_t in slot t+1 of
-// `pf`, the reverse chain stores R_t in slot t-1 of `pb`, each already bridged by the reading frame's decay; slot 0
-// of pf and slot T-1 of pb receive the initial state (zero unless a text state is passed).  The read-out kernel adds the two in its accumulator (Eq. 1a).
+// Gather (Eq. A.4).  A chain covers the scanned frames win.first .. win.last (all frames, or the interior ones when
+// the clip has boundary anchors).  Slot t of `pf` is what query frame t reads from the forward scan,
+// P_{l_t - 1} Diag(prod_{r=l_t..t} alpha_r), slot t of `pb` what it reads from the reverse scan,
+// R_{h_t + 1} Diag(prod_{r=t..h_t} alpha_r), [l_t, h_t] being the frame's local window: whenever a chain reaches a
+// state that some frames read, it writes those frames' slots, bridged by their decay (with the default window
+// {t} that is one slot per step: P_t into slot t+1, R_t into slot t-1).  Frames whose window leaves no distant
+// frame on a side read the initial state (zero unless a text state is passed).  A chain stops after the last
+// state that anybody reads.  The read-out kernel adds the two slots in its accumulator (Eq. 1a).
 #pragma once
 #include <cuda_bf16.h>
 
@@ -43,7 +48,7 @@ __global__ void __launch_bounds__(ScanTc::THREADS, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict__ stats,
                __nv_bfloat16* __restrict__ pf, __nv_bfloat16* __restrict__ pb, int T,
                const float* __restrict__ alpha, const float* __restrict__ s0, int H, float additive_bscale,
-               int* status) {
+               int* status, Window win) {
   using namespace tc;
   using S = ScanTc;
   constexpr int D = S::D;
@@ -61,7 +66,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int bh = blockIdx.x >> 1, dir = blockIdx.x & 1;
-  auto frame_of = [&](int s) { return dir == 0 ? s : T - 1 - s; };   // frame folded in at scan step s
+  auto frame_of = [&](int s) { return dir == 0 ? win.first + s : win.last - s; };   // frame folded in at scan step s
+  // steps this chain runs: up to the last state that some frame reads (P_{l-1} of the last frame's window,
+  // R_{h+1} of the first frame's)
+  const int nfold = dir == 0 ? win.lo(win.last) - win.first : win.last - win.hi(win.first);
 
   if (threadIdx.x == 0) {
     for (int p = 0; p < 3; ++p) { mbar_init(CFULL(p), 1); mbar_init(CFREE(p), 1); }
@@ -87,7 +95,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     // of this step's MMA time plus the state warps' turn to arrive.
     if (lane == 0) {
       bool ok = true;
-      for (int s = 0; s + 1 < T && ok; ++s) {     // the last frame of a chain is never folded in: nobody reads it
+      for (int s = 0; s < nfold && ok; ++s) {
         const long long n = (long long)bh * T + frame_of(s);
 #pragma unroll
         for (int p = 2; p >= 0; --p) {
@@ -105,7 +113,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
       bool ok = true;
-      for (int s = 0; s + 1 < T && ok; ++s) {
+      for (int s = 0; s < nfold && ok; ++s) {
         if (!mbar_wait(XREADY, s & 1, wc)) break;
         tc_fence_after_sync();
         // C3 X1, then C2 (X2, X1), then C1 (X3, X2, X1): smallest contributions first
@@ -178,34 +186,55 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     // C_t = I - A_t / F prepared by the host's choice of kernel; the same MMAs, the write added after them.
     const bool additive = additive_bscale > 0.f;
     const int lead = additive ? 0 : 1;       // bt holds B^T of frame_of(step + lead) when step's MMAs retire
+
+    // Gather: `z` is the state that the frames t with l_t = bound (forward chain) / h_t = bound (reverse chain)
+    // read; write their slots, each bridged by the decay of the frames between the state and the query
+    // (Eq. A.4).  Readers are visited walking away from the state, so the bridge is a running product.
+    auto store_readers = [&](int bound, const float (&z)[CW]) {
+      __nv_bfloat16* slots = (dir == 0 ? pf : pb) + (size_t)bh * T * (D * D) + (size_t)col0 * D + row;
+      float bridge = 1.0f;
+      int r = bound;                           // next frame whose decay enters the bridge
+      // only a chunk edge (or the end of the scanned range) is the end of anybody's window
+      if (dir == 0 ? (bound != win.first && bound % win.chunk != 0) : (bound != win.last && (bound + 1) % win.chunk != 0))
+        return;
+      const int far = dir == 0 ? min(win.last, bound + win.span()) : max(win.first, bound - win.span());
+      for (int t = bound; dir == 0 ? t <= far : t >= far; t += dir == 0 ? 1 : -1) {
+        if ((dir == 0 ? win.lo(t) : win.hi(t)) != bound) continue;
+        for (; dir == 0 ? r <= t : r >= t; r += dir == 0 ? 1 : -1) bridge *= alpha_of(r);
+        __nv_bfloat16* dst = slots + (size_t)t * (D * D);
+#pragma unroll
+        for (int e = 0; e < CW; e += 2) {
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(bridge * z[e], bridge * z[e + 1]);
+          dst[(size_t)e * D] = v2.x;
+          dst[(size_t)(e + 1) * D] = v2.y;
+        }
+      }
+    };
+
     float bt[CW];
-    load_bt(frame_of(0), bt);
+    if (nfold > 0) load_bt(frame_of(0), bt);
     {
-      // the chain's first read slot holds the (bridged) initial state, and X_0 = alpha_0 * Z_init (+ B_0^T)
-      const float a0 = alpha_of(frame_of(0));
-      __nv_bfloat16* z0 = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(0)) * (D * D) + (size_t)col0 * D + row;
-      if (additive) {
-        float x0[CW];
+      // the frames with no distant frame on this chain's side read the initial state; X_0 = alpha_0 * Z_init (+ B_0^T)
+      float zi[CW];
 #pragma unroll
-        for (int e = 0; e < CW; ++e) {
-          const float zi = s0 ? 0.5f * __ldg(s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
-          z0[(size_t)e * D] = __float2bfloat16_rn(a0 * zi);
-          x0[e] = a0 * zi;
-        }
-        publish_x(x0);
-      } else {
+      for (int e = 0; e < CW; ++e) zi[e] = s0 ? 0.5f * __ldg(s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
+      store_readers(dir == 0 ? win.first : win.last, zi);
+      if (nfold > 0) {
+        const float a0 = alpha_of(frame_of(0));
+        if (additive) {
 #pragma unroll
-        for (int e = 0; e < CW; ++e) {
-          const float zi = s0 ? 0.5f * __ldg(s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
-          z0[(size_t)e * D] = __float2bfloat16_rn(a0 * zi);
-          bt[e] = fmaf(a0, zi, bt[e]);
+          for (int e = 0; e < CW; ++e) zi[e] *= a0;
+          publish_x(zi);
+        } else {
+#pragma unroll
+          for (int e = 0; e < CW; ++e) bt[e] = fmaf(a0, zi[e], bt[e]);
+          publish_x(bt);
         }
-        publish_x(bt);
       }
     }
-    if (!additive && T > 1) load_bt(frame_of(1), bt);
-    float a_next = T > 1 ? alpha_of(frame_of(1)) : 1.0f;
-    for (int s = 0; s + 1 < T; ++s) {
+    if (!additive && nfold > 1) load_bt(frame_of(1), bt);
+    float a_next = nfold > 1 ? alpha_of(frame_of(1)) : 1.0f;
+    for (int s = 0; s < nfold; ++s) {
       if (!mbar_wait(ACCFULL, s & 1, wc)) break;
       tc_fence_after_sync();
       float z[CW];
@@ -216,25 +245,18 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
         for (int e = 0; e < CW; ++e) z[e] = fmaf(additive_bscale, bt[e], z[e]);
       }
       // first what the next MMAs are waiting for: X = alpha * Z (+ B^T of the next frame), split, into shared memory
-      if (s + 2 < T) {                       // in place: bt is dead once it has been added
+      if (s + 1 < nfold) {                   // in place: bt is dead once it has been added
 #pragma unroll
         for (int e = 0; e < CW; ++e) bt[e] = additive ? a_next * z[e] : fmaf(a_next, z[e], bt[e]);
         publish_x(bt);
       }
-      // then, under the next step's MMAs: the state after step s is what the next frame in scan order reads.
+      // then, under the next step's MMAs: the state after step s goes to the frames that read it.
       // Stored as bf16 [d_v][d_k] (the paper's orientation), so the 32 lanes of a warp (consecutive key
       // channels) write 64 contiguous bytes per value column.
-      __nv_bfloat16* dst = (dir == 0 ? pf : pb) + ((size_t)bh * T + frame_of(s + 1)) * (D * D) + (size_t)col0 * D + row;
-#pragma unroll
-      for (int e = 0; e < CW; e += 2) {
-        const __nv_bfloat162 v2 = __floats2bfloat162_rn(a_next * z[e], a_next * z[e + 1]);   // decay bridge of the reader
-        dst[(size_t)e * D] = v2.x;
-        dst[(size_t)(e + 1) * D] = v2.y;
-      }
-      if (s + 2 < T) {                                 // B^T and decay for the step after, also under the MMAs
-        load_bt(frame_of(s + 1 + lead), bt);
-        a_next = alpha_of(frame_of(s + 2));
-      }
+      store_readers(dir == 0 ? frame_of(s) + 1 : frame_of(s) - 1, z);
+      // B^T and decay for the step after, also under the MMAs
+      if (s + 1 + lead < nfold) load_bt(frame_of(s + 1 + lead), bt);
+      if (s + 2 < nfold) a_next = alpha_of(frame_of(s + 2));
     }
   }
 

@@ -42,6 +42,16 @@ struct StagingLayout {
   size_t q, k, v, out, beta, gate, total;
 };
 
+// The optional inputs of vdn_vda_forward_opt, checked and with defaults filled in.
+struct Extras {
+  const float* alpha = nullptr;
+  const float* s0 = nullptr;
+  const void* gate_elem = nullptr;
+  const float* norm_weight = nullptr;
+  vdn::Window win{1, 0, 0, -1};
+  bool anchors = false;
+};
+
 }  // namespace
 
 // Optional per-kernel timing: a ring of CUDA-event sets recorded on the caller's stream, one set per
@@ -197,7 +207,7 @@ vdn_status set_attrs_simt(vdn_vda_t h) {
 // The plain-fp32 path: four launches.
 template <typename Tio, int D>
 vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
-                        const float* gate, const float* alpha, const float* s0, void* out, const Shape& s,
+                        const float* gate, const Extras& x, void* out, const Shape& s,
                         const Layout& L, cudaStream_t st) {
   if (!h->attrs_set) {
     vdn_status r = set_attrs_simt<Tio, D>(h);
@@ -218,17 +228,18 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
   const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
   const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
   if (additive) {
-    vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n, 1.0f / (float)s.F);
+    vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n, 1.0f / (float)s.F, s);
     prof_mark(h, st, 1, "additive_transition");
   } else {
-    vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n);
+    vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n, s);
     prof_mark(h, st, 1, "resolve");
   }
   vdn::scan_kernel<D, 32><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
-      stats, inv, fwd, read, s.T, alpha, s0, s.H, bscale);
+      stats, inv, fwd, read, s.T, x.alpha, x.s0, s.H, bscale, x.win);
   prof_mark(h, st, 2, "scan");
   vdn::readout_simt_kernel<Tio, D><<<dim3((unsigned)n, (s.F + 63) / 64), 256, sizeof(vdn::ReadoutSimtSmem<D>), st>>>(
-      static_cast<const Tio*>(q), read, gate, static_cast<Tio*>(out), s, h->cfg.rms_eps);
+      static_cast<const Tio*>(q), read, gate, static_cast<Tio*>(out), s, h->cfg.rms_eps,
+      static_cast<const Tio*>(x.gate_elem), x.norm_weight);
   prof_mark(h, st, 3, "readout_simt");
   h->launches = 4;
   VDN_CUDA(h, cudaGetLastError());
@@ -269,14 +280,16 @@ vdn_status make_matrix_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, long lo
 }
 
 vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
-                      const float* gate, const float* alpha, const float* s0, void* out, const Shape& s,
+                      const float* gate, const Extras& x, void* out, const Shape& s,
                       const Layout& L, cudaStream_t st) {
   constexpr int D = 128;
   if (!h->encode) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   if (!h->tc_attrs_set) {
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::GramTc::SMEM_BYTES));
-    VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::ReadoutTc::SMEM_BYTES));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ReadoutTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
@@ -300,7 +313,8 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   if ((r = make_matrix_map(h, &tmS, pf, 2 * n * D)) != VDN_OK) return r;      // pf then pb
   if ((r = make_matrix_map(h, &tmC, csplit, 3 * n * D)) != VDN_OK) return r;
 
-  const unsigned persistent = (unsigned)(n < h->sm_count ? n : h->sm_count);
+  const long long nwork = s.work_items();
+  const unsigned persistent = (unsigned)(nwork < h->sm_count ? nwork : h->sm_count);
   prof_begin(h, st);
   int nk = 0;
   vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
@@ -309,22 +323,27 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
   const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
   if (additive) {
-    vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n, 1.0f / (float)s.F);
+    vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n, 1.0f / (float)s.F, s);
     prof_mark(h, st, nk++, "additive_transition");
   } else {
     vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
-        stats, csplit, n, h->status_dev);
+        stats, csplit, n, h->status_dev, s);
     prof_mark(h, st, nk++, "resolve_tc");
   }
   vdn::scan_tc_kernel<<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS, vdn::ScanTc::SMEM_BYTES, st>>>(
-      tmC, stats, pf, pb, s.T, alpha, s0, s.H, bscale, h->status_dev);
+      tmC, stats, pf, pb, s.T, x.alpha, x.s0, s.H, bscale, h->status_dev, x.win);
   prof_mark(h, st, nk++, "scan_tc");
   // The read-out streams reads and writes in equal parts and is fastest on about five SMs out of six
   // (measured on three workloads: 124 CTAs beat 148 by 5 %; fewer interleaved read/write streams at the DRAM).
   const long long ro_target = ((long long)h->sm_count * 27 + 16) / 32;
-  const unsigned persistent_ro = (unsigned)(n < ro_target ? n : ro_target);
-  vdn::readout_tc_kernel<<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
-      tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev);
+  const unsigned persistent_ro = (unsigned)(nwork < ro_target ? nwork : ro_target);
+  if (x.gate_elem || x.norm_weight || !gate)
+    vdn::readout_tc_kernel<true><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
+        tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
+        x.norm_weight);
+  else
+    vdn::readout_tc_kernel<false><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
+        tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev, nullptr, nullptr);
   prof_mark(h, st, nk++, "readout_tc");
   h->launches = nk;
   VDN_CUDA(h, cudaGetLastError());
@@ -352,8 +371,8 @@ vdn_status launch_scan_static(const float* stats, const float* inv, float* read,
   cudaError_t e = cudaFuncSetAttribute(vdn::scan_kernel<D, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)sizeof(vdn::ScanSmem<D, 32>));
   if (e != cudaSuccess) { *why = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return VDN_ERR_CUDA; }
-  vdn::scan_kernel<D, 32><<<dim3((unsigned)BH, D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(stats, inv, scratch,
-                                                                                               read, T);
+  vdn::scan_kernel<D, 32><<<dim3((unsigned)BH, D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
+      stats, inv, scratch, read, T, nullptr, nullptr, 1, 0.f, vdn::Window{1, 0, 0, T - 1});
   e = cudaGetLastError();
   if (e != cudaSuccess) { *why = std::string("kernel launch: ") + cudaGetErrorString(e); return VDN_ERR_CUDA; }
   return VDN_OK;
@@ -436,31 +455,75 @@ vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes) {
   return VDN_OK;
 }
 
-vdn_status vdn_vda_forward_ex(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
-                              const float* gate, const float* alpha, const float* s0, void* out, int B, int T,
-                              int F, int H, int d, void* cuda_stream) {
+vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                               const float* gate, void* out, int B, int T, int F, int H, int d,
+                               const vdn_vda_options* opt, void* cuda_stream) {
   if (!h) return VDN_ERR_INVALID_ARG;
-  if (!q || !k || !v || !beta || !gate || !out) return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
+  Extras x;
+  if (opt) {
+    if (opt->struct_size != sizeof(vdn_vda_options))
+      return fail(h, VDN_ERR_INVALID_ARG, "vdn_vda_options.struct_size does not match this library");
+    if (opt->chunk < 0 || opt->radius < 0) return fail(h, VDN_ERR_INVALID_ARG, "chunk and radius must be non-negative");
+    x.alpha = opt->alpha;
+    x.s0 = opt->s0;
+    x.gate_elem = opt->gate_elem;
+    x.norm_weight = opt->norm_weight;
+    x.win.chunk = opt->chunk > 0 ? opt->chunk : 1;
+    x.win.radius = opt->radius;
+    x.anchors = opt->anchors != 0;
+  }
+  if (!q || !k || !v || !beta || !out || (!gate && !x.gate_elem))
+    return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(beta) ||
-      !aligned16(alpha) || !aligned16(s0))
-    return fail(h, VDN_ERR_INVALID_ARG, "q, k, v, beta, alpha, s0, out must be 16-byte aligned");
-  if (out == q || out == k || out == v) return fail(h, VDN_ERR_INVALID_ARG, "out must not alias an input");
+      !aligned16(x.alpha) || !aligned16(x.s0) || !aligned16(x.gate_elem) || !aligned16(x.norm_weight))
+    return fail(h, VDN_ERR_INVALID_ARG, "q, k, v, beta, alpha, s0, gate_elem, norm_weight, out must be 16-byte aligned");
+  if (out == q || out == k || out == v || out == x.gate_elem)
+    return fail(h, VDN_ERR_INVALID_ARG, "out must not alias an input");
   std::string why;
   if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
+  if ((long long)(x.win.radius + 1) * x.win.chunk > (1 << 20))
+    return fail(h, VDN_ERR_INVALID_ARG, "(radius + 1) * chunk is unreasonably large");
   const Layout L = make_layout(h, B, T, H, d);
   if (!h->workspace || h->workspace_bytes < L.total)
     return fail(h, VDN_ERR_WORKSPACE, "workspace not set or smaller than vdn_vda_workspace_bytes");
   DeviceGuard guard(h->cfg.device);
   if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const Shape s{B, T, F, H, d};
-  if (use_tensor_cores(h, d)) return forward_tc(h, q, k, v, beta, gate, alpha, s0, out, s, L, st);
-  if (h->cfg.io_dtype == VDN_F32) {
-    return d == 64 ? forward_simt<float, 64>(h, q, k, v, beta, gate, alpha, s0, out, s, L, st)
-                   : forward_simt<float, 128>(h, q, k, v, beta, gate, alpha, s0, out, s, L, st);
+  // The scanned frames: all of them, or the interior ones when frames 0 and T-1 are boundary anchors.
+  x.win.first = x.anchors ? 1 : 0;
+  x.win.last = x.anchors ? T - 2 : T - 1;
+  const Shape s{B, T, F, H, d, x.win.first, x.win.last - x.win.first + 1};
+  h->launches = 0;
+  if (x.anchors) {
+    // Alg. 1 step 7: anchor rows of the linear output are zero (frames 0 and T-1 of every clip)
+    const size_t frame_bytes = (size_t)F * H * d * elem_size(h);
+    char* o = static_cast<char*>(out);
+    for (int b = 0; b < B; ++b) {
+      VDN_CUDA(h, cudaMemsetAsync(o + (size_t)b * T * frame_bytes, 0, frame_bytes, st));
+      if (T > 1) VDN_CUDA(h, cudaMemsetAsync(o + ((size_t)b * T + T - 1) * frame_bytes, 0, frame_bytes, st));
+    }
+    if (s.Tn <= 0) return VDN_OK;      // a clip of anchor frames only has no linear output (Sec. A.4)
   }
-  return d == 64 ? forward_simt<__nv_bfloat16, 64>(h, q, k, v, beta, gate, alpha, s0, out, s, L, st)
-                 : forward_simt<__nv_bfloat16, 128>(h, q, k, v, beta, gate, alpha, s0, out, s, L, st);
+  if (use_tensor_cores(h, d)) return forward_tc(h, q, k, v, beta, gate, x, out, s, L, st);
+  if (h->cfg.io_dtype == VDN_F32) {
+    return d == 64 ? forward_simt<float, 64>(h, q, k, v, beta, gate, x, out, s, L, st)
+                   : forward_simt<float, 128>(h, q, k, v, beta, gate, x, out, s, L, st);
+  }
+  return d == 64 ? forward_simt<__nv_bfloat16, 64>(h, q, k, v, beta, gate, x, out, s, L, st)
+                 : forward_simt<__nv_bfloat16, 128>(h, q, k, v, beta, gate, x, out, s, L, st);
+}
+
+vdn_status vdn_vda_forward_ex(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                              const float* gate, const float* alpha, const float* s0, void* out, int B, int T,
+                              int F, int H, int d, void* cuda_stream) {
+  if (!gate) return h ? fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer") : VDN_ERR_INVALID_ARG;
+  vdn_vda_options opt;
+  std::memset(&opt, 0, sizeof(opt));
+  opt.struct_size = sizeof(opt);
+  opt.alpha = alpha;
+  opt.s0 = s0;
+  opt.chunk = 1;
+  return vdn_vda_forward_opt(h, q, k, v, beta, gate, out, B, T, F, H, d, &opt, cuda_stream);
 }
 
 vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,

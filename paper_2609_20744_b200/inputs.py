@@ -132,6 +132,17 @@ def generate_recurrence_extras(w: VdaWorkload, device="cpu"):
     return alpha.contiguous(), s0.contiguous()
 
 
+def generate_output_extras(w: VdaWorkload, device="cpu"):
+    """Seeded element-wise output gate gate_elem [B,T,F,H,d] = sigmoid(N(0,1)) in the I/O dtype (the output of a
+    content-dependent gate network) and a per-channel norm scale norm_weight [H,d] = 1 + 0.1 N(0,1), float32."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(_seed(w.seed, 0x6A7E))
+    gate_elem = torch.sigmoid(torch.randn((w.B, w.T, w.F, w.H, w.d), generator=g, device=dev)).to(w.torch_dtype)
+    norm_weight = 1.0 + 0.1 * torch.randn((w.H, w.d), generator=g, device=dev)
+    return gate_elem.contiguous(), norm_weight.contiguous()
+
+
 def head_slice(x: dict, b: int, h: int):
     """Host float64 numpy copies of one (batch, head) slice: q,k,v [T,F,d], beta [T,F], gate scalar."""
     import numpy as np

@@ -1,0 +1,174 @@
+"""Parity of vdn_vda_forward_opt (chunk windows, boundary anchors, decay bridge, element-wise gate, norm
+weight) against the fp64 checker, element by element, on every kernel path.
+
+Tolerances as in test_gpu_parity.py: 1e-4 for f32 I/O, 2e-2 for bf16 I/O (oracle.slice_error).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import vda_oracle as orc
+from paper_2609_20744_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+SIMT = binding.VDN_FLAG_FORCE_SIMT
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    binding.load_library()
+
+
+def check(w, x, out, alpha=None, s0=None, gate_elem=None, norm_weight=None, use_gate=True, rule="vda", **win):
+    worst = 0.0
+    for b in range(w.B):
+        for h in range(w.H):
+            q, k, v, beta, gate = inputs.head_slice(x, b, h)
+            if gate_elem is not None:
+                ge = gate_elem[b, :, :, h, :].double().cpu().numpy()
+                gate = ge * gate if use_gate else ge
+            a = None if alpha is None else alpha[b, :, h, :].double().cpu().numpy()
+            s = None if s0 is None else s0[b, h].double().cpu().numpy()
+            nw = None if norm_weight is None else norm_weight[h].double().cpu().numpy()
+            ref = orc.vda_slice(q, k, v, beta, gate, 1e-6, alpha=a, s0=s, rule=rule, norm_weight=nw, **win)["out"]
+            got = out[b, :, :, h, :].double().cpu().numpy()
+            assert np.isfinite(got).all()
+            e = orc.slice_error(got, ref)
+            worst = max(worst, e)
+            assert e <= TOL[w.dtype], f"slice (b={b}, h={h}) error {e:.3e} > {TOL[w.dtype]}"
+    return worst
+
+
+@pytest.mark.parametrize("dtype,d,flags", [("f32", 64, 0), ("bf16", 128, 0), ("bf16", 128, SIMT)])
+@pytest.mark.parametrize("T,chunk,radius,anchors", [
+    (12, 5, 1, True),      # the release setting on a short clip: every window touches a clip end
+    (23, 5, 1, True),      # long enough for full 15-frame windows in the middle
+    (9, 2, 0, True), (10, 2, 1, False), (7, 3, 0, False), (6, 1, 1, True), (5, 1, 0, True),
+    (4, 5, 1, True),       # one window covers every scanned frame: both sides read the text state
+    (3, 1, 0, True),       # a single scanned frame
+])
+def test_window_anchor_bridge_matches_oracle(dtype, d, flags, T, chunk, radius, anchors):
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=1, H=2, T=T, F=140, seed=100 * T + 10 * chunk + radius)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0,
+                      chunk=chunk, radius=radius, anchors=anchors)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK and vda.launch_count() > 0
+    check(w, x, out, alpha, s0, chunk=chunk, radius=radius, anchors=anchors)
+    if anchors:
+        assert torch.count_nonzero(out[:, 0]) == 0 and torch.count_nonzero(out[:, -1]) == 0
+
+
+@pytest.mark.parametrize("dtype,d,flags", [("f32", 128, 0), ("bf16", 128, 0)])
+def test_window_without_decay_or_text_state(dtype, d, flags):
+    # alpha = 1, S_T = 0: frames of one chunk read the same pair of states; frames near a clip end read zero on that side
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=2, H=2, T=17, F=130, seed=5)
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], chunk=5, radius=1, anchors=True)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    check(w, x, out, chunk=5, radius=1, anchors=True)
+
+
+@pytest.mark.parametrize("T", [1, 2])
+def test_clip_of_anchor_frames_only_has_no_linear_output(T):
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=T, F=70, H=2)
+    x = inputs.generate(w, "cuda")
+    _, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    out = torch.full_like(x["q"], 3.0)
+    vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out, s0=s0, anchors=True)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(out) == 0
+
+
+@pytest.mark.parametrize("dtype,d,flags", [("f32", 64, 0), ("bf16", 128, 0), ("bf16", 128, SIMT)])
+@pytest.mark.parametrize("use_gate_elem,use_weight,use_head_gate", [
+    (True, True, True), (True, False, False), (False, True, True)])
+def test_elementwise_gate_and_norm_weight_match_oracle(dtype, d, flags, use_gate_elem, use_weight, use_head_gate):
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=2, H=3, T=4, F=150, seed=31)
+    x = inputs.generate(w, "cuda")
+    ge, nw = inputs.generate_output_extras(w, "cuda")
+    ge = ge if use_gate_elem else None
+    nw = nw if use_weight else None
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"] if use_head_gate else None,
+                      gate_elem=ge, norm_weight=nw)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    check(w, x, out, gate_elem=ge, norm_weight=nw, use_gate=use_head_gate)
+    plain = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
+    torch.cuda.synchronize()
+    assert not torch.allclose(plain.float(), out.float(), atol=1e-2)
+
+
+def test_everything_at_once_on_the_tensor_core_path():
+    # release setting (chunk 5, radius 1, anchors, decay bridge, text state) + content-dependent gate + norm weight,
+    # several token tiles with a ragged tail, two batches
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=2, H=2, T=13, F=300, seed=8)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    ge, nw = inputs.generate_output_extras(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    assert vda.uses_tensor_cores()
+    kw = dict(chunk=5, radius=1, anchors=True)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0, gate_elem=ge,
+                      norm_weight=nw, **kw)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    check(w, x, out, alpha, s0, ge, nw, **kw)
+    # bit-identical run to run
+    out2 = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0, gate_elem=ge,
+                       norm_weight=nw, **kw)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+
+
+def test_additive_rule_with_window():
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=1, H=2, T=11, F=200, seed=12)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    for flags in (0, SIMT):
+        vda = binding.Vda(w.d, w.dtype, flags=flags | binding.VDN_FLAG_ADDITIVE_RULE)
+        out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0,
+                          chunk=2, radius=1, anchors=True)
+        torch.cuda.synchronize()
+        assert vda.status() == binding.VDN_OK
+        check(w, x, out, alpha, s0, rule="additive", chunk=2, radius=1, anchors=True)
+
+
+def test_default_window_through_the_options_entry_is_bitwise_the_plain_call():
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=6, F=260, H=2)
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    a = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"]).clone()
+    nw = torch.ones((w.H, w.d), device="cuda")
+    b = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], norm_weight=nw)     # forces forward_opt, extras path
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+
+
+def test_options_argument_errors():
+    import ctypes
+    w = inputs.TINY
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    vda.ensure_workspace(w.B, w.T, w.F, w.H)
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    out = torch.empty_like(x["q"])
+    opt = binding.VdnOptions(ctypes.sizeof(binding.VdnOptions) - 4, 1, 0, 0, None, None, None, None)
+    args = (vda.h, p(x["q"]), p(x["k"]), p(x["v"]), p(x["beta"]), p(x["gate"]), p(out), w.B, w.T, w.F, w.H, w.d)
+    assert vda.lib.vdn_vda_forward_opt(*args, ctypes.byref(opt), None) == 1          # struct_size mismatch
+    opt = binding.VdnOptions(ctypes.sizeof(binding.VdnOptions), 1, -1, 0, None, None, None, None)
+    assert vda.lib.vdn_vda_forward_opt(*args, ctypes.byref(opt), None) == 1          # negative radius
+    args_nogate = args[:5] + (None,) + args[6:]
+    opt = binding.VdnOptions(ctypes.sizeof(binding.VdnOptions), 1, 0, 0, None, None, None, None)
+    assert vda.lib.vdn_vda_forward_opt(*args_nogate, ctypes.byref(opt), None) == 1   # neither gate given
+    assert vda.lib.vdn_vda_forward_opt(*args, None, None) == 0                       # NULL options = plain forward
+    torch.cuda.synchronize()
