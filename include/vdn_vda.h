@@ -74,6 +74,11 @@ typedef enum { VDN_F32 = 0, VDN_BF16 = 1 } vdn_dtype;
                                   /* update with 1/sqrt(F) key scaling, S_t = S_bar (I - A_t/F) + B_t/sqrt(F)   */
                                   /* (Eq. 3c, Sec. 3.3), no resolve; everything else unchanged                  */
 
+#define VDN_FLAG_SCAN_CHUNKWISE 8u  /* vdn_vda_forward_opt with chunk >= 2 on the tensor-core kernels: always run the */
+                                   /* scan chunk-wise (Sec. 5, "Chunk-wise scans"); without this flag the library    */
+                                   /* chooses by the number of chains and chunks, given a large enough workspace     */
+#define VDN_FLAG_SCAN_FRAMEWISE 16u /* never run the scan chunk-wise                                                 */
+
 typedef struct {
   uint32_t struct_size; /* sizeof(vdn_vda_config), checked                                            */
   int32_t io_dtype;     /* vdn_dtype of q, k, v, out                                                  */
@@ -165,6 +170,17 @@ typedef struct {
 vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
                                const float* gate, void* out, int B, int T, int F, int H, int d,
                                const vdn_vda_options* opt, void* cuda_stream);
+
+/* Workspace for vdn_vda_forward_opt with room for the chunk-wise scan (Sec. 5, "Chunk-wise scans": the frames of a
+ * temporal chunk are composed into S_out = S_in M_chunk + J_chunk, all chunks side by side, and the chunk sequence
+ * is scanned; states are read at chunk edges only, so nothing is lost, and the chain is about `chunk` times
+ * shorter at about four times the arithmetic).  With opt->chunk >= 2 on the tensor-core kernels this is
+ * vdn_vda_workspace_bytes plus the composites (per batch, head, direction and chunk: M as three bf16 parts, J in
+ * fp32); otherwise it equals vdn_vda_workspace_bytes.  Given such a workspace, vdn_vda_forward_opt runs the scan
+ * chunk-wise when that shortens it (few chains, many chunks: e.g. heads sharded over several GPUs), or always
+ * under VDN_FLAG_SCAN_CHUNKWISE; with the smaller workspace it scans frame by frame.  The text state enters the
+ * chunk-level scan as its initial state.  Pure function; 0 on invalid arguments. */
+size_t vdn_vda_workspace_bytes_opt(vdn_vda_t h, int B, int T, int F, int H, int d, const vdn_vda_options* opt);
 
 /* The same layer for callers whose tensors live in HOST memory (pinned memory recommended): copies
  * q, k, v, beta, gate to the staging buffer, runs vdn_vda_forward, copies `out` back, all on

@@ -19,11 +19,13 @@ STATUS_NAMES = {0: "VDN_OK", 1: "VDN_ERR_INVALID_ARG", 2: "VDN_ERR_UNSUPPORTED",
 VDN_F32, VDN_BF16 = 0, 1
 VDN_FLAG_FORCE_SIMT = 1
 VDN_FLAG_ADDITIVE_RULE = 4
+VDN_FLAG_SCAN_CHUNKWISE = 8
+VDN_FLAG_SCAN_FRAMEWISE = 16
 VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_READ_BWD = range(7)
 
 EXPORTS = (
     "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward", "vdn_vda_forward_ex",
-    "vdn_vda_forward_opt",
+    "vdn_vda_forward_opt", "vdn_vda_workspace_bytes_opt",
     "vdn_vda_staging_bytes", "vdn_vda_set_staging", "vdn_vda_forward_host", "vdn_vda_workspace_view",
     "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_scan_static", "vdn_vda_status", "vdn_vda_last_error", "vdn_vda_destroy",
 )
@@ -78,6 +80,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.vdn_vda_forward_ex.restype = ci
     lib.vdn_vda_forward_opt.argtypes = [vp, vp, vp, vp, vp, vp, vp, *shape, ctypes.POINTER(VdnOptions), vp]
     lib.vdn_vda_forward_opt.restype = ci
+    lib.vdn_vda_workspace_bytes_opt.argtypes = [vp, *shape, ctypes.POINTER(VdnOptions)]
+    lib.vdn_vda_workspace_bytes_opt.restype = sz
     lib.vdn_vda_forward_host.argtypes = fwd_args
     lib.vdn_vda_forward_host.restype = ci
     lib.vdn_vda_workspace_view.argtypes = [vp, ci, *shape, ctypes.POINTER(sz), ctypes.POINTER(sz)]
@@ -161,12 +165,15 @@ class Vda:
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
         return ctypes.c_void_p(s.cuda_stream)
 
-    def workspace_bytes(self, B, T, F, H) -> int:
+    def workspace_bytes(self, B, T, F, H, chunk=1) -> int:
+        if chunk > 1:
+            opt = VdnOptions(ctypes.sizeof(VdnOptions), chunk, 0, 0, None, None, None, None)
+            return int(self.lib.vdn_vda_workspace_bytes_opt(self.h, B, T, F, H, self.d, ctypes.byref(opt)))
         return int(self.lib.vdn_vda_workspace_bytes(self.h, B, T, F, H, self.d))
 
-    def ensure_workspace(self, B, T, F, H):
+    def ensure_workspace(self, B, T, F, H, chunk=1):
         torch = self._torch
-        need = self.workspace_bytes(B, T, F, H)
+        need = self.workspace_bytes(B, T, F, H, chunk)
         if need == 0:
             raise VdnError(1, "invalid shape")
         if self._ws is None or self._ws.numel() < need:
@@ -213,7 +220,7 @@ class Vda:
             raise ValueError("gate_elem must be [B, T, F, H, d] of the I/O dtype")
         if out is None:
             out = torch.empty_like(q)
-        self.ensure_workspace(B, T, F, H)
+        self.ensure_workspace(B, T, F, H, chunk)
         p = lambda x: ctypes.c_void_p(x.data_ptr()) if x is not None else None
         a = lambda x: x.data_ptr() if x is not None else None
         if (chunk, radius, bool(anchors)) != (1, 0, False) or gate_elem is not None or norm_weight is not None \

@@ -24,6 +24,17 @@
 // {t} that is one slot per step: P_t into slot t+1, R_t into slot t-1).  Frames whose window leaves no distant
 // frame on a side read the initial state (zero unless a text state is passed).  A chain stops after the last
 // state that anybody reads.  The read-out kernel adds the two slots in its accumulator (Eq. 1a).
+//
+// Chunk-wise scan (Sec. 5, "Chunk-wise scans").  With a chunk window, states are read at chunk edges only, so the
+// frames of a chunk can be composed first:  Z_out = M Z_in + J  with  M = C_n D_n ... C_1 D_1  (D = Diag(alpha)) and
+// J the chunk folded from a zero state.  The same pipeline runs in three modes:
+//   SCAN_FRAMES   one CTA per chain, one step per frame (above).
+//   SCAN_COMPOSE  one CTA per (chain, direction, chunk, half): the chunk's frames folded from Z = I without writes
+//                 (-> M, written as three bf16 parts, the operand format of the scan) or from Z = 0 (-> J, fp32).
+//                 All chunks run side by side, which is what shortens the critical path.
+//   SCAN_CHUNKS   one CTA per chain, one step per chunk:  Z <- M Z + J,  the gather as above at chunk edges.
+// The composed scan pays about four times the arithmetic of the frame scan for a chain of
+// chunk + T/chunk steps instead of T: it wins when the chains leave most SMs idle (few heads per GPU).
 #pragma once
 #include <cuda_bf16.h>
 
@@ -44,11 +55,33 @@ struct ScanTc {
   static constexpr int THREADS = 64 + 4 * 32 * (D / CW);  // producer + MMA + state warps
 };
 
+enum { SCAN_FRAMES = 0, SCAN_CHUNKS = 1, SCAN_COMPOSE = 2 };
+
+struct ScanTcArgs {
+  const float* stats;        // [B*H*T][2d][d] per-frame statistics; the scan reads the B_t half
+  __nv_bfloat16* pf;         // [B*H*T][d_v][d_k] read slots of the forward scan
+  __nv_bfloat16* pb;         // ... of the reverse scan
+  const float* alpha;        // [B,T,H,d] or null
+  const float* s0;           // [B,H,d_v,d_k] or null
+  int T, H;
+  float additive_bscale;     // > 0: the additive baseline, Z_t = C_t (alpha Z) + bscale B_t^T
+  Window win;
+  // chunk composites (SCAN_COMPOSE writes, SCAN_CHUNKS reads); position p of a chain's direction is the p-th chunk
+  // that direction folds
+  int nseg;                  // chunks that overlap the scanned frames
+  __nv_bfloat16* comp_m;     // [B*H][2][nseg][3][d][d]  M as three bf16 parts, row-major
+  float* comp_j;             // [B*H][2][nseg][d_v][d_k] J (in the orientation of the B_t block)
+};
+
+// Chunks a direction's chunk-level scan folds: up to the last state that some frame reads.
+__host__ __device__ inline int scan_chunk_steps(const Window& w, int dir) {
+  if (dir == 0) return w.lo(w.last) == w.first ? 0 : w.lo(w.last) / w.chunk - w.first / w.chunk;
+  return w.hi(w.first) == w.last ? 0 : w.last / w.chunk - w.hi(w.first) / w.chunk;
+}
+
+template <int MODE>
 __global__ void __launch_bounds__(ScanTc::THREADS, 1)
-scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict__ stats,
-               __nv_bfloat16* __restrict__ pf, __nv_bfloat16* __restrict__ pb, int T,
-               const float* __restrict__ alpha, const float* __restrict__ s0, int H, float additive_bscale,
-               int* status, Window win) {
+scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int* status) {
   using namespace tc;
   using S = ScanTc;
   constexpr int D = S::D;
@@ -64,12 +97,40 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + S::OFF_BAR + 72);
   const WaitCtx wc{abort_flag, status};
 
+  const Window& win = a.win;
+  const int T = a.T;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bh = blockIdx.x >> 1, dir = blockIdx.x & 1;
-  auto frame_of = [&](int s) { return dir == 0 ? win.first + s : win.last - s; };   // frame folded in at scan step s
-  // steps this chain runs: up to the last state that some frame reads (P_{l-1} of the last frame's window,
-  // R_{h+1} of the first frame's)
-  const int nfold = dir == 0 ? win.lo(win.last) - win.first : win.last - win.hi(win.first);
+
+  // ---- which sequence this CTA folds
+  int bh, dir, nsteps;
+  int f_lo = win.first, f_hi = win.last;     // frames of this CTA's sequence (SCAN_FRAMES, SCAN_COMPOSE)
+  int half = 0, pos = 0;                     // SCAN_COMPOSE: 0 = J (from zero, with writes), 1 = M (from I, no writes)
+  const int kfirst = win.first / win.chunk, klast = win.last / win.chunk;
+  if constexpr (MODE == SCAN_COMPOSE) {
+    half = blockIdx.x & 1;
+    dir = (blockIdx.x >> 1) & 1;
+    const int rest = blockIdx.x >> 2;
+    pos = rest % a.nseg;
+    bh = rest / a.nseg;
+    if (pos >= scan_chunk_steps(win, dir)) return;           // nobody reads past this chunk
+    const int kc = dir == 0 ? kfirst + pos : klast - pos;
+    f_lo = max(win.first, kc * win.chunk);
+    f_hi = min(win.last, (kc + 1) * win.chunk - 1);
+    nsteps = f_hi - f_lo + 1;
+  } else {
+    bh = blockIdx.x >> 1;
+    dir = blockIdx.x & 1;
+    // steps this chain runs: up to the last state that some frame reads (P_{l-1} of the last frame's window,
+    // R_{h+1} of the first frame's)
+    if constexpr (MODE == SCAN_FRAMES) nsteps = dir == 0 ? win.lo(win.last) - win.first : win.last - win.hi(win.first);
+    else nsteps = scan_chunk_steps(win, dir);
+  }
+  auto frame_of = [&](int s) { return dir == 0 ? f_lo + s : f_hi - s; };   // frame folded in at step s
+  // index of step s's transition (three bf16 parts, 3*D rows of the tensor map) and of its write
+  auto item_of = [&](int s) -> long long {
+    if constexpr (MODE == SCAN_CHUNKS) return ((long long)bh * 2 + dir) * a.nseg + s;
+    else return (long long)bh * T + frame_of(s);
+  };
 
   if (threadIdx.x == 0) {
     for (int p = 0; p < 3; ++p) { mbar_init(CFULL(p), 1); mbar_init(CFREE(p), 1); }
@@ -95,8 +156,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     // of this step's MMA time plus the state warps' turn to arrive.
     if (lane == 0) {
       bool ok = true;
-      for (int s = 0; s < nfold && ok; ++s) {
-        const long long n = (long long)bh * T + frame_of(s);
+      for (int s = 0; s < nsteps && ok; ++s) {
+        const long long n = item_of(s);
 #pragma unroll
         for (int p = 2; p >= 0; --p) {
           if (!mbar_wait(CFREE(p), (s & 1) ^ 1, wc)) { ok = false; break; }
@@ -113,7 +174,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
       bool ok = true;
-      for (int s = 0; s < nfold && ok; ++s) {
+      for (int s = 0; s < nsteps && ok; ++s) {
         if (!mbar_wait(XREADY, s & 1, wc)) break;
         tc_fence_after_sync();
         // C3 X1, then C2 (X2, X1), then C1 (X3, X2, X1): smallest contributions first
@@ -149,10 +210,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     const int ch0 = (col0 & 63) >> 3;        // first 16-byte chunk of this thread inside the 64-column box
     const int sw = row & 7;
 
-    auto load_bt = [&](int frame, float (&bt)[CW]) {
-      // B_t is stored [d_v][d_k]; lanes read consecutive key channels (scalar but coalesced: measured
+    auto load_bt = [&](int s, float (&bt)[CW]) {
+      // the write of step s, stored [d_v][d_k]; lanes read consecutive key channels (scalar but coalesced: measured
       // faster than 16-byte loads of a thread-contiguous layout, whose lanes sit 512 bytes apart)
-      const float* src = stats + ((size_t)bh * T + frame) * (2 * D * D) + (size_t)(D + col0) * D + row;
+      const float* src;
+      if constexpr (MODE == SCAN_CHUNKS) src = a.comp_j + (size_t)item_of(s) * (D * D) + (size_t)col0 * D + row;
+      else src = a.stats + (size_t)item_of(s) * (2 * D * D) + (size_t)(D + col0) * D + row;
 #pragma unroll
       for (int e = 0; e < CW; ++e) bt[e] = __ldg(src + (size_t)e * D);
     };
@@ -179,24 +242,29 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
     // state before a frame is folded in, and bridges the state that frame reads; s0 [B,H,d_v,d_k] is the text
     // state, each scan starting from half of it.  Both act on a thread's own row: one scalar per step.
     auto alpha_of = [&](int frame) {
-      return alpha ? __ldg(alpha + (((size_t)(bh / H) * T + frame) * H + (bh % H)) * D + row) : 1.0f;
+      return a.alpha ? __ldg(a.alpha + (((size_t)(bh / a.H) * T + frame) * a.H + (bh % a.H)) * D + row) : 1.0f;
     };
-    // Additive baseline (additive_bscale = 1/sqrt(F) > 0; Eq. 3c with the key scaling of Sec. 3.3): the frame's
-    // write is not resolved against its keys,  Z_t = C_t (alpha_t * Z_{t-1}) + B_t^T / sqrt(F)  with
-    // C_t = I - A_t / F prepared by the host's choice of kernel; the same MMAs, the write added after them.
-    const bool additive = additive_bscale > 0.f;
-    const int lead = additive ? 0 : 1;       // bt holds B^T of frame_of(step + lead) when step's MMAs retire
+    // decay applied to the inherited state at step s (inside M for a composed chunk)
+    auto step_decay = [&](int s) { return MODE == SCAN_CHUNKS ? 1.0f : alpha_of(frame_of(s)); };
+    // Additive form of a step: the write is added after the product, Z = C (decay * Z) + bscale * B^T.  That is the
+    // additive baseline (additive_bscale = 1/sqrt(F) > 0; Eq. 3c with the key scaling of Sec. 3.3, C_t = I - A_t/F
+    // prepared by the host's choice of kernel) and, with bscale = 1, a composed chunk (Z = M Z + J).
+    // Otherwise Z = C (decay * Z + B^T), the joint solve of Eq. 5.
+    const bool additive = MODE == SCAN_CHUNKS || a.additive_bscale > 0.f;
+    const float bscale = MODE == SCAN_CHUNKS ? 1.0f : a.additive_bscale;
+    const bool writes = !(MODE == SCAN_COMPOSE && half == 1);     // M is the chunk without its writes
+    const int lead = additive ? 0 : 1;       // bt holds the write of step (s + lead) when step s's MMAs retire
 
     // Gather: `z` is the state that the frames t with l_t = bound (forward chain) / h_t = bound (reverse chain)
     // read; write their slots, each bridged by the decay of the frames between the state and the query
     // (Eq. A.4).  Readers are visited walking away from the state, so the bridge is a running product.
     auto store_readers = [&](int bound, const float (&z)[CW]) {
-      __nv_bfloat16* slots = (dir == 0 ? pf : pb) + (size_t)bh * T * (D * D) + (size_t)col0 * D + row;
-      float bridge = 1.0f;
-      int r = bound;                           // next frame whose decay enters the bridge
       // only a chunk edge (or the end of the scanned range) is the end of anybody's window
       if (dir == 0 ? (bound != win.first && bound % win.chunk != 0) : (bound != win.last && (bound + 1) % win.chunk != 0))
         return;
+      __nv_bfloat16* slots = (dir == 0 ? a.pf : a.pb) + (size_t)bh * T * (D * D) + (size_t)col0 * D + row;
+      float bridge = 1.0f;
+      int r = bound;                           // next frame whose decay enters the bridge
       const int far = dir == 0 ? min(win.last, bound + win.span()) : max(win.first, bound - win.span());
       for (int t = bound; dir == 0 ? t <= far : t >= far; t += dir == 0 ? 1 : -1) {
         if ((dir == 0 ? win.lo(t) : win.hi(t)) != bound) continue;
@@ -210,18 +278,56 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
         }
       }
     };
+    // the state that the frames beyond step s's last frame read sits at this window bound
+    auto bound_after = [&](int s) {
+      if constexpr (MODE == SCAN_CHUNKS) {
+        const int kc = dir == 0 ? kfirst + s : klast - s;
+        return dir == 0 ? min(win.last, (kc + 1) * win.chunk - 1) + 1 : max(win.first, kc * win.chunk) - 1;
+      } else {
+        return dir == 0 ? frame_of(s) + 1 : frame_of(s) - 1;
+      }
+    };
+    // SCAN_COMPOSE: the folded chunk goes to position `pos` of this direction's composites
+    auto store_composite = [&](const float (&z)[CW]) {
+      const size_t slot = ((size_t)bh * 2 + dir) * a.nseg + pos;
+      if (half == 0) {
+        float* dst = a.comp_j + slot * (D * D) + (size_t)col0 * D + row;      // [d_v][d_k], as the B_t block
+#pragma unroll
+        for (int e = 0; e < CW; ++e) dst[(size_t)e * D] = z[e];
+      } else {
+        // row `row`, columns col0 .. col0+31 of M, three bf16 parts, row-major (the K-major A operand of the scan)
+        __nv_bfloat16* dst = a.comp_m + slot * (3 * D * D) + (size_t)row * D + col0;
+#pragma unroll
+        for (int ch = 0; ch < CW / 8; ++ch) {
+          uint4 w1, w2, w3;
+          uint32_t* a1 = reinterpret_cast<uint32_t*>(&w1);
+          uint32_t* a2 = reinterpret_cast<uint32_t*>(&w2);
+          uint32_t* a3 = reinterpret_cast<uint32_t*>(&w3);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) split3_pair(z[ch * 8 + 2 * e], z[ch * 8 + 2 * e + 1], a1[e], a2[e], a3[e]);
+          *reinterpret_cast<uint4*>(dst + ch * 8) = w1;
+          *reinterpret_cast<uint4*>(dst + (size_t)D * D + ch * 8) = w2;
+          *reinterpret_cast<uint4*>(dst + (size_t)2 * D * D + ch * 8) = w3;
+        }
+      }
+    };
 
     float bt[CW];
-    if (nfold > 0) load_bt(frame_of(0), bt);
+    if (nsteps > 0 && writes) load_bt(0, bt);
     {
-      // the frames with no distant frame on this chain's side read the initial state; X_0 = alpha_0 * Z_init (+ B_0^T)
+      // the state the sequence starts from: half the text state for a scan (the frames with no distant frame on
+      // this chain's side read it), zero or the identity for the two halves of a composed chunk
       float zi[CW];
 #pragma unroll
-      for (int e = 0; e < CW; ++e) zi[e] = s0 ? 0.5f * __ldg(s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
-      store_readers(dir == 0 ? win.first : win.last, zi);
-      if (nfold > 0) {
-        const float a0 = alpha_of(frame_of(0));
-        if (additive) {
+      for (int e = 0; e < CW; ++e) {
+        if constexpr (MODE == SCAN_COMPOSE) zi[e] = (half == 1 && col0 + e == row) ? 1.0f : 0.0f;
+        else zi[e] = a.s0 ? 0.5f * __ldg(a.s0 + ((size_t)bh * D + col0 + e) * D + row) : 0.f;
+      }
+      if constexpr (MODE != SCAN_COMPOSE) store_readers(dir == 0 ? win.first : win.last, zi);
+      if (nsteps > 0) {
+        // X_0 = decay_0 * Z_init (+ the first write)
+        const float a0 = step_decay(0);
+        if (additive || !writes) {
 #pragma unroll
           for (int e = 0; e < CW; ++e) zi[e] *= a0;
           publish_x(zi);
@@ -232,31 +338,42 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const float* __restrict_
         }
       }
     }
-    if (!additive && nfold > 1) load_bt(frame_of(1), bt);
-    float a_next = nfold > 1 ? alpha_of(frame_of(1)) : 1.0f;
-    for (int s = 0; s < nfold; ++s) {
+    if (!additive && writes && nsteps > 1) load_bt(1, bt);
+    float a_next = nsteps > 1 ? step_decay(1) : 1.0f;
+    for (int s = 0; s < nsteps; ++s) {
       if (!mbar_wait(ACCFULL, s & 1, wc)) break;
       tc_fence_after_sync();
       float z[CW];
       tmem_ld32(taddr, z);
       tmem_wait_ld();
-      if (additive) {
+      if (additive && writes) {
 #pragma unroll
-        for (int e = 0; e < CW; ++e) z[e] = fmaf(additive_bscale, bt[e], z[e]);
+        for (int e = 0; e < CW; ++e) z[e] = fmaf(bscale, bt[e], z[e]);
       }
-      // first what the next MMAs are waiting for: X = alpha * Z (+ B^T of the next frame), split, into shared memory
-      if (s + 1 < nfold) {                   // in place: bt is dead once it has been added
+      // first what the next MMAs are waiting for: X = decay * Z (+ the next write), split, into shared memory
+      if (s + 1 < nsteps) {
+        if (additive || !writes) {
+          float xn[CW];
 #pragma unroll
-        for (int e = 0; e < CW; ++e) bt[e] = additive ? a_next * z[e] : fmaf(a_next, z[e], bt[e]);
-        publish_x(bt);
+          for (int e = 0; e < CW; ++e) xn[e] = a_next * z[e];
+          publish_x(xn);
+        } else {                               // in place: bt is dead once it has been added
+#pragma unroll
+          for (int e = 0; e < CW; ++e) bt[e] = fmaf(a_next, z[e], bt[e]);
+          publish_x(bt);
+        }
       }
       // then, under the next step's MMAs: the state after step s goes to the frames that read it.
       // Stored as bf16 [d_v][d_k] (the paper's orientation), so the 32 lanes of a warp (consecutive key
       // channels) write 64 contiguous bytes per value column.
-      store_readers(dir == 0 ? frame_of(s) + 1 : frame_of(s) - 1, z);
-      // B^T and decay for the step after, also under the MMAs
-      if (s + 1 + lead < nfold) load_bt(frame_of(s + 1 + lead), bt);
-      if (s + 2 < nfold) a_next = alpha_of(frame_of(s + 2));
+      if constexpr (MODE == SCAN_COMPOSE) {
+        if (s + 1 == nsteps) store_composite(z);
+      } else {
+        store_readers(bound_after(s), z);
+      }
+      // the write and the decay for the step after, also under the MMAs
+      if (writes && s + 1 + lead < nsteps) load_bt(s + 1 + lead, bt);
+      if (s + 2 < nsteps) a_next = step_decay(s + 2);
     }
   }
 

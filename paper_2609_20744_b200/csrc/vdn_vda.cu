@@ -36,6 +36,8 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct Layout {
   size_t stats, inv, fwd, read, total;
   size_t inv_bytes, state_bytes;
+  size_t comp_m = 0, comp_j = 0;   // chunk composites of the chunk-wise scan (0 = not laid out)
+  int nseg_max = 0;
 };
 
 struct StagingLayout {
@@ -50,6 +52,7 @@ struct Extras {
   const float* norm_weight = nullptr;
   vdn::Window win{1, 0, 0, -1};
   bool anchors = false;
+  bool composed = false;   // run the scan chunk-wise (tensor-core path, chunk >= 2)
 };
 
 }  // namespace
@@ -110,7 +113,9 @@ bool shape_ok(const vdn_vda_s* h, int B, int T, int F, int H, int d, std::string
   return true;
 }
 
-Layout make_layout(const vdn_vda_s* h, int B, int T, int H, int d) {
+// chunk >= 2 adds room for the composites of the chunk-wise scan (tensor-core path): per (batch, head, direction)
+// and chunk, M as three bf16 parts and J in fp32.
+Layout make_layout(const vdn_vda_s* h, int B, int T, int H, int d, int chunk = 1) {
   const size_t n = (size_t)B * H * T;
   const size_t dd = (size_t)d * d;
   Layout L;
@@ -122,6 +127,12 @@ Layout make_layout(const vdn_vda_s* h, int B, int T, int H, int d) {
   L.inv = off;   off += align_up(L.inv_bytes);
   L.fwd = off;   off += L.state_bytes;             // fwd and read stay contiguous (n*d*d*es is 256-aligned)
   L.read = off;  off += align_up(L.state_bytes);
+  if (tcp && chunk >= 2 && !(h->cfg.flags & VDN_FLAG_SCAN_FRAMEWISE)) {
+    L.nseg_max = (T - 1) / chunk + 1;
+    const size_t nc = (size_t)B * H * 2 * L.nseg_max;
+    L.comp_m = off; off += align_up(nc * dd * 3 * 2);
+    L.comp_j = off; off += align_up(nc * dd * sizeof(float));
+  }
   L.total = off;
   return L;
 }
@@ -291,7 +302,11 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
                                      vdn::ReadoutTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ReadoutTc::SMEM_BYTES));
-    VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::ScanTc::SMEM_BYTES));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_CHUNKS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::ScanTc::SMEM_BYTES));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_COMPOSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::resolve_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ResolveTc::SMEM_BYTES));
@@ -330,9 +345,27 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
         stats, csplit, n, h->status_dev, s);
     prof_mark(h, st, nk++, "resolve_tc");
   }
-  vdn::scan_tc_kernel<<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS, vdn::ScanTc::SMEM_BYTES, st>>>(
-      tmC, stats, pf, pb, s.T, x.alpha, x.s0, s.H, bscale, h->status_dev, x.win);
-  prof_mark(h, st, nk++, "scan_tc");
+  vdn::ScanTcArgs sa{};
+  sa.stats = stats; sa.pf = pf; sa.pb = pb; sa.alpha = x.alpha; sa.s0 = x.s0;
+  sa.T = s.T; sa.H = s.H; sa.additive_bscale = bscale; sa.win = x.win;
+  if (x.composed) {
+    // chunk-wise scan: compose every chunk (all at once), then scan the chunk sequence
+    sa.nseg = x.win.last / x.win.chunk - x.win.first / x.win.chunk + 1;
+    sa.comp_m = reinterpret_cast<__nv_bfloat16*>(ws + L.comp_m);
+    sa.comp_j = reinterpret_cast<float*>(ws + L.comp_j);
+    CUtensorMap tmM;
+    if ((r = make_matrix_map(h, &tmM, sa.comp_m, (long long)3 * s.B * s.H * 2 * sa.nseg * D)) != VDN_OK) return r;
+    vdn::scan_tc_kernel<vdn::SCAN_COMPOSE><<<(unsigned)(4 * s.B * s.H * sa.nseg), vdn::ScanTc::THREADS,
+                                             vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
+    prof_mark(h, st, nk++, "compose_tc");
+    vdn::scan_tc_kernel<vdn::SCAN_CHUNKS><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
+                                            vdn::ScanTc::SMEM_BYTES, st>>>(tmM, sa, h->status_dev);
+    prof_mark(h, st, nk++, "scan_chunks_tc");
+  } else {
+    vdn::scan_tc_kernel<vdn::SCAN_FRAMES><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
+                                            vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
+    prof_mark(h, st, nk++, "scan_tc");
+  }
   // The read-out streams reads and writes in equal parts and is fastest on about five SMs out of six
   // (measured on three workloads: 124 CTAs beat 148 by 5 %; fewer interleaved read/write streams at the DRAM).
   const long long ro_target = ((long long)h->sm_count * 27 + 16) / 32;
@@ -431,6 +464,13 @@ size_t vdn_vda_workspace_bytes(vdn_vda_t h, int B, int T, int F, int H, int d) {
   return make_layout(h, B, T, H, d).total;
 }
 
+size_t vdn_vda_workspace_bytes_opt(vdn_vda_t h, int B, int T, int F, int H, int d, const vdn_vda_options* opt) {
+  std::string why;
+  if (!h || !shape_ok(h, B, T, F, H, d, &why)) return 0;
+  if (opt && (opt->struct_size != sizeof(vdn_vda_options) || opt->chunk < 0)) return 0;
+  return make_layout(h, B, T, H, d, opt ? opt->chunk : 1).total;
+}
+
 vdn_status vdn_vda_set_workspace(vdn_vda_t h, void* dev_ptr, size_t bytes) {
   if (!h) return VDN_ERR_INVALID_ARG;
   if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) != 0)
@@ -483,15 +523,34 @@ vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const 
   if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
   if ((long long)(x.win.radius + 1) * x.win.chunk > (1 << 20))
     return fail(h, VDN_ERR_INVALID_ARG, "(radius + 1) * chunk is unreasonably large");
-  const Layout L = make_layout(h, B, T, H, d);
-  if (!h->workspace || h->workspace_bytes < L.total)
-    return fail(h, VDN_ERR_WORKSPACE, "workspace not set or smaller than vdn_vda_workspace_bytes");
-  DeviceGuard guard(h->cfg.device);
-  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   // The scanned frames: all of them, or the interior ones when frames 0 and T-1 are boundary anchors.
   x.win.first = x.anchors ? 1 : 0;
   x.win.last = x.anchors ? T - 2 : T - 1;
+  Layout L = make_layout(h, B, T, H, d);
+  if (!h->workspace || h->workspace_bytes < L.total)
+    return fail(h, VDN_ERR_WORKSPACE, "workspace not set or smaller than vdn_vda_workspace_bytes");
+  if (use_tensor_cores(h, d) && x.win.chunk >= 2 && x.win.last >= x.win.first &&
+      !(h->cfg.flags & VDN_FLAG_SCAN_FRAMEWISE)) {
+    // Chunk-wise scan (Sec. 5): worth it when the chains leave most SMs idle.  Costs in scan steps: one chain
+    // step per frame, against the waves of chunk compositions plus one chain step per chunk plus a launch.
+    const Layout Lc = make_layout(h, B, T, H, d, x.win.chunk);
+    const bool forced = (h->cfg.flags & VDN_FLAG_SCAN_CHUNKWISE) != 0;
+    const int cf = vdn::scan_chunk_steps(x.win, 0), cb = vdn::scan_chunk_steps(x.win, 1);
+    const int ff = x.win.lo(x.win.last) - x.win.first, fb = x.win.last - x.win.hi(x.win.first);
+    const long long ctas = (long long)B * H * (cf + cb) * 2;
+    const long long waves = (ctas + h->sm_count - 1) / h->sm_count;
+    const long long cost_chunks = waves * x.win.chunk + (cf > cb ? cf : cb) + 2;
+    const long long cost_frames = ff > fb ? ff : fb;
+    if (forced && h->workspace_bytes < Lc.total)
+      return fail(h, VDN_ERR_WORKSPACE, "VDN_FLAG_SCAN_CHUNKWISE needs a workspace of vdn_vda_workspace_bytes_opt");
+    if ((forced || cost_chunks < cost_frames) && h->workspace_bytes >= Lc.total && cf + cb > 0) {
+      x.composed = true;
+      L = Lc;
+    }
+  }
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const Shape s{B, T, F, H, d, x.win.first, x.win.last - x.win.first + 1};
   h->launches = 0;
   if (x.anchors) {

@@ -172,3 +172,91 @@ def test_options_argument_errors():
     assert vda.lib.vdn_vda_forward_opt(*args_nogate, ctypes.byref(opt), None) == 1   # neither gate given
     assert vda.lib.vdn_vda_forward_opt(*args, None, None) == 0                       # NULL options = plain forward
     torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------------------ chunk-wise scan (Sec. 5)
+CHUNKWISE = binding.VDN_FLAG_SCAN_CHUNKWISE
+
+
+@pytest.mark.parametrize("T,chunk,radius,anchors,extras", [
+    (23, 5, 1, True, True),       # release setting; first and last chunk clipped by the anchors
+    (23, 5, 1, True, False),      # alpha = 1, zero text state
+    (20, 5, 0, False, True),      # exact chunks, no anchors
+    (14, 2, 1, False, True), (17, 3, 0, True, True), (9, 4, 0, True, True),
+    (12, 5, 1, True, True),       # one (clipped) chunk folded each way
+    (9, 5, 1, True, True),        # no chunk is ever folded: every frame reads the text state on both sides
+])
+def test_chunkwise_scan_matches_oracle(T, chunk, radius, anchors, extras):
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=1, H=2, T=T, F=140, seed=7 * T + chunk)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda") if extras else (None, None)
+    vda = binding.Vda(w.d, w.dtype, flags=CHUNKWISE)
+    kw = dict(chunk=chunk, radius=radius, anchors=anchors)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0, **kw)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    names = [n for (n, _, _) in _kernel_names(vda, x, alpha, s0, kw)]
+    folds = any(orc.local_window(t, T, chunk, radius, anchors)[0] > (1 if anchors else 0) for t in range(T))
+    assert ("compose_tc" in names) == folds
+    check(w, x, out, alpha, s0, **kw)
+    # frame by frame on the same inputs: the same result up to rounding
+    vda2 = binding.Vda(w.d, w.dtype, flags=binding.VDN_FLAG_SCAN_FRAMEWISE)
+    out2 = vda2.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0, **kw)
+    torch.cuda.synchronize()
+    scale = out2.float().abs().amax()
+    assert float((out.float() - out2.float()).abs().amax() / scale) < 2e-2
+
+
+def _kernel_names(vda, x, alpha, s0, kw):
+    vda.profile(True)
+    vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0, **kw)
+    torch.cuda.synchronize()
+    times = vda.kernel_times()
+    vda.profile(False)
+    return times
+
+
+def test_chunkwise_scan_with_the_additive_rule():
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=1, H=2, T=16, F=200, seed=3)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype, flags=CHUNKWISE | binding.VDN_FLAG_ADDITIVE_RULE)
+    kw = dict(chunk=3, radius=0, anchors=True)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0, **kw)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    check(w, x, out, alpha, s0, rule="additive", **kw)
+
+
+def test_chunkwise_scan_is_chosen_for_few_chains_and_needs_its_workspace():
+    import ctypes
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=1, H=1, T=52, F=64, seed=9)
+    x = inputs.generate(w, "cuda")
+    kw = dict(chunk=5, radius=1, anchors=True)
+    vda = binding.Vda(w.d, w.dtype)                                   # no flag: the library decides
+    assert vda.workspace_bytes(w.B, w.T, w.F, w.H, chunk=5) > vda.workspace_bytes(w.B, w.T, w.F, w.H)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], **kw)
+    torch.cuda.synchronize()
+    assert "compose_tc" in [n for (n, _, _) in _kernel_names(vda, x, None, None, kw)]   # 2 chains, 9 chunks each way
+    check(w, x, out, **kw)
+    # with the plain workspace the same call scans frame by frame
+    vda2 = binding.Vda(w.d, w.dtype)
+    vda2.ensure_workspace(w.B, w.T, w.F, w.H)
+    small = vda2._ws[: vda2.workspace_bytes(w.B, w.T, w.F, w.H)]
+    vda2.lib.vdn_vda_set_workspace(vda2.h, ctypes.c_void_p(small.data_ptr()), small.numel())
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    opt = binding.VdnOptions(ctypes.sizeof(binding.VdnOptions), 5, 1, 1, None, None, None, None)
+    out2 = torch.empty_like(x["q"])
+    vda2.profile(True)
+    st = vda2.lib.vdn_vda_forward_opt(vda2.h, p(x["q"]), p(x["k"]), p(x["v"]), p(x["beta"]), p(x["gate"]), p(out2),
+                                      w.B, w.T, w.F, w.H, w.d, ctypes.byref(opt), None)
+    torch.cuda.synchronize()
+    assert st == 0 and "scan_tc" in [n for (n, _, _) in vda2.kernel_times()]
+    check(w, x, out2, **kw)
+    # forcing it without the room is an error, and nothing runs
+    vda3 = binding.Vda(w.d, w.dtype, flags=CHUNKWISE)
+    vda3.lib.vdn_vda_set_workspace(vda3.h, ctypes.c_void_p(small.data_ptr()), small.numel())
+    st = vda3.lib.vdn_vda_forward_opt(vda3.h, p(x["q"]), p(x["k"]), p(x["v"]), p(x["beta"]), p(x["gate"]), p(out2),
+                                      w.B, w.T, w.F, w.H, w.d, ctypes.byref(opt), None)
+    assert st == 3
+    torch.cuda.synchronize()
