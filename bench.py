@@ -238,12 +238,15 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     x = inputs.generate(w, dev)
-    vda = binding.Vda(w.d, w.dtype, device=local_rank)
+    flags = {"auto": 0, "frames": binding.VDN_FLAG_SCAN_FRAMEWISE, "chunks": binding.VDN_FLAG_SCAN_CHUNKWISE}[args.scan]
+    vda = binding.Vda(w.d, w.dtype, device=local_rank, flags=flags)
     out = torch.empty_like(x["q"])
     stream = torch.cuda.current_stream()
+    # the headline configuration is the plain entry point; --chunk/--radius/--anchors time the windowed gather
+    win = dict(chunk=args.chunk, radius=args.radius, anchors=bool(args.anchors))
 
     def step():
-        vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out)
+        vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out, **win)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -289,7 +292,7 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
         errs = []
         for (b, hh) in pairs:
             qs, ks, vs, bs, gs = inputs.head_slice(x, b, hh)
-            ref = vda_oracle.vda_slice(qs, ks, vs, bs, gs, 1e-6)["out"]
+            ref = vda_oracle.vda_slice(qs, ks, vs, bs, gs, 1e-6, **win)["out"]
             errs.append(vda_oracle.slice_error(out[b, :, :, hh, :].double().cpu().numpy(), ref))
             del qs, ks, vs, ref
         parity = {"metric": "max over a (batch, head) slice of |gpu - oracle| / max |oracle|", "slices": pairs,
@@ -300,6 +303,8 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     try:
         if args.skip_e2e:
             raise RuntimeError("skipped (--skip-e2e)")
+        if win != dict(chunk=1, radius=0, anchors=False):
+            raise RuntimeError("the host-buffer entry point has no window options")
         xh = {n: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for n, t in x.items()}
         outh = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
         e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -366,7 +371,8 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
                    "seed": w.seed, "parallelism": "single GPU" if world == 1 else f"{world} independent replicas",
                    "l2": "inputs+outputs far larger than the 126 MB L2; no flush" if ab["total"] > 1e9
                          else "inputs smaller than L2: numbers are L2-warm",
-                   "path": "tensor-core" if vda.launch_count() and any("tc" in n for n in kt) else "plain-fp32"},
+                   "path": "tensor-core" if vda.launch_count() and any("tc" in n for n in kt) else "plain-fp32",
+                   "window": win},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "parity": parity,
         "roofline": roof,
         "layer_roofline": {"t_roof_ms_measured_peaks": t_roof_ms, "frac_of_measured": t_roof_ms / (ms_max / 1.0),
@@ -389,6 +395,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--heads", type=int, default=0, help="override H (smaller cases for profiler captures)")
     ap.add_argument("--frames", type=int, default=0, help="override T (smaller cases for profiler captures)")
+    ap.add_argument("--chunk", type=int, default=1, help="frames per temporal chunk of the local window (1 = headline)")
+    ap.add_argument("--radius", type=int, default=0, help="chunks on either side inside the local window")
+    ap.add_argument("--anchors", type=int, default=0, help="1: first and last frame are boundary anchors")
+    ap.add_argument("--scan", default="auto", choices=["auto", "frames", "chunks"],
+                    help="scan schedule for chunk >= 2 (frame by frame / chunk-wise / the library's choice)")
     ap.add_argument("--skip-e2e", action="store_true", help="no host-buffer pass (profiler captures)")
     ap.add_argument("--skip-cpu", action="store_true", help="no CPU-oracle timing (profiler captures)")
     args = ap.parse_args()

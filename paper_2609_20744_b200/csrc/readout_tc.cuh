@@ -42,7 +42,8 @@ template <bool EXTRAS>
 __global__ void __launch_bounds__(ReadoutTc::THREADS, 1)
 readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmS,
                   const __grid_constant__ CUtensorMap tmO, const float* __restrict__ gate, Shape s, float eps,
-                  int* status, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight) {
+                  int* status, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight,
+                  Window win, int bridged) {
   using namespace tc;
   using R = ReadoutTc;
   extern __shared__ unsigned char smem_dyn[];
@@ -94,10 +95,13 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!mbar_wait(STEMPTY(0), (si & 1) ^ 1, wc)) { ok = false; break; }
         mbar_arrive_expect_tx(STFULL(0), 2 * R::TILE_BYTES);
         const uint32_t sdst = base + R::OFF_STATE;
-        // rows [n*128, +128) hold the forward state, rows [(frames+n)*128, +128) the reverse state
-        const long long nrev = s.frames() + n;
-        tma_load_2d(sdst, &tmS, STFULL(0), 0, (int)(n * R::D));
-        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(n * R::D));
+        // Slot of the forward state in rows [nf*128, +128), of the reverse state in rows [nrev*128, +128).  With
+        // decay gates every frame has its own (bridged) pair; without, the frames of a window share the states
+        // stored at the window's ends (slot l_t of the forward scan, slot h_t of the reverse scan; Eq. A.4).
+        const long long nf = bridged ? n : n - t + win.lo(t);
+        const long long nrev = s.frames() + (bridged ? n : n - t + win.hi(t));
+        tma_load_2d(sdst, &tmS, STFULL(0), 0, (int)(nf * R::D));
+        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(nf * R::D));
         tma_load_2d(sdst + 2 * R::BOX_BYTES, &tmS, STFULL(0), 0, (int)(nrev * R::D));
         tma_load_2d(sdst + 3 * R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(nrev * R::D));
         for (int tile = 0; tile < ntiles; ++tile, ++qi) {

@@ -21,7 +21,9 @@
 // P_{l_t - 1} Diag(prod_{r=l_t..t} alpha_r), slot t of `pb` what it reads from the reverse scan,
 // R_{h_t + 1} Diag(prod_{r=t..h_t} alpha_r), [l_t, h_t] being the frame's local window: whenever a chain reaches a
 // state that some frames read, it writes those frames' slots, bridged by their decay (with the default window
-// {t} that is one slot per step: P_t into slot t+1, R_t into slot t-1).  Frames whose window leaves no distant
+// {t} that is one slot per step: P_t into slot t+1, R_t into slot t-1).  Without a decay gate all readers of a
+// state read the same matrix; it is then stored once, in slot l_t (forward) / h_t (reverse), where the read-out
+// looks it up.  Frames whose window leaves no distant
 // frame on a side read the initial state (zero unless a text state is passed).  A chain stops after the last
 // state that anybody reads.  The read-out kernel adds the two slots in its accumulator (Eq. 1a).
 //
@@ -263,6 +265,18 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
       if (dir == 0 ? (bound != win.first && bound % win.chunk != 0) : (bound != win.last && (bound + 1) % win.chunk != 0))
         return;
       __nv_bfloat16* slots = (dir == 0 ? a.pf : a.pb) + (size_t)bh * T * (D * D) + (size_t)col0 * D + row;
+      if (a.alpha == nullptr) {
+        // no decay, no bridge: every reader of this state reads the same matrix, stored once in slot `bound`
+        // (the read-out looks up slot l_t / h_t)
+        __nv_bfloat16* dst = slots + (size_t)bound * (D * D);
+#pragma unroll
+        for (int e = 0; e < CW; e += 2) {
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(z[e], z[e + 1]);
+          dst[(size_t)e * D] = v2.x;
+          dst[(size_t)(e + 1) * D] = v2.y;
+        }
+        return;
+      }
       float bridge = 1.0f;
       int r = bound;                           // next frame whose decay enters the bridge
       const int far = dir == 0 ? min(win.last, bound + win.span()) : max(win.first, bound - win.span());
@@ -366,14 +380,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
       // then, under the next step's MMAs: the state after step s goes to the frames that read it.
       // Stored as bf16 [d_v][d_k] (the paper's orientation), so the 32 lanes of a warp (consecutive key
       // channels) write 64 contiguous bytes per value column.
+      // (the write and the decay for the step after are requested first: their latency passes under the stores)
+      if (writes && s + 1 + lead < nsteps) load_bt(s + 1 + lead, bt);
+      if (s + 2 < nsteps) a_next = step_decay(s + 2);
       if constexpr (MODE == SCAN_COMPOSE) {
         if (s + 1 == nsteps) store_composite(z);
       } else {
         store_readers(bound_after(s), z);
       }
-      // the write and the decay for the step after, also under the MMAs
-      if (writes && s + 1 + lead < nsteps) load_bt(s + 1 + lead, bt);
-      if (s + 2 < nsteps) a_next = step_decay(s + 2);
     }
   }
 

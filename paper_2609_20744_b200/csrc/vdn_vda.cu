@@ -373,10 +373,10 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   if (x.gate_elem || x.norm_weight || !gate)
     vdn::readout_tc_kernel<true><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
         tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
-        x.norm_weight);
+        x.norm_weight, x.win, x.alpha != nullptr);
   else
     vdn::readout_tc_kernel<false><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
-        tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev, nullptr, nullptr);
+        tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev, nullptr, nullptr, x.win, x.alpha != nullptr);
   prof_mark(h, st, nk++, "readout_tc");
   h->launches = nk;
   VDN_CUDA(h, cudaGetLastError());
