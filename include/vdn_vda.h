@@ -182,6 +182,36 @@ vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const 
  * chunk-level scan as its initial state.  Pure function; 0 on invalid arguments. */
 size_t vdn_vda_workspace_bytes_opt(vdn_vda_t h, int B, int T, int F, int H, int d, const vdn_vda_options* opt);
 
+/* Feature preparation in front of the layer (Sec. 2.3; the "VDA-Prep" kernel of Sec. 5): turns the projected
+ * q, k, v into the prepared features that vdn_vda_forward takes.
+ *      k' = L2norm( SiLU( conv(k) ) ),    v' = SiLU( conv(v) ),    q' = L2norm(q)
+ * conv is the separable short convolution of Sec. 2.3: per channel a 5 x 5 spatial filter over the frame's
+ * Y x X token grid and a five-tap temporal filter over the frames, applied as cross-correlations with centred
+ * taps and zero padding:  out[t,y,x,c] = sum_{i,j,l} wt[c,l] ws[c,i,j] in[t+l-2, y+i-2, x+j-2, c].
+ * L2norm(x) = x / sqrt(sum_j x_j^2 + l2_eps) over the d channels of a (token, head).  All arithmetic in fp32.
+ *
+ *   q_in, k_in, v_in, q_out, k_out, v_out : [B,T,F,H,d] of cfg.io_dtype, DEVICE, 16-byte aligned.  k_out and v_out
+ *        must not alias any input (the filters read neighbours); q_out may be q_in.
+ *   p->Y, p->X   the spatial grid: F = Y * X, tokens of a frame in row-major (y, x) order
+ *   p->wk_spatial, p->wv_spatial   float [H*d][5][5];   p->wk_temporal, p->wv_temporal   float [H*d][5]  (DEVICE)
+ *   p->anchors   non-zero: frames 0 and T-1 are boundary anchors, removed before the preparation (Alg. 1
+ *        step 2): the temporal filter sees zeros beyond frames 1 and T-2, and the anchor frames of all three
+ *        outputs are zero.
+ * Needs no workspace.  Enqueues on cuda_stream and returns; does not synchronise. */
+typedef struct {
+  uint32_t struct_size;      /* sizeof(vdn_vda_prep_params), checked */
+  int32_t Y, X;
+  int32_t anchors;
+  float l2_eps;              /* <= 0 selects 1e-6 */
+  const float* wk_spatial;
+  const float* wk_temporal;
+  const float* wv_spatial;
+  const float* wv_temporal;
+} vdn_vda_prep_params;
+vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const void* v_in, void* q_out,
+                           void* k_out, void* v_out, int B, int T, int F, int H, int d,
+                           const vdn_vda_prep_params* p, void* cuda_stream);
+
 /* The same layer for callers whose tensors live in HOST memory (pinned memory recommended): copies
  * q, k, v, beta, gate to the staging buffer, runs vdn_vda_forward, copies `out` back, all on
  * cuda_stream, and returns without synchronising.  All six tensor pointers are HOST pointers.  The

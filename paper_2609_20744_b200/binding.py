@@ -25,7 +25,7 @@ VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_R
 
 EXPORTS = (
     "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward", "vdn_vda_forward_ex",
-    "vdn_vda_forward_opt", "vdn_vda_workspace_bytes_opt",
+    "vdn_vda_forward_opt", "vdn_vda_workspace_bytes_opt", "vdn_vda_prepare",
     "vdn_vda_staging_bytes", "vdn_vda_set_staging", "vdn_vda_forward_host", "vdn_vda_workspace_view",
     "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_scan_static", "vdn_vda_status", "vdn_vda_last_error", "vdn_vda_destroy",
 )
@@ -40,6 +40,12 @@ class VdnOptions(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("chunk", ctypes.c_int32), ("radius", ctypes.c_int32),
                 ("anchors", ctypes.c_int32), ("alpha", ctypes.c_void_p), ("s0", ctypes.c_void_p),
                 ("gate_elem", ctypes.c_void_p), ("norm_weight", ctypes.c_void_p)]
+
+
+class VdnPrepParams(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("Y", ctypes.c_int32), ("X", ctypes.c_int32),
+                ("anchors", ctypes.c_int32), ("l2_eps", ctypes.c_float), ("wk_spatial", ctypes.c_void_p),
+                ("wk_temporal", ctypes.c_void_p), ("wv_spatial", ctypes.c_void_p), ("wv_temporal", ctypes.c_void_p)]
 
 
 class VdnError(RuntimeError):
@@ -82,6 +88,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.vdn_vda_forward_opt.restype = ci
     lib.vdn_vda_workspace_bytes_opt.argtypes = [vp, *shape, ctypes.POINTER(VdnOptions)]
     lib.vdn_vda_workspace_bytes_opt.restype = sz
+    lib.vdn_vda_prepare.argtypes = [vp, vp, vp, vp, vp, vp, vp, *shape, ctypes.POINTER(VdnPrepParams), vp]
+    lib.vdn_vda_prepare.restype = ci
     lib.vdn_vda_forward_host.argtypes = fwd_args
     lib.vdn_vda_forward_host.restype = ci
     lib.vdn_vda_workspace_view.argtypes = [vp, ci, *shape, ctypes.POINTER(sz), ctypes.POINTER(sz)]
@@ -237,6 +245,30 @@ class Vda:
                                           B, T, F, H, d, self._stream(stream))
         self._check(st)
         return out
+
+    def prepare(self, q, k, v, filters, Y, X, anchors=False, l2_eps=1e-6, out=None, stream=None):
+        """vdn_vda_prepare: projected q, k, v [B,T,F,H,d] -> prepared (q', k', v') (Sec. 2.3).
+
+        filters = dict(wk_spatial [H*d,5,5], wk_temporal [H*d,5], wv_spatial, wv_temporal), float32 CUDA tensors.
+        `out` = optional (q_out, k_out, v_out); q_out may be q itself.
+        """
+        torch = self._torch
+        B, T, F, H, d = q.shape
+        names = ("wk_spatial", "wk_temporal", "wv_spatial", "wv_temporal")
+        for x in (q, k, v, *(filters[n] for n in names)):
+            if not (x.is_cuda and x.is_contiguous()):
+                raise ValueError("vdn_vda_prepare needs contiguous CUDA tensors")
+        for n in names:
+            want = (H * d, 5, 5) if n.endswith("spatial") else (H * d, 5)
+            if tuple(filters[n].shape) != want or filters[n].dtype != torch.float32:
+                raise ValueError(f"{n} must be float32 {want}")
+        qo, ko, vo = out if out is not None else (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v))
+        p = lambda x: ctypes.c_void_p(x.data_ptr())
+        prm = VdnPrepParams(ctypes.sizeof(VdnPrepParams), Y, X, 1 if anchors else 0, l2_eps,
+                            *(filters[n].data_ptr() for n in names))
+        self._check(self.lib.vdn_vda_prepare(self.h, p(q), p(k), p(v), p(qo), p(ko), p(vo), B, T, F, H, d,
+                                             ctypes.byref(prm), self._stream(stream)))
+        return qo, ko, vo
 
     def forward_host(self, q, k, v, beta, gate, out, stream=None):
         """vdn_vda_forward_host on HOST tensors (pinned recommended); `out` is a host tensor too."""

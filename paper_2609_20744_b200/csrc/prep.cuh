@@ -1,0 +1,272 @@
+// Feature preparation in front of the recurrence (Sec. 2.3; "VDA-Prep", Sec. 5):
+//     K, V : depthwise 5 x 5 spatial filter and five-tap temporal filter (one pair per channel, taps centred,
+//            zero padding), then SiLU;      K, Q : L2 normalisation over the d channels of a (token, head).
+// One pass over K and V: every input element is read once from HBM (its halo re-reads hit L2), nothing
+// intermediate is written.
+//
+// prep_kv_kernel: one CTA per (head, spatial tile of ROWS x 8 tokens, batch, tensor) walks the frames in order.
+// A thread owns two neighbouring channels of the head (the two lanes of every packed fp32 FMA) and one tile row of
+// 8 tokens.  Per frame: the tile and its 2-token halo arrive in shared memory (cp.async, double buffered); the
+// thread slides along its row, five inputs per column, scattering each column into the (up to) five outputs it
+// touches, so an input is read from shared memory once per output row, not once per tap; the spatial result
+// enters a five-frame ring in registers, from which the temporal filter produces the frame two steps back;
+// SiLU; for K the sum of squares over the head's channels (warp shuffles, plus one shared-memory exchange when
+// the head spans two warps); store.  30 fused multiply-adds per element: this kernel is bound by the fp32 pipe.
+//
+// prep_q_kernel: L2 normalisation of Q, one warp per (token, head); bound by HBM.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace vdn {
+
+// ---- packed fp32 pairs (the two channels a thread owns)
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// two neighbouring channels from shared / to global memory
+__device__ __forceinline__ f32x2 load_pair(const __nv_bfloat16* p) {
+  const uint32_t u = *reinterpret_cast<const uint32_t*>(p);
+  return pack2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+}
+__device__ __forceinline__ f32x2 load_pair(const float* p) {
+  const float2 v = *reinterpret_cast<const float2*>(p);
+  return pack2(v.x, v.y);
+}
+__device__ __forceinline__ void store_pair(__nv_bfloat16* p, float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  *reinterpret_cast<__nv_bfloat162*>(p) = v;
+}
+__device__ __forceinline__ void store_pair(float* p, float lo, float hi) {
+  *reinterpret_cast<float2*>(p) = make_float2(lo, hi);
+}
+
+__device__ __forceinline__ float silu_f(float x) { return x * __frcp_rn(1.0f + __expf(-x)); }
+
+struct PrepKv {
+  static constexpr int TX = 8;          // tile columns = tokens per thread
+  static constexpr int HALO = 2;
+  static constexpr int THREADS = 256;
+  __host__ __device__ static constexpr int rows(int D) { return THREADS / (D / 2); }            // tile rows
+  __host__ __device__ static constexpr int tile_tokens(int D) { return (rows(D) + 2 * HALO) * (TX + 2 * HALO); }
+  static constexpr size_t smem_bytes(int D, int es) { return (size_t)2 * tile_tokens(D) * D * es + 64 * sizeof(float); }
+};
+
+struct PrepArgs {
+  const void* in[2];          // k, v   [B,T,F,H,d]
+  void* out[2];
+  const float* ws[2];         // spatial filters  [H*d][5][5]
+  const float* wt[2];         // temporal filters [H*d][5]
+  int Y, X;                   // F = Y * X, tokens of a frame in row-major (y, x) order
+  float l2_eps;
+};
+
+template <typename Tio, int D>
+__global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a, Shape s) {
+  using P = PrepKv;
+  constexpr int ROWS = P::rows(D);
+  constexpr int TX = P::TX, HALO = P::HALO;
+  constexpr int SW = TX + 2 * HALO, SH = ROWS + 2 * HALO;       // tile with halo
+  constexpr int GT = D / 2;                                      // threads per tile row (one head's channel pairs)
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Tio* tile = reinterpret_cast<Tio*>(smem_raw);                  // [2][SH][SW][D]
+  float* red = reinterpret_cast<float*>(smem_raw + (size_t)2 * SH * SW * D * sizeof(Tio));   // [ROWS][TX] exchange
+
+  const int h = blockIdx.x;
+  const int tiles_x = (a.X + TX - 1) / TX;
+  const int x0 = (blockIdx.y % tiles_x) * TX, y0 = (blockIdx.y / tiles_x) * ROWS;
+  const int which = blockIdx.z & 1;                              // 0 = K (normalised), 1 = V
+  const int b = blockIdx.z >> 1;
+  const Tio* __restrict__ src = static_cast<const Tio*>(a.in[which]);
+  Tio* __restrict__ dst = static_cast<Tio*>(a.out[which]);
+
+  const int tid = threadIdx.x;
+  const int g = tid / GT;                   // tile row of this thread
+  const int cp = tid % GT;                  // channel pair within the head
+  const int ch = h * D + 2 * cp;            // first of this thread's two channels, [H*d] index
+
+  // this thread's filters, both channels packed: 25 spatial + 5 temporal taps
+  f32x2 wsp[5][5], wtp[5];
+  {
+    const float* w0 = a.ws[which] + (size_t)ch * 25;
+#pragma unroll
+    for (int i = 0; i < 5; ++i)
+#pragma unroll
+      for (int j = 0; j < 5; ++j) wsp[i][j] = pack2(__ldg(w0 + i * 5 + j), __ldg(w0 + 25 + i * 5 + j));
+    const float* t0 = a.wt[which] + (size_t)ch * 5;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) wtp[i] = pack2(__ldg(t0 + i), __ldg(t0 + 5 + i));
+  }
+
+  const int first = s.t0, last = s.t0 + s.Tn - 1;
+
+  // frame t's tile (with halo) -> buffer t & 1; tokens outside the frame are zeros
+  auto stage = [&](int t) {
+    Tio* buf = tile + (size_t)(t & 1) * SH * SW * D;
+    constexpr int CHUNKS = D * (int)sizeof(Tio) / 16;            // 16-byte pieces per token
+    for (int e = tid; e < SH * SW * CHUNKS; e += P::THREADS) {
+      const int c = e % CHUNKS, tok = e / CHUNKS;
+      const int yy = y0 - HALO + tok / SW, xx = x0 - HALO + tok % SW;
+      unsigned char* d8 = reinterpret_cast<unsigned char*>(buf + (size_t)tok * D) + c * 16;
+      if (yy >= 0 && yy < a.Y && xx >= 0 && xx < a.X) {
+        const Tio* p = src + token_offset(s, b, t, yy * a.X + xx, h);
+        cp_async16(d8, reinterpret_cast<const unsigned char*>(p) + c * 16);
+      } else {
+        *reinterpret_cast<uint4*>(d8) = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+    cp_async_commit();
+  };
+
+  f32x2 ring[5][TX];                        // spatial results of the last five frames (slot = step % 5)
+#pragma unroll
+  for (int i = 0; i < 5; ++i)
+#pragma unroll
+    for (int j = 0; j < TX; ++j) ring[i][j] = 0ull;
+
+  const int nsteps = s.Tn + HALO;           // two extra steps flush the last two output frames
+  stage(first);
+#pragma unroll 1
+  for (int sb = 0; sb < nsteps; sb += 5) {
+#pragma unroll
+    for (int r = 0; r < 5; ++r) {           // ring slot r is static: sb is a multiple of five
+      const int step = sb + r;
+      if (step >= nsteps) break;
+      const int t = first + step;           // input frame of this step; the output frame is t - 2
+      if (t <= last) {
+        if (t + 1 <= last) { stage(t + 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+        __syncthreads();
+        // ---- spatial filter of frame t for this thread's row: slide over the SW input columns
+        const Tio* base = tile + (size_t)(t & 1) * SH * SW * D + (size_t)g * SW * D + 2 * cp;
+        f32x2 acc[TX];
+#pragma unroll
+        for (int j = 0; j < TX; ++j) acc[j] = 0ull;
+#pragma unroll
+        for (int xi = 0; xi < SW; ++xi) {   // input column xi sits at x0 - 2 + xi
+          f32x2 in[5];
+#pragma unroll
+          for (int i = 0; i < 5; ++i) in[i] = load_pair(base + ((size_t)i * SW + xi) * D);
+#pragma unroll
+          for (int j = 0; j < 5; ++j) {     // tap column j: output column xo = xi - j
+            const int xo = xi - j;
+            if (xo < 0 || xo >= TX) continue;
+#pragma unroll
+            for (int i = 0; i < 5; ++i) acc[xo] = fma2(wsp[i][j], in[i], acc[xo]);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < TX; ++j) ring[r][j] = acc[j];
+        __syncthreads();                    // the buffer may be overwritten by the copy issued two steps on
+      } else {
+#pragma unroll
+        for (int j = 0; j < TX; ++j) ring[r][j] = 0ull;
+      }
+      // ---- temporal filter: output frame to = t - 2 = sum_i wt[i] S[to + i - 2]; S[to + i - 2] sits in slot (r + i + 1) % 5
+      const int to = t - HALO;
+      if (to < first) continue;
+      float o0[TX], o1[TX];
+#pragma unroll
+      for (int j = 0; j < TX; ++j) {
+        f32x2 o = mul2(wtp[0], ring[(r + 1) % 5][j]);
+#pragma unroll
+        for (int i = 1; i < 5; ++i) o = fma2(wtp[i], ring[(r + i + 1) % 5][j], o);
+        unpack2(o, o0[j], o1[j]);
+        o0[j] = silu_f(o0[j]);
+        o1[j] = silu_f(o1[j]);
+      }
+      const int y = y0 + g;
+      if (which == 0) {
+        // ---- L2 normalisation over the head's d channels (Sec. 2.3)
+        float ss[TX];
+#pragma unroll
+        for (int j = 0; j < TX; ++j) {
+          ss[j] = fmaf(o0[j], o0[j], o1[j] * o1[j]);
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) ss[j] += __shfl_xor_sync(0xffffffffu, ss[j], off);
+        }
+        if constexpr (GT == 64) {           // the head spans two warps: exchange the partial sums
+          const int wv = (tid >> 5) & 1;
+          float* mine = red + (g * 2 + wv) * TX;
+          if ((tid & 31) == 0) {
+#pragma unroll
+            for (int j = 0; j < TX; ++j) mine[j] = ss[j];
+          }
+          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(GT) : "memory");
+          const float* other = red + (g * 2 + (wv ^ 1)) * TX;
+#pragma unroll
+          for (int j = 0; j < TX; ++j) ss[j] += other[j];
+          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(GT) : "memory");
+        }
+#pragma unroll
+        for (int j = 0; j < TX; ++j) {
+          const float sc = rsqrtf(ss[j] + a.l2_eps);
+          o0[j] *= sc;
+          o1[j] *= sc;
+        }
+      }
+      if (y < a.Y) {
+#pragma unroll
+        for (int j = 0; j < TX; ++j) {
+          const int x = x0 + j;
+          if (x < a.X) store_pair(dst + token_offset(s, b, to, y * a.X + x, h) + 2 * cp, o0[j], o1[j]);
+        }
+      }
+    }
+  }
+}
+
+// L2 normalisation of Q over the d channels of each (token, head); one warp per (token, head), 16-byte accesses
+// for bf16 at d = 128.  In place is fine.
+template <typename Tio, int D>
+__global__ void __launch_bounds__(256) prep_q_kernel(const Tio* __restrict__ q, Tio* __restrict__ out, Shape s,
+                                                      float eps) {
+  constexpr int PER = D / 32;                  // channels per lane: 4 (d = 128) or 2 (d = 64)
+  const int lane = threadIdx.x & 31;
+  const long long per_frame = (long long)s.F * s.H;
+  const long long total = (long long)s.B * s.Tn * per_frame;
+  for (long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); w < total; w += (long long)gridDim.x * 8) {
+    const long long bt = w / per_frame;
+    const int b = (int)(bt / s.Tn), t = s.t0 + (int)(bt % s.Tn);
+    const size_t off = (((size_t)b * s.T + t) * per_frame + (size_t)(w % per_frame)) * D + lane * PER;
+    float x[PER];
+    if constexpr (PER == 4) {
+      const float4 v = load4(q + off);
+      x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    } else {
+      x[0] = to_float(q[off]);
+      x[1] = to_float(q[off + 1]);
+    }
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) ss = fmaf(x[i], x[i], ss);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const float sc = rsqrtf(ss + eps);
+    if constexpr (PER == 4) {
+      store4(out + off, make_float4(x[0] * sc, x[1] * sc, x[2] * sc, x[3] * sc));
+    } else {
+      out[off] = from_float<Tio>(x[0] * sc);
+      out[off + 1] = from_float<Tio>(x[1] * sc);
+    }
+  }
+}
+
+}  // namespace vdn

@@ -15,6 +15,7 @@
 #include "common.cuh"
 #include "gram_simt.cuh"
 #include "gram_tc.cuh"
+#include "prep.cuh"
 #include "readout_simt.cuh"
 #include "readout_tc.cuh"
 #include "resolve.cuh"
@@ -413,6 +414,32 @@ vdn_status launch_scan_static(const float* stats, const float* inv, float* read,
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Feature preparation: two launches (K and V in one, Q in the other).
+template <typename Tio, int D>
+vdn_status launch_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const void* v_in, void* q_out, void* k_out,
+                          void* v_out, const Shape& s, const vdn_vda_prep_params& p, cudaStream_t st) {
+  using P = vdn::PrepKv;
+  const size_t smem = P::smem_bytes(D, (int)sizeof(Tio));
+  VDN_CUDA(h, cudaFuncSetAttribute(vdn::prep_kv_kernel<Tio, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  vdn::PrepArgs a;
+  a.in[0] = k_in; a.in[1] = v_in; a.out[0] = k_out; a.out[1] = v_out;
+  a.ws[0] = p.wk_spatial; a.ws[1] = p.wv_spatial; a.wt[0] = p.wk_temporal; a.wt[1] = p.wv_temporal;
+  a.Y = p.Y; a.X = p.X;
+  a.l2_eps = p.l2_eps > 0.f ? p.l2_eps : 1e-6f;
+  const int tiles = ((p.X + P::TX - 1) / P::TX) * ((p.Y + P::rows(D) - 1) / P::rows(D));
+  prof_begin(h, st);
+  vdn::prep_kv_kernel<Tio, D><<<dim3((unsigned)s.H, (unsigned)tiles, (unsigned)(2 * s.B)), P::THREADS, smem, st>>>(a, s);
+  prof_mark(h, st, 0, "prep_kv");
+  const long long rows = (long long)s.B * s.Tn * s.F * s.H;
+  const long long want = (rows + 7) / 8;
+  const unsigned grid = (unsigned)(want < (long long)h->sm_count * 16 ? want : (long long)h->sm_count * 16);
+  vdn::prep_q_kernel<Tio, D><<<grid, 256, 0, st>>>(static_cast<const Tio*>(q_in), static_cast<Tio*>(q_out), s, a.l2_eps);
+  prof_mark(h, st, 1, "prep_q");
+  h->launches = 2;
+  VDN_CUDA(h, cudaGetLastError());
+  return VDN_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -570,6 +597,53 @@ vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const 
   }
   return d == 64 ? forward_simt<__nv_bfloat16, 64>(h, q, k, v, beta, gate, x, out, s, L, st)
                  : forward_simt<__nv_bfloat16, 128>(h, q, k, v, beta, gate, x, out, s, L, st);
+}
+
+vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const void* v_in, void* q_out, void* k_out,
+                           void* v_out, int B, int T, int F, int H, int d, const vdn_vda_prep_params* p,
+                           void* cuda_stream) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  if (!p || p->struct_size != sizeof(vdn_vda_prep_params))
+    return fail(h, VDN_ERR_INVALID_ARG, "vdn_vda_prep_params missing or of the wrong struct_size");
+  if (!q_in || !k_in || !v_in || !q_out || !k_out || !v_out || !p->wk_spatial || !p->wk_temporal || !p->wv_spatial ||
+      !p->wv_temporal)
+    return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
+  if (!aligned16(q_in) || !aligned16(k_in) || !aligned16(v_in) || !aligned16(q_out) || !aligned16(k_out) ||
+      !aligned16(v_out) || !aligned16(p->wk_spatial) || !aligned16(p->wk_temporal) || !aligned16(p->wv_spatial) ||
+      !aligned16(p->wv_temporal))
+    return fail(h, VDN_ERR_INVALID_ARG, "tensors and filters must be 16-byte aligned");
+  if (k_out == k_in || k_out == v_in || v_out == k_in || v_out == v_in || k_out == v_out || k_out == q_in ||
+      v_out == q_in || q_out == k_in || q_out == v_in || q_out == k_out || q_out == v_out)
+    return fail(h, VDN_ERR_INVALID_ARG, "k_out and v_out must not alias anything (only q_out may equal q_in)");
+  std::string why;
+  if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
+  if (p->Y <= 0 || p->X <= 0 || (long long)p->Y * p->X != F)
+    return fail(h, VDN_ERR_INVALID_ARG, "Y * X must equal F");
+  if (H > 65535 || 2LL * B > 65535 || ((long long)(p->X + 7) / 8) * ((p->Y + 3) / 4) > 65535)
+    return fail(h, VDN_ERR_UNSUPPORTED, "grid too large for the preparation kernel");
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const bool anchors = p->anchors != 0;
+  const Shape s{B, T, F, H, d, anchors ? 1 : 0, anchors ? T - 2 : T};
+  h->launches = 0;
+  if (anchors) {
+    // anchor frames are removed before the preparation (Alg. 1 step 2): they come out as zeros
+    const size_t frame_bytes = (size_t)F * H * d * elem_size(h);
+    void* outs[3] = {q_out, k_out, v_out};
+    for (void* o : outs)
+      for (int b = 0; b < B; ++b) {
+        VDN_CUDA(h, cudaMemsetAsync(static_cast<char*>(o) + (size_t)b * T * frame_bytes, 0, frame_bytes, st));
+        if (T > 1)
+          VDN_CUDA(h, cudaMemsetAsync(static_cast<char*>(o) + ((size_t)b * T + T - 1) * frame_bytes, 0, frame_bytes, st));
+      }
+    if (s.Tn <= 0) return VDN_OK;
+  }
+  if (h->cfg.io_dtype == VDN_F32)
+    return d == 64 ? launch_prepare<float, 64>(h, q_in, k_in, v_in, q_out, k_out, v_out, s, *p, st)
+                   : launch_prepare<float, 128>(h, q_in, k_in, v_in, q_out, k_out, v_out, s, *p, st);
+  return d == 64 ? launch_prepare<__nv_bfloat16, 64>(h, q_in, k_in, v_in, q_out, k_out, v_out, s, *p, st)
+                 : launch_prepare<__nv_bfloat16, 128>(h, q_in, k_in, v_in, q_out, k_out, v_out, s, *p, st);
 }
 
 vdn_status vdn_vda_forward_ex(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,

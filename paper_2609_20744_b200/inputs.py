@@ -143,6 +143,33 @@ def generate_output_extras(w: VdaWorkload, device="cpu"):
     return gate_elem.contiguous(), norm_weight.contiguous()
 
 
+def generate_projected(w: VdaWorkload, device="cpu"):
+    """Seeded stand-ins for the projected (not yet prepared) q, k, v [B,T,F,H,d] ~ N(0,1) in the I/O dtype and
+    for the short-convolution filters of the feature preparation: per channel a 5 x 5 spatial and a five-tap
+    temporal filter, drawn as a unit centre tap plus N(0, 0.15^2) on every tap (a trained short filter stays
+    close to the identity it is initialised with).  Filters are float32."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    out = {}
+    for i, n in enumerate(("q", "k", "v")):
+        x = torch.empty((w.B, w.T, w.F, w.H, w.d), device=dev, dtype=w.torch_dtype)
+        for b in range(w.B):
+            for t in range(w.T):
+                g.manual_seed(_seed(w.seed, 0x9E0 + i, b, t))
+                x[b, t].copy_(torch.randn((w.F, w.H, w.d), generator=g, device=dev))
+        out[n] = x
+    g.manual_seed(_seed(w.seed, 0xF17))
+    C = w.H * w.d
+    for n in ("wk", "wv"):
+        ws = 0.15 * torch.randn((C, 5, 5), generator=g, device=dev)
+        ws[:, 2, 2] += 1.0
+        wt = 0.15 * torch.randn((C, 5), generator=g, device=dev)
+        wt[:, 2] += 1.0
+        out[n + "_spatial"] = ws.contiguous()
+        out[n + "_temporal"] = wt.contiguous()
+    return out
+
+
 def head_slice(x: dict, b: int, h: int):
     """Host float64 numpy copies of one (batch, head) slice: q,k,v [T,F,d], beta [T,F], gate scalar."""
     import numpy as np
