@@ -385,6 +385,110 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     print(json.dumps(line), flush=True)
 
 
+def run_prep(args, w, local_rank: int):
+    """--stage prep: the feature preparation in front of the layer (Sec. 2.3), timed on the same shape.  Not part
+    of the headline step; one JSON line of the same form, `roofline` against the fp32 pipe that bounds it."""
+    import torch
+    from paper_2609_20744_b200 import binding, build, inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the VDA library has no CPU fallback")
+    build.build()
+    torch.cuda.set_device(local_rank)
+    Y, X = args.grid
+    if Y * X != w.F:
+        raise SystemExit(f"--grid {Y}x{X} does not give F = {w.F}")
+    p = inputs.generate_projected(w, f"cuda:{local_rank}")
+    vda = binding.Vda(w.d, w.dtype, device=local_rank)
+    outs = tuple(torch.empty_like(p[n]) for n in "qkv")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        vda.prepare(p["q"], p["k"], p["v"], p, Y, X, out=outs)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    vda.profile(True)
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    kt = {n: m for n, m, _ in vda.kernel_times()}
+    vda.profile(False)
+    clocks = sampler.summary(t0, t1)
+    sampler.stop()
+
+    # parity of this launch on a sample the oracle can afford: one head, one output frame in the middle of the
+    # clip (the oracle gets the five frames the temporal filter reaches), every token of that frame
+    parity = None
+    if not args.skip_cpu:
+        from oracle import prep_oracle, vda_oracle
+        tol = 1e-4 if w.dtype == "f32" else 2e-2
+        b, h, tc = w.B - 1, w.H - 1, w.T // 2
+        lo, hi = max(0, tc - 2), min(w.T, tc + 3)
+        f = lambda t: t.detach().double().cpu().numpy()
+        sl = slice(h * w.d, (h + 1) * w.d)
+        ref = prep_oracle.prepare(f(p["q"][b, lo:hi, :, h]), f(p["k"][b, lo:hi, :, h]), f(p["v"][b, lo:hi, :, h]),
+                                  f(p["wk_spatial"][sl]), f(p["wk_temporal"][sl]), f(p["wv_spatial"][sl]),
+                                  f(p["wv_temporal"][sl]), Y, X)
+        errs = [vda_oracle.slice_error(f(o[b, tc, :, h]), r[tc - lo]) for o, r in zip(outs, ref)]
+        parity = {"metric": "max |gpu - oracle| / max |oracle| over the sampled frame, for q', k', v'",
+                  "sample": f"batch {b}, head {h}, frame {tc} (needs frames {lo}..{hi - 1} of the input)",
+                  "errors": errs, "tolerance": tol, "ok": bool(max(errs) <= tol)}
+
+    es = 4 if w.dtype == "f32" else 2
+    elems = w.B * w.T * w.F * w.H * w.d
+    alg_bytes = 6 * elems * es                       # q, k, v read once and written once
+    flops = 2 * elems * 2 * 30                       # K and V: 25 + 5 fused multiply-adds per element
+    prop = torch.cuda.get_device_properties(local_rank)
+    alu_peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+    peaks = measured_peaks()
+    dom = max(kt, key=kt.get) if kt else None
+    roof = None
+    if dom == "prep_kv":
+        achieved = flops / (kt[dom] / 1e3) / 1e12
+        roof = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
+                "frac": achieved / alu_peak, "traffic": None,
+                "peak_source": f"{prop.multi_processor_count} SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                "kernel_ms": kt[dom], "hbm_GBps_of_this_kernel": 4 * elems * es / (kt[dom] / 1e3) / 1e9}
+    base = None
+    if not args.skip_cpu:
+        from oracle import prep_oracle
+        f = lambda t: t.detach().double().cpu().numpy()
+        nfr = min(w.T, 6)
+        sl = slice(0, w.d)
+        args_o = (f(p["q"][0, :nfr, :, 0]), f(p["k"][0, :nfr, :, 0]), f(p["v"][0, :nfr, :, 0]), f(p["wk_spatial"][sl]),
+                  f(p["wk_temporal"][sl]), f(p["wv_spatial"][sl]), f(p["wv_temporal"][sl]), Y, X)
+        c0 = time.perf_counter()
+        prep_oracle.prepare(*args_o)
+        sec = time.perf_counter() - c0
+        base = {"value": w.tokens / (sec * w.B * w.H * w.T / nfr), "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                "sample": f"1 of {w.B * w.H} (batch, head) slices x {nfr} of {w.T} frames; rate scaled by the unit count",
+                "seconds_sample": sec}
+    line = {
+        "metric": "vda_prep_tokens_per_s", "value": w.tokens / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 arithmetic on bf16 I/O" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "stage": "prep", "B": w.B, "T": w.T, "F": w.F, "Y": Y, "X": X, "H": w.H, "d": w.d,
+                   "io_dtype": w.dtype, "l2": "inputs+outputs far larger than the 126 MB L2; no flush"},
+        "clocks": clocks, "gpu_launches": vda.launch_count() * args.steps, "parity": parity, "roofline": roof,
+        "stage_roofline": {"t_alu_ms": flops / (alu_peak * 1e12) * 1e3, "t_hbm_ms": alg_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                           "algorithmic_bytes": alg_bytes, "fp32_flops": flops},
+        "kernel_ms": kt, "cpu_baseline": base,
+        "context": "paper (context only): VDA-Prep 17.1 -> 3.4 ms on B200 at 102 latent frames (Sec. 4.3)",
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -400,6 +504,10 @@ def main():
     ap.add_argument("--anchors", type=int, default=0, help="1: first and last frame are boundary anchors")
     ap.add_argument("--scan", default="auto", choices=["auto", "frames", "chunks"],
                     help="scan schedule for chunk >= 2 (frame by frame / chunk-wise / the library's choice)")
+    ap.add_argument("--stage", default="layer", choices=["layer", "prep"],
+                    help="layer = the headline step; prep = the feature preparation in front of it (1 GPU)")
+    ap.add_argument("--grid", type=lambda v: tuple(int(x) for x in v.split("x")), default=(48, 85),
+                    help="YxX token grid of a frame for --stage prep (768p: 48x85)")
     ap.add_argument("--skip-e2e", action="store_true", help="no host-buffer pass (profiler captures)")
     ap.add_argument("--skip-cpu", action="store_true", help="no CPU-oracle timing (profiler captures)")
     args = ap.parse_args()
@@ -417,6 +525,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, w, rank, world)
+        return
+    if args.stage == "prep":
+        if rank == 0:
+            run_prep(args, w, local_rank)
         return
     if world > 1:
         import torch

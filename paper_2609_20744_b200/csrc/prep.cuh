@@ -59,7 +59,14 @@ __device__ __forceinline__ void store_pair(float* p, float lo, float hi) {
   *reinterpret_cast<float2*>(p) = make_float2(lo, hi);
 }
 
-__device__ __forceinline__ float silu_f(float x) { return x * __frcp_rn(1.0f + __expf(-x)); }
+// SiLU(x) = x / (1 + 2^(-x log2 e)) with the hardware exponential and reciprocal (each good to about 2^-22
+// relative): five instructions per element, and this kernel is bound by instruction issue.
+__device__ __forceinline__ float silu_f(float x) {
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-1.4426950408889634f * x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return x * r;
+}
 
 struct PrepKv {
   static constexpr int TX = 8;          // tile columns = tokens per thread
@@ -95,8 +102,8 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
   const int x0 = (blockIdx.y % tiles_x) * TX, y0 = (blockIdx.y / tiles_x) * ROWS;
   const int which = blockIdx.z & 1;                              // 0 = K (normalised), 1 = V
   const int b = blockIdx.z >> 1;
-  const Tio* __restrict__ src = static_cast<const Tio*>(a.in[which]);
-  Tio* __restrict__ dst = static_cast<Tio*>(a.out[which]);
+  const Tio* __restrict__ src = static_cast<const Tio*>(which == 0 ? a.in[0] : a.in[1]);
+  Tio* __restrict__ dst = static_cast<Tio*>(which == 0 ? a.out[0] : a.out[1]);
 
   const int tid = threadIdx.x;
   const int g = tid / GT;                   // tile row of this thread
@@ -106,31 +113,44 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
   // this thread's filters, both channels packed: 25 spatial + 5 temporal taps
   f32x2 wsp[5][5], wtp[5];
   {
-    const float* w0 = a.ws[which] + (size_t)ch * 25;
+    const float* w0 = (which == 0 ? a.ws[0] : a.ws[1]) + (size_t)ch * 25;
 #pragma unroll
     for (int i = 0; i < 5; ++i)
 #pragma unroll
       for (int j = 0; j < 5; ++j) wsp[i][j] = pack2(__ldg(w0 + i * 5 + j), __ldg(w0 + 25 + i * 5 + j));
-    const float* t0 = a.wt[which] + (size_t)ch * 5;
+    const float* t0 = (which == 0 ? a.wt[0] : a.wt[1]) + (size_t)ch * 5;
 #pragma unroll
     for (int i = 0; i < 5; ++i) wtp[i] = pack2(__ldg(t0 + i), __ldg(t0 + 5 + i));
   }
 
   const int first = s.t0, last = s.t0 + s.Tn - 1;
+  // this thread's first output element of frame 0: token (y0 + g, x0), its channel pair
+  Tio* dst_b = dst + token_offset(s, b, 0, min(y0 + g, a.Y - 1) * a.X + x0, h) + 2 * cp;
 
-  // frame t's tile (with halo) -> buffer t & 1; tokens outside the frame are zeros
+  // Frame t's tile (with halo) -> buffer t & 1; tokens outside the frame are zeros.  A thread copies the same
+  // 16-byte pieces of every frame, so their offsets inside a frame are worked out once (-1: outside the frame).
+  constexpr int CHUNKS = D * (int)sizeof(Tio) / 16;              // 16-byte pieces per token
+  constexpr int NPIECE = (SH * SW * CHUNKS + P::THREADS - 1) / P::THREADS;
+  int goff[NPIECE];                                              // byte offset inside the frame, or -1
+#pragma unroll
+  for (int i = 0; i < NPIECE; ++i) {
+    const int e = tid + i * P::THREADS;
+    const int c = e % CHUNKS, tok = e / CHUNKS;
+    const int yy = y0 - HALO + tok / SW, xx = x0 - HALO + tok % SW;
+    const bool in = e < SH * SW * CHUNKS && yy >= 0 && yy < a.Y && xx >= 0 && xx < a.X;
+    goff[i] = in ? (int)((((size_t)(yy * a.X + xx) * s.H + h) * D) * sizeof(Tio)) + c * 16 : -1;
+  }
+  const size_t frame_bytes = (size_t)s.F * s.H * D * sizeof(Tio);
+  const unsigned char* src_b = reinterpret_cast<const unsigned char*>(src) + (size_t)b * s.T * frame_bytes;
   auto stage = [&](int t) {
-    Tio* buf = tile + (size_t)(t & 1) * SH * SW * D;
-    constexpr int CHUNKS = D * (int)sizeof(Tio) / 16;            // 16-byte pieces per token
-    for (int e = tid; e < SH * SW * CHUNKS; e += P::THREADS) {
-      const int c = e % CHUNKS, tok = e / CHUNKS;
-      const int yy = y0 - HALO + tok / SW, xx = x0 - HALO + tok % SW;
-      unsigned char* d8 = reinterpret_cast<unsigned char*>(buf + (size_t)tok * D) + c * 16;
-      if (yy >= 0 && yy < a.Y && xx >= 0 && xx < a.X) {
-        const Tio* p = src + token_offset(s, b, t, yy * a.X + xx, h);
-        cp_async16(d8, reinterpret_cast<const unsigned char*>(p) + c * 16);
-      } else {
-        *reinterpret_cast<uint4*>(d8) = make_uint4(0u, 0u, 0u, 0u);
+    unsigned char* buf = reinterpret_cast<unsigned char*>(tile) + (size_t)(t & 1) * SH * SW * D * sizeof(Tio);
+    const unsigned char* fr = src_b + (size_t)t * frame_bytes;
+#pragma unroll
+    for (int i = 0; i < NPIECE; ++i) {
+      const int e = tid + i * P::THREADS;
+      if (e < SH * SW * CHUNKS) {
+        if (goff[i] >= 0) cp_async16(buf + (size_t)e * 16, fr + goff[i]);
+        else *reinterpret_cast<uint4*>(buf + (size_t)e * 16) = make_uint4(0u, 0u, 0u, 0u);
       }
     }
     cp_async_commit();
@@ -165,11 +185,13 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
 #pragma unroll
           for (int i = 0; i < 5; ++i) in[i] = load_pair(base + ((size_t)i * SW + xi) * D);
 #pragma unroll
-          for (int j = 0; j < 5; ++j) {     // tap column j: output column xo = xi - j
-            const int xo = xi - j;
-            if (xo < 0 || xo >= TX) continue;
+          for (int i = 0; i < 5; ++i) {     // neighbouring instructions update different accumulators
 #pragma unroll
-            for (int i = 0; i < 5; ++i) acc[xo] = fma2(wsp[i][j], in[i], acc[xo]);
+            for (int j = 0; j < 5; ++j) {   // tap column j: output column xo = xi - j
+              const int xo = xi - j;
+              if (xo < 0 || xo >= TX) continue;
+              acc[xo] = fma2(wsp[i][j], in[i], acc[xo]);
+            }
           }
         }
 #pragma unroll
@@ -223,48 +245,76 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
         }
       }
       if (y < a.Y) {
+        Tio* orow = dst_b + (size_t)to * ((size_t)s.F * s.H * D);
 #pragma unroll
-        for (int j = 0; j < TX; ++j) {
-          const int x = x0 + j;
-          if (x < a.X) store_pair(dst + token_offset(s, b, to, y * a.X + x, h) + 2 * cp, o0[j], o1[j]);
-        }
+        for (int j = 0; j < TX; ++j)
+          if (x0 + j < a.X) store_pair(orow + (size_t)j * (s.H * D), o0[j], o1[j]);
       }
     }
   }
 }
 
-// L2 normalisation of Q over the d channels of each (token, head); one warp per (token, head), 16-byte accesses
-// for bf16 at d = 128.  In place is fine.
+// L2 normalisation of Q over the d channels of each (token, head).  A (token, head) row is D * sizeof(Tio) / 16
+// 16-byte pieces, one per lane; a warp covers 32 / that many rows at once and four such groups per trip, so that
+// enough loads are in flight to stream from HBM.  In place is fine.
 template <typename Tio, int D>
 __global__ void __launch_bounds__(256) prep_q_kernel(const Tio* __restrict__ q, Tio* __restrict__ out, Shape s,
                                                       float eps) {
-  constexpr int PER = D / 32;                  // channels per lane: 4 (d = 128) or 2 (d = 64)
+  constexpr int EPL = 16 / (int)sizeof(Tio);   // elements per lane
+  constexpr int LPR = D / EPL;                 // lanes per row
+  constexpr int RPW = 32 / LPR;                // rows per warp
+  constexpr int UN = 4;
   const int lane = threadIdx.x & 31;
+  const int sub = lane / LPR, li = lane % LPR;
   const long long per_frame = (long long)s.F * s.H;
   const long long total = (long long)s.B * s.Tn * per_frame;
-  for (long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); w < total; w += (long long)gridDim.x * 8) {
-    const long long bt = w / per_frame;
-    const int b = (int)(bt / s.Tn), t = s.t0 + (int)(bt % s.Tn);
-    const size_t off = (((size_t)b * s.T + t) * per_frame + (size_t)(w % per_frame)) * D + lane * PER;
-    float x[PER];
-    if constexpr (PER == 4) {
-      const float4 v = load4(q + off);
-      x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-    } else {
-      x[0] = to_float(q[off]);
-      x[1] = to_float(q[off + 1]);
+  const long long stride = (long long)gridDim.x * 8 * RPW * UN;
+  for (long long w0 = ((long long)blockIdx.x * 8 + (threadIdx.x >> 5)) * RPW * UN; w0 < total; w0 += stride) {
+    uint4 raw[UN];
+    size_t off[UN];
+    bool ok[UN];
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      const long long w = w0 + u * RPW + sub;
+      ok[u] = w < total;
+      const long long ww = ok[u] ? w : 0;
+      const long long bt = ww / per_frame;
+      const int b = (int)(bt / s.Tn), t = s.t0 + (int)(bt % s.Tn);
+      off[u] = (((size_t)b * s.T + t) * per_frame + (size_t)(ww % per_frame)) * D + li * EPL;
+      raw[u] = ok[u] ? __ldg(reinterpret_cast<const uint4*>(q + off[u])) : make_uint4(0u, 0u, 0u, 0u);
     }
-    float ss = 0.f;
 #pragma unroll
-    for (int i = 0; i < PER; ++i) ss = fmaf(x[i], x[i], ss);
+    for (int u = 0; u < UN; ++u) {
+      float x[EPL];
+      if constexpr (sizeof(Tio) == 2) {
+        const uint32_t* r = reinterpret_cast<const uint32_t*>(&raw[u]);
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    const float sc = rsqrtf(ss + eps);
-    if constexpr (PER == 4) {
-      store4(out + off, make_float4(x[0] * sc, x[1] * sc, x[2] * sc, x[3] * sc));
-    } else {
-      out[off] = from_float<Tio>(x[0] * sc);
-      out[off + 1] = from_float<Tio>(x[1] * sc);
+        for (int i = 0; i < 4; ++i) { x[2 * i] = __uint_as_float(r[i] << 16); x[2 * i + 1] = __uint_as_float(r[i] & 0xFFFF0000u); }
+      } else {
+        const float* r = reinterpret_cast<const float*>(&raw[u]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) x[i] = r[i];
+      }
+      float ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < EPL; ++i) ss = fmaf(x[i], x[i], ss);
+#pragma unroll
+      for (int o = LPR / 2; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      const float sc = rsqrtf(ss + eps);
+      uint4 res;
+      if constexpr (sizeof(Tio) == 2) {
+        uint32_t* r = reinterpret_cast<uint32_t*>(&res);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const __nv_bfloat162 v = __floats2bfloat162_rn(x[2 * i] * sc, x[2 * i + 1] * sc);
+          r[i] = *reinterpret_cast<const uint32_t*>(&v);
+        }
+      } else {
+        float* r = reinterpret_cast<float*>(&res);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) r[i] = x[i] * sc;
+      }
+      if (ok[u]) *reinterpret_cast<uint4*>(out + off[u]) = res;
     }
   }
 }

@@ -431,8 +431,9 @@ vdn_status launch_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const
   vdn::prep_kv_kernel<Tio, D><<<dim3((unsigned)s.H, (unsigned)tiles, (unsigned)(2 * s.B)), P::THREADS, smem, st>>>(a, s);
   prof_mark(h, st, 0, "prep_kv");
   const long long rows = (long long)s.B * s.Tn * s.F * s.H;
-  const long long want = (rows + 7) / 8;
-  const unsigned grid = (unsigned)(want < (long long)h->sm_count * 16 ? want : (long long)h->sm_count * 16);
+  const long long per_cta = 8LL * (32 / (D * (int)sizeof(Tio) / 16)) * 4;       // rows one CTA covers per trip
+  const long long want = (rows + per_cta - 1) / per_cta;
+  const unsigned grid = (unsigned)(want < (long long)h->sm_count * 8 ? want : (long long)h->sm_count * 8);
   vdn::prep_q_kernel<Tio, D><<<grid, 256, 0, st>>>(static_cast<const Tio*>(q_in), static_cast<Tio*>(q_out), s, a.l2_eps);
   prof_mark(h, st, 1, "prep_q");
   h->launches = 2;
@@ -619,6 +620,8 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
   if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
   if (p->Y <= 0 || p->X <= 0 || (long long)p->Y * p->X != F)
     return fail(h, VDN_ERR_INVALID_ARG, "Y * X must equal F");
+  if ((long long)F * H * d * (long long)elem_size(h) > 0x7fffffffLL)
+    return fail(h, VDN_ERR_UNSUPPORTED, "one frame of a tensor must stay below 2 GiB");
   if (H > 65535 || 2LL * B > 65535 || ((long long)(p->X + 7) / 8) * ((p->Y + 3) / 4) > 65535)
     return fail(h, VDN_ERR_UNSUPPORTED, "grid too large for the preparation kernel");
   DeviceGuard guard(h->cfg.device);
