@@ -194,6 +194,9 @@ size_t vdn_vda_workspace_bytes_opt(vdn_vda_t h, int B, int T, int F, int H, int 
  *        must not alias any input (the filters read neighbours); q_out may be q_in.
  *   p->Y, p->X   the spatial grid: F = Y * X, tokens of a frame in row-major (y, x) order
  *   p->wk_spatial, p->wv_spatial   float [H*d][5][5];   p->wk_temporal, p->wv_temporal   float [H*d][5]  (DEVICE)
+ *        Both spatial filters may be NULL: the spatial part is then the identity (temporal filter, SiLU and
+ *        normalisation only -- the operation the paper's VDA-Prep kernel fuses, Sec. 5), a streaming pass bound
+ *        by HBM instead of by the 25 extra multiply-adds per element.
  *   p->anchors   non-zero: frames 0 and T-1 are boundary anchors, removed before the preparation (Alg. 1
  *        step 2): the temporal filter sees zeros beyond frames 1 and T-2, and the anchor frames of all three
  *        outputs are zero.

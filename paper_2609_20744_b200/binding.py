@@ -255,17 +255,18 @@ class Vda:
         torch = self._torch
         B, T, F, H, d = q.shape
         names = ("wk_spatial", "wk_temporal", "wv_spatial", "wv_temporal")
-        for x in (q, k, v, *(filters[n] for n in names)):
+        given = [n for n in names if filters.get(n) is not None]      # spatial filters may be left out (identity)
+        for x in (q, k, v, *(filters[n] for n in given)):
             if not (x.is_cuda and x.is_contiguous()):
                 raise ValueError("vdn_vda_prepare needs contiguous CUDA tensors")
-        for n in names:
+        for n in given:
             want = (H * d, 5, 5) if n.endswith("spatial") else (H * d, 5)
             if tuple(filters[n].shape) != want or filters[n].dtype != torch.float32:
                 raise ValueError(f"{n} must be float32 {want}")
         qo, ko, vo = out if out is not None else (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v))
         p = lambda x: ctypes.c_void_p(x.data_ptr())
         prm = VdnPrepParams(ctypes.sizeof(VdnPrepParams), Y, X, 1 if anchors else 0, l2_eps,
-                            *(filters[n].data_ptr() for n in names))
+                            *(filters[n].data_ptr() if filters.get(n) is not None else None for n in names))
         self._check(self.lib.vdn_vda_prepare(self.h, p(q), p(k), p(v), p(qo), p(ko), p(vo), B, T, F, H, d,
                                              ctypes.byref(prm), self._stream(stream)))
         return qo, ko, vo

@@ -13,7 +13,8 @@
 // SiLU; for K the sum of squares over the head's channels (warp shuffles, plus one shared-memory exchange when
 // the head spans two warps); store.  30 fused multiply-adds per element: this kernel is bound by the fp32 pipe.
 //
-// prep_q_kernel: L2 normalisation of Q, one warp per (token, head); bound by HBM.
+// prep_kv_temporal_kernel: the same without the spatial filter (a streaming kernel, bound by HBM).
+// prep_q_kernel: L2 normalisation of Q; bound by HBM.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -250,6 +251,130 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
         for (int j = 0; j < TX; ++j)
           if (x0 + j < a.X) store_pair(orow + (size_t)j * (s.H * D), o0[j], o1[j]);
       }
+    }
+  }
+}
+
+// The same preparation without the spatial filter (its filters passed as null: the spatial part is then the
+// identity, e.g. because it was applied elsewhere): five-tap temporal filter, SiLU, L2 normalisation of K.  This is
+// the operation the paper's VDA-Prep kernel fuses (Sec. 5).  No neighbours in space, so no shared memory: a thread
+// owns one 16-byte piece of a (token, head) row and walks the frames with a five-frame ring in registers; the
+// lanes that share a row reduce the sum of squares by shuffles.  One read and one write of K and V: bound by HBM.
+struct PrepKvTemporal {
+  static constexpr int PF = 8;                                   // frames in flight per thread
+  static constexpr int SMEM_BYTES = PF * 256 * 16;
+};
+
+template <typename Tio, int D>
+__global__ void __launch_bounds__(256, 2) prep_kv_temporal_kernel(PrepArgs a, Shape s) {
+  constexpr int EPL = 16 / (int)sizeof(Tio);   // channels per thread
+  constexpr int LPR = D / EPL;                 // lanes per (token, head) row
+  const int which = blockIdx.y & 1;            // 0 = K (normalised), 1 = V
+  const int b = blockIdx.y >> 1;
+  const long long gid = (long long)blockIdx.x * 256 + threadIdx.x;
+  const long long rows = (long long)s.F * s.H;
+  // whole warps stay together for the shuffles: threads past the end work on the last row and do not store
+  const bool live = gid < rows * LPR;
+  const long long g2 = live ? gid : rows * LPR - 1;
+  const int piece = (int)(g2 % LPR);
+  const long long row = g2 / LPR;              // u * H + h
+  const int h = (int)(row % s.H);
+  const int ch = h * D + piece * EPL;
+
+  float wt[5][EPL];
+  {
+    const float* t0 = (which == 0 ? a.wt[0] : a.wt[1]) + (size_t)ch * 5;
+#pragma unroll
+    for (int c = 0; c < EPL; ++c)
+#pragma unroll
+      for (int i = 0; i < 5; ++i) wt[i][c] = __ldg(t0 + c * 5 + i);
+  }
+  const size_t frame_elems = (size_t)rows * D;
+  const Tio* src = static_cast<const Tio*>(which == 0 ? a.in[0] : a.in[1]) + (size_t)b * s.T * frame_elems +
+                   (size_t)row * D + piece * EPL;
+  Tio* dst = static_cast<Tio*>(which == 0 ? a.out[0] : a.out[1]) + (size_t)b * s.T * frame_elems + (size_t)row * D +
+             piece * EPL;
+  const int first = s.t0, last = s.t0 + s.Tn - 1;
+
+  float ring[5][EPL];
+#pragma unroll
+  for (int i = 0; i < 5; ++i)
+#pragma unroll
+    for (int c = 0; c < EPL; ++c) ring[i][c] = 0.f;
+
+  // Frames arrive through a queue of asynchronous copies in shared memory, PF frames ahead; a thread only ever
+  // reads the 16 bytes it copied itself, so no barrier is needed.  (Held in registers, the same number of bytes
+  // in flight would cost a quarter of the register file.)
+  constexpr int PF = PrepKvTemporal::PF;
+  extern __shared__ uint4 stg[];               // [PF][256]
+  const int nsteps = s.Tn + 2;
+#pragma unroll
+  for (int i = 0; i < PF - 1; ++i) {
+    if (first + i <= last) cp_async16(&stg[i * 256 + threadIdx.x], src + (size_t)(first + i) * frame_elems);
+    cp_async_commit();
+  }
+#pragma unroll 1
+  for (int sb = 0; sb < nsteps; sb += 5) {
+#pragma unroll
+    for (int r = 0; r < 5; ++r) {              // ring slot r is static: sb is a multiple of five
+      const int step = sb + r;
+      if (step >= nsteps) break;
+      const int t = first + step;
+      if (t + PF - 1 <= last)
+        cp_async16(&stg[((step + PF - 1) % PF) * 256 + threadIdx.x], src + (size_t)(t + PF - 1) * frame_elems);
+      cp_async_commit();
+      cp_async_wait<PF - 1>();                 // frame t has landed
+      if (t <= last) {
+        const uint4 cur = stg[(step % PF) * 256 + threadIdx.x];
+        if constexpr (sizeof(Tio) == 2) {
+          const uint32_t* u = reinterpret_cast<const uint32_t*>(&cur);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            ring[r][2 * i] = __uint_as_float(u[i] << 16);
+            ring[r][2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+          }
+        } else {
+          const float* u = reinterpret_cast<const float*>(&cur);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) ring[r][i] = u[i];
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < EPL; ++c) ring[r][c] = 0.f;
+      }
+      const int to = t - 2;                    // output frame: sum_i wt[i] x[to + i - 2], x[to + i - 2] in slot (r + i + 1) % 5
+      if (to < first) continue;
+      float o[EPL];
+      float ss = 0.f;
+#pragma unroll
+      for (int c = 0; c < EPL; ++c) {
+        float v = wt[0][c] * ring[(r + 1) % 5][c];
+#pragma unroll
+        for (int i = 1; i < 5; ++i) v = fmaf(wt[i][c], ring[(r + i + 1) % 5][c], v);
+        o[c] = silu_f(v);
+        ss = fmaf(o[c], o[c], ss);
+      }
+      if (which == 0) {
+#pragma unroll
+        for (int off = LPR / 2; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        const float sc = rsqrtf(ss + a.l2_eps);
+#pragma unroll
+        for (int c = 0; c < EPL; ++c) o[c] *= sc;
+      }
+      uint4 res;
+      if constexpr (sizeof(Tio) == 2) {
+        uint32_t* w = reinterpret_cast<uint32_t*>(&res);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+          w[i] = *reinterpret_cast<const uint32_t*>(&v2);
+        }
+      } else {
+        float* w = reinterpret_cast<float*>(&res);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w[i] = o[i];
+      }
+      if (live) *reinterpret_cast<uint4*>(dst + (size_t)to * frame_elems) = res;
     }
   }
 }

@@ -428,8 +428,15 @@ vdn_status launch_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const
   a.l2_eps = p.l2_eps > 0.f ? p.l2_eps : 1e-6f;
   const int tiles = ((p.X + P::TX - 1) / P::TX) * ((p.Y + P::rows(D) - 1) / P::rows(D));
   prof_begin(h, st);
-  vdn::prep_kv_kernel<Tio, D><<<dim3((unsigned)s.H, (unsigned)tiles, (unsigned)(2 * s.B)), P::THREADS, smem, st>>>(a, s);
-  prof_mark(h, st, 0, "prep_kv");
+  if (p.wk_spatial) {
+    vdn::prep_kv_kernel<Tio, D><<<dim3((unsigned)s.H, (unsigned)tiles, (unsigned)(2 * s.B)), P::THREADS, smem, st>>>(a, s);
+    prof_mark(h, st, 0, "prep_kv");
+  } else {
+    const long long threads = (long long)s.F * s.H * (D * (int)sizeof(Tio) / 16);
+    vdn::prep_kv_temporal_kernel<Tio, D><<<dim3((unsigned)((threads + 255) / 256), (unsigned)(2 * s.B)), 256,
+                                           vdn::PrepKvTemporal::SMEM_BYTES, st>>>(a, s);
+    prof_mark(h, st, 0, "prep_kv_temporal");
+  }
   const long long rows = (long long)s.B * s.Tn * s.F * s.H;
   const long long per_cta = 8LL * (32 / (D * (int)sizeof(Tio) / 16)) * 4;       // rows one CTA covers per trip
   const long long want = (rows + per_cta - 1) / per_cta;
@@ -606,9 +613,10 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
   if (!h) return VDN_ERR_INVALID_ARG;
   if (!p || p->struct_size != sizeof(vdn_vda_prep_params))
     return fail(h, VDN_ERR_INVALID_ARG, "vdn_vda_prep_params missing or of the wrong struct_size");
-  if (!q_in || !k_in || !v_in || !q_out || !k_out || !v_out || !p->wk_spatial || !p->wk_temporal || !p->wv_spatial ||
-      !p->wv_temporal)
+  if (!q_in || !k_in || !v_in || !q_out || !k_out || !v_out || !p->wk_temporal || !p->wv_temporal)
     return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
+  if ((p->wk_spatial == nullptr) != (p->wv_spatial == nullptr))
+    return fail(h, VDN_ERR_INVALID_ARG, "pass both spatial filters or neither");
   if (!aligned16(q_in) || !aligned16(k_in) || !aligned16(v_in) || !aligned16(q_out) || !aligned16(k_out) ||
       !aligned16(v_out) || !aligned16(p->wk_spatial) || !aligned16(p->wk_temporal) || !aligned16(p->wv_spatial) ||
       !aligned16(p->wv_temporal))

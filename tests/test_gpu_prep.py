@@ -63,6 +63,22 @@ def test_prepare_matches_oracle(dtype, d, T, Y, X, anchors):
             assert torch.count_nonzero(g[:, 0]) == 0 and torch.count_nonzero(g[:, -1]) == 0
 
 
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("f32", 128), ("bf16", 128), ("bf16", 64)])
+@pytest.mark.parametrize("T,Y,X,anchors", [(6, 9, 11, False), (1, 3, 5, False), (2, 1, 1, False), (9, 5, 7, True)])
+def test_prepare_without_spatial_filter_matches_oracle(dtype, d, T, Y, X, anchors):
+    # spatial filters left out: temporal filter + SiLU + normalisation; the checker gets centre-tap spatial filters
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=2, H=3, T=T, F=Y * X, seed=T * 100 + Y * 10 + X + 1)
+    p = inputs.generate_projected(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    flt = dict(wk_temporal=p["wk_temporal"], wv_temporal=p["wv_temporal"])
+    got = vda.prepare(p["q"], p["k"], p["v"], flt, Y, X, anchors=anchors)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    for n in ("wk", "wv"):
+        p[n + "_spatial"].zero_(); p[n + "_spatial"][:, 2, 2] = 1.0
+    check(w, p, got, Y, X, anchors)
+
+
 def test_prepare_identity_filters_and_in_place_q():
     # centre-tap filters: k' = L2norm(SiLU(k)), v' = SiLU(v); q normalised in place
     w = inputs.TINY.scaled(dtype="f32", d=64, B=1, H=2, T=3, F=6 * 7)
