@@ -80,3 +80,73 @@ def test_cfg_long_clip_full_size():
     if free < need:
         pytest.skip(f"needs {need >> 30} GiB of free device memory")
     run_and_check(w, 2)
+
+
+def test_768p_release_window_full_size():
+    # the release setting of the paper (chunk 5, radius 1, boundary anchors, decay bridge, text state) at the
+    # benchmark's size; both scan schedules
+    w = inputs.CLIP_768P
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    kw = dict(chunk=5, radius=1, anchors=True)
+    pairs = sampled_pairs(w, 2)
+    refs = {}
+    for (b, h) in pairs:
+        q, k, v, beta, gate = inputs.head_slice(x, b, h)
+        refs[(b, h)] = orc.vda_slice(q, k, v, beta, gate, 1e-6, alpha=alpha[b, :, h].double().cpu().numpy(),
+                                     s0=s0[b, h].double().cpu().numpy(), **kw)["out"]
+        del q, k, v
+    for flags in (binding.VDN_FLAG_SCAN_FRAMEWISE, binding.VDN_FLAG_SCAN_CHUNKWISE):
+        vda = binding.Vda(w.d, w.dtype, flags=flags)
+        out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0, **kw)
+        torch.cuda.synchronize()
+        assert vda.status() == binding.VDN_OK
+        for (b, h) in pairs:
+            e = orc.slice_error(out[b, :, :, h, :].double().cpu().numpy(), refs[(b, h)])
+            assert e <= TOL_BF16, f"flags={flags} slice (b={b}, h={h}): error {e:.3e}"
+        assert torch.count_nonzero(out[:, 0]) == 0 and torch.count_nonzero(out[:, -1]) == 0
+        assert torch.isfinite(out.float()).all()
+        del out, vda
+    del x
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("spatial", [True, False])
+def test_768p_preparation_full_size(spatial):
+    # vdn_vda_prepare on the 768p shape (48 x 85 tokens per frame): sampled output frames of sampled heads against
+    # the checker (which gets the five input frames the temporal filter reaches), plus properties on everything
+    from oracle import prep_oracle as po
+    w = inputs.CLIP_768P
+    Y, X = 48, 85
+    p = inputs.generate_projected(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    flt = p if spatial else dict(wk_temporal=p["wk_temporal"], wv_temporal=p["wv_temporal"])
+    q, k, v = vda.prepare(p["q"], p["k"], p["v"], flt, Y, X)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    if not spatial:
+        for n in ("wk", "wv"):
+            p[n + "_spatial"].zero_(); p[n + "_spatial"][:, 2, 2] = 1.0
+    f = lambda t: t.detach().double().cpu().numpy()
+    for (b, h, tc) in [(0, 0, 0), (0, w.H - 1, w.T - 1), (0, 17, 40), (0, 5, 1)]:
+        lo, hi = max(0, tc - 2), min(w.T, tc + 3)
+        sl = slice(h * w.d, (h + 1) * w.d)
+        # frames outside the clip are zero padding for the checker too: hand it exactly the frames that exist
+        ref = po.prepare(f(p["q"][b, lo:hi, :, h]), f(p["k"][b, lo:hi, :, h]), f(p["v"][b, lo:hi, :, h]),
+                         f(p["wk_spatial"][sl]), f(p["wk_temporal"][sl]), f(p["wv_spatial"][sl]),
+                         f(p["wv_temporal"][sl]), Y, X)
+        # the cropped clip pads with zeros where the real clip has frames: only exact when the crop reaches as far
+        # as the filter does, i.e. at the clip's own ends or with two frames on either side
+        assert lo == max(0, tc - 2) and hi == min(w.T, tc + 3)
+        for name, g, r in zip("qkv", (q, k, v), ref):
+            e = orc.slice_error(f(g[b, tc, :, h]), r[tc - lo])
+            assert e <= TOL_BF16, f"{name}' (b={b}, h={h}, t={tc}): error {e:.3e}"
+    for t0 in range(0, w.T, 16):
+        assert torch.isfinite(v[:, t0:t0 + 16].float()).all()
+        for g in (q, k):
+            n2 = g[:, t0:t0 + 16].float().pow(2).sum(-1)
+            assert torch.allclose(n2, torch.ones_like(n2), atol=2e-2)       # unit rows (bf16 rounding)
+    del p, q, k, v
+    gc.collect()
+    torch.cuda.empty_cache()
