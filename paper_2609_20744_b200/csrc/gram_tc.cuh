@@ -11,9 +11,9 @@
 //   warp 0      TMA producer: K and V tiles (4 boxes of 16 KB) into a 3-stage ring
 //   warp 1      MMA issuer (one thread) and TMEM owner
 //   warps 2-5   weighting: K' = bf16(beta) * K in packed bf16 arithmetic, written to a second buffer in two halves of
-//               64 tokens so the MMA of one half overlaps the weighting of the other.  Once per frame (after the
-//               first tile of the next frame is with the MMA) the same warps drain the finished accumulator:
-//               TMEM -> registers -> global fp32 [2d][d] (A_t, then B_t); there are two accumulators
+//               64 tokens so the MMA of one half overlaps the weighting of the other
+//   warps 6-9   drain: once per frame, the finished accumulator (of two) TMEM -> registers -> global fp32 [2d][d]
+//               (A_t, then B_t), while the other warps are already on the next frame
 // Rows past the end of a frame are zero-filled by TMA (the map has F as its own dimension) and their
 // beta is forced to zero.  Every mbarrier wait is bounded.
 #pragma once
@@ -36,7 +36,7 @@ struct GramTc {
   static constexpr int USED_BYTES = OFF_BAR + 128;
   static constexpr int SMEM_BYTES = 232448;                // everything an SM offers one CTA; the slack
                                                            // absorbs the 1024-byte alignment
-  static constexpr int THREADS = 192;
+  static constexpr int THREADS = 320;
 };
 
 __global__ void __launch_bounds__(GramTc::THREADS, 1)
@@ -72,8 +72,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 3; ++i) { mbar_init(FULL(i), 1); mbar_init(EMPTY(i), 1); }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(SCALED(i), 128); mbar_init(KPFREE(i), 1);
-      mbar_init(ACCFULL(i), 1);  mbar_init(ACCEMPTY(i), 128);
+      mbar_init(SCALED(i), 4); mbar_init(KPFREE(i), 1);      // one arrival per weighting warp
+      mbar_init(ACCFULL(i), 1);  mbar_init(ACCEMPTY(i), 4);   // ... per drain warp
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -148,25 +148,20 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (ok) mma_commit(ACCFULL(a));
       }
     }
-  } else {
-    // ------------------------------------------------------------------ weighting warps: K' = beta * K,
-    // and, once per frame, the drain of the previous frame's accumulator
-    const int ts = threadIdx.x - 64;          // 0..127
-    const int r = ts >> 1, c = ts & 1;        // row within the half, 64-channel box
-    const int qd = warp & 3;                  // TMEM lane quarter this warp may read
-    const int row = qd * 32 + lane;           // accumulator row drained by this thread
-    uint32_t it = 0, ai = 0;
-    bool ok = true;
-
+  } else if (warp >= 6) {
+    // ------------------------------------------------------------------ drain warps
     // TMEM -> registers -> global fp32 [2d][d].  Accumulator lane = key channel i, column = column of [K|V];
     // stored transposed so that the 32 lanes of a warp write 32 consecutive floats.
-    auto drain = [&](long long ditem, uint32_t dai) -> bool {
-      const int a = dai & 1;
-      if (!mbar_wait(ACCFULL(a), (dai >> 1) & 1, wc)) return false;
+    const int qd = warp & 3;                  // TMEM lane quarter this warp may read
+    const int row = qd * 32 + lane;           // accumulator row drained by this thread
+    uint32_t ai = 0;
+    for (long long item = blockIdx.x; item < nitems; item += gridDim.x, ++ai) {
+      const int a = ai & 1;
+      if (!mbar_wait(ACCFULL(a), (ai >> 1) & 1, wc)) break;
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 256;
       int b, h, t;
-      const long long n = split_work(s, ditem, b, h, t);
+      const long long n = split_work(s, item, b, h, t);
       float* dst = stats + (size_t)n * (2 * G::D * G::D) + row;
 #pragma unroll 1
       for (int cc = 0; cc < 8; ++cc) {
@@ -177,9 +172,14 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         for (int e = 0; e < 32; ++e) dst[(size_t)(cc * 32 + e) * G::D] = v[e];
       }
       tc_fence_before_sync();
-      mbar_arrive(ACCEMPTY(a));                 // the accumulator is free for the frame after next
-      return true;
-    };
+      mbar_arrive_warp(ACCEMPTY(a));            // the accumulator is free for the frame after next
+    }
+  } else {
+    // ------------------------------------------------------------------ weighting warps: K' = beta * K
+    const int ts = threadIdx.x - 64;          // 0..127
+    const int r = ts >> 1, c = ts & 1;        // row within the half, 64-channel box
+    uint32_t it = 0;
+    bool ok = true;
 
     // beta of (frame, tile), one value per half for this thread's row; zero past the end of the frame.
     // Fetched one tile ahead: the loads are scattered 4-byte reads (one head out of H) whose L2 latency would
@@ -196,7 +196,6 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     };
 
-    long long prev_item = -1;
     float bnext[2];
     load_beta(blockIdx.x, 0, bnext);
     for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
@@ -230,18 +229,10 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           for (int j = 0; j < 8; ++j)            // chunks staggered across rows: conflict-free
             *reinterpret_cast<uint4*>(dst + ((j ^ (r & 7)) * 16)) = raw[j];
           fence_proxy_async_smem();
-          mbar_arrive(SCALED(half));
-        }
-        // the first tile of this frame is with the MMA: now empty the previous frame's accumulator
-        if (ok && tile == 0 && prev_item >= 0) {
-          ok = drain(prev_item, ai - 1);
-          prev_item = -1;
+          mbar_arrive_warp(SCALED(half));
         }
       }
-      prev_item = item;
-      ++ai;
     }
-    if (ok && prev_item >= 0) drain(prev_item, ai - 1);
   }
 
   // ------------------------------------------------------------------ teardown

@@ -68,7 +68,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (threadIdx.x == 0) {
     for (int i = 0; i < 3; ++i) { mbar_init(QFULL(i), 1); mbar_init(QEMPTY(i), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(STFULL(i), 1); mbar_init(STEMPTY(i), 1); }
-    for (int i = 0; i < 4; ++i) { mbar_init(ACCFULL(i), 1); mbar_init(ACCEMPTY(i), 128); }
+    for (int i = 0; i < 4; ++i) { mbar_init(ACCFULL(i), 1); mbar_init(ACCEMPTY(i), 4); }   // one arrival per epilogue warp
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
@@ -186,7 +186,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tmem_ld32(taddr + 96, v[3]);
         tmem_wait_ld();
         tc_fence_before_sync();
-        mbar_arrive(ACCEMPTY(a));
+        mbar_arrive_warp(ACCEMPTY(a));
 
         float ss = 0.f;
 #pragma unroll

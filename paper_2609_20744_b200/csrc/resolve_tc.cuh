@@ -36,17 +36,18 @@ __device__ __forceinline__ float fast_rcp(float x) {
 struct ResolveTc {
   static constexpr int D = 128;
   static constexpr int NB = 16;                       // pivots per step
-  static constexpr int CM_PART = 128 * 128;           // coefficient part: 128 rows x 128 B (32 B used), K-major
+  static constexpr int CM_BYTES = 128 * 128;          // coefficients, K-major: 128 rows x 128 B; part p of a row sits in
+                                                      // bytes [32 p, 32 p + 32) (K = 16 bf16), 32 B unused
   static constexpr int PR_PART = 2 * NB * 128;        // pivot-row part: 2 boxes x 16 rows x 128 B, MN-major
   static constexpr int OFF_CM = 0;
-  static constexpr int OFF_PR = 3 * CM_PART;
+  static constexpr int OFF_PR = CM_BYTES;
   static constexpr int OFF_GI = OFF_PR + 3 * PR_PART; // Gi, 16 x 16 floats
   static constexpr int OFF_BAR = OFF_GI + 1024;
   static constexpr int SMEM_BYTES = OFF_BAR + 64 + 1024;
   static constexpr int THREADS = 160;                 // 4 row warps + 1 MMA warp
 };
 
-__global__ void __launch_bounds__(ResolveTc::THREADS, 3)
+__global__ void __launch_bounds__(ResolveTc::THREADS, 4)
 resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ csplit, long long nframes,
                   int* status, Shape shp) {
   using namespace tc;
@@ -67,7 +68,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
   if ((int)(n % shp.T) < shp.t0 || (int)(n % shp.T) >= shp.t0 + shp.Tn) return;   // an anchor frame: not scanned
 
   if (threadIdx.x == 0) {
-    mbar_init(OPREADY, 128);
+    mbar_init(OPREADY, 4);                    // one arrival per row warp
     mbar_init(MMADONE, 1);
     *abort_flag = 0;
     mbar_fence_init();
@@ -76,7 +77,6 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
     tmem_alloc(smem_u32(tmem_slot), 128);
     tmem_relinquish();
   }
-  // the unused 96 bytes of every coefficient row are never read by the MMA (K = 16 = 32 bytes)
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -93,7 +93,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
         tc_fence_after_sync();
 #pragma unroll
         for (int pr = 0; pr < 6; ++pr) {
-          const uint64_t adesc = make_smem_desc(base + R::OFF_CM + PA[pr] * R::CM_PART, 16, 1024);
+          const uint64_t adesc = make_smem_desc(base + R::OFF_CM + PA[pr] * 32, 16, 1024);
           const uint64_t bdesc = make_smem_desc(base + R::OFF_PR + PB[pr] * R::PR_PART, R::NB * 128, 1024);
           mma_bf16_ss(tmem_base, adesc, bdesc, idesc, 1u);
         }
@@ -208,8 +208,8 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
         unsigned char* crow = base_ptr + R::OFF_CM + row * 128;
 #pragma unroll
         for (int part = 0; part < 3; ++part) {
-          *reinterpret_cast<uint4*>(crow + part * R::CM_PART + ((0 ^ (row & 7)) * 16)) = w[part][0];
-          *reinterpret_cast<uint4*>(crow + part * R::CM_PART + ((1 ^ (row & 7)) * 16)) = w[part][1];
+          *reinterpret_cast<uint4*>(crow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
+          *reinterpret_cast<uint4*>(crow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
         }
       }
       // ---- B operand: the 16 pivot rows, three bf16 parts, MN-major.  M is symmetric up to the sign pattern
@@ -236,7 +236,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       }
       fence_proxy_async_smem();
       tc_fence_before_sync();
-      mbar_arrive(OPREADY);
+      mbar_arrive_warp(OPREADY);
       if (!mbar_wait(MMADONE, step & 1, wc)) { ok = false; break; }
       tc_fence_after_sync();
       // ---- column fix: M[i][P] = c (for a pivot row: Gi[a])
@@ -244,7 +244,6 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       tmem_wait_st();
       done |= 1u << blk;
     }
-
     if (ok) {
       // ---- the inverse as three bf16 parts; this thread holds column `row` of it
       __nv_bfloat16* c1 = csplit + (size_t)n * (3 * D * D) + row;
@@ -268,7 +267,6 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       }
     }
   }
-
   __syncwarp();
   tc_fence_before_sync();
   __syncthreads();

@@ -136,7 +136,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
 
   if (threadIdx.x == 0) {
     for (int p = 0; p < 3; ++p) { mbar_init(CFULL(p), 1); mbar_init(CFREE(p), 1); }
-    mbar_init(XREADY, S::THREADS - 64);
+    mbar_init(XREADY, (S::THREADS - 64) / 32);     // one arrival per state warp
     mbar_init(ACCFULL, 1);
     *abort_flag = 0;
     mbar_fence_init();
@@ -237,7 +237,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
       }
       fence_proxy_async_smem();
       tc_fence_before_sync();
-      mbar_arrive(XREADY);
+      mbar_arrive_warp(XREADY);
     };
 
     // Optional extras (Eq. A.1, Eq. 1b, Eq. A.4): alpha [B,T,H,d] decays key channel `row` of the inherited
