@@ -215,10 +215,14 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
                            void* k_out, void* v_out, int B, int T, int F, int H, int d,
                            const vdn_vda_prep_params* p, void* cuda_stream);
 
-/* The same layer for callers whose tensors live in HOST memory (pinned memory recommended): copies
- * q, k, v, beta, gate to the staging buffer, runs vdn_vda_forward, copies `out` back, all on
- * cuda_stream, and returns without synchronising.  All six tensor pointers are HOST pointers.  The
- * staging buffer is a caller-owned DEVICE buffer of at least vdn_vda_staging_bytes, set beforehand. */
+/* The same layer for callers whose tensors live in HOST memory (pinned memory recommended; with pageable
+ * memory the copies are not asynchronous).  All six tensor pointers are HOST pointers.  The staging buffer is a
+ * caller-owned DEVICE buffer of at least vdn_vda_staging_bytes, set beforehand.  Order of work on cuda_stream:
+ * k, v, beta, gate are copied in; statistics, resolve and both scans run; then, for each of up to eight groups of
+ * frames, that group's queries are copied in and read out, and its output rows are copied back on a second
+ * stream owned by the handle, beside the next group's copy in (the host link is full duplex, and out needs the
+ * scans of the whole clip, so this is all the overlap there is).  cuda_stream waits for the last copy back:
+ * synchronising it is enough.  The first call creates the second stream and nine events (no device memory). */
 size_t vdn_vda_staging_bytes(vdn_vda_t h, int B, int T, int F, int H, int d);
 vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes);
 vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const void* v,

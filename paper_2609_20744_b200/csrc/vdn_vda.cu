@@ -54,6 +54,10 @@ struct Extras {
   vdn::Window win{1, 0, 0, -1};
   bool anchors = false;
   bool composed = false;   // run the scan chunk-wise (tensor-core path, chunk >= 2)
+  // vdn_vda_forward_host runs the layer in pieces: everything up to the scans once the keys and values have
+  // arrived, then the read-out of one group of frames after another as their queries arrive
+  int phase = 0;           // 0 = whole layer, 1 = statistics, resolve and scans only, 2 = read-out only
+  int ro_first = 0, ro_count = 0;   // phase 2: the frames to read out
 };
 
 }  // namespace
@@ -87,6 +91,10 @@ struct vdn_vda_s {
   bool attrs_set = false;
   bool tc_attrs_set = false;
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;  // driver entry point, resolved at create
+  // vdn_vda_forward_host: frame groups whose results are copied back on a second stream (made on first use)
+  static constexpr int kHostGroups = 8;
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t copy_ev[kHostGroups + 1] = {};
   std::string err = "no error";
 };
 
@@ -233,27 +241,36 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
   float* read = reinterpret_cast<float*>(ws + L.read);
   const long long n = s.frames();
 
-  prof_begin(h, st);
-  vdn::gram_simt_kernel<Tio, D><<<dim3((unsigned)n, 2 * D / 64), 256, 0, st>>>(
-      static_cast<const Tio*>(k), static_cast<const Tio*>(v), beta, stats, s);
-  prof_mark(h, st, 0, "gram_simt");
-  const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
-  const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
-  if (additive) {
-    vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n, 1.0f / (float)s.F, s);
-    prof_mark(h, st, 1, "additive_transition");
+  if (x.phase != 2) {
+    prof_begin(h, st);
+    vdn::gram_simt_kernel<Tio, D><<<dim3((unsigned)n, 2 * D / 64), 256, 0, st>>>(
+        static_cast<const Tio*>(k), static_cast<const Tio*>(v), beta, stats, s);
+    prof_mark(h, st, 0, "gram_simt");
+    const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
+    const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
+    if (additive) {
+      vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n, 1.0f / (float)s.F, s);
+      prof_mark(h, st, 1, "additive_transition");
+    } else {
+      vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n, s);
+      prof_mark(h, st, 1, "resolve");
+    }
+    vdn::scan_kernel<D, 32><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
+        stats, inv, fwd, read, s.T, x.alpha, x.s0, s.H, bscale, x.win);
+    prof_mark(h, st, 2, "scan");
+    h->launches = 3;
   } else {
-    vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, inv, nullptr, n, s);
-    prof_mark(h, st, 1, "resolve");
+    h->prof.cur = -1;
   }
-  vdn::scan_kernel<D, 32><<<dim3((unsigned)(s.B * s.H), D / 32), 256, sizeof(vdn::ScanSmem<D, 32>), st>>>(
-      stats, inv, fwd, read, s.T, x.alpha, x.s0, s.H, bscale, x.win);
-  prof_mark(h, st, 2, "scan");
-  vdn::readout_simt_kernel<Tio, D><<<dim3((unsigned)n, (s.F + 63) / 64), 256, sizeof(vdn::ReadoutSimtSmem<D>), st>>>(
-      static_cast<const Tio*>(q), read, gate, static_cast<Tio*>(out), s, h->cfg.rms_eps,
-      static_cast<const Tio*>(x.gate_elem), x.norm_weight);
-  prof_mark(h, st, 3, "readout_simt");
-  h->launches = 4;
+  if (x.phase != 1) {
+    Shape sr = s;                                     // the frames to read out (the kernel skips the others)
+    if (x.phase == 2) { sr.t0 = x.ro_first; sr.Tn = x.ro_count; }
+    vdn::readout_simt_kernel<Tio, D><<<dim3((unsigned)n, (s.F + 63) / 64), 256, sizeof(vdn::ReadoutSimtSmem<D>), st>>>(
+        static_cast<const Tio*>(q), read, gate, static_cast<Tio*>(out), sr, h->cfg.rms_eps,
+        static_cast<const Tio*>(x.gate_elem), x.norm_weight);
+    prof_mark(h, st, 3, "readout_simt");
+    h->launches += 1;
+  }
   VDN_CUDA(h, cudaGetLastError());
   return VDN_OK;
 }
@@ -331,53 +348,63 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
 
   const long long nwork = s.work_items();
   const unsigned persistent = (unsigned)(nwork < h->sm_count ? nwork : h->sm_count);
-  prof_begin(h, st);
   int nk = 0;
-  vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
-                                                                                       h->status_dev);
-  prof_mark(h, st, nk++, "gram_tc");
-  const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
-  const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
-  if (additive) {
-    vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n, 1.0f / (float)s.F, s);
-    prof_mark(h, st, nk++, "additive_transition");
+  if (x.phase != 2) {
+    prof_begin(h, st);
+    vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
+                                                                                         h->status_dev);
+    prof_mark(h, st, nk++, "gram_tc");
+    const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
+    const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
+    if (additive) {
+      vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n, 1.0f / (float)s.F, s);
+      prof_mark(h, st, nk++, "additive_transition");
+    } else {
+      vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
+          stats, csplit, n, h->status_dev, s);
+      prof_mark(h, st, nk++, "resolve_tc");
+    }
+    vdn::ScanTcArgs sa{};
+    sa.stats = stats; sa.pf = pf; sa.pb = pb; sa.alpha = x.alpha; sa.s0 = x.s0;
+    sa.T = s.T; sa.H = s.H; sa.additive_bscale = bscale; sa.win = x.win;
+    if (x.composed) {
+      // chunk-wise scan: compose every chunk (all at once), then scan the chunk sequence
+      sa.nseg = x.win.last / x.win.chunk - x.win.first / x.win.chunk + 1;
+      sa.comp_m = reinterpret_cast<__nv_bfloat16*>(ws + L.comp_m);
+      sa.comp_j = reinterpret_cast<float*>(ws + L.comp_j);
+      CUtensorMap tmM;
+      if ((r = make_matrix_map(h, &tmM, sa.comp_m, (long long)3 * s.B * s.H * 2 * sa.nseg * D)) != VDN_OK) return r;
+      vdn::scan_tc_kernel<vdn::SCAN_COMPOSE><<<(unsigned)(4 * s.B * s.H * sa.nseg), vdn::ScanTc::THREADS,
+                                               vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
+      prof_mark(h, st, nk++, "compose_tc");
+      vdn::scan_tc_kernel<vdn::SCAN_CHUNKS><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
+                                              vdn::ScanTc::SMEM_BYTES, st>>>(tmM, sa, h->status_dev);
+      prof_mark(h, st, nk++, "scan_chunks_tc");
+    } else {
+      vdn::scan_tc_kernel<vdn::SCAN_FRAMES><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
+                                              vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
+      prof_mark(h, st, nk++, "scan_tc");
+    }
+    h->launches = nk;
   } else {
-    vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
-        stats, csplit, n, h->status_dev, s);
-    prof_mark(h, st, nk++, "resolve_tc");
+    h->prof.cur = -1;
+    nk = h->launches;
   }
-  vdn::ScanTcArgs sa{};
-  sa.stats = stats; sa.pf = pf; sa.pb = pb; sa.alpha = x.alpha; sa.s0 = x.s0;
-  sa.T = s.T; sa.H = s.H; sa.additive_bscale = bscale; sa.win = x.win;
-  if (x.composed) {
-    // chunk-wise scan: compose every chunk (all at once), then scan the chunk sequence
-    sa.nseg = x.win.last / x.win.chunk - x.win.first / x.win.chunk + 1;
-    sa.comp_m = reinterpret_cast<__nv_bfloat16*>(ws + L.comp_m);
-    sa.comp_j = reinterpret_cast<float*>(ws + L.comp_j);
-    CUtensorMap tmM;
-    if ((r = make_matrix_map(h, &tmM, sa.comp_m, (long long)3 * s.B * s.H * 2 * sa.nseg * D)) != VDN_OK) return r;
-    vdn::scan_tc_kernel<vdn::SCAN_COMPOSE><<<(unsigned)(4 * s.B * s.H * sa.nseg), vdn::ScanTc::THREADS,
-                                             vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
-    prof_mark(h, st, nk++, "compose_tc");
-    vdn::scan_tc_kernel<vdn::SCAN_CHUNKS><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
-                                            vdn::ScanTc::SMEM_BYTES, st>>>(tmM, sa, h->status_dev);
-    prof_mark(h, st, nk++, "scan_chunks_tc");
-  } else {
-    vdn::scan_tc_kernel<vdn::SCAN_FRAMES><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
-                                            vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
-    prof_mark(h, st, nk++, "scan_tc");
-  }
+  if (x.phase == 1) { VDN_CUDA(h, cudaGetLastError()); return VDN_OK; }
   // The read-out streams reads and writes in equal parts and is fastest on about five SMs out of six
   // (measured on three workloads: 124 CTAs beat 148 by 5 %; fewer interleaved read/write streams at the DRAM).
+  Shape sr = s;                                       // the frames to read out
+  if (x.phase == 2) { sr.t0 = x.ro_first; sr.Tn = x.ro_count; }
+  const long long nread = sr.work_items();
   const long long ro_target = ((long long)h->sm_count * 27 + 16) / 32;
-  const unsigned persistent_ro = (unsigned)(nwork < ro_target ? nwork : ro_target);
+  const unsigned persistent_ro = (unsigned)(nread < ro_target ? nread : ro_target);
   if (x.gate_elem || x.norm_weight || !gate)
     vdn::readout_tc_kernel<true><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
-        tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
+        tmQ, tmS, tmO, gate, sr, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
         x.norm_weight, x.win, x.alpha != nullptr);
   else
     vdn::readout_tc_kernel<false><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
-        tmQ, tmS, tmO, gate, s, h->cfg.rms_eps, h->status_dev, nullptr, nullptr, x.win, x.alpha != nullptr);
+        tmQ, tmS, tmO, gate, sr, h->cfg.rms_eps, h->status_dev, nullptr, nullptr, x.win, x.alpha != nullptr);
   prof_mark(h, st, nk++, "readout_tc");
   h->launches = nk;
   VDN_CUDA(h, cudaGetLastError());
@@ -530,11 +557,18 @@ vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes) {
   return VDN_OK;
 }
 
-vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
-                               const float* gate, void* out, int B, int T, int F, int H, int d,
-                               const vdn_vda_options* opt, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+// The layer, whole (phase 0) or in the two pieces vdn_vda_forward_host interleaves with its copies (phase 1:
+// statistics, resolve, scans; phase 2: read-out of frames ro_first .. ro_first + ro_count - 1).
+vdn_status forward_core(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                        const float* gate, void* out, int B, int T, int F, int H, int d,
+                        const vdn_vda_options* opt, void* cuda_stream, int phase, int ro_first, int ro_count) {
   if (!h) return VDN_ERR_INVALID_ARG;
   Extras x;
+  x.phase = phase;
   if (opt) {
     if (opt->struct_size != sizeof(vdn_vda_options))
       return fail(h, VDN_ERR_INVALID_ARG, "vdn_vda_options.struct_size does not match this library");
@@ -587,8 +621,17 @@ vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const 
   if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const Shape s{B, T, F, H, d, x.win.first, x.win.last - x.win.first + 1};
-  h->launches = 0;
-  if (x.anchors) {
+  if (phase == 2) {
+    // clip the requested frames to the scanned ones (anchor rows were zeroed in phase 1)
+    const int lo = ro_first > x.win.first ? ro_first : x.win.first;
+    const int hi = ro_first + ro_count - 1 < x.win.last ? ro_first + ro_count - 1 : x.win.last;
+    if (hi < lo) return VDN_OK;
+    x.ro_first = lo;
+    x.ro_count = hi - lo + 1;
+  } else {
+    h->launches = 0;
+  }
+  if (x.anchors && phase != 2) {
     // Alg. 1 step 7: anchor rows of the linear output are zero (frames 0 and T-1 of every clip)
     const size_t frame_bytes = (size_t)F * H * d * elem_size(h);
     char* o = static_cast<char*>(out);
@@ -605,6 +648,16 @@ vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const 
   }
   return d == 64 ? forward_simt<__nv_bfloat16, 64>(h, q, k, v, beta, gate, x, out, s, L, st)
                  : forward_simt<__nv_bfloat16, 128>(h, q, k, v, beta, gate, x, out, s, L, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                               const float* gate, void* out, int B, int T, int F, int H, int d,
+                               const vdn_vda_options* opt, void* cuda_stream) {
+  return forward_core(h, q, k, v, beta, gate, out, B, T, F, H, d, opt, cuda_stream, 0, 0, 0);
 }
 
 vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const void* v_in, void* q_out, void* k_out,
@@ -688,20 +741,51 @@ vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const
     return fail(h, VDN_ERR_WORKSPACE, "staging buffer not set or smaller than vdn_vda_staging_bytes");
   DeviceGuard guard(h->cfg.device);
   if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
+  if (!h->copy_stream) {
+    // a second stream and a few events, made on first use: results travel back while later queries still arrive
+    VDN_CUDA(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i <= vdn_vda_s::kHostGroups; ++i)
+      VDN_CUDA(h, cudaEventCreateWithFlags(&h->copy_ev[i], cudaEventDisableTiming));
+  }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   char* sg = static_cast<char*>(h->staging);
   const size_t tokh = (size_t)B * T * F * H;
   const size_t big = tokh * d * elem_size(h);
+  const size_t frame_bytes = (size_t)F * H * d * elem_size(h);
+  // Keys, values and write gates first: the statistics, the resolve and both scans need nothing else.
   VDN_CUDA(h, cudaMemcpyAsync(sg + S.k, k, big, cudaMemcpyHostToDevice, st));
   VDN_CUDA(h, cudaMemcpyAsync(sg + S.v, v, big, cudaMemcpyHostToDevice, st));
   VDN_CUDA(h, cudaMemcpyAsync(sg + S.beta, beta, tokh * sizeof(float), cudaMemcpyHostToDevice, st));
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.q, q, big, cudaMemcpyHostToDevice, st));
   VDN_CUDA(h, cudaMemcpyAsync(sg + S.gate, gate, (size_t)H * sizeof(float), cudaMemcpyHostToDevice, st));
-  vdn_status r = vdn_vda_forward(h, sg + S.q, sg + S.k, sg + S.v, reinterpret_cast<const float*>(sg + S.beta),
-                                 reinterpret_cast<const float*>(sg + S.gate), sg + S.out, B, T, F, H, d,
-                                 cuda_stream);
+  const float* dbeta = reinterpret_cast<const float*>(sg + S.beta);
+  const float* dgate = reinterpret_cast<const float*>(sg + S.gate);
+  vdn_status r = forward_core(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, B, T, F, H, d, nullptr,
+                              cuda_stream, 1, 0, 0);
   if (r != VDN_OK) return r;
-  VDN_CUDA(h, cudaMemcpyAsync(out, sg + S.out, big, cudaMemcpyDeviceToHost, st));
+  // Then the queries, one group of frames after another: copy in, read out, and hand the finished rows to the
+  // second stream, whose copy back to the host runs beside the next group's copy in (the link is full duplex).
+  const int groups = T < vdn_vda_s::kHostGroups ? T : vdn_vda_s::kHostGroups;
+  for (int g = 0; g < groups; ++g) {
+    const int t0 = (int)((long long)T * g / groups), t1 = (int)((long long)T * (g + 1) / groups);
+    const size_t off = (size_t)t0 * frame_bytes, len = (size_t)(t1 - t0) * frame_bytes;
+    for (int b = 0; b < B; ++b) {
+      const size_t o = (size_t)b * T * frame_bytes + off;
+      VDN_CUDA(h, cudaMemcpyAsync(sg + S.q + o, static_cast<const char*>(q) + o, len, cudaMemcpyHostToDevice, st));
+    }
+    r = forward_core(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, B, T, F, H, d, nullptr, cuda_stream,
+                     2, t0, t1 - t0);
+    if (r != VDN_OK) return r;
+    VDN_CUDA(h, cudaEventRecord(h->copy_ev[g], st));
+    VDN_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->copy_ev[g], 0));
+    for (int b = 0; b < B; ++b) {
+      const size_t o = (size_t)b * T * frame_bytes + off;
+      VDN_CUDA(h, cudaMemcpyAsync(static_cast<char*>(out) + o, sg + S.out + o, len, cudaMemcpyDeviceToHost,
+                                  h->copy_stream));
+    }
+  }
+  // the caller's stream is done when the last rows have landed
+  VDN_CUDA(h, cudaEventRecord(h->copy_ev[vdn_vda_s::kHostGroups], h->copy_stream));
+  VDN_CUDA(h, cudaStreamWaitEvent(st, h->copy_ev[vdn_vda_s::kHostGroups], 0));
   return VDN_OK;
 }
 
@@ -823,6 +907,11 @@ const char* vdn_vda_last_error(vdn_vda_t h) { return h ? h->err.c_str() : "null 
 vdn_status vdn_vda_destroy(vdn_vda_t h) {
   if (!h) return VDN_ERR_INVALID_ARG;
   if (h->prof.on) vdn_vda_profile(h, 0);
+  if (h->copy_stream) {
+    for (cudaEvent_t e : h->copy_ev)
+      if (e) cudaEventDestroy(e);
+    cudaStreamDestroy(h->copy_stream);
+  }
   if (h->status_host) cudaFreeHost(h->status_host);
   delete h;
   return VDN_OK;

@@ -295,15 +295,20 @@ def test_output_rows_have_gate_sized_rms():
 
 
 # ------------------------------------------------------------------------------ host-buffer entry point
-def test_forward_host_matches_device_entry_point():
-    w = inputs.TINY.scaled(dtype="bf16", d=128, T=3, F=200, H=2)
+@pytest.mark.parametrize("dtype,d,B,T", [("bf16", 128, 1, 3), ("bf16", 128, 2, 11), ("f32", 64, 2, 9), ("bf16", 128, 1, 1)])
+def test_forward_host_matches_device_entry_point(dtype, d, B, T):
+    # the host entry point copies the queries in and the results out in groups of frames, on two streams
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=B, T=T, F=200, H=2)
     xh = inputs.generate(w, "cpu", pin=True)
     xd = {n: t.cuda() for n, t in xh.items()}
     vda, out_d = run_gpu(w, xd)
     out_h = torch.empty_like(xh["q"]).pin_memory()
-    vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], out_h)
-    torch.cuda.synchronize()
-    assert torch.equal(out_h, out_d.cpu())
+    out_h.fill_(7.0)
+    for _ in range(2):                                  # twice: the second call reuses the stream and events
+        vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], out_h)
+        torch.cuda.current_stream().synchronize()       # the caller's stream alone covers the copies back
+        assert torch.equal(out_h, out_d.cpu())
+        out_h.fill_(7.0)
 
 
 # ------------------------------------------------------------------------------ argument errors (host side)
