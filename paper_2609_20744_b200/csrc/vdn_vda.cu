@@ -278,15 +278,15 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
 // ---------------------------------------------------------------------------------------------------
 // Tensor-core path (bf16, d = 128): TMA tensor maps + four launches.
 
-// [B,T,F,H,d] bf16 tensor as a 5-D map (d, H, F, T, B) with a (64, 1, 128, 1, 1) box and the 128-byte
-// swizzle: one box is 128 tokens x 64 channels of one head.  F is its own dimension so that a tile
+// [B,T,F,H,d] bf16 tensor as a 5-D map (d, H, F, T, B) with a (64, 1, box_tokens, 1, 1) box and the 128-byte
+// swizzle: one box is box_tokens tokens x 64 channels of one head.  F is its own dimension so that a tile
 // hanging over the end of a frame is zero-filled on load and clipped on store.
-vdn_status make_token_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, const Shape& s) {
+vdn_status make_token_map(vdn_vda_t h, CUtensorMap* m, const void* ptr, const Shape& s, unsigned box_tokens = 128) {
   const cuuint64_t dims[5] = {(cuuint64_t)s.d, (cuuint64_t)s.H, (cuuint64_t)s.F, (cuuint64_t)s.T, (cuuint64_t)s.B};
   const cuuint64_t es = 2;
   const cuuint64_t strides[4] = {s.d * es, (cuuint64_t)s.H * s.d * es, (cuuint64_t)s.F * s.H * s.d * es,
                                  (cuuint64_t)s.T * s.F * s.H * s.d * es};
-  const cuuint32_t box[5] = {64, 1, 128, 1, 1};
+  const cuuint32_t box[5] = {64, 1, box_tokens, 1, 1};
   const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   CUresult r = h->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -339,8 +339,8 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
 
   CUtensorMap tmQ, tmK, tmV, tmO, tmS, tmC;
   vdn_status r;
-  if ((r = make_token_map(h, &tmK, k, s)) != VDN_OK) return r;
-  if ((r = make_token_map(h, &tmV, v, s)) != VDN_OK) return r;
+  if ((r = make_token_map(h, &tmK, k, s, vdn::GramTc::TILE)) != VDN_OK) return r;
+  if ((r = make_token_map(h, &tmV, v, s, vdn::GramTc::TILE)) != VDN_OK) return r;
   if ((r = make_token_map(h, &tmQ, q, s)) != VDN_OK) return r;
   if ((r = make_token_map(h, &tmO, out, s)) != VDN_OK) return r;
   if ((r = make_matrix_map(h, &tmS, pf, 2 * n * D)) != VDN_OK) return r;      // pf then pb
