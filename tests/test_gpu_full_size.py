@@ -65,7 +65,7 @@ def run_and_check(w, nheads):
 
 
 def test_768p_config_full_size():
-    run_and_check(inputs.CLIP_768P, 3)
+    run_and_check(inputs.CLIP_768P, 4)       # first, last and two seeded (batch, head) slices
 
 
 @pytest.mark.parametrize("idx", [0, 1, 2, 3])
