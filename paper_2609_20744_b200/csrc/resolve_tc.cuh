@@ -13,7 +13,8 @@
 //     rows travelling by shuffle;
 //   * every thread owns one matrix row (its TMEM lane), forms its 16 coefficients from Gi, and -- the matrix
 //     being symmetric up to the sign pattern of in-place elimination -- also supplies its column of the 16
-//     pivot rows, so nobody has to read whole rows back.
+//     pivot rows, so nobody has to read whole rows back.  Both MMA operands are K-major with one row per
+//     thread, so each thread writes its 16 values of a part as 32 contiguous bytes.
 // The matrix that is inverted is I + (A_t + A_t^T)/2: the stored statistics are symmetric only up to the bf16
 // rounding of one factor, and the symmetric part is the natural reading of Eq. 3b (and keeps Proposition 1).
 // The inverse is written as three bf16 parts C1 + C2 + C3 for the tensor-core scan.
@@ -38,10 +39,11 @@ struct ResolveTc {
   static constexpr int NB = 16;                       // pivots per step
   static constexpr int CM_BYTES = 128 * 128;          // coefficients, K-major: 128 rows x 128 B; part p of a row sits in
                                                       // bytes [32 p, 32 p + 32) (K = 16 bf16), 32 B unused
-  static constexpr int PR_PART = 2 * NB * 128;        // pivot-row part: 2 boxes x 16 rows x 128 B, MN-major
+  static constexpr int PR_BYTES = 128 * 128;          // pivot rows, K-major as well: row j = column j of the 16 pivot
+                                                      // rows, parts laid out like the coefficients
   static constexpr int OFF_CM = 0;
   static constexpr int OFF_PR = CM_BYTES;
-  static constexpr int OFF_GI = OFF_PR + 3 * PR_PART; // Gi, 16 x 16 floats
+  static constexpr int OFF_GI = OFF_PR + PR_BYTES;    // Gi, 16 x 16 floats
   static constexpr int OFF_BAR = OFF_GI + 1024;
   static constexpr int SMEM_BYTES = OFF_BAR + 64 + 1024;
   static constexpr int THREADS = 160;                 // 4 row warps + 1 MMA warp
@@ -85,7 +87,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
   if (warp == 4) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
+      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
       constexpr int PA[6] = {0, 2, 1, 0, 1, 0};   // (coefficient part, pivot-row part), smallest first
       constexpr int PB[6] = {2, 0, 1, 1, 0, 0};
       for (int step = 0; step < D / R::NB; ++step) {
@@ -94,7 +96,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
 #pragma unroll
         for (int pr = 0; pr < 6; ++pr) {
           const uint64_t adesc = make_smem_desc(base + R::OFF_CM + PA[pr] * 32, 16, 1024);
-          const uint64_t bdesc = make_smem_desc(base + R::OFF_PR + PB[pr] * R::PR_PART, R::NB * 128, 1024);
+          const uint64_t bdesc = make_smem_desc(base + R::OFF_PR + PB[pr] * 32, 16, 1024);
           mma_bf16_ss(tmem_base, adesc, bdesc, idesc, 1u);
         }
         mma_commit(MMADONE);
@@ -212,26 +214,26 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           *reinterpret_cast<uint4*>(crow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
         }
       }
-      // ---- B operand: the 16 pivot rows, three bf16 parts, MN-major.  M is symmetric up to the sign pattern
-      // of in-place elimination: M[P_k][j] = M[j][P_k] for rows j not yet eliminated and -M[j][P_k] for rows
-      // already eliminated (`done`).  So thread j owns column j of the pivot rows: its own x, signed.
+      // ---- B operand: the 16 pivot rows, three bf16 parts.  M is symmetric up to the sign pattern of in-place
+      // elimination: M[P_k][j] = M[j][P_k] for rows j not yet eliminated and -M[j][P_k] for rows already
+      // eliminated (`done`).  So thread j owns column j of the pivot rows: its own x, signed -- which is one row
+      // of the K-major operand (row = output column, 16 contiguous pivot indices): two 16-byte stores per part.
       {
         const float sgn = ((done >> (row >> 4)) & 1u) ? -1.0f : 1.0f;
-        const int jj = row & 63;
-        unsigned char* pcol = base_ptr + R::OFF_PR + (row >> 6) * (R::NB * 128) + (jj & 7) * 2;
-        const int ch = jj >> 3;
+        uint4 w[3][2];
 #pragma unroll
-        for (int k = 0; k < 16; k += 2) {
-          uint32_t w1, w2, w3;
-          split3_pair(sgn * x[k], sgn * x[k + 1], w1, w2, w3);
-          unsigned char* r0 = pcol + k * 128 + ((ch ^ (k & 7)) * 16);
-          unsigned char* r1 = pcol + (k + 1) * 128 + ((ch ^ ((k + 1) & 7)) * 16);
-          *reinterpret_cast<unsigned short*>(r0) = (unsigned short)(w1 & 0xFFFFu);
-          *reinterpret_cast<unsigned short*>(r1) = (unsigned short)(w1 >> 16);
-          *reinterpret_cast<unsigned short*>(r0 + R::PR_PART) = (unsigned short)(w2 & 0xFFFFu);
-          *reinterpret_cast<unsigned short*>(r1 + R::PR_PART) = (unsigned short)(w2 >> 16);
-          *reinterpret_cast<unsigned short*>(r0 + 2 * R::PR_PART) = (unsigned short)(w3 & 0xFFFFu);
-          *reinterpret_cast<unsigned short*>(r1 + 2 * R::PR_PART) = (unsigned short)(w3 >> 16);
+        for (int q = 0; q < 8; ++q) {
+          uint32_t a1, a2, a3;
+          split3_pair(sgn * x[2 * q], sgn * x[2 * q + 1], a1, a2, a3);
+          reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
+          reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
+          reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
+        }
+        unsigned char* prow = base_ptr + R::OFF_PR + row * 128;
+#pragma unroll
+        for (int part = 0; part < 3; ++part) {
+          *reinterpret_cast<uint4*>(prow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
+          *reinterpret_cast<uint4*>(prow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
         }
       }
       fence_proxy_async_smem();
@@ -245,7 +247,8 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       done |= 1u << blk;
     }
     if (ok) {
-      // ---- the inverse as three bf16 parts; this thread holds column `row` of it
+      // ---- the inverse as three bf16 parts; this thread holds row `row` of it and stores it transposed (the
+      // inverse is symmetric), so that the 32 lanes of a warp write 32 consecutive elements
       __nv_bfloat16* c1 = csplit + (size_t)n * (3 * D * D) + row;
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
