@@ -8,13 +8,17 @@
 // i.e. one rank-16 update  M += Cm * M[P][:]  of the whole matrix plus a 128 x 16 column fix.  The rank-16
 // update is a 128 x 128 x 16 MMA accumulating into the TMEM-resident matrix.  Both factors are fp32 values
 // split three-way into bf16 parts (24 mantissa bits); the six partial products of weight >= 2^-24 are
-// accumulated in fp32, so the update carries fp32 accuracy.  Everything else is plain fp32:
-//   * the 16 x 16 pivot block is inverted inside the warp that owns those rows, one row per lane, the pivot
-//     rows travelling by shuffle;
-//   * every thread owns one matrix row (its TMEM lane), forms its 16 coefficients from Gi, and -- the matrix
-//     being symmetric up to the sign pattern of in-place elimination -- also supplies its column of the 16
-//     pivot rows, so nobody has to read whole rows back.  Both MMA operands are K-major with one row per
-//     thread, so each thread writes its 16 values of a part as 32 contiguous bytes.
+// accumulated in fp32, so the update carries fp32 accuracy.
+//   * The 16 x 16 pivot block is inverted in plain fp32 inside the warp that owns those rows, one row per lane,
+//     the pivot rows travelling by shuffle.
+//   * Every thread owns one matrix row (its TMEM lane) and -- the matrix being symmetric up to the sign pattern of
+//     in-place elimination -- supplies its column of the 16 pivot rows (its own 16 pivot-column entries, signed),
+//     so nobody has to read whole rows back.  Both MMA operands are K-major with one row per thread: a thread
+//     writes its 16 values of a part as 32 contiguous bytes.
+//   * The 128 x 16 coefficients Cm = -M[:, P] Gi are a matrix product as well: the pivot-row operand the threads
+//     have just written, times Gi (split three-way by the pivot warp), in a first, 128 x 16 x 16 MMA into the
+//     pivot columns themselves; each thread reads its row back and applies its sign.  Formed with fp32 FMAs
+//     (256 per thread and step) they were the largest item of a kernel that is bound by instruction issue.
 // The matrix that is inverted is I + (A_t + A_t^T)/2: the stored statistics are symmetric only up to the bf16
 // rounding of one factor, and the symmetric part is the natural reading of Eq. 3b (and keeps Proposition 1).
 // The inverse is written as three bf16 parts C1 + C2 + C3 for the tensor-core scan.
@@ -43,7 +47,8 @@ struct ResolveTc {
                                                       // rows, parts laid out like the coefficients
   static constexpr int OFF_CM = 0;
   static constexpr int OFF_PR = CM_BYTES;
-  static constexpr int OFF_GI = OFF_PR + PR_BYTES;    // Gi, 16 x 16 floats
+  static constexpr int OFF_GIB = OFF_PR + PR_BYTES;   // Gi as an MMA operand: 16 rows x 128 B, three parts per row
+  static constexpr int OFF_GI = OFF_GIB + 2048;       // Gi, 16 x 16 floats (for the pivot rows themselves)
   static constexpr int OFF_BAR = OFF_GI + 1024;
   static constexpr int SMEM_BYTES = OFF_BAR + 64 + 1024;
   static constexpr int THREADS = 160;                 // 4 row warps + 1 MMA warp
@@ -59,8 +64,9 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
   const uint32_t OPREADY = base + R::OFF_BAR, MMADONE = base + R::OFF_BAR + 8;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 16);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 20);
+  const uint32_t XREADY = base + R::OFF_BAR + 16, CDONE = base + R::OFF_BAR + 24;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 36);
   float* gi = reinterpret_cast<float*>(base_ptr + R::OFF_GI);
   const WaitCtx wc{abort_flag, status};
 
@@ -72,6 +78,8 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
   if (threadIdx.x == 0) {
     mbar_init(OPREADY, 4);                    // one arrival per row warp
     mbar_init(MMADONE, 1);
+    mbar_init(XREADY, 4);
+    mbar_init(CDONE, 1);
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -90,7 +98,21 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
       constexpr int PA[6] = {0, 2, 1, 0, 1, 0};   // (coefficient part, pivot-row part), smallest first
       constexpr int PB[6] = {2, 0, 1, 1, 0, 0};
+      constexpr uint32_t idesc_c = make_idesc_bf16(128, 16, false, false);
       for (int step = 0; step < D / R::NB; ++step) {
+        // ---- coefficients: M[:, P] <- Xs Gi (128 x 16 x 16), Xs = the signed pivot columns the row threads just
+        // wrote as the pivot-row operand, Gi = the inverse of the pivot block; each thread negates / signs its row
+        const int p0c = (((int)(blockIdx.x & 3) * 2 + step) & 7) * R::NB;
+        if (!mbar_wait(XREADY, step & 1, wc)) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int pr = 0; pr < 6; ++pr) {
+          const uint64_t adesc = make_smem_desc(base + R::OFF_PR + PA[pr] * 32, 16, 1024);
+          const uint64_t bdesc = make_smem_desc(base + R::OFF_GIB + PB[pr] * 32, 16, 1024);
+          mma_bf16_ss(tmem_base + p0c, adesc, bdesc, idesc_c, pr == 0 ? 0u : 1u);
+        }
+        mma_commit(CDONE);
+        // ---- the rank-16 update of the whole matrix
         if (!mbar_wait(OPREADY, step & 1, wc)) break;
         tc_fence_after_sync();
 #pragma unroll
@@ -149,6 +171,29 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       tmem_ld16(trow + p0, x);
       tmem_wait_ld();
 
+      // ---- the 16 pivot rows as an MMA operand, three bf16 parts.  M is symmetric up to the sign pattern of
+      // in-place elimination: M[P_k][j] = M[j][P_k] for rows j not yet eliminated and -M[j][P_k] for rows already
+      // eliminated (`done`).  So thread j owns column j of the pivot rows: its own x, signed -- which is one row
+      // of the K-major operand (row = output column, 16 contiguous pivot indices): two 16-byte stores per part.
+      // The same rows, times Gi, give the update coefficients (below).
+      const float sgn = ((done >> (row >> 4)) & 1u) ? -1.0f : 1.0f;
+      {
+        uint4 w[3][2];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          uint32_t a1, a2, a3;
+          split3_pair(sgn * x[2 * q], sgn * x[2 * q + 1], a1, a2, a3);
+          reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
+          reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
+          reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
+        }
+        unsigned char* prow = base_ptr + R::OFF_PR + row * 128;
+#pragma unroll
+        for (int part = 0; part < 3; ++part) {
+          *reinterpret_cast<uint4*>(prow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
+          *reinterpret_cast<uint4*>(prow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
+        }
+      }
       if (warp == (blk >> 1)) {
         // ---- invert the 16 x 16 pivot block: lane (l0 + a) holds row a; pivot rows travel by shuffle
         const int l0 = (blk & 1) * 16;
@@ -170,28 +215,49 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           g[p] = prow ? ip : -fi;
         }
         if (owner) {
-          float* dst = gi + (row & 15) * 16;
+          // Gi row a: in fp32 for this pivot row's own coefficients, and as three bf16 parts for the tensor cores
+          // (Gi is symmetric, so its rows serve as the rows of the K-major operand, which wants columns)
+          const int a = row & 15;
+          float* dst = gi + a * 16;
 #pragma unroll
           for (int j = 0; j < 16; j += 4) store4(dst + j, make_float4(g[j], g[j + 1], g[j + 2], g[j + 3]));
+          uint4 w[3][2];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            uint32_t a1, a2, a3;
+            split3_pair(g[2 * q], g[2 * q + 1], a1, a2, a3);
+            reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
+            reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
+            reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
+          }
+          unsigned char* grow = base_ptr + R::OFF_GIB + a * 128;
+#pragma unroll
+          for (int part = 0; part < 3; ++part) {
+            *reinterpret_cast<uint4*>(grow + (((2 * part) ^ (a & 7)) * 16)) = w[part][0];
+            *reinterpret_cast<uint4*>(grow + (((2 * part + 1) ^ (a & 7)) * 16)) = w[part][1];
+          }
         }
       }
-      named_barrier_sync(1, 128);
+      fence_proxy_async_smem();
+      tc_fence_before_sync();
+      mbar_arrive_warp(XREADY);
 
-      // ---- coefficients: c = -xx Gi  with xx = M[i][P] (other rows) or -e_a (pivot row a, giving Gi[a])
+      // ---- coefficients: c = -M[i][P] Gi = -sgn (Xs Gi) from the tensor cores; a pivot row a takes Gi[a]
+      if (!mbar_wait(CDONE, step & 1, wc)) { ok = false; break; }
+      tc_fence_after_sync();
       float c[16];
-#pragma unroll
-      for (int k = 0; k < 16; ++k) c[k] = 0.f;
-#pragma unroll
-      for (int l = 0; l < 16; ++l) {
-        const float xl = owner ? ((row & 15) == l ? 1.0f : 0.0f) : -x[l];
+      tmem_ld16(trow + p0, c);
+      tmem_wait_ld();
+      if (owner) {
+        const float* src = gi + (row & 15) * 16;
 #pragma unroll
         for (int k = 0; k < 16; k += 4) {
-          const float4 gq = load4(gi + l * 16 + k);
-          c[k] = fmaf(xl, gq.x, c[k]);
-          c[k + 1] = fmaf(xl, gq.y, c[k + 1]);
-          c[k + 2] = fmaf(xl, gq.z, c[k + 2]);
-          c[k + 3] = fmaf(xl, gq.w, c[k + 3]);
+          const float4 gq = load4(src + k);
+          c[k] = gq.x; c[k + 1] = gq.y; c[k + 2] = gq.z; c[k + 3] = gq.w;
         }
+      } else {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) c[k] *= -sgn;
       }
       // ---- A operand: this row's 16 update coefficients (pivot rows: Gi[a] - e_a), three bf16 parts
       {
@@ -212,28 +278,6 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
         for (int part = 0; part < 3; ++part) {
           *reinterpret_cast<uint4*>(crow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
           *reinterpret_cast<uint4*>(crow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
-        }
-      }
-      // ---- B operand: the 16 pivot rows, three bf16 parts.  M is symmetric up to the sign pattern of in-place
-      // elimination: M[P_k][j] = M[j][P_k] for rows j not yet eliminated and -M[j][P_k] for rows already
-      // eliminated (`done`).  So thread j owns column j of the pivot rows: its own x, signed -- which is one row
-      // of the K-major operand (row = output column, 16 contiguous pivot indices): two 16-byte stores per part.
-      {
-        const float sgn = ((done >> (row >> 4)) & 1u) ? -1.0f : 1.0f;
-        uint4 w[3][2];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          uint32_t a1, a2, a3;
-          split3_pair(sgn * x[2 * q], sgn * x[2 * q + 1], a1, a2, a3);
-          reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
-          reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
-          reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
-        }
-        unsigned char* prow = base_ptr + R::OFF_PR + row * 128;
-#pragma unroll
-        for (int part = 0; part < 3; ++part) {
-          *reinterpret_cast<uint4*>(prow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
-          *reinterpret_cast<uint4*>(prow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
         }
       }
       fence_proxy_async_smem();
