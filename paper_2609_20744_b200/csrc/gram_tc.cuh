@@ -10,9 +10,11 @@
 // Persistent CTAs, one per SM, loop over frames (b,h,t).  Warp roles:
 //   warp 0      TMA producer: K and V tiles (4 boxes of 16 KB) into a 3-stage ring
 //   warp 1      MMA issuer (one thread) and TMEM owner
-//   warps 2-5   weighting: K' = bf16(beta) * K in packed bf16 arithmetic, written to a second buffer in two halves of
-//               64 tokens so the MMA of one half overlaps the weighting of the other
-//   warps 6-9   drain: once per frame, the finished accumulator (of two) TMEM -> registers -> global fp32 [2d][d]
+//   warps 2-9   weighting: K' = bf16(beta) * K in packed bf16 arithmetic, written to a second buffer in two halves of
+//               64 tokens so the MMA of one half overlaps the weighting of the other.  A thread does 64 bytes of a
+//               token row: the stage is held for the length of this chain (load, multiply, store, proxy fence,
+//               arrive), and eight warps make it shorter than four (-3 %; sixteen are slower again)
+//   warps 10-13 drain: once per frame, the finished accumulator (of two) TMEM -> registers -> global fp32 [2d][d]
 //               (A_t, then B_t), while the other warps are already on the next frame
 // Rows past the end of a frame are zero-filled by TMA (the map has F as its own dimension) and their
 // beta is forced to zero.  Every mbarrier wait is bounded.
@@ -36,7 +38,7 @@ struct GramTc {
   static constexpr int USED_BYTES = OFF_BAR + 128;
   static constexpr int SMEM_BYTES = 232448;                // everything an SM offers one CTA; the slack
                                                            // absorbs the 1024-byte alignment
-  static constexpr int THREADS = 320;
+  static constexpr int THREADS = 448;
 };
 
 __global__ void __launch_bounds__(GramTc::THREADS, 1)
@@ -72,7 +74,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 3; ++i) { mbar_init(FULL(i), 1); mbar_init(EMPTY(i), 1); }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(SCALED(i), 4); mbar_init(KPFREE(i), 1);      // one arrival per weighting warp
+      mbar_init(SCALED(i), 8); mbar_init(KPFREE(i), 1);      // one arrival per weighting warp
       mbar_init(ACCFULL(i), 1);  mbar_init(ACCEMPTY(i), 4);   // ... per drain warp
     }
     *abort_flag = 0;
@@ -148,7 +150,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (ok) mma_commit(ACCFULL(a));
       }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= 10) {
     // ------------------------------------------------------------------ drain warps
     // TMEM -> registers -> global fp32 [2d][d].  Accumulator lane = key channel i, column = column of [K|V];
     // stored transposed so that the 32 lanes of a warp write 32 consecutive floats.
@@ -176,8 +178,9 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------------ weighting warps: K' = beta * K
-    const int ts = threadIdx.x - 64;          // 0..127
-    const int r = ts >> 1, c = ts & 1;        // row within the half, 64-channel box
+    const int ts = threadIdx.x - 64;          // 0..255
+    const int r = ts >> 2, c = (ts >> 1) & 1; // row within the half, 64-channel box
+    const int q4 = (ts & 1) * 4;              // which four 16-byte chunks of the 128-byte row
     uint32_t it = 0;
     bool ok = true;
 
@@ -216,18 +219,18 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           // all eight loads first, then the stores: written as one load-store pair per chunk the compiler
           // must keep them in order (the two shared-memory pointers might alias) and every chunk pays the
           // full shared-memory latency
-          uint4 raw[8];
+          uint4 raw[4];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) raw[j] = *reinterpret_cast<const uint4*>(src + ((j ^ (r & 7)) * 16));
+          for (int j = 0; j < 4; ++j) raw[j] = *reinterpret_cast<const uint4*>(src + (((q4 + j) ^ (r & 7)) * 16));
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
+          for (int j = 0; j < 4; ++j) {
             __nv_bfloat162* x = reinterpret_cast<__nv_bfloat162*>(&raw[j]);
 #pragma unroll
             for (int e = 0; e < 4; ++e) x[e] = __hmul2(x[e], w2);
           }
 #pragma unroll
-          for (int j = 0; j < 8; ++j)            // chunks staggered across rows: conflict-free
-            *reinterpret_cast<uint4*>(dst + ((j ^ (r & 7)) * 16)) = raw[j];
+          for (int j = 0; j < 4; ++j)            // chunks staggered across rows: conflict-free
+            *reinterpret_cast<uint4*>(dst + (((q4 + j) ^ (r & 7)) * 16)) = raw[j];
           fence_proxy_async_smem();
           mbar_arrive_warp(SCALED(half));
         }
