@@ -260,3 +260,35 @@ def test_chunkwise_scan_is_chosen_for_few_chains_and_needs_its_workspace():
                                       w.B, w.T, w.F, w.H, w.d, ctypes.byref(opt), None)
     assert st == 3
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64), ("f32", 128)])
+def test_random_window_settings_on_every_scan_schedule(dtype, d):
+    # seeded sweep over (T, chunk, radius, anchors, alpha?, s0?) on small frames: the bookkeeping of which state a
+    # frame reads, where a chain may stop, and which chunks get composed, against the checker every time
+    import random
+    rnd = random.Random(20744)
+    for trial in range(24):
+        T = rnd.randint(1, 27)
+        chunk = rnd.choice([1, 2, 3, 4, 5, 7])
+        radius = rnd.choice([0, 0, 1, 1, 2])
+        anchors = rnd.random() < 0.5
+        use_alpha = rnd.random() < 0.6
+        use_s0 = rnd.random() < 0.6
+        flags = rnd.choice([0, binding.VDN_FLAG_SCAN_FRAMEWISE, CHUNKWISE])
+        w = inputs.TINY.scaled(dtype=dtype, d=d, B=1, H=1, T=T, F=48, seed=1000 + trial)
+        x = inputs.generate(w, "cuda")
+        alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+        alpha = alpha if use_alpha else None
+        s0 = s0 if use_s0 else None
+        vda = binding.Vda(w.d, w.dtype, flags=flags)
+        kw = dict(chunk=chunk, radius=radius, anchors=anchors)
+        out = torch.full_like(x["q"], 9.0)
+        vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out, alpha=alpha, s0=s0, **kw)
+        torch.cuda.synchronize()
+        assert vda.status() == binding.VDN_OK, (trial, T, kw, flags)
+        try:
+            check(w, x, out, alpha, s0, **kw)
+        except AssertionError as e:
+            raise AssertionError(f"trial {trial}: T={T} {kw} alpha={use_alpha} s0={use_s0} flags={flags}: {e}")
+        vda.close()
