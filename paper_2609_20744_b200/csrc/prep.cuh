@@ -69,6 +69,17 @@ __device__ __forceinline__ float silu_f(float x) {
   return x * r;
 }
 
+// the same for a packed pair: the scale, the "+ 1" and the final product as packed operations
+__device__ __forceinline__ void silu2(f32x2 x, float& y0, float& y1) {
+  float t0, t1, e0, e1, r0, r1;
+  unpack2(mul2(x, pack2(-1.4426950408889634f, -1.4426950408889634f)), t0, t1);
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(t0));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(t1));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(1.0f + e0));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(1.0f + e1));
+  unpack2(mul2(x, pack2(r0, r1)), y0, y1);
+}
+
 struct PrepKv {
   static constexpr int TX = 8;          // tile columns = tokens per thread
   static constexpr int HALO = 2;
@@ -177,7 +188,7 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
         __syncthreads();
         // ---- spatial filter of frame t for this thread's row: slide over the SW input columns
         const Tio* base = tile + (size_t)(t & 1) * SH * SW * D + (size_t)g * SW * D + 2 * cp;
-        f32x2 acc[TX];
+        f32x2 (&acc)[TX] = ring[r];         // the spatial result accumulates straight into this step's ring slot
 #pragma unroll
         for (int j = 0; j < TX; ++j) acc[j] = 0ull;
 #pragma unroll
@@ -195,8 +206,6 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
             }
           }
         }
-#pragma unroll
-        for (int j = 0; j < TX; ++j) ring[r][j] = acc[j];
         __syncthreads();                    // the buffer may be overwritten by the copy issued two steps on
       } else {
 #pragma unroll
@@ -211,9 +220,7 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
         f32x2 o = mul2(wtp[0], ring[(r + 1) % 5][j]);
 #pragma unroll
         for (int i = 1; i < 5; ++i) o = fma2(wtp[i], ring[(r + i + 1) % 5][j], o);
-        unpack2(o, o0[j], o1[j]);
-        o0[j] = silu_f(o0[j]);
-        o1[j] = silu_f(o1[j]);
+        silu2(o, o0[j], o1[j]);
       }
       const int y = y0 + g;
       if (which == 0) {
