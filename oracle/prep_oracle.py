@@ -7,7 +7,7 @@ What the linear branch does to the projected q, k, v before the recurrence (Sec.
     K, V : a separable short convolution -- a depthwise 5 x 5 spatial filter and a five-tap temporal filter,
            one filter pair per channel -- followed by SiLU;
     Q, K : L2 normalisation over the d channels of each (token, head).
-Readings where the text is silent (also listed in the design doc):
+Readings where the text is silent:
   * "convolution" is the cross-correlation of deep-learning libraries, taps centred on the output position
     (the model is bidirectional, so the temporal filter is centred too), zero padding, no bias;
   * the SiLU belongs to the convolved tensors (K and V); Q is only normalised;
