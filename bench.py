@@ -202,8 +202,8 @@ def run_reference(args, w, rank: int, world: int):
     """The reference arm is the fp64 oracle on the host cores (rank 0 only)."""
     if rank != 0:
         return
-    budget = 60.0                                         # seconds for the whole --steps/--warmup run
-    heads, frames = plan_sample(w, budget / max(1, args.steps + args.warmup))
+    seconds_total = 60.0                                  # for the whole --steps/--warmup run
+    heads, frames = plan_sample(w, seconds_total / max(1, args.steps + args.warmup))
     _, slices = oracle_sample(w, heads, frames)
     for _ in range(args.warmup):
         time_oracle(slices)
