@@ -55,6 +55,7 @@ struct ScanTc {
   static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
   static constexpr int CW = 32;                      // value columns per state thread
   static constexpr int THREADS = 64 + 4 * 32 * (D / CW);  // producer + MMA + state warps
+  static constexpr int threads(int ns) { return 64 + 4 * 32 * (D / ns / CW); }
 };
 
 enum { SCAN_FRAMES = 0, SCAN_CHUNKS = 1, SCAN_COMPOSE = 2 };
@@ -81,7 +82,10 @@ __host__ __device__ inline int scan_chunk_steps(const Window& w, int dir) {
   return w.hi(w.first) == w.last ? 0 : w.last / w.chunk - w.hi(w.first) / w.chunk;
 }
 
-template <int MODE>
+// NS = 2 splits the value columns of a chain over two CTAs (the columns of Z evolve independently; each CTA
+// loads the whole C_t): for shapes whose chains would leave more than half of the SMs idle.  Such a CTA has half
+// the state warps (launch it with threads(NS) threads) and issues MMAs of N = 64.
+template <int MODE, int NS = 1>
 __global__ void __launch_bounds__(ScanTc::THREADS, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int* status) {
   using namespace tc;
@@ -120,8 +124,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
     f_hi = min(win.last, (kc + 1) * win.chunk - 1);
     nsteps = f_hi - f_lo + 1;
   } else {
-    bh = blockIdx.x >> 1;
-    dir = blockIdx.x & 1;
+    bh = (blockIdx.x / NS) >> 1;
+    dir = (blockIdx.x / NS) & 1;
     // steps this chain runs: up to the last state that some frame reads (P_{l-1} of the last frame's window,
     // R_{h+1} of the first frame's)
     if constexpr (MODE == SCAN_FRAMES) nsteps = dir == 0 ? win.lo(win.last) - win.first : win.last - win.hi(win.first);
@@ -136,7 +140,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
 
   if (threadIdx.x == 0) {
     for (int p = 0; p < 3; ++p) { mbar_init(CFULL(p), 1); mbar_init(CFREE(p), 1); }
-    mbar_init(XREADY, (S::THREADS - 64) / 32);     // one arrival per state warp
+    mbar_init(XREADY, (blockDim.x - 64) / 32);     // one arrival per state warp
     mbar_init(ACCFULL, 1);
     *abort_flag = 0;
     mbar_fence_init();
@@ -174,7 +178,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, true);
+      constexpr uint32_t idesc = make_idesc_bf16(128, 128 / NS, false, true);
       bool ok = true;
       for (int s = 0; s < nsteps && ok; ++s) {
         if (!mbar_wait(XREADY, s & 1, wc)) break;
@@ -205,11 +209,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
     constexpr int CW = S::CW;
     const int qd = warp & 3;                 // TMEM lane quarter
     const int row = qd * 32 + lane;          // key channel (row of Z, row of X)
-    const int slice = (warp - 2) >> 2;       // value columns [CW*slice, CW*slice + CW)
-    const int col0 = slice * CW;
-    const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + col0;
-    unsigned char* xrow = base_ptr + S::OFF_X + (col0 >> 6) * S::BOX_BYTES + row * 128;
-    const int ch0 = (col0 & 63) >> 3;        // first 16-byte chunk of this thread inside the 64-column box
+    const int slice = (warp - 2) >> 2;       // this CTA's value columns [CW*slice, CW*slice + CW)
+    const int lc0 = slice * CW;              // ... counted inside the CTA (TMEM column, operand column)
+    const int col0 = (MODE == SCAN_COMPOSE ? 0 : (int)(blockIdx.x % NS) * (D / NS)) + lc0;   // ... inside the state
+    const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + lc0;
+    unsigned char* xrow = base_ptr + S::OFF_X + (lc0 >> 6) * S::BOX_BYTES + row * 128;
+    const int ch0 = (lc0 & 63) >> 3;         // first 16-byte chunk of this thread inside the 64-column box
     const int sw = row & 7;
 
     auto load_bt = [&](int s, float (&bt)[CW]) {

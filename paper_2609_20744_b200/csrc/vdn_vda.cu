@@ -322,6 +322,8 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
                                      vdn::ReadoutTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
+    VDN_CUDA(h, (cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      vdn::ScanTc::SMEM_BYTES)));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_CHUNKS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_COMPOSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -380,6 +382,11 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
       vdn::scan_tc_kernel<vdn::SCAN_CHUNKS><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
                                               vdn::ScanTc::SMEM_BYTES, st>>>(tmM, sa, h->status_dev);
       prof_mark(h, st, nk++, "scan_chunks_tc");
+    } else if (4LL * s.B * s.H <= h->sm_count) {
+      // few chains: two CTAs per chain, half of the value columns each
+      vdn::scan_tc_kernel<vdn::SCAN_FRAMES, 2><<<(unsigned)(4 * s.B * s.H), vdn::ScanTc::threads(2),
+                                                 vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
+      prof_mark(h, st, nk++, "scan_tc");
     } else {
       vdn::scan_tc_kernel<vdn::SCAN_FRAMES><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
                                               vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
