@@ -230,7 +230,8 @@ def test_stagewise_intermediates_tensor_core_kernels():
             # that rounding only; the resolve inverts I + its symmetric part)
             a_sym = 0.5 * (stats[0, h, t, :d, :] + stats[0, h, t, :d, :].T)
             inv_g = np.linalg.inv(np.eye(d) + a_sym)
-            assert rel(split[0, h, t].sum(axis=0), inv_g) < 1e-5            # three parts carry fp32 accuracy
+            # three parts carry fp32 accuracy: an fp32 inverse is good to a few eps times the condition number
+            assert rel(split[0, h, t].sum(axis=0), inv_g) < 5e-6 * np.linalg.cond(np.eye(d) + a_sym)
             assert rel(split[0, h, t, 0], inv_g) < 8e-3                     # the leading part alone: bf16, truncated (2^-7)
             want_f = ref["P"][t - 1] if t > 0 else np.zeros((d, d))
             want_b = ref["R"][t + 1] if t + 1 < T else np.zeros((d, d))
