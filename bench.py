@@ -178,8 +178,8 @@ def plan_sample(w, seconds_per_step: float):
     time_oracle(sl)                                       # page in numpy / BLAS
     per_frame = time_oracle(sl) / probe_T                 # seconds per (head, frame)
     per_head = per_frame * w.T
-    if per_head <= seconds_per_step:                      # at most 4 slices: drawing them on the CPU costs time too
-        return max(1, min(w.B * w.H, 4, int(seconds_per_step / per_head))), w.T
+    if per_head <= seconds_per_step:                      # at most 8 slices: drawing them on the CPU costs time too
+        return max(1, min(w.B * w.H, 8, int(seconds_per_step / per_head))), w.T
     return 1, max(2, min(w.T, int(seconds_per_step / per_frame)))
 
 
