@@ -43,6 +43,15 @@ def check_heads(w, x, out, pairs, tol):
     return worst
 
 
+def kernel_names(vda, x):
+    vda.profile(True)
+    vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
+    torch.cuda.synchronize()
+    times = vda.kernel_times()
+    vda.profile(False)
+    return times
+
+
 def all_pairs(w):
     return [(b, h) for b in range(w.B) for h in range(w.H)]
 
@@ -56,6 +65,7 @@ def all_pairs(w):
     ("tiny", dict(B=2, H=1, T=3, F=257)),                      # several tiles + tail, two batches
     ("tiny", dict(dtype="bf16", d=128, T=6, F=300, H=2)),      # bf16 I/O
     ("tiny", dict(dtype="bf16", d=64, T=3, F=70, H=2)),
+    ("tiny", dict(dtype="bf16", d=128, B=2, T=5, F=3100, H=3)),  # long frames, ragged last tile
 ])
 def test_forward_matches_oracle_small(name, kw):
     w = inputs.WORKLOADS[name].scaled(**kw)
@@ -204,11 +214,13 @@ def test_stagewise_intermediates_plain_fp32_kernels(dtype, d, flags):
             assert rel(read[0, h, t].T, want) < 1e-5
 
 
-def test_stagewise_intermediates_tensor_core_kernels():
+@pytest.mark.parametrize("F", [300, 3200])
+def test_stagewise_intermediates_tensor_core_kernels(F):
     d = 128
-    w = inputs.TINY.scaled(dtype="bf16", d=d, T=6, F=300, H=2)
+    w = inputs.TINY.scaled(dtype="bf16", d=d, T=6, F=F, H=2)
     x = inputs.generate(w, "cuda")
     vda, out = run_gpu(w, x)
+    assert [n for (n, _, _) in kernel_names(vda, x)] == ["gram_tc", "resolve_tc", "scan_tc", "readout_tc"]
     assert vda.uses_tensor_cores()
     B, T, F, H = w.B, w.T, w.F, w.H
     stats = vda.view(binding.VIEW_STATS, B, T, F, H).double().cpu().numpy()
@@ -242,11 +254,12 @@ def test_stagewise_intermediates_tensor_core_kernels():
             if t == T - 1:
                 assert not pb[0, h, t].any()
             # against the checker fed with the GPU's statistics the stored states differ by their own bf16
-            # rounding only (2^-9 relative per element): the scan itself runs at fp32 accuracy
+            # rounding (2^-9 relative per element) plus an fp32-level absolute term (a few eps times the condition
+            # number, relative to the largest entry): the inverse and the scan run at fp32 accuracy
             if t > 0:
-                assert np.max(np.abs(pf[0, h, t] - Pg[t - 1]) / (np.abs(Pg[t - 1]) + 1e-3 * np.abs(Pg[t - 1]).max())) < 2.0 ** -8
+                assert np.all(np.abs(pf[0, h, t] - Pg[t - 1]) <= 2.0 ** -8 * np.abs(Pg[t - 1]) + 2e-5 * np.abs(Pg[t - 1]).max())
             if t + 1 < T:
-                assert np.max(np.abs(pb[0, h, t] - Rg[t + 1]) / (np.abs(Rg[t + 1]) + 1e-3 * np.abs(Rg[t + 1]).max())) < 2.0 ** -8
+                assert np.all(np.abs(pb[0, h, t] - Rg[t + 1]) <= 2.0 ** -8 * np.abs(Rg[t + 1]) + 2e-5 * np.abs(Rg[t + 1]).max())
 
 
 # ------------------------------------------------------------------------------ properties
