@@ -128,3 +128,32 @@ def test_prepare_argument_errors():
     with pytest.raises(binding.VdnError):
         vda.prepare(p["q"], p["k"], p["v"], p, 4, 5, out=(p["q"], p["k"], torch.empty_like(p["v"])))   # k in place
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_random_preparation_shapes(dtype, d):
+    # seeded sweep over clip length, token grid (whole tiles, ragged tiles, single rows and columns), anchors and the
+    # two variants (with and without the spatial filter)
+    import random
+    rnd = random.Random(744)
+    for trial in range(12):
+        T = rnd.randint(1, 9)
+        Y, X = rnd.choice([(1, 1), (1, 9), (9, 1), (4, 8), (5, 9), (8, 16), (3, 17), (13, 5)])
+        anchors = rnd.random() < 0.4
+        spatial = rnd.random() < 0.6
+        w = inputs.TINY.scaled(dtype=dtype, d=d, B=rnd.choice([1, 2]), H=rnd.choice([1, 2, 3]), T=T, F=Y * X,
+                               seed=3000 + trial)
+        p = inputs.generate_projected(w, "cuda")
+        vda = binding.Vda(w.d, w.dtype)
+        flt = p if spatial else dict(wk_temporal=p["wk_temporal"], wv_temporal=p["wv_temporal"])
+        got = vda.prepare(p["q"], p["k"], p["v"], flt, Y, X, anchors=anchors)
+        torch.cuda.synchronize()
+        assert vda.status() == binding.VDN_OK
+        if not spatial:
+            for n in ("wk", "wv"):
+                p[n + "_spatial"].zero_(); p[n + "_spatial"][:, 2, 2] = 1.0
+        try:
+            check(w, p, got, Y, X, anchors)
+        except AssertionError as e:
+            raise AssertionError(f"trial {trial}: T={T} grid={Y}x{X} anchors={anchors} spatial={spatial}: {e}")
+        vda.close()
