@@ -21,31 +21,38 @@
 
 namespace vdn {
 
-struct ReadoutTc {
+template <bool EXTRAS>
+struct ReadoutTcCfg {
   static constexpr int D = 128;
   static constexpr int TILE = 128;
-  static constexpr int QSTAGES = 3;
+  // EXTRAS: gate tiles arrive by TMA in the output staging tiles (a third one takes the place of a Q stage)
+  static constexpr int QSTAGES = EXTRAS ? 2 : 3;       // (3 Q stages, 2 staging tiles and a one-tile gate lookahead:
+  static constexpr int NOUT = EXTRAS ? 3 : 2;          //  2.74 ms instead of 2.07 ms on the 768p clip)
   static constexpr int BOX_BYTES = 128 * 128;          // 128 rows x 128 B
   static constexpr int TILE_BYTES = 2 * BOX_BYTES;     // 32 KB: state, Q tile or output tile
   static constexpr int OFF_STATE = 0;
   static constexpr int OFF_Q = 2 * TILE_BYTES;
   static constexpr int OFF_OUT = OFF_Q + QSTAGES * TILE_BYTES;
-  static constexpr int OFF_BAR = OFF_OUT + 2 * TILE_BYTES;
+  static constexpr int OFF_NW = OFF_OUT + NOUT * TILE_BYTES;   // norm weights of the current head, 128 floats
+  static constexpr int OFF_BAR = OFF_NW + 512;
   static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
   static constexpr int THREADS = 192;
 };
+using ReadoutTc = ReadoutTcCfg<false>;
 
 // EXTRAS = true adds the two optional factors of Eq. 1c to the epilogue: an element-wise (content-dependent) gate
-// gate_elem [B,T,F,H,d] bf16 and a per-channel norm scale norm_weight [H,d]; either may be null, and so may the
-// per-head gate (read as 1).  The plain instantiation carries none of that code.
+// gate_elem [B,T,F,H,d] bf16 (tensor map tmG; its tiles arrive by TMA in the very staging tile the output is then
+// written to, two tiles ahead) and a per-channel norm scale norm_weight [H,d] (kept in shared memory per frame);
+// either may be null, and so may the per-head gate (read as 1).  The plain instantiation carries none of that code.
 template <bool EXTRAS>
-__global__ void __launch_bounds__(ReadoutTc::THREADS, 1)
+__global__ void __launch_bounds__(ReadoutTcCfg<EXTRAS>::THREADS, 1)
 readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmS,
-                  const __grid_constant__ CUtensorMap tmO, const float* __restrict__ gate, Shape s, float eps,
+                  const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmG,
+                  const float* __restrict__ gate, Shape s, float eps,
                   int* status, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight,
                   Window win, int bridged) {
   using namespace tc;
-  using R = ReadoutTc;
+  using R = ReadoutTcCfg<EXTRAS>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -57,8 +64,9 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   auto STEMPTY = [&](int i) { return bar0 + 8u * (8 + i); };     // 2
   auto ACCFULL = [&](int i) { return bar0 + 8u * (10 + i); };    // 4
   auto ACCEMPTY = [&](int i) { return bar0 + 8u * (14 + i); };   // 4
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 8 * 18);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 8 * 18 + 8);
+  auto GFULL = [&](int i) { return bar0 + 8u * (18 + i); };      // 3 (EXTRAS: gate tile landed)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 8 * 21);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 8 * 21 + 8);
   const WaitCtx wc{abort_flag, status};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -69,11 +77,13 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     for (int i = 0; i < 3; ++i) { mbar_init(QFULL(i), 1); mbar_init(QEMPTY(i), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(STFULL(i), 1); mbar_init(STEMPTY(i), 1); }
     for (int i = 0; i < 4; ++i) { mbar_init(ACCFULL(i), 1); mbar_init(ACCEMPTY(i), 4); }   // one arrival per epilogue warp
+    for (int i = 0; i < 3; ++i) mbar_init(GFULL(i), 1);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmS);
     tma_prefetch_desc(&tmO);
+    if (EXTRAS) tma_prefetch_desc(&tmG);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), 512);
@@ -158,24 +168,37 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int et = threadIdx.x - 64;            // 0..127
     uint32_t qi = 0;
     bool ok = true;
+    const bool use_ge = EXTRAS && gate_elem != nullptr;
+    float* nws = reinterpret_cast<float*>(base_ptr + R::OFF_NW);
+    // EXTRAS: the gate tile of tile number q (counted over this CTA's tiles) is copied into staging tile q % NOUT,
+    // where the output of that tile is then written; issued by one thread, two tiles ahead
+    auto issue_gate = [&](uint32_t q, long long gitem, int gtile) {
+      while (gtile >= ntiles) { gtile -= ntiles; gitem += gridDim.x; }
+      if (gitem >= nitems) return;
+      int gb, gh, gt;
+      split_work(s, gitem, gb, gh, gt);
+      const int ob = q % R::NOUT;
+      const uint32_t dstg = base + R::OFF_OUT + ob * R::TILE_BYTES;
+      mbar_arrive_expect_tx(GFULL(ob), R::TILE_BYTES);
+      tma_load_5d(dstg, &tmG, GFULL(ob), 0, gh, gtile * R::TILE, gt, gb);
+      tma_load_5d(dstg + R::BOX_BYTES, &tmG, GFULL(ob), 64, gh, gtile * R::TILE, gt, gb);
+    };
+    if (use_ge && et == 0) {
+      for (int i = 0; i < R::NOUT - 1; ++i) issue_gate(i, blockIdx.x, i);
+    }
     for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
       int b, h, t;
       split_work(s, item, b, h, t);
       const float g = (!EXTRAS || gate) ? __ldg(gate + h) : 1.0f;
+      const bool use_nw = EXTRAS && norm_weight != nullptr;
+      if (use_nw) {
+        // this head's norm weights into shared memory (all epilogue threads are past the previous frame's reads:
+        // they met at the barrier before its last store)
+        nws[et] = __ldg(norm_weight + (size_t)h * R::D + et);
+        named_barrier_sync(1, 128);
+      }
       for (int tile = 0; tile < ntiles; ++tile, ++qi) {
         const int a = qi & 3;
-        // the token's 128 gate values (256 contiguous bytes), requested before the accumulator is waited for
-        uint4 graw[EXTRAS ? 16 : 1];
-        bool has_ge = false;
-        if constexpr (EXTRAS) {
-          const int u = tile * R::TILE + row;
-          has_ge = gate_elem != nullptr && u < s.F;
-          if (has_ge) {
-            const uint4* gp = reinterpret_cast<const uint4*>(gate_elem + token_offset(s, b, t, u, h));
-#pragma unroll
-            for (int j = 0; j < 16; ++j) graw[j] = __ldg(gp + j);
-          }
-        }
         if (!mbar_wait(ACCFULL(a), (qi >> 2) & 1, wc)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 128;
@@ -194,52 +217,52 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
           for (int e = 0; e < 32; ++e) ss = fmaf(v[c][e], v[c][e], ss);
         const float scale = g * rsqrtf(ss * (1.0f / R::D) + eps);
-        if constexpr (EXTRAS) {
-          // v <- v * norm_weight[c] * gate_elem[c]; the common factor `scale` is applied while packing
-          if (norm_weight != nullptr) {
-            const float4* wp = reinterpret_cast<const float4*>(norm_weight + (size_t)h * R::D);
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-              for (int e = 0; e < 32; e += 4) {
-                const float4 w4 = __ldg(wp + c * 8 + (e >> 2));
-                v[c][e] *= w4.x; v[c][e + 1] *= w4.y; v[c][e + 2] *= w4.z; v[c][e + 3] *= w4.w;
-              }
-          }
-          if (has_ge) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const __nv_bfloat162* gp2 = reinterpret_cast<const __nv_bfloat162*>(&graw[c * 4 + j]);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  const float2 gf = __bfloat1622float2(gp2[e]);
-                  v[c][j * 8 + 2 * e] *= gf.x;
-                  v[c][j * 8 + 2 * e + 1] *= gf.y;
-                }
-              }
-          }
-        }
 
-        const int ob = qi & 1;
-        if (et == 0) tma_store_wait_read<1>();   // the store that last used this staging tile has read it
-        named_barrier_sync(1, 128);
+        const int ob = qi % R::NOUT;
+        if (use_ge) {
+          // the gate tile sits in the staging tile (its copy was issued after the store that last used the tile
+          // had been read)
+          if (!mbar_wait(GFULL(ob), (qi / R::NOUT) & 1, wc)) { ok = false; break; }
+        } else {
+          if (et == 0) tma_store_wait_read<R::NOUT - 1>();   // the store that last used this staging tile has read it
+          named_barrier_sync(1, 128);
+        }
         unsigned char* orow = base_ptr + R::OFF_OUT + ob * R::TILE_BYTES + row * 128;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
+            const int chunk = (c & 1) * 4 + j;          // 16-byte chunk inside the 64-channel box
+            const int boxi = c >> 1;                    // channels 0-63 / 64-127
+            uint4* slot = reinterpret_cast<uint4*>(orow + boxi * R::BOX_BYTES + ((chunk ^ (row & 7)) * 16));
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = v[c][j * 8 + e] * scale;
+            if constexpr (EXTRAS) {
+              if (use_nw) {
+                const float4 w0 = *reinterpret_cast<const float4*>(nws + c * 32 + j * 8);
+                const float4 w1 = *reinterpret_cast<const float4*>(nws + c * 32 + j * 8 + 4);
+                f[0] *= w0.x; f[1] *= w0.y; f[2] *= w0.z; f[3] *= w0.w;
+                f[4] *= w1.x; f[5] *= w1.y; f[6] *= w1.z; f[7] *= w1.w;
+              }
+              if (use_ge) {
+                const uint4 gr = *slot;                 // this token's eight gate values for these channels
+                const uint32_t* gu = reinterpret_cast<const uint32_t*>(&gr);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  f[2 * e] *= __uint_as_float(gu[e] << 16);
+                  f[2 * e + 1] *= __uint_as_float(gu[e] & 0xFFFF0000u);
+                }
+              }
+            }
             uint4 pk;
             uint32_t* x = reinterpret_cast<uint32_t*>(&pk);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              __nv_bfloat162 p = __floats2bfloat162_rn(v[c][j * 8 + 2 * e] * scale, v[c][j * 8 + 2 * e + 1] * scale);
-              x[e] = *reinterpret_cast<uint32_t*>(&p);
+              __nv_bfloat162 p2 = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+              x[e] = *reinterpret_cast<uint32_t*>(&p2);
             }
-            const int chunk = (c & 1) * 4 + j;          // 16-byte chunk inside the 64-channel box
-            const int boxi = c >> 1;                    // channels 0-63 / 64-127
-            *reinterpret_cast<uint4*>(orow + boxi * R::BOX_BYTES + ((chunk ^ (row & 7)) * 16)) = pk;
+            *slot = pk;
           }
         }
         fence_proxy_async_smem();
@@ -249,6 +272,12 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           tma_store_5d(&tmO, src, 0, h, tile * R::TILE, t, b);
           tma_store_5d(&tmO, src + R::BOX_BYTES, 64, h, tile * R::TILE, t, b);
           tma_store_commit();
+          if (use_ge) {
+            // the staging tile of the tile after next was last used by the previous tile's store: once that one
+            // has been read (only the newest may still be pending), the next gate tile may land there
+            tma_store_wait_read<1>();
+            issue_gate(qi + R::NOUT - 1, item, tile + R::NOUT - 1);
+          }
         }
       }
     }

@@ -319,7 +319,7 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ReadoutTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     vdn::ReadoutTc::SMEM_BYTES));
+                                     vdn::ReadoutTcCfg<true>::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
     VDN_CUDA(h, (cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -405,13 +405,17 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   const long long nread = sr.work_items();
   const long long ro_target = ((long long)h->sm_count * 27 + 16) / 32;
   const unsigned persistent_ro = (unsigned)(nread < ro_target ? nread : ro_target);
-  if (x.gate_elem || x.norm_weight || !gate)
-    vdn::readout_tc_kernel<true><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
-        tmQ, tmS, tmO, gate, sr, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
+  if (x.gate_elem || x.norm_weight || !gate) {
+    CUtensorMap tmG = tmO;                                      // the gate tensor has the layout of the output
+    if (x.gate_elem && (r = make_token_map(h, &tmG, x.gate_elem, s)) != VDN_OK) return r;
+    using RX = vdn::ReadoutTcCfg<true>;
+    vdn::readout_tc_kernel<true><<<persistent_ro, RX::THREADS, RX::SMEM_BYTES, st>>>(
+        tmQ, tmS, tmO, tmG, gate, sr, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
         x.norm_weight, x.win, x.alpha != nullptr);
-  else
+  } else {
     vdn::readout_tc_kernel<false><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
-        tmQ, tmS, tmO, gate, sr, h->cfg.rms_eps, h->status_dev, nullptr, nullptr, x.win, x.alpha != nullptr);
+        tmQ, tmS, tmO, tmO, gate, sr, h->cfg.rms_eps, h->status_dev, nullptr, nullptr, x.win, x.alpha != nullptr);
+  }
   prof_mark(h, st, nk++, "readout_tc");
   h->launches = nk;
   VDN_CUDA(h, cudaGetLastError());
