@@ -18,6 +18,8 @@
 #pragma once
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace vdn {
@@ -268,17 +270,20 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
 // owns one 16-byte piece of a (token, head) row and walks the frames with a five-frame ring in registers; the
 // lanes that share a row reduce the sum of squares by shuffles.  One read and one write of K and V: bound by HBM.
 struct PrepKvTemporal {
-  static constexpr int PF = 8;                                   // frames in flight per thread (12: 7 % slower)
-  static constexpr int SMEM_BYTES = PF * 256 * 16;
+  static constexpr int PF = 5;                                   // queue slots per thread (4, 6, 8: the same; 12: 7 % slower)
+  static constexpr int THREADS = 256;
+  static constexpr int SMEM_BYTES = PF * THREADS * 16;
 };
 
 template <typename Tio, int D>
-__global__ void __launch_bounds__(256, 2) prep_kv_temporal_kernel(PrepArgs a, Shape s) {
+__global__ void __launch_bounds__(PrepKvTemporal::THREADS, 512 / PrepKvTemporal::THREADS)
+prep_kv_temporal_kernel(PrepArgs a, Shape s) {
+  constexpr int NT = PrepKvTemporal::THREADS;
   constexpr int EPL = 16 / (int)sizeof(Tio);   // channels per thread
   constexpr int LPR = D / EPL;                 // lanes per (token, head) row
   const int which = blockIdx.y & 1;            // 0 = K (normalised), 1 = V
   const int b = blockIdx.y >> 1;
-  const long long gid = (long long)blockIdx.x * 256 + threadIdx.x;
+  const long long gid = (long long)blockIdx.x * NT + threadIdx.x;
   const long long rows = (long long)s.F * s.H;
   // whole warps stay together for the shuffles: threads past the end work on the last row and do not store
   const bool live = gid < rows * LPR;
@@ -288,13 +293,24 @@ __global__ void __launch_bounds__(256, 2) prep_kv_temporal_kernel(PrepArgs a, Sh
   const int h = (int)(row % s.H);
   const int ch = h * D + piece * EPL;
 
-  float wt[5][EPL];
+  // Channels are handled two at a time as packed fp32 pairs (fma.rn.f32x2 and friends): the kernel would
+  // otherwise be bound by instruction issue, at about 22 instructions per element, not by HBM.
+  constexpr int NP = EPL / 2;                  // channel pairs per thread
+  f32x2 wt[5][NP];
   {
-    const float* t0 = (which == 0 ? a.wt[0] : a.wt[1]) + (size_t)ch * 5;
+    // the thread's EPL x 5 taps are contiguous (and 16-byte aligned): 16-byte loads, a quarter of the L1 wavefronts
+    // of tap-by-tap loads, which otherwise cost a fifth of a CTA's lifetime
+    const float4* t0 = reinterpret_cast<const float4*>((which == 0 ? a.wt[0] : a.wt[1]) + (size_t)ch * 5);
+    float w[EPL * 5];
 #pragma unroll
-    for (int c = 0; c < EPL; ++c)
+    for (int i = 0; i < EPL * 5 / 4; ++i) {
+      const float4 x = __ldg(t0 + i);
+      w[4 * i] = x.x; w[4 * i + 1] = x.y; w[4 * i + 2] = x.z; w[4 * i + 3] = x.w;
+    }
 #pragma unroll
-      for (int i = 0; i < 5; ++i) wt[i][c] = __ldg(t0 + c * 5 + i);
+    for (int c = 0; c < NP; ++c)
+#pragma unroll
+      for (int i = 0; i < 5; ++i) wt[i][c] = pack2(w[(2 * c) * 5 + i], w[(2 * c + 1) * 5 + i]);
   }
   const size_t frame_elems = (size_t)rows * D;
   const Tio* src = static_cast<const Tio*>(which == 0 ? a.in[0] : a.in[1]) + (size_t)b * s.T * frame_elems +
@@ -303,85 +319,116 @@ __global__ void __launch_bounds__(256, 2) prep_kv_temporal_kernel(PrepArgs a, Sh
              piece * EPL;
   const int first = s.t0, last = s.t0 + s.Tn - 1;
 
-  float ring[5][EPL];
+  f32x2 ring[5][NP];
 #pragma unroll
   for (int i = 0; i < 5; ++i)
 #pragma unroll
-    for (int c = 0; c < EPL; ++c) ring[i][c] = 0.f;
+    for (int c = 0; c < NP; ++c) ring[i][c] = 0ull;
 
-  // Frames arrive through a queue of asynchronous copies in shared memory, PF frames ahead; a thread only ever
+  // Frames arrive through a queue of asynchronous copies in shared memory, PF - 1 frames ahead; a thread only ever
   // reads the 16 bytes it copied itself, so no barrier is needed.  (Held in registers, the same number of bytes
-  // in flight would cost a quarter of the register file.)
+  // in flight would cost a quarter of the register file.)  The queue is as long as the ring, so both slots of a
+  // step are static in the loop unrolled by five.
   constexpr int PF = PrepKvTemporal::PF;
-  extern __shared__ uint4 stg[];               // [PF][256]
+  static_assert(PF == 5, "queue slot = ring slot = step % 5");
+  extern __shared__ uint4 stg[];               // [PF][NT]
+  uint4* const myq = stg + threadIdx.x;
   const int nsteps = s.Tn + 2;
+  const Tio* psrc = src + (size_t)first * frame_elems;      // next frame to request
+  Tio* pdst = dst + (size_t)first * frame_elems;            // next frame to write
 #pragma unroll
   for (int i = 0; i < PF - 1; ++i) {
-    if (first + i <= last) cp_async16(&stg[i * 256 + threadIdx.x], src + (size_t)(first + i) * frame_elems);
+    if (first + i <= last) cp_async16(myq + i * NT, psrc);
+    psrc += frame_elems;
     cp_async_commit();
   }
+
+  // One step: request frame t + 4, take frame t = first + step into ring slot r, write frame t - 2.  EDGE = false
+  // is the steady state, where every frame involved exists; EDGE = true checks each of them.
+  auto one_step = [&](auto rc, auto ec, int step) {
+    constexpr int r = decltype(rc)::value;
+    constexpr bool EDGE = decltype(ec)::value;
+    const int t = first + step;
+    if (!EDGE || t + PF - 1 <= last) cp_async16(myq + ((r + PF - 1) % PF) * NT, psrc);
+    psrc += frame_elems;
+    cp_async_commit();
+    cp_async_wait<PF - 1>();                   // frame t has landed
+    if (!EDGE || t <= last) {
+      const uint4 cur = myq[r * NT];
+      if constexpr (sizeof(Tio) == 2) {
+        const uint32_t* u = reinterpret_cast<const uint32_t*>(&cur);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          ring[r][i] = pack2(__uint_as_float(u[i] << 16), __uint_as_float(u[i] & 0xFFFF0000u));
+      } else {
+        const float* u = reinterpret_cast<const float*>(&cur);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) ring[r][i] = pack2(u[2 * i], u[2 * i + 1]);
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < NP; ++c) ring[r][c] = 0ull;
+    }
+    // output frame to = t - 2: sum_i wt[i] x[to + i - 2], x[to + i - 2] in slot (r + i + 1) % 5
+    if (EDGE && step < 2) return;
+    f32x2 y[NP];
+    f32x2 ss2 = 0ull;
+#pragma unroll
+    for (int c = 0; c < NP; ++c) {
+      f32x2 v = mul2(wt[0][c], ring[(r + 1) % 5][c]);
+#pragma unroll
+      for (int i = 1; i < 5; ++i) v = fma2(wt[i][c], ring[(r + i + 1) % 5][c], v);
+      float y0, y1;
+      silu2(v, y0, y1);
+      y[c] = pack2(y0, y1);
+      ss2 = fma2(y[c], y[c], ss2);
+    }
+    if (which == 0) {
+      float s0, s1;
+      unpack2(ss2, s0, s1);
+      float ss = s0 + s1;
+#pragma unroll
+      for (int off = LPR / 2; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+      const float sc = rsqrtf(ss + a.l2_eps);
+      const f32x2 sc2 = pack2(sc, sc);
+#pragma unroll
+      for (int c = 0; c < NP; ++c) y[c] = mul2(y[c], sc2);
+    }
+    float o[EPL];
+#pragma unroll
+    for (int c = 0; c < NP; ++c) unpack2(y[c], o[2 * c], o[2 * c + 1]);
+    uint4 res;
+    if constexpr (sizeof(Tio) == 2) {
+      uint32_t* w = reinterpret_cast<uint32_t*>(&res);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 v2 = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+        w[i] = *reinterpret_cast<const uint32_t*>(&v2);
+      }
+    } else {
+      float* w = reinterpret_cast<float*>(&res);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) w[i] = o[i];
+    }
+    if (live) *reinterpret_cast<uint4*>(pdst) = res;
+    pdst += frame_elems;
+  };
+  using std::integral_constant;
 #pragma unroll 1
   for (int sb = 0; sb < nsteps; sb += 5) {
-#pragma unroll
-    for (int r = 0; r < 5; ++r) {              // ring slot r is static: sb is a multiple of five
-      const int step = sb + r;
-      if (step >= nsteps) break;
-      const int t = first + step;
-      if (t + PF - 1 <= last)
-        cp_async16(&stg[((step + PF - 1) % PF) * 256 + threadIdx.x], src + (size_t)(t + PF - 1) * frame_elems);
-      cp_async_commit();
-      cp_async_wait<PF - 1>();                 // frame t has landed
-      if (t <= last) {
-        const uint4 cur = stg[(step % PF) * 256 + threadIdx.x];
-        if constexpr (sizeof(Tio) == 2) {
-          const uint32_t* u = reinterpret_cast<const uint32_t*>(&cur);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            ring[r][2 * i] = __uint_as_float(u[i] << 16);
-            ring[r][2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
-          }
-        } else {
-          const float* u = reinterpret_cast<const float*>(&cur);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) ring[r][i] = u[i];
-        }
-      } else {
-#pragma unroll
-        for (int c = 0; c < EPL; ++c) ring[r][c] = 0.f;
-      }
-      const int to = t - 2;                    // output frame: sum_i wt[i] x[to + i - 2], x[to + i - 2] in slot (r + i + 1) % 5
-      if (to < first) continue;
-      float o[EPL];
-      float ss = 0.f;
-#pragma unroll
-      for (int c = 0; c < EPL; ++c) {
-        float v = wt[0][c] * ring[(r + 1) % 5][c];
-#pragma unroll
-        for (int i = 1; i < 5; ++i) v = fmaf(wt[i][c], ring[(r + i + 1) % 5][c], v);
-        o[c] = silu_f(v);
-        ss = fmaf(o[c], o[c], ss);
-      }
-      if (which == 0) {
-#pragma unroll
-        for (int off = LPR / 2; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-        const float sc = rsqrtf(ss + a.l2_eps);
-#pragma unroll
-        for (int c = 0; c < EPL; ++c) o[c] *= sc;
-      }
-      uint4 res;
-      if constexpr (sizeof(Tio) == 2) {
-        uint32_t* w = reinterpret_cast<uint32_t*>(&res);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const __nv_bfloat162 v2 = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
-          w[i] = *reinterpret_cast<const uint32_t*>(&v2);
-        }
-      } else {
-        float* w = reinterpret_cast<float*>(&res);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) w[i] = o[i];
-      }
-      if (live) *reinterpret_cast<uint4*>(dst + (size_t)to * frame_elems) = res;
+    // ring slot r = step % 5 is static: sb is a multiple of five
+    if (sb >= 5 && sb + 4 + PF - 1 <= s.Tn - 1) {
+      one_step(integral_constant<int, 0>{}, integral_constant<bool, false>{}, sb);
+      one_step(integral_constant<int, 1>{}, integral_constant<bool, false>{}, sb + 1);
+      one_step(integral_constant<int, 2>{}, integral_constant<bool, false>{}, sb + 2);
+      one_step(integral_constant<int, 3>{}, integral_constant<bool, false>{}, sb + 3);
+      one_step(integral_constant<int, 4>{}, integral_constant<bool, false>{}, sb + 4);
+    } else {
+      if (sb + 0 < nsteps) one_step(integral_constant<int, 0>{}, integral_constant<bool, true>{}, sb);
+      if (sb + 1 < nsteps) one_step(integral_constant<int, 1>{}, integral_constant<bool, true>{}, sb + 1);
+      if (sb + 2 < nsteps) one_step(integral_constant<int, 2>{}, integral_constant<bool, true>{}, sb + 2);
+      if (sb + 3 < nsteps) one_step(integral_constant<int, 3>{}, integral_constant<bool, true>{}, sb + 3);
+      if (sb + 4 < nsteps) one_step(integral_constant<int, 4>{}, integral_constant<bool, true>{}, sb + 4);
     }
   }
 }

@@ -473,7 +473,8 @@ vdn_status launch_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::prep_kv_temporal_kernel<Tio, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::PrepKvTemporal::SMEM_BYTES));
     const long long threads = (long long)s.F * s.H * (D * (int)sizeof(Tio) / 16);
-    vdn::prep_kv_temporal_kernel<Tio, D><<<dim3((unsigned)((threads + 255) / 256), (unsigned)(2 * s.B)), 256,
+    constexpr int NT = vdn::PrepKvTemporal::THREADS;
+    vdn::prep_kv_temporal_kernel<Tio, D><<<dim3((unsigned)((threads + NT - 1) / NT), (unsigned)(2 * s.B)), NT,
                                            vdn::PrepKvTemporal::SMEM_BYTES, st>>>(a, s);
     prof_mark(h, st, 0, "prep_kv_temporal");
   }
