@@ -166,6 +166,10 @@ typedef struct {
   const float* s0;
   const void* gate_elem;
   const float* norm_weight;
+  float q_l2_eps;           /* 0: q arrives L2-normalised.  > 0: q arrives as projected and the read-out uses
+                             * q / sqrt(sum_j q_j^2 + q_l2_eps), the q' of vdn_vda_prepare (Sec. 2.3), which may then
+                             * be called without queries: one pass over Q less */
+  uint32_t reserved;        /* 0 */
 } vdn_vda_options;
 vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
                                const float* gate, void* out, int B, int T, int F, int H, int d,
@@ -191,7 +195,8 @@ size_t vdn_vda_workspace_bytes_opt(vdn_vda_t h, int B, int T, int F, int H, int 
  * L2norm(x) = x / sqrt(sum_j x_j^2 + l2_eps) over the d channels of a (token, head).  All arithmetic in fp32.
  *
  *   q_in, k_in, v_in, q_out, k_out, v_out : [B,T,F,H,d] of cfg.io_dtype, DEVICE, 16-byte aligned.  k_out and v_out
- *        must not alias any input (the filters read neighbours); q_out may be q_in.
+ *        must not alias any input (the filters read neighbours); q_out may be q_in.  q_in and q_out may both be
+ *        NULL: the queries are then left alone (vdn_vda_options.q_l2_eps makes the read-out normalise them).
  *   p->Y, p->X   the spatial grid: F = Y * X, tokens of a frame in row-major (y, x) order
  *   p->wk_spatial, p->wv_spatial   float [H*d][5][5];   p->wk_temporal, p->wv_temporal   float [H*d][5]  (DEVICE)
  *        Both spatial filters may be NULL: the spatial part is then the identity (temporal filter, SiLU and

@@ -39,7 +39,8 @@ class VdnConfig(ctypes.Structure):
 class VdnOptions(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("chunk", ctypes.c_int32), ("radius", ctypes.c_int32),
                 ("anchors", ctypes.c_int32), ("alpha", ctypes.c_void_p), ("s0", ctypes.c_void_p),
-                ("gate_elem", ctypes.c_void_p), ("norm_weight", ctypes.c_void_p)]
+                ("gate_elem", ctypes.c_void_p), ("norm_weight", ctypes.c_void_p), ("q_l2_eps", ctypes.c_float),
+                ("reserved", ctypes.c_uint32)]
 
 
 class VdnPrepParams(ctypes.Structure):
@@ -201,12 +202,13 @@ class Vda:
 
     # -- the two entry points -----------------------------------------------------------------
     def forward(self, q, k, v, beta, gate, out=None, stream=None, alpha=None, s0=None,
-                chunk=1, radius=0, anchors=False, gate_elem=None, norm_weight=None):
+                chunk=1, radius=0, anchors=False, gate_elem=None, norm_weight=None, q_l2_eps=0.0):
         """vdn_vda_forward on device tensors q,k,v [B,T,F,H,d], beta [B,T,F,H], gate [H].
 
         With alpha [B,T,H,d] (decay gates) and/or s0 [B,H,d,d] (text state) the call goes to vdn_vda_forward_ex;
         with a chunk window (chunk, radius), boundary anchors, an element-wise gate gate_elem [B,T,F,H,d] (then
-        `gate` may be None) or a norm weight norm_weight [H,d] it goes to vdn_vda_forward_opt.
+        `gate` may be None), a norm weight norm_weight [H,d] or q_l2_eps > 0 (q arrives without its L2
+        normalisation; the read-out applies it) it goes to vdn_vda_forward_opt.
         """
         torch = self._torch
         B, T, F, H, d = q.shape
@@ -232,9 +234,9 @@ class Vda:
         p = lambda x: ctypes.c_void_p(x.data_ptr()) if x is not None else None
         a = lambda x: x.data_ptr() if x is not None else None
         if (chunk, radius, bool(anchors)) != (1, 0, False) or gate_elem is not None or norm_weight is not None \
-                or gate is None:
+                or gate is None or q_l2_eps:
             opt = VdnOptions(ctypes.sizeof(VdnOptions), chunk, radius, 1 if anchors else 0, a(alpha), a(s0),
-                             a(gate_elem), a(norm_weight))
+                             a(gate_elem), a(norm_weight), float(q_l2_eps), 0)
             st = self.lib.vdn_vda_forward_opt(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
                                               B, T, F, H, d, ctypes.byref(opt), self._stream(stream))
         elif alpha is not None or s0 is not None:
@@ -250,21 +252,23 @@ class Vda:
         """vdn_vda_prepare: projected q, k, v [B,T,F,H,d] -> prepared (q', k', v') (Sec. 2.3).
 
         filters = dict(wk_spatial [H*d,5,5], wk_temporal [H*d,5], wv_spatial, wv_temporal), float32 CUDA tensors.
-        `out` = optional (q_out, k_out, v_out); q_out may be q itself.
+        `out` = optional (q_out, k_out, v_out); q_out may be q itself.  q may be None: the queries are then left
+        to the read-out (forward(..., q_l2_eps=l2_eps)) and the first element of the result is None.
         """
         torch = self._torch
-        B, T, F, H, d = q.shape
+        B, T, F, H, d = k.shape
         names = ("wk_spatial", "wk_temporal", "wv_spatial", "wv_temporal")
         given = [n for n in names if filters.get(n) is not None]      # spatial filters may be left out (identity)
-        for x in (q, k, v, *(filters[n] for n in given)):
+        for x in (*([q] if q is not None else []), k, v, *(filters[n] for n in given)):
             if not (x.is_cuda and x.is_contiguous()):
                 raise ValueError("vdn_vda_prepare needs contiguous CUDA tensors")
         for n in given:
             want = (H * d, 5, 5) if n.endswith("spatial") else (H * d, 5)
             if tuple(filters[n].shape) != want or filters[n].dtype != torch.float32:
                 raise ValueError(f"{n} must be float32 {want}")
-        qo, ko, vo = out if out is not None else (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v))
-        p = lambda x: ctypes.c_void_p(x.data_ptr())
+        qo, ko, vo = out if out is not None else (torch.empty_like(q) if q is not None else None,
+                                                  torch.empty_like(k), torch.empty_like(v))
+        p = lambda x: ctypes.c_void_p(x.data_ptr()) if x is not None else None
         prm = VdnPrepParams(ctypes.sizeof(VdnPrepParams), Y, X, 1 if anchors else 0, l2_eps,
                             *(filters[n].data_ptr() if filters.get(n) is not None else None for n in names))
         self._check(self.lib.vdn_vda_prepare(self.h, p(q), p(k), p(v), p(qo), p(ko), p(vo), B, T, F, H, d,

@@ -20,7 +20,8 @@ __global__ void __launch_bounds__(256) readout_simt_kernel(const Tio* __restrict
                                                             const float* __restrict__ gate,
                                                             Tio* __restrict__ out, Shape s, float eps,
                                                             const Tio* __restrict__ gate_elem,
-                                                            const float* __restrict__ norm_weight) {
+                                                            const float* __restrict__ norm_weight,
+                                                            float q_l2_eps) {
   constexpr int TU = 64;
   constexpr int DC = D / 16;   // output channels per thread
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -71,6 +72,24 @@ __global__ void __launch_bounds__(256) readout_simt_kernel(const Tio* __restrict
     for (int r = 0; r < 4; ++r)
 #pragma unroll
       for (int c = 0; c < DC; ++c) acc[r][c] = fmaf(qa[r], zc[c], acc[r][c]);
+  }
+
+  // queries that arrive without their L2 normalisation (q_l2_eps > 0): o is linear in q, so scale the rows now
+  if (q_l2_eps > 0.f) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      float qs = 0.f;
+#pragma unroll
+      for (int i = 0; i < DC; ++i) {
+        const float x = sm.Q[tu * 4 + r][tc * DC + i];
+        qs = fmaf(x, x, qs);
+      }
+#pragma unroll
+      for (int off = 8; off >= 1; off >>= 1) qs += __shfl_xor_sync(0xffffffffu, qs, off);
+      const float rs = rsqrtf(qs + q_l2_eps);
+#pragma unroll
+      for (int c = 0; c < DC; ++c) acc[r][c] *= rs;
+    }
   }
 
   // Eq. 1c: per-head gate (null = 1), optional element-wise gate [B,T,F,H,d] and per-channel norm scale [H,d]

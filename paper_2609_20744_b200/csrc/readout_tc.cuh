@@ -12,6 +12,9 @@
 //   warps 2-5   epilogue: tcgen05.ld gives every thread one whole token row, so the sum of squares is
 //               thread-local; the scaled row is packed to bf16, written to a swizzled staging tile and
 //               sent out with a TMA store whose map has F as its own dimension (the tail is clipped)
+//   warps 6-9   (QNORM only) the queries' L2 normalisation, for callers that skip the preparation pass over Q:
+//               a thread sums the squares of one token's row of the Q tile in shared memory and leaves
+//               1 / sqrt(|q|^2 + eps_q) for the epilogue thread of that token, which scales its row before the norm
 // Every mbarrier wait is bounded.
 #pragma once
 #include <cuda_bf16.h>
@@ -21,7 +24,7 @@
 
 namespace vdn {
 
-template <bool EXTRAS>
+template <bool EXTRAS, bool QNORM = false>
 struct ReadoutTcCfg {
   static constexpr int D = 128;
   static constexpr int TILE = 128;
@@ -34,9 +37,11 @@ struct ReadoutTcCfg {
   static constexpr int OFF_Q = 2 * TILE_BYTES;
   static constexpr int OFF_OUT = OFF_Q + QSTAGES * TILE_BYTES;
   static constexpr int OFF_NW = OFF_OUT + NOUT * TILE_BYTES;   // norm weights of the current head, 128 floats
-  static constexpr int OFF_BAR = OFF_NW + 512;
+  static constexpr int OFF_QN = OFF_NW + (EXTRAS ? 512 : 0);   // QNORM: 1/|q| of the tokens of two tiles, 2 x 128 floats
+  static constexpr int OFF_BAR = OFF_QN + (QNORM ? 1024 : 0);
   static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
-  static constexpr int THREADS = 192;
+  static constexpr int THREADS = QNORM ? 320 : 192;
+  static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one SM");
 };
 using ReadoutTc = ReadoutTcCfg<false>;
 
@@ -44,15 +49,15 @@ using ReadoutTc = ReadoutTcCfg<false>;
 // gate_elem [B,T,F,H,d] bf16 (tensor map tmG; its tiles arrive by TMA in the very staging tile the output is then
 // written to, two tiles ahead) and a per-channel norm scale norm_weight [H,d] (kept in shared memory per frame);
 // either may be null, and so may the per-head gate (read as 1).  The plain instantiation carries none of that code.
-template <bool EXTRAS>
-__global__ void __launch_bounds__(ReadoutTcCfg<EXTRAS>::THREADS, 1)
+template <bool EXTRAS, bool QNORM = false>
+__global__ void __launch_bounds__(ReadoutTcCfg<EXTRAS, QNORM>::THREADS, 1)
 readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmS,
                   const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmG,
                   const float* __restrict__ gate, Shape s, float eps,
                   int* status, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight,
-                  Window win, int bridged) {
+                  Window win, int bridged, float q_l2_eps) {
   using namespace tc;
-  using R = ReadoutTcCfg<EXTRAS>;
+  using R = ReadoutTcCfg<EXTRAS, QNORM>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -65,8 +70,9 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   auto ACCFULL = [&](int i) { return bar0 + 8u * (10 + i); };    // 4
   auto ACCEMPTY = [&](int i) { return bar0 + 8u * (14 + i); };   // 4
   auto GFULL = [&](int i) { return bar0 + 8u * (18 + i); };      // 3 (EXTRAS: gate tile landed)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 8 * 21);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 8 * 21 + 8);
+  auto QNFULL = [&](int i) { return bar0 + 8u * (21 + i); };     // 2 (QNORM: 1/|q| of a tile written)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 8 * 23);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 8 * 23 + 8);
   const WaitCtx wc{abort_flag, status};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -74,10 +80,12 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const long long nitems = s.work_items();
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 3; ++i) { mbar_init(QFULL(i), 1); mbar_init(QEMPTY(i), 1); }
+    // a Q stage is handed back by the MMA commit and, with QNORM, by the four warps that read its rows
+    for (int i = 0; i < 3; ++i) { mbar_init(QFULL(i), 1); mbar_init(QEMPTY(i), QNORM ? 5 : 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(STFULL(i), 1); mbar_init(STEMPTY(i), 1); }
     for (int i = 0; i < 4; ++i) { mbar_init(ACCFULL(i), 1); mbar_init(ACCEMPTY(i), 4); }   // one arrival per epilogue warp
     for (int i = 0; i < 3; ++i) mbar_init(GFULL(i), 1);
+    for (int i = 0; i < 2; ++i) mbar_init(QNFULL(i), 4);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
@@ -161,6 +169,57 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (ok) mma_commit(STEMPTY(0));
       }
     }
+  } else if (QNORM && warp >= 6) {
+    // ------------------------------------------------------------------ query norms
+    const int qrow = threadIdx.x - 192;         // token row inside the tile
+    float* qn = reinterpret_cast<float*>(base_ptr + R::OFF_QN);
+    uint32_t qi = 0;
+    bool ok = true;
+    for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
+      for (int tile = 0; tile < ntiles; ++tile, ++qi) {
+        const int st = qi % R::QSTAGES;
+        // Slot qi & 1 was last read for tile qi - 2, whose epilogue threads arrived on that tile's ACCEMPTY after
+        // the read (tile qi + 2 cannot have completed that barrier again: it needs this slot first).  One lane
+        // polls, so that the other 31 take no issue slots from the epilogue warp on the same scheduler; then every
+        // lane observes the completed phases itself.
+        if (lane == 0)
+          ok = mbar_wait(QFULL(st), (qi / R::QSTAGES) & 1, wc) &&
+               (qi < 2 || mbar_wait(ACCEMPTY((qi - 2) & 3), ((qi - 2) >> 2) & 1, wc));
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (!mbar_wait(QFULL(st), (qi / R::QSTAGES) & 1, wc)) { ok = false; break; }
+        if (qi >= 2 && !mbar_wait(ACCEMPTY((qi - 2) & 3), ((qi - 2) >> 2) & 1, wc)) { ok = false; break; }
+        const unsigned char* qrowp = base_ptr + R::OFF_Q + st * R::TILE_BYTES + qrow * 128;
+        // packed fp32 pairs: these warps share their schedulers with the epilogue warps, whose per-tile chain sets
+        // the pace of the kernel, so every instruction here counts
+        unsigned long long acc2[2] = {0ull, 0ull};
+#pragma unroll
+        for (int bx = 0; bx < 2; ++bx)
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            // the order of the channels does not matter here; walking the chunks in swizzled order keeps the
+            // eight rows of a quarter-warp on different banks
+            const uint4 x = *reinterpret_cast<const uint4*>(qrowp + bx * R::BOX_BYTES + ((c ^ (qrow & 7)) * 16));
+            const uint32_t* u = reinterpret_cast<const uint32_t*>(&x);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              unsigned long long pr;
+              asm("mov.b64 %0, {%1, %2};" : "=l"(pr) : "r"(u[e] << 16), "r"(u[e] & 0xFFFF0000u));
+              asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(acc2[e & 1]) : "l"(pr));
+            }
+          }
+        float ss;
+        {
+          float a0, a1, b0, b1;
+          asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(acc2[0]));
+          asm("mov.b64 {%0, %1}, %2;" : "=f"(b0), "=f"(b1) : "l"(acc2[1]));
+          ss = (a0 + a1) + (b0 + b1);
+        }
+        qn[(qi & 1) * 128 + qrow] = rsqrtf(ss + q_l2_eps);
+        mbar_arrive_warp(QEMPTY(st));
+        mbar_arrive_warp(QNFULL(qi & 1));
+      }
+    }
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int qd = warp & 3;
@@ -201,6 +260,11 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const int a = qi & 3;
         if (!mbar_wait(ACCFULL(a), (qi >> 2) & 1, wc)) { ok = false; break; }
         tc_fence_after_sync();
+        float qrs = 1.0f;
+        if constexpr (QNORM) {
+          if (!mbar_wait(QNFULL(qi & 1), (qi >> 1) & 1, wc)) { ok = false; break; }
+          qrs = reinterpret_cast<const float*>(base_ptr + R::OFF_QN)[(qi & 1) * 128 + row];
+        }
         const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 128;
         float v[4][32];
         tmem_ld32(taddr + 0, v[0]);
@@ -216,7 +280,8 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int c = 0; c < 4; ++c)
 #pragma unroll
           for (int e = 0; e < 32; ++e) ss = fmaf(v[c][e], v[c][e], ss);
-        const float scale = g * rsqrtf(ss * (1.0f / R::D) + eps);
+        // with o = qrs * v (the read-out of the normalised query): mean o^2 = qrs^2 mean v^2
+        const float scale = g * qrs * rsqrtf(ss * (qrs * qrs) * (1.0f / R::D) + eps);
 
         const int ob = qi % R::NOUT;
         if (use_ge) {

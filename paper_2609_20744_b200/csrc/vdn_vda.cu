@@ -51,6 +51,7 @@ struct Extras {
   const float* s0 = nullptr;
   const void* gate_elem = nullptr;
   const float* norm_weight = nullptr;
+  float q_l2_eps = 0.f;    // > 0: the read-out normalises the queries itself
   vdn::Window win{1, 0, 0, -1};
   bool anchors = false;
   bool composed = false;   // run the scan chunk-wise (tensor-core path, chunk >= 2)
@@ -267,7 +268,7 @@ vdn_status forward_simt(vdn_vda_t h, const void* q, const void* k, const void* v
     if (x.phase == 2) { sr.t0 = x.ro_first; sr.Tn = x.ro_count; }
     vdn::readout_simt_kernel<Tio, D><<<dim3((unsigned)n, (s.F + 63) / 64), 256, sizeof(vdn::ReadoutSimtSmem<D>), st>>>(
         static_cast<const Tio*>(q), read, gate, static_cast<Tio*>(out), sr, h->cfg.rms_eps,
-        static_cast<const Tio*>(x.gate_elem), x.norm_weight);
+        static_cast<const Tio*>(x.gate_elem), x.norm_weight, x.q_l2_eps);
     prof_mark(h, st, 3, "readout_simt");
     h->launches += 1;
   }
@@ -320,6 +321,10 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
                                      vdn::ReadoutTc::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ReadoutTcCfg<true>::SMEM_BYTES));
+    VDN_CUDA(h, (cudaFuncSetAttribute(vdn::readout_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      vdn::ReadoutTcCfg<false, true>::SMEM_BYTES)));
+    VDN_CUDA(h, (cudaFuncSetAttribute(vdn::readout_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      vdn::ReadoutTcCfg<true, true>::SMEM_BYTES)));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
     VDN_CUDA(h, (cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -405,16 +410,22 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   const long long nread = sr.work_items();
   const long long ro_target = ((long long)h->sm_count * 27 + 16) / 32;
   const unsigned persistent_ro = (unsigned)(nread < ro_target ? nread : ro_target);
-  if (x.gate_elem || x.norm_weight || !gate) {
-    CUtensorMap tmG = tmO;                                      // the gate tensor has the layout of the output
-    if (x.gate_elem && (r = make_token_map(h, &tmG, x.gate_elem, s)) != VDN_OK) return r;
-    using RX = vdn::ReadoutTcCfg<true>;
-    vdn::readout_tc_kernel<true><<<persistent_ro, RX::THREADS, RX::SMEM_BYTES, st>>>(
+  const bool extras = x.gate_elem || x.norm_weight || !gate;
+  CUtensorMap tmG = tmO;                                        // the gate tensor has the layout of the output
+  if (x.gate_elem && (r = make_token_map(h, &tmG, x.gate_elem, s)) != VDN_OK) return r;
+  auto launch_readout = [&](auto ex, auto qn) {
+    constexpr bool EX = decltype(ex)::value, QN = decltype(qn)::value;
+    using RX = vdn::ReadoutTcCfg<EX, QN>;
+    vdn::readout_tc_kernel<EX, QN><<<persistent_ro, RX::THREADS, RX::SMEM_BYTES, st>>>(
         tmQ, tmS, tmO, tmG, gate, sr, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
-        x.norm_weight, x.win, x.alpha != nullptr);
+        x.norm_weight, x.win, x.alpha != nullptr, x.q_l2_eps);
+  };
+  using std::true_type;
+  using std::false_type;
+  if (x.q_l2_eps > 0.f) {
+    if (extras) launch_readout(true_type{}, true_type{}); else launch_readout(false_type{}, true_type{});
   } else {
-    vdn::readout_tc_kernel<false><<<persistent_ro, vdn::ReadoutTc::THREADS, vdn::ReadoutTc::SMEM_BYTES, st>>>(
-        tmQ, tmS, tmO, tmO, gate, sr, h->cfg.rms_eps, h->status_dev, nullptr, nullptr, x.win, x.alpha != nullptr);
+    if (extras) launch_readout(true_type{}, false_type{}); else launch_readout(false_type{}, false_type{});
   }
   prof_mark(h, st, nk++, "readout_tc");
   h->launches = nk;
@@ -478,6 +489,8 @@ vdn_status launch_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const
                                            vdn::PrepKvTemporal::SMEM_BYTES, st>>>(a, s);
     prof_mark(h, st, 0, "prep_kv_temporal");
   }
+  h->launches = 1;
+  if (!q_in) { VDN_CUDA(h, cudaGetLastError()); return VDN_OK; }   // the queries are normalised by the read-out
   const long long rows = (long long)s.B * s.Tn * s.F * s.H;
   const long long per_cta = 8LL * (32 / (D * (int)sizeof(Tio) / 16)) * 4;       // rows one CTA covers per trip
   const long long want = (rows + per_cta - 1) / per_cta;
@@ -591,6 +604,9 @@ vdn_status forward_core(vdn_vda_t h, const void* q, const void* k, const void* v
     x.s0 = opt->s0;
     x.gate_elem = opt->gate_elem;
     x.norm_weight = opt->norm_weight;
+    if (!(opt->q_l2_eps >= 0.f) || opt->q_l2_eps > 1e30f)
+      return fail(h, VDN_ERR_INVALID_ARG, "q_l2_eps must be a finite non-negative number");
+    x.q_l2_eps = opt->q_l2_eps;
     x.win.chunk = opt->chunk > 0 ? opt->chunk : 1;
     x.win.radius = opt->radius;
     x.anchors = opt->anchors != 0;
@@ -680,7 +696,7 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
   if (!h) return VDN_ERR_INVALID_ARG;
   if (!p || p->struct_size != sizeof(vdn_vda_prep_params))
     return fail(h, VDN_ERR_INVALID_ARG, "vdn_vda_prep_params missing or of the wrong struct_size");
-  if (!q_in || !k_in || !v_in || !q_out || !k_out || !v_out || !p->wk_temporal || !p->wv_temporal)
+  if (!k_in || !v_in || !k_out || !v_out || !p->wk_temporal || !p->wv_temporal || (q_in == nullptr) != (q_out == nullptr))
     return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
   if ((p->wk_spatial == nullptr) != (p->wv_spatial == nullptr))
     return fail(h, VDN_ERR_INVALID_ARG, "pass both spatial filters or neither");
@@ -689,7 +705,7 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
       !aligned16(p->wv_temporal))
     return fail(h, VDN_ERR_INVALID_ARG, "tensors and filters must be 16-byte aligned");
   if (k_out == k_in || k_out == v_in || v_out == k_in || v_out == v_in || k_out == v_out || k_out == q_in ||
-      v_out == q_in || q_out == k_in || q_out == v_in || q_out == k_out || q_out == v_out)
+      v_out == q_in || (q_out && (q_out == k_in || q_out == v_in || q_out == k_out || q_out == v_out)))
     return fail(h, VDN_ERR_INVALID_ARG, "k_out and v_out must not alias anything (only q_out may equal q_in)");
   std::string why;
   if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
@@ -710,7 +726,7 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
     const size_t frame_bytes = (size_t)F * H * d * elem_size(h);
     void* outs[3] = {q_out, k_out, v_out};
     for (void* o : outs)
-      for (int b = 0; b < B; ++b) {
+      for (int b = 0; o && b < B; ++b) {
         VDN_CUDA(h, cudaMemsetAsync(static_cast<char*>(o) + (size_t)b * T * frame_bytes, 0, frame_bytes, st));
         if (T > 1)
           VDN_CUDA(h, cudaMemsetAsync(static_cast<char*>(o) + ((size_t)b * T + T - 1) * frame_bytes, 0, frame_bytes, st));

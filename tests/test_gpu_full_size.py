@@ -112,6 +112,39 @@ def test_768p_release_window_full_size():
     torch.cuda.empty_cache()
 
 
+def test_768p_queries_normalised_by_the_readout_full_size():
+    # projected queries (token norms spread over two decades) with vdn_vda_options.q_l2_eps: the read-out applies
+    # the preparation's L2 normalisation itself; checker = that normalisation in fp64 in front of the layer
+    from oracle import prep_oracle as po
+    w = inputs.CLIP_768P
+    x = inputs.generate(w, "cuda")
+    g = torch.Generator(device="cuda")
+    g.manual_seed(991)
+    scale = torch.exp(torch.empty((w.B, w.T, w.F, w.H, 1), device="cuda").uniform_(-2.3, 2.3, generator=g))
+    q_raw = (x["q"].float() * scale).to(x["q"].dtype)
+    del scale
+    vda = binding.Vda(w.d, w.dtype)
+    out = vda.forward(q_raw, x["k"], x["v"], x["beta"], x["gate"], q_l2_eps=1e-6)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    assert vda.uses_tensor_cores()
+    for (b, h) in sampled_pairs(w, 2):
+        q, k, v, beta, gate = inputs.head_slice(x, b, h)
+        qn = po.l2_normalise(q_raw[b, :, :, h, :].double().cpu().numpy(), 1e-6)
+        ref = orc.vda_slice(qn, k, v, beta, gate, 1e-6)["out"]
+        e = orc.slice_error(out[b, :, :, h, :].double().cpu().numpy(), ref)
+        assert e <= TOL_BF16, f"slice (b={b}, h={h}): error {e:.3e}"
+        del q, k, v, qn, ref
+    for t0 in range(0, w.T, 16):
+        blk = out[:, t0:t0 + 16].float()
+        assert torch.isfinite(blk).all()
+        ms = blk.pow(2).mean(dim=-1)
+        assert torch.allclose(ms, x["gate"].pow(2)[None, None, None, :].expand_as(ms), rtol=2e-2)
+    del x, out, q_raw, vda
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
 @pytest.mark.parametrize("spatial", [True, False])
 def test_768p_preparation_full_size(spatial):
     # vdn_vda_prepare on the 768p shape (48 x 85 tokens per frame): sampled output frames of sampled heads against

@@ -118,6 +118,54 @@ def test_prepared_features_feed_the_layer():
     check(w, p, (q, k, v), Y, X, anchors=True)
 
 
+@pytest.mark.parametrize("dtype,d,F,extras", [
+    ("bf16", 128, 300, False),     # tensor-core read-out, three tiles with a ragged tail
+    ("bf16", 128, 130, True),      # ... with the element-wise gate and the norm weight on top
+    ("bf16", 64, 70, False),       # plain-fp32 kernels
+    ("f32", 128, 45, True),
+])
+def test_readout_normalises_the_queries(dtype, d, F, extras):
+    # q arrives as projected (norms far from one); with q_l2_eps the read-out applies q / sqrt(|q|^2 + eps) itself.
+    # Checker: the preparation's L2 normalisation in fp64, unrounded, in front of the layer.  A large RMSNorm eps
+    # makes the scale of q matter (with a tiny eps the norm would hide a wrong or missing factor).
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=2, H=2, T=5, F=F, seed=77)
+    x = inputs.generate(w, "cuda")
+    p = inputs.generate_projected(w, "cuda")
+    scale = torch.linspace(0.05, 20.0, w.T * w.F, device="cuda").view(1, w.T, w.F, 1, 1)
+    q_raw = (p["q"].float() * scale).to(p["q"].dtype)
+    rms_eps = 1e-2
+    vda = binding.Vda(w.d, w.dtype, rms_eps=rms_eps)
+    kw = {}
+    if extras:
+        ge, nw = inputs.generate_output_extras(w, "cuda")
+        kw = dict(gate_elem=ge, norm_weight=nw)
+    out = vda.forward(q_raw, x["k"], x["v"], x["beta"], x["gate"], chunk=2, radius=1, q_l2_eps=1e-6, **kw)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    for b in range(w.B):
+        for h in range(w.H):
+            qn = po.l2_normalise(f64(q_raw[b, :, :, h]), 1e-6)
+            gate = float(x["gate"][h]) * (f64(kw["gate_elem"][b, :, :, h]) if extras else 1.0)
+            ref = orc.vda_slice(qn, f64(x["k"][b, :, :, h]), f64(x["v"][b, :, :, h]), f64(x["beta"][b, :, :, h]),
+                                gate, rms_eps, chunk=2, radius=1,
+                                norm_weight=f64(kw["norm_weight"][h]) if extras else None)["out"]
+            assert orc.slice_error(f64(out[b, :, :, h]), ref) <= TOL[dtype]
+    # and it is not a no-op: without the option the same inputs give a different answer
+    out2 = vda.forward(q_raw, x["k"], x["v"], x["beta"], x["gate"], chunk=2, radius=1, **kw)
+    torch.cuda.synchronize()
+    assert (out2.float() - out.float()).abs().max() > 1e-2 * out.float().abs().max()
+
+
+def test_prepare_without_queries():
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=1, H=2, T=4, F=6 * 7, seed=5)
+    p = inputs.generate_projected(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    q1, k1, v1 = vda.prepare(p["q"], p["k"], p["v"], p, 6, 7)
+    q2, k2, v2 = vda.prepare(None, p["k"], p["v"], p, 6, 7)
+    torch.cuda.synchronize()
+    assert q2 is None and torch.equal(k1, k2) and torch.equal(v1, v2)
+
+
 def test_prepare_argument_errors():
     import ctypes
     w = inputs.TINY.scaled(F=4 * 5)
