@@ -88,7 +88,9 @@ struct PrepKv {
   static constexpr int THREADS = 256;
   __host__ __device__ static constexpr int rows(int D) { return THREADS / (D / 2); }            // tile rows
   __host__ __device__ static constexpr int tile_tokens(int D) { return (rows(D) + 2 * HALO) * (TX + 2 * HALO); }
-  static constexpr size_t smem_bytes(int D, int es) { return (size_t)2 * tile_tokens(D) * D * es + 64 * sizeof(float); }
+  // two tiles (the asynchronous copies' double buffer) and the exchange area of the norm
+  static constexpr size_t RED_BYTES = 1024;
+  static constexpr size_t smem_bytes(int D, int es) { return (size_t)2 * tile_tokens(D) * D * es + RED_BYTES; }
 };
 
 struct PrepArgs {
@@ -107,9 +109,11 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
   constexpr int TX = P::TX, HALO = P::HALO;
   constexpr int SW = TX + 2 * HALO, SH = ROWS + 2 * HALO;       // tile with halo
   constexpr int GT = D / 2;                                      // threads per tile row (one head's channel pairs)
+  constexpr int NW = GT / 32;                                    // warps per tile row
+  static_assert(TX == 8, "the norm's reduction is written for eight tokens per thread");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Tio* tile = reinterpret_cast<Tio*>(smem_raw);                  // [2][SH][SW][D]
-  float* red = reinterpret_cast<float*>(smem_raw + (size_t)2 * SH * SW * D * sizeof(Tio));   // [ROWS][TX] exchange
+  float* red = reinterpret_cast<float*>(smem_raw + (size_t)2 * SH * SW * D * sizeof(Tio));     // [2][ROWS][NW][TX]
 
   const int h = blockIdx.x;
   const int tiles_x = (a.X + TX - 1) / TX;
@@ -119,7 +123,7 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
   const Tio* __restrict__ src = static_cast<const Tio*>(which == 0 ? a.in[0] : a.in[1]);
   Tio* __restrict__ dst = static_cast<Tio*>(which == 0 ? a.out[0] : a.out[1]);
 
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int g = tid / GT;                   // tile row of this thread
   const int cp = tid % GT;                  // channel pair within the head
   const int ch = h * D + 2 * cp;            // first of this thread's two channels, [H*d] index
@@ -138,10 +142,12 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
   }
 
   const int first = s.t0, last = s.t0 + s.Tn - 1;
-  // this thread's first output element of frame 0: token (y0 + g, x0), its channel pair
-  Tio* dst_b = dst + token_offset(s, b, 0, min(y0 + g, a.Y - 1) * a.X + x0, h) + 2 * cp;
+  const size_t frame_elems = (size_t)s.F * s.H * D;
+  // this thread's first output element: token (y0 + g, x0) of the first scanned frame, its channel pair
+  Tio* pdst = dst + token_offset(s, b, first, min(y0 + g, a.Y - 1) * a.X + x0, h) + 2 * cp;
+  const bool row_ok = y0 + g < a.Y;
 
-  // Frame t's tile (with halo) -> buffer t & 1; tokens outside the frame are zeros.  A thread copies the same
+  // Frame t's tile (with halo) -> raw buffer t & 1; tokens outside the frame are zeros.  A thread copies the same
   // 16-byte pieces of every frame, so their offsets inside a frame are worked out once (-1: outside the frame).
   constexpr int CHUNKS = D * (int)sizeof(Tio) / 16;              // 16-byte pieces per token
   constexpr int NPIECE = (SH * SW * CHUNKS + P::THREADS - 1) / P::THREADS;
@@ -154,7 +160,7 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
     const bool in = e < SH * SW * CHUNKS && yy >= 0 && yy < a.Y && xx >= 0 && xx < a.X;
     goff[i] = in ? (int)((((size_t)(yy * a.X + xx) * s.H + h) * D) * sizeof(Tio)) + c * 16 : -1;
   }
-  const size_t frame_bytes = (size_t)s.F * s.H * D * sizeof(Tio);
+  const size_t frame_bytes = frame_elems * sizeof(Tio);
   const unsigned char* src_b = reinterpret_cast<const unsigned char*>(src) + (size_t)b * s.T * frame_bytes;
   auto stage = [&](int t) {
     unsigned char* buf = reinterpret_cast<unsigned char*>(tile) + (size_t)(t & 1) * SH * SW * D * sizeof(Tio);
@@ -176,90 +182,121 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
 #pragma unroll
     for (int j = 0; j < TX; ++j) ring[i][j] = 0ull;
 
+  int par = 0;                              // which half of the norm's exchange area this step uses
+
+  // One step: spatial filter of frame t = first + step into ring slot r, then the temporal filter, SiLU, norm and
+  // store of frame t - 2.  EDGE = false is the steady state, where all the frames involved exist.
+  auto one_step = [&](auto rc, auto ec, int step) {
+    constexpr int r = decltype(rc)::value;
+    constexpr bool EDGE = decltype(ec)::value;
+    const int t = first + step;             // input frame of this step; the output frame is t - 2
+    if (!EDGE || t <= last) {
+      if (!EDGE || t + 1 <= last) { stage(t + 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+      __syncthreads();                      // frame t's tile is complete
+      // (Widening a 16-bit tile to fp32 once per frame, so that the loop below reads ready pairs, was slower:
+      // 12.8 ms instead of 10.4 ms on the 768p clip; the shared-memory port is the scarcer resource here.)
+      const Tio* base = tile + (size_t)(t & 1) * SH * SW * D + (size_t)g * SW * D + 2 * cp;
+      // ---- spatial filter of frame t for this thread's row: slide over the SW input columns
+      f32x2 (&acc)[TX] = ring[r];           // the spatial result accumulates straight into this step's ring slot
+#pragma unroll
+      for (int j = 0; j < TX; ++j) acc[j] = 0ull;
+#pragma unroll
+      for (int xi = 0; xi < SW; ++xi) {     // input column xi sits at x0 - 2 + xi
+        f32x2 in[5];
+#pragma unroll
+        for (int i = 0; i < 5; ++i) in[i] = load_pair(base + ((size_t)i * SW + xi) * D);
+#pragma unroll
+        for (int i = 0; i < 5; ++i) {       // neighbouring instructions update different accumulators
+#pragma unroll
+          for (int j = 0; j < 5; ++j) {     // tap column j: output column xo = xi - j
+            const int xo = xi - j;
+            if (xo < 0 || xo >= TX) continue;
+            acc[xo] = fma2(wsp[i][j], in[i], acc[xo]);
+          }
+        }
+      }
+      __syncthreads();                      // the buffer is overwritten by the copy issued at the start of the next step
+    } else {
+#pragma unroll
+      for (int j = 0; j < TX; ++j) ring[r][j] = 0ull;
+    }
+    // ---- temporal filter: output frame to = t - 2 = sum_i wt[i] S[to + i - 2]; S[to + i - 2] sits in slot (r + i + 1) % 5
+    if (EDGE && step < HALO) return;
+    float o0[TX], o1[TX];
+#pragma unroll
+    for (int j = 0; j < TX; ++j) {
+      f32x2 o = mul2(wtp[0], ring[(r + 1) % 5][j]);
+#pragma unroll
+      for (int i = 1; i < 5; ++i) o = fma2(wtp[i], ring[(r + i + 1) % 5][j], o);
+      silu2(o, o0[j], o1[j]);
+    }
+    if (which == 0) {
+      // ---- L2 normalisation over the head's d channels (Sec. 2.3).  Eight sums over the row's lanes at once:
+      // each exchange halves the number of tokens a lane still carries, so a warp needs 9 shuffles instead of 40;
+      // the totals go through shared memory to every thread of the row.
+      float v4[4], v2[2], v1;
+      const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float lo = fmaf(o0[j], o0[j], o1[j] * o1[j]), hi = fmaf(o0[j + 4], o0[j + 4], o1[j + 4] * o1[j + 4]);
+        v4[j] = (b16 ? hi : lo) + __shfl_xor_sync(0xffffffffu, b16 ? lo : hi, 16);
+      }
+#pragma unroll
+      for (int j = 0; j < 2; ++j) v2[j] = (b8 ? v4[j + 2] : v4[j]) + __shfl_xor_sync(0xffffffffu, b8 ? v4[j] : v4[j + 2], 8);
+      v1 = (b4 ? v2[1] : v2[0]) + __shfl_xor_sync(0xffffffffu, b4 ? v2[0] : v2[1], 4);
+      v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
+      v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+      // this lane now holds the warp's sum for token 4 [lane & 16] + 2 [lane & 8] + [lane & 4]
+      float* mine = red + ((par * ROWS + g) * NW) * TX;
+      if ((lane & 3) == 0) mine[((tid >> 5) % NW) * TX + (b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)] = v1;
+      if constexpr (NW == 1) __syncwarp();
+      else asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(GT) : "memory");
+      float ss[TX];
+      {
+        const float4 x0 = *reinterpret_cast<const float4*>(mine), x1 = *reinterpret_cast<const float4*>(mine + 4);
+        ss[0] = x0.x; ss[1] = x0.y; ss[2] = x0.z; ss[3] = x0.w; ss[4] = x1.x; ss[5] = x1.y; ss[6] = x1.z; ss[7] = x1.w;
+      }
+#pragma unroll
+      for (int w = 1; w < NW; ++w) {
+        const float4 x0 = *reinterpret_cast<const float4*>(mine + w * TX), x1 = *reinterpret_cast<const float4*>(mine + w * TX + 4);
+        ss[0] += x0.x; ss[1] += x0.y; ss[2] += x0.z; ss[3] += x0.w; ss[4] += x1.x; ss[5] += x1.y; ss[6] += x1.z; ss[7] += x1.w;
+      }
+      par ^= 1;                             // the next step writes the other half: no second barrier (the block-wide
+                                            // barriers of the steps in between order the reuse)
+#pragma unroll
+      for (int j = 0; j < TX; ++j) {
+        float sc;
+        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(sc) : "f"(ss[j] + a.l2_eps));
+        o0[j] *= sc;
+        o1[j] *= sc;
+      }
+    }
+    if (row_ok) {
+#pragma unroll
+      for (int j = 0; j < TX; ++j)
+        if (x0 + j < a.X) store_pair(pdst + (size_t)j * (s.H * D), o0[j], o1[j]);
+    }
+    pdst += frame_elems;
+  };
+
+  using std::integral_constant;
   const int nsteps = s.Tn + HALO;           // two extra steps flush the last two output frames
   stage(first);
 #pragma unroll 1
   for (int sb = 0; sb < nsteps; sb += 5) {
-#pragma unroll
-    for (int r = 0; r < 5; ++r) {           // ring slot r is static: sb is a multiple of five
-      const int step = sb + r;
-      if (step >= nsteps) break;
-      const int t = first + step;           // input frame of this step; the output frame is t - 2
-      if (t <= last) {
-        if (t + 1 <= last) { stage(t + 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
-        __syncthreads();
-        // ---- spatial filter of frame t for this thread's row: slide over the SW input columns
-        const Tio* base = tile + (size_t)(t & 1) * SH * SW * D + (size_t)g * SW * D + 2 * cp;
-        f32x2 (&acc)[TX] = ring[r];         // the spatial result accumulates straight into this step's ring slot
-#pragma unroll
-        for (int j = 0; j < TX; ++j) acc[j] = 0ull;
-#pragma unroll
-        for (int xi = 0; xi < SW; ++xi) {   // input column xi sits at x0 - 2 + xi
-          f32x2 in[5];
-#pragma unroll
-          for (int i = 0; i < 5; ++i) in[i] = load_pair(base + ((size_t)i * SW + xi) * D);
-#pragma unroll
-          for (int i = 0; i < 5; ++i) {     // neighbouring instructions update different accumulators
-#pragma unroll
-            for (int j = 0; j < 5; ++j) {   // tap column j: output column xo = xi - j
-              const int xo = xi - j;
-              if (xo < 0 || xo >= TX) continue;
-              acc[xo] = fma2(wsp[i][j], in[i], acc[xo]);
-            }
-          }
-        }
-        __syncthreads();                    // the buffer may be overwritten by the copy issued two steps on
-      } else {
-#pragma unroll
-        for (int j = 0; j < TX; ++j) ring[r][j] = 0ull;
-      }
-      // ---- temporal filter: output frame to = t - 2 = sum_i wt[i] S[to + i - 2]; S[to + i - 2] sits in slot (r + i + 1) % 5
-      const int to = t - HALO;
-      if (to < first) continue;
-      float o0[TX], o1[TX];
-#pragma unroll
-      for (int j = 0; j < TX; ++j) {
-        f32x2 o = mul2(wtp[0], ring[(r + 1) % 5][j]);
-#pragma unroll
-        for (int i = 1; i < 5; ++i) o = fma2(wtp[i], ring[(r + i + 1) % 5][j], o);
-        silu2(o, o0[j], o1[j]);
-      }
-      const int y = y0 + g;
-      if (which == 0) {
-        // ---- L2 normalisation over the head's d channels (Sec. 2.3)
-        float ss[TX];
-#pragma unroll
-        for (int j = 0; j < TX; ++j) {
-          ss[j] = fmaf(o0[j], o0[j], o1[j] * o1[j]);
-#pragma unroll
-          for (int off = 16; off >= 1; off >>= 1) ss[j] += __shfl_xor_sync(0xffffffffu, ss[j], off);
-        }
-        if constexpr (GT == 64) {           // the head spans two warps: exchange the partial sums
-          const int wv = (tid >> 5) & 1;
-          float* mine = red + (g * 2 + wv) * TX;
-          if ((tid & 31) == 0) {
-#pragma unroll
-            for (int j = 0; j < TX; ++j) mine[j] = ss[j];
-          }
-          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(GT) : "memory");
-          const float* other = red + (g * 2 + (wv ^ 1)) * TX;
-#pragma unroll
-          for (int j = 0; j < TX; ++j) ss[j] += other[j];
-          asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(GT) : "memory");
-        }
-#pragma unroll
-        for (int j = 0; j < TX; ++j) {
-          const float sc = rsqrtf(ss[j] + a.l2_eps);
-          o0[j] *= sc;
-          o1[j] *= sc;
-        }
-      }
-      if (y < a.Y) {
-        Tio* orow = dst_b + (size_t)to * ((size_t)s.F * s.H * D);
-#pragma unroll
-        for (int j = 0; j < TX; ++j)
-          if (x0 + j < a.X) store_pair(orow + (size_t)j * (s.H * D), o0[j], o1[j]);
-      }
+    // ring slot r = step % 5 is static: sb is a multiple of five
+    if (sb >= 5 && sb + 4 + 1 <= s.Tn - 1) {
+      one_step(integral_constant<int, 0>{}, integral_constant<bool, false>{}, sb);
+      one_step(integral_constant<int, 1>{}, integral_constant<bool, false>{}, sb + 1);
+      one_step(integral_constant<int, 2>{}, integral_constant<bool, false>{}, sb + 2);
+      one_step(integral_constant<int, 3>{}, integral_constant<bool, false>{}, sb + 3);
+      one_step(integral_constant<int, 4>{}, integral_constant<bool, false>{}, sb + 4);
+    } else {
+      if (sb + 0 < nsteps) one_step(integral_constant<int, 0>{}, integral_constant<bool, true>{}, sb);
+      if (sb + 1 < nsteps) one_step(integral_constant<int, 1>{}, integral_constant<bool, true>{}, sb + 1);
+      if (sb + 2 < nsteps) one_step(integral_constant<int, 2>{}, integral_constant<bool, true>{}, sb + 2);
+      if (sb + 3 < nsteps) one_step(integral_constant<int, 3>{}, integral_constant<bool, true>{}, sb + 3);
+      if (sb + 4 < nsteps) one_step(integral_constant<int, 4>{}, integral_constant<bool, true>{}, sb + 4);
     }
   }
 }
