@@ -178,17 +178,12 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x) {
       for (int tile = 0; tile < ntiles; ++tile, ++qi) {
         const int st = qi % R::QSTAGES;
-        // Slot qi & 1 was last read for tile qi - 2, whose epilogue threads arrived on that tile's ACCEMPTY after
-        // the read (tile qi + 2 cannot have completed that barrier again: it needs this slot first).  One lane
-        // polls, so that the other 31 take no issue slots from the epilogue warp on the same scheduler; then every
-        // lane observes the completed phases itself.
-        if (lane == 0)
-          ok = mbar_wait(QFULL(st), (qi / R::QSTAGES) & 1, wc) &&
-               (qi < 2 || mbar_wait(ACCEMPTY((qi - 2) & 3), ((qi - 2) >> 2) & 1, wc));
+        // One lane polls, so that the other 31 take no issue slots from the epilogue warp on the same scheduler;
+        // then every lane observes the completed phase itself.
+        if (lane == 0) ok = mbar_wait(QFULL(st), (qi / R::QSTAGES) & 1, wc);
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
         if (!mbar_wait(QFULL(st), (qi / R::QSTAGES) & 1, wc)) { ok = false; break; }
-        if (qi >= 2 && !mbar_wait(ACCEMPTY((qi - 2) & 3), ((qi - 2) >> 2) & 1, wc)) { ok = false; break; }
         const unsigned char* qrowp = base_ptr + R::OFF_Q + st * R::TILE_BYTES + qrow * 128;
         // packed fp32 pairs: these warps share their schedulers with the epilogue warps, whose per-tile chain sets
         // the pace of the kernel, so every instruction here counts
@@ -215,6 +210,11 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           asm("mov.b64 {%0, %1}, %2;" : "=f"(b0), "=f"(b1) : "l"(acc2[1]));
           ss = (a0 + a1) + (b0 + b1);
         }
+        // Slot qi & 1 was last read for tile qi - 2, whose epilogue threads arrived on that tile's ACCEMPTY after
+        // the read (tile qi + 2 cannot have completed that barrier again: it needs this slot first).  The Q stage
+        // goes back only after this wait: measured, handing it back before the wait is slower (768p clip, 148
+        // CTAs: 1.39 instead of 1.25 ms) -- the producer running further ahead of the epilogue does not help.
+        if (qi >= 2 && !mbar_wait(ACCEMPTY((qi - 2) & 3), ((qi - 2) >> 2) & 1, wc)) { ok = false; break; }
         qn[(qi & 1) * 128 + qrow] = rsqrtf(ss + q_l2_eps);
         mbar_arrive_warp(QEMPTY(st));
         mbar_arrive_warp(QNFULL(qi & 1));
@@ -275,11 +275,16 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tc_fence_before_sync();
         mbar_arrive_warp(ACCEMPTY(a));
 
-        float ss = 0.f;
+        // eight partial sums: one running sum would be a chain of 128 dependent FMAs (about 500 cycles) in the
+        // per-tile critical path of these warps
+        float sp[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sp[e] = 0.f;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
-          for (int e = 0; e < 32; ++e) ss = fmaf(v[c][e], v[c][e], ss);
+          for (int e = 0; e < 32; ++e) sp[e & 7] = fmaf(v[c][e], v[c][e], sp[e & 7]);
+        const float ss = ((sp[0] + sp[1]) + (sp[2] + sp[3])) + ((sp[4] + sp[5]) + (sp[6] + sp[7]));
         // with o = qrs * v (the read-out of the normalised query): mean o^2 = qrs^2 mean v^2
         const float scale = g * qrs * rsqrtf(ss * (qrs * qrs) * (1.0f / R::D) + eps);
 

@@ -403,14 +403,16 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
     nk = h->launches;
   }
   if (x.phase == 1) { VDN_CUDA(h, cudaGetLastError()); return VDN_OK; }
-  // The read-out streams reads and writes in equal parts and is fastest on about five SMs out of six
+  // The plain read-out streams reads and writes in equal parts and is fastest on about five SMs out of six
   // (measured on three workloads: 124 CTAs beat 148 by 5 %; fewer interleaved read/write streams at the DRAM).
+  // With the optional factors or the query norms it is paced by its epilogue warps and wants every SM (768p clip,
+  // warm GPU, 124 -> 148 CTAs: queries normalised 1.36 -> 1.25 ms, gate + norm weight 2.09 -> 1.87 ms).
   Shape sr = s;                                       // the frames to read out
   if (x.phase == 2) { sr.t0 = x.ro_first; sr.Tn = x.ro_count; }
   const long long nread = sr.work_items();
-  const long long ro_target = ((long long)h->sm_count * 27 + 16) / 32;
-  const unsigned persistent_ro = (unsigned)(nread < ro_target ? nread : ro_target);
   const bool extras = x.gate_elem || x.norm_weight || !gate;
+  const long long ro_target = (extras || x.q_l2_eps > 0.f) ? h->sm_count : ((long long)h->sm_count * 27 + 16) / 32;
+  const unsigned persistent_ro = (unsigned)(nread < ro_target ? nread : ro_target);
   CUtensorMap tmG = tmO;                                        // the gate tensor has the layout of the output
   if (x.gate_elem && (r = make_token_map(h, &tmG, x.gate_elem, s)) != VDN_OK) return r;
   auto launch_readout = [&](auto ex, auto qn) {
