@@ -280,6 +280,35 @@ def test_run_to_run_bitwise_determinism_and_canaries():
     assert torch.all(buf[:pad] == 7.0) and torch.all(buf[pad + n:] == 7.0)
 
 
+def test_forward_can_be_captured_in_a_cuda_graph():
+    # the layer only enqueues kernels and memsets on the caller's stream (tensor maps travel as kernel parameters):
+    # after one eager call (which sets the kernels' attributes) it can be captured and replayed; replays are
+    # bitwise the eager result, also after the inputs change in place
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=6, F=200, H=3, seed=12)
+    x = inputs.generate(w, "cuda")
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    kw = dict(alpha=alpha, s0=s0, chunk=2, radius=1, anchors=True)
+    out = torch.empty_like(x["q"])
+    eager = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], **kw).clone()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out, stream=side, **kw)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    assert torch.equal(out, eager)
+    x["v"].mul_(0.5)                       # same buffers, new contents
+    graph.replay()
+    torch.cuda.synchronize()
+    eager2 = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], **kw)
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager2) and not torch.equal(out, eager)
+
+
 def test_token_permutation_within_frames_permutes_rows_only():
     w = inputs.TINY.scaled(d=128, T=3, F=96, H=2)
     x = inputs.generate(w, "cuda")
