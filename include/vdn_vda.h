@@ -225,7 +225,7 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
 /* The same layer for callers whose tensors live in HOST memory (pinned memory recommended; with pageable
  * memory the copies are not asynchronous).  All six tensor pointers are HOST pointers.  The staging buffer is a
  * caller-owned DEVICE buffer of at least vdn_vda_staging_bytes, set beforehand.  Order of work on cuda_stream:
- * k, v, beta, gate are copied in; statistics, resolve and both scans run; then, for each of up to eight groups of
+ * k, v, beta, gate are copied in; statistics, resolve and both scans run; then, for each of up to 32 groups of
  * frames, that group's queries are copied in and read out, and its output rows are copied back on a second
  * stream owned by the handle, beside the next group's copy in (the host link is full duplex, and out needs the
  * scans of the whole clip, so this is all the overlap there is).  cuda_stream waits for the last copy back:

@@ -93,7 +93,7 @@ struct vdn_vda_s {
   bool tc_attrs_set = false;
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;  // driver entry point, resolved at create
   // vdn_vda_forward_host: frame groups whose results are copied back on a second stream (made on first use)
-  static constexpr int kHostGroups = 8;
+  static constexpr int kHostGroups = 32;
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t copy_ev[kHostGroups + 1] = {};
   std::string err = "no error";
