@@ -224,12 +224,14 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
 
 /* The same layer for callers whose tensors live in HOST memory (pinned memory recommended; with pageable
  * memory the copies are not asynchronous).  All six tensor pointers are HOST pointers.  The staging buffer is a
- * caller-owned DEVICE buffer of at least vdn_vda_staging_bytes, set beforehand.  Order of work on cuda_stream:
- * k, v, beta, gate are copied in; statistics, resolve and both scans run; then, for each of up to 32 groups of
- * frames, that group's queries are copied in and read out, and its output rows are copied back on a second
- * stream owned by the handle, beside the next group's copy in (the host link is full duplex, and out needs the
- * scans of the whole clip, so this is all the overlap there is).  cuda_stream waits for the last copy back:
- * synchronising it is enough.  The first call creates the second stream and nine events (no device memory). */
+ * caller-owned DEVICE buffer of at least vdn_vda_staging_bytes, set beforehand.  The copies in run on an input
+ * stream owned by the handle, which starts where cuda_stream stands at the call and is queued in one go, so the
+ * host link never waits for a kernel: k, v, beta, gate, then the queries in up to 32 groups of frames.  On
+ * cuda_stream: statistics, resolve and both scans once k, v, beta have landed; then each group is read out as
+ * soon as its queries have landed.  Each group's output rows are copied back on a third stream, beside the
+ * copies in (the host link is full duplex, and out needs the scans of the whole clip, so this is all the
+ * overlap there is).  cuda_stream waits for the last copy back: synchronising it is enough.  The first call
+ * creates the two streams and their events (no device memory). */
 size_t vdn_vda_staging_bytes(vdn_vda_t h, int B, int T, int F, int H, int d);
 vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes);
 vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const void* v,

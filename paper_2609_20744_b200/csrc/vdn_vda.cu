@@ -92,10 +92,13 @@ struct vdn_vda_s {
   bool attrs_set = false;
   bool tc_attrs_set = false;
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;  // driver entry point, resolved at create
-  // vdn_vda_forward_host: frame groups whose results are copied back on a second stream (made on first use)
+  // vdn_vda_forward_host: inputs arrive on one stream of the handle's own and results leave on another, in groups of
+  // frames (streams and events made on first use)
   static constexpr int kHostGroups = 32;
-  cudaStream_t copy_stream = nullptr;
+  cudaStream_t copy_stream = nullptr;                  // device -> host
   cudaEvent_t copy_ev[kHostGroups + 1] = {};
+  cudaStream_t in_stream = nullptr;                    // host -> device
+  cudaEvent_t in_ev[kHostGroups + 2] = {};             // call entered, keys/values landed, query group g landed
   std::string err = "no error";
 };
 
@@ -778,32 +781,49 @@ vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const
     VDN_CUDA(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
     for (int i = 0; i <= vdn_vda_s::kHostGroups; ++i)
       VDN_CUDA(h, cudaEventCreateWithFlags(&h->copy_ev[i], cudaEventDisableTiming));
+    VDN_CUDA(h, cudaStreamCreateWithFlags(&h->in_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < vdn_vda_s::kHostGroups + 2; ++i)
+      VDN_CUDA(h, cudaEventCreateWithFlags(&h->in_ev[i], cudaEventDisableTiming));
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   char* sg = static_cast<char*>(h->staging);
   const size_t tokh = (size_t)B * T * F * H;
   const size_t big = tokh * d * elem_size(h);
   const size_t frame_bytes = (size_t)F * H * d * elem_size(h);
-  // Keys, values and write gates first: the statistics, the resolve and both scans need nothing else.
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.k, k, big, cudaMemcpyHostToDevice, st));
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.v, v, big, cudaMemcpyHostToDevice, st));
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.beta, beta, tokh * sizeof(float), cudaMemcpyHostToDevice, st));
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.gate, gate, (size_t)H * sizeof(float), cudaMemcpyHostToDevice, st));
-  const float* dbeta = reinterpret_cast<const float*>(sg + S.beta);
-  const float* dgate = reinterpret_cast<const float*>(sg + S.gate);
-  vdn_status r = forward_core(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, B, T, F, H, d, nullptr,
-                              cuda_stream, 1, 0, 0);
-  if (r != VDN_OK) return r;
-  // Then the queries, one group of frames after another: copy in, read out, and hand the finished rows to the
-  // second stream, whose copy back to the host runs beside the next group's copy in (the link is full duplex).
+  // All copies in are queued at once on the handle's input stream, in the order the layer needs them, so that the
+  // host link never waits for a kernel: keys, values and write gates first (the statistics, the resolve and both
+  // scans need nothing else), then the queries, one group of frames after another.  The input stream starts where
+  // the caller's stream stands now (earlier work on it may still be reading the staging buffer).
+  cudaStream_t in = h->in_stream;
+  VDN_CUDA(h, cudaEventRecord(h->in_ev[0], st));
+  VDN_CUDA(h, cudaStreamWaitEvent(in, h->in_ev[0], 0));
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.k, k, big, cudaMemcpyHostToDevice, in));
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.v, v, big, cudaMemcpyHostToDevice, in));
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.beta, beta, tokh * sizeof(float), cudaMemcpyHostToDevice, in));
+  VDN_CUDA(h, cudaMemcpyAsync(sg + S.gate, gate, (size_t)H * sizeof(float), cudaMemcpyHostToDevice, in));
+  VDN_CUDA(h, cudaEventRecord(h->in_ev[1], in));
   const int groups = T < vdn_vda_s::kHostGroups ? T : vdn_vda_s::kHostGroups;
   for (int g = 0; g < groups; ++g) {
     const int t0 = (int)((long long)T * g / groups), t1 = (int)((long long)T * (g + 1) / groups);
     const size_t off = (size_t)t0 * frame_bytes, len = (size_t)(t1 - t0) * frame_bytes;
     for (int b = 0; b < B; ++b) {
       const size_t o = (size_t)b * T * frame_bytes + off;
-      VDN_CUDA(h, cudaMemcpyAsync(sg + S.q + o, static_cast<const char*>(q) + o, len, cudaMemcpyHostToDevice, st));
+      VDN_CUDA(h, cudaMemcpyAsync(sg + S.q + o, static_cast<const char*>(q) + o, len, cudaMemcpyHostToDevice, in));
     }
+    VDN_CUDA(h, cudaEventRecord(h->in_ev[2 + g], in));
+  }
+  const float* dbeta = reinterpret_cast<const float*>(sg + S.beta);
+  const float* dgate = reinterpret_cast<const float*>(sg + S.gate);
+  VDN_CUDA(h, cudaStreamWaitEvent(st, h->in_ev[1], 0));
+  vdn_status r = forward_core(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, B, T, F, H, d, nullptr,
+                              cuda_stream, 1, 0, 0);
+  if (r != VDN_OK) return r;
+  // Each group is read out as soon as its queries have landed, and its finished rows go to the second stream,
+  // whose copy back to the host runs beside the copies in (the link is full duplex).
+  for (int g = 0; g < groups; ++g) {
+    const int t0 = (int)((long long)T * g / groups), t1 = (int)((long long)T * (g + 1) / groups);
+    const size_t off = (size_t)t0 * frame_bytes, len = (size_t)(t1 - t0) * frame_bytes;
+    VDN_CUDA(h, cudaStreamWaitEvent(st, h->in_ev[2 + g], 0));
     r = forward_core(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, B, T, F, H, d, nullptr, cuda_stream,
                      2, t0, t1 - t0);
     if (r != VDN_OK) return r;
@@ -943,6 +963,9 @@ vdn_status vdn_vda_destroy(vdn_vda_t h) {
     for (cudaEvent_t e : h->copy_ev)
       if (e) cudaEventDestroy(e);
     cudaStreamDestroy(h->copy_stream);
+    for (cudaEvent_t e : h->in_ev)
+      if (e) cudaEventDestroy(e);
+    if (h->in_stream) cudaStreamDestroy(h->in_stream);
   }
   if (h->status_host) cudaFreeHost(h->status_host);
   delete h;
