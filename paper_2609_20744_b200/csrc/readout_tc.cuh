@@ -24,40 +24,47 @@
 
 namespace vdn {
 
-template <bool EXTRAS, bool QNORM = false>
+template <bool EXTRAS, bool QNORM = false, bool GATE = false>
 struct ReadoutTcCfg {
+  static_assert(EXTRAS || !GATE, "the element-wise gate is one of the optional factors");
   static constexpr int D = 128;
   static constexpr int TILE = 128;
-  // EXTRAS: gate tiles arrive by TMA in the output staging tiles (a third one takes the place of a Q stage)
-  static constexpr int QSTAGES = EXTRAS ? 2 : 3;       // (3 Q stages, 2 staging tiles and a one-tile gate lookahead:
-  static constexpr int NOUT = EXTRAS ? 3 : 2;          //  2.74 ms instead of 2.07 ms on the 768p clip)
+  // GATE: gate tiles arrive by TMA in the output staging tiles, two tiles ahead; a third staging tile takes the
+  // place of a Q stage (with 3 Q stages, 2 staging tiles and a one-tile lookahead the gate path takes 2.47 ms
+  // instead of 1.76 ms on the 768p clip; without a gate the third Q stage is worth more: 1.24 against 1.37 ms)
+  static constexpr int QSTAGES = GATE ? 2 : 3;
+  static constexpr int NOUT = GATE ? 3 : 2;
   static constexpr int BOX_BYTES = 128 * 128;          // 128 rows x 128 B
   static constexpr int TILE_BYTES = 2 * BOX_BYTES;     // 32 KB: state, Q tile or output tile
   static constexpr int OFF_STATE = 0;
   static constexpr int OFF_Q = 2 * TILE_BYTES;
   static constexpr int OFF_OUT = OFF_Q + QSTAGES * TILE_BYTES;
   static constexpr int OFF_NW = OFF_OUT + NOUT * TILE_BYTES;   // norm weights of the current head, 128 floats
-  static constexpr int OFF_QN = OFF_NW + (EXTRAS ? 512 : 0);   // QNORM: 1/|q| of the tokens of two tiles, 2 x 128 floats
-  static constexpr int OFF_BAR = OFF_QN + (QNORM ? 1024 : 0);
-  static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
+  // QNORM: 1/|q| of the tokens of QSLOTS tiles, 128 floats each.  (Four slots instead of two for the variant with
+  // two Q stages: no faster, 2.16 against 2.06 ms on the 768p clip.)
+  static constexpr int QSLOTS = 2;
+  static constexpr int OFF_QN = OFF_NW + (EXTRAS ? 512 : 0);
+  static constexpr int OFF_BAR = OFF_QN + (QNORM ? QSLOTS * 512 : 0);
+  static constexpr int USED_BYTES = OFF_BAR + 256;
+  static constexpr int SMEM_BYTES = USED_BYTES + 1024 <= 227 * 1024 ? USED_BYTES + 1024 : 227 * 1024;
   static constexpr int THREADS = QNORM ? 320 : 192;
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one SM");
 };
 using ReadoutTc = ReadoutTcCfg<false>;
 
-// EXTRAS = true adds the two optional factors of Eq. 1c to the epilogue: an element-wise (content-dependent) gate
-// gate_elem [B,T,F,H,d] bf16 (tensor map tmG; its tiles arrive by TMA in the very staging tile the output is then
-// written to, two tiles ahead) and a per-channel norm scale norm_weight [H,d] (kept in shared memory per frame);
-// either may be null, and so may the per-head gate (read as 1).  The plain instantiation carries none of that code.
-template <bool EXTRAS, bool QNORM = false>
-__global__ void __launch_bounds__(ReadoutTcCfg<EXTRAS, QNORM>::THREADS, 1)
+// EXTRAS = true adds the optional factors of Eq. 1c to the epilogue: a per-channel norm scale norm_weight [H,d]
+// (kept in shared memory per frame; may be null), a per-head gate that may be null (read as 1) and, with GATE, an
+// element-wise (content-dependent) gate gate_elem [B,T,F,H,d] bf16 (tensor map tmG; its tiles arrive by TMA in the
+// very staging tile the output is then written to, two tiles ahead).  The plain instantiation carries none of that.
+template <bool EXTRAS, bool QNORM = false, bool GATE = false>
+__global__ void __launch_bounds__(ReadoutTcCfg<EXTRAS, QNORM, GATE>::THREADS, 1)
 readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmS,
                   const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmG,
                   const float* __restrict__ gate, Shape s, float eps,
                   int* status, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight,
                   Window win, int bridged, float q_l2_eps) {
   using namespace tc;
-  using R = ReadoutTcCfg<EXTRAS, QNORM>;
+  using R = ReadoutTcCfg<EXTRAS, QNORM, GATE>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -70,11 +77,17 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   auto ACCFULL = [&](int i) { return bar0 + 8u * (10 + i); };    // 4
   auto ACCEMPTY = [&](int i) { return bar0 + 8u * (14 + i); };   // 4
   auto GFULL = [&](int i) { return bar0 + 8u * (18 + i); };      // 3 (EXTRAS: gate tile landed)
-  auto QNFULL = [&](int i) { return bar0 + 8u * (21 + i); };     // 2 (QNORM: 1/|q| of a tile written)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 8 * 23);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 8 * 23 + 8);
+  auto QNFULL = [&](int i) { return bar0 + 8u * (21 + i); };     // up to 4 (QNORM: 1/|q| of a tile written)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 8 * 25);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 8 * 25 + 8);
+  constexpr uint32_t QS = R::QSLOTS;
   const WaitCtx wc{abort_flag, status};
 
+  if ((base - smem_u32(smem_dyn)) + R::USED_BYTES > (uint32_t)R::SMEM_BYTES) {
+    // the dynamic shared memory window starts too far from a 1024-byte boundary for the layout to fit
+    if (threadIdx.x == 0) atomicExch(status, kStatusTimeout);
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ntiles = (s.F + R::TILE - 1) / R::TILE;
   const long long nitems = s.work_items();
@@ -85,13 +98,13 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     for (int i = 0; i < 2; ++i) { mbar_init(STFULL(i), 1); mbar_init(STEMPTY(i), 1); }
     for (int i = 0; i < 4; ++i) { mbar_init(ACCFULL(i), 1); mbar_init(ACCEMPTY(i), 4); }   // one arrival per epilogue warp
     for (int i = 0; i < 3; ++i) mbar_init(GFULL(i), 1);
-    for (int i = 0; i < 2; ++i) mbar_init(QNFULL(i), 4);
+    for (int i = 0; i < R::QSLOTS; ++i) mbar_init(QNFULL(i), 4);
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmS);
     tma_prefetch_desc(&tmO);
-    if (EXTRAS) tma_prefetch_desc(&tmG);
+    if (GATE) tma_prefetch_desc(&tmG);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), 512);
@@ -210,14 +223,14 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           asm("mov.b64 {%0, %1}, %2;" : "=f"(b0), "=f"(b1) : "l"(acc2[1]));
           ss = (a0 + a1) + (b0 + b1);
         }
-        // Slot qi & 1 was last read for tile qi - 2, whose epilogue threads arrived on that tile's ACCEMPTY after
-        // the read (tile qi + 2 cannot have completed that barrier again: it needs this slot first).  The Q stage
+        // Slot qi % QS was last read for tile qi - QS, whose epilogue threads arrived on that tile's ACCEMPTY after
+        // the read (a later tile cannot have completed that barrier again: it needs this slot first).  The Q stage
         // goes back only after this wait: measured, handing it back before the wait is slower (768p clip, 148
         // CTAs: 1.39 instead of 1.25 ms) -- the producer running further ahead of the epilogue does not help.
-        if (qi >= 2 && !mbar_wait(ACCEMPTY((qi - 2) & 3), ((qi - 2) >> 2) & 1, wc)) { ok = false; break; }
-        qn[(qi & 1) * 128 + qrow] = rsqrtf(ss + q_l2_eps);
+        if (qi >= QS && !mbar_wait(ACCEMPTY((qi - QS) & 3), ((qi - QS) >> 2) & 1, wc)) { ok = false; break; }
+        qn[(qi % QS) * 128 + qrow] = rsqrtf(ss + q_l2_eps);
         mbar_arrive_warp(QEMPTY(st));
-        mbar_arrive_warp(QNFULL(qi & 1));
+        mbar_arrive_warp(QNFULL(qi % QS));
       }
     }
   } else {
@@ -227,7 +240,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int et = threadIdx.x - 64;            // 0..127
     uint32_t qi = 0;
     bool ok = true;
-    const bool use_ge = EXTRAS && gate_elem != nullptr;
+    constexpr bool use_ge = GATE;            // (gate_elem itself is read through its tensor map)
     float* nws = reinterpret_cast<float*>(base_ptr + R::OFF_NW);
     // EXTRAS: the gate tile of tile number q (counted over this CTA's tiles) is copied into staging tile q % NOUT,
     // where the output of that tile is then written; issued by one thread, two tiles ahead
@@ -262,8 +275,8 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tc_fence_after_sync();
         float qrs = 1.0f;
         if constexpr (QNORM) {
-          if (!mbar_wait(QNFULL(qi & 1), (qi >> 1) & 1, wc)) { ok = false; break; }
-          qrs = reinterpret_cast<const float*>(base_ptr + R::OFF_QN)[(qi & 1) * 128 + row];
+          if (!mbar_wait(QNFULL(qi % QS), (qi / QS) & 1, wc)) { ok = false; break; }
+          qrs = reinterpret_cast<const float*>(base_ptr + R::OFF_QN)[(qi % QS) * 128 + row];
         }
         const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 128;
         float v[4][32];

@@ -91,6 +91,7 @@ struct vdn_vda_s {
   int launches = 0;
   bool attrs_set = false;
   bool tc_attrs_set = false;
+  unsigned ro_attrs_set = 0;       // read-out instantiations whose shared-memory attribute has been set
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;  // driver entry point, resolved at create
   // vdn_vda_forward_host: inputs arrive on one stream of the handle's own and results leave on another, in groups of
   // frames (streams and events made on first use)
@@ -320,14 +321,6 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   if (!h->tc_attrs_set) {
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::GramTc::SMEM_BYTES));
-    VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     vdn::ReadoutTc::SMEM_BYTES));
-    VDN_CUDA(h, cudaFuncSetAttribute(vdn::readout_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     vdn::ReadoutTcCfg<true>::SMEM_BYTES));
-    VDN_CUDA(h, (cudaFuncSetAttribute(vdn::readout_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      vdn::ReadoutTcCfg<false, true>::SMEM_BYTES)));
-    VDN_CUDA(h, (cudaFuncSetAttribute(vdn::readout_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      vdn::ReadoutTcCfg<true, true>::SMEM_BYTES)));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
     VDN_CUDA(h, (cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -418,20 +411,34 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   const unsigned persistent_ro = (unsigned)(nread < ro_target ? nread : ro_target);
   CUtensorMap tmG = tmO;                                        // the gate tensor has the layout of the output
   if (x.gate_elem && (r = make_token_map(h, &tmG, x.gate_elem, s)) != VDN_OK) return r;
-  auto launch_readout = [&](auto ex, auto qn) {
-    constexpr bool EX = decltype(ex)::value, QN = decltype(qn)::value;
-    using RX = vdn::ReadoutTcCfg<EX, QN>;
-    vdn::readout_tc_kernel<EX, QN><<<persistent_ro, RX::THREADS, RX::SMEM_BYTES, st>>>(
+  auto launch_readout = [&](auto ex, auto qn, auto ge) {
+    constexpr bool EX = decltype(ex)::value, QN = decltype(qn)::value, GE = decltype(ge)::value;
+    using RX = vdn::ReadoutTcCfg<EX, QN, GE>;
+    constexpr unsigned bit = 1u << ((EX ? 1 : 0) | (QN ? 2 : 0) | (GE ? 4 : 0));
+    if (!(h->ro_attrs_set & bit)) {        // per handle, i.e. per device
+      if (cudaFuncSetAttribute(vdn::readout_tc_kernel<EX, QN, GE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               RX::SMEM_BYTES) != cudaSuccess)
+        return false;
+      h->ro_attrs_set |= bit;
+    }
+    vdn::readout_tc_kernel<EX, QN, GE><<<persistent_ro, RX::THREADS, RX::SMEM_BYTES, st>>>(
         tmQ, tmS, tmO, tmG, gate, sr, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
         x.norm_weight, x.win, x.alpha != nullptr, x.q_l2_eps);
+    return true;
   };
   using std::true_type;
   using std::false_type;
+  bool launched;
   if (x.q_l2_eps > 0.f) {
-    if (extras) launch_readout(true_type{}, true_type{}); else launch_readout(false_type{}, true_type{});
+    if (x.gate_elem) launched = launch_readout(true_type{}, true_type{}, true_type{});
+    else if (extras) launched = launch_readout(true_type{}, true_type{}, false_type{});
+    else launched = launch_readout(false_type{}, true_type{}, false_type{});
   } else {
-    if (extras) launch_readout(true_type{}, false_type{}); else launch_readout(false_type{}, false_type{});
+    if (x.gate_elem) launched = launch_readout(true_type{}, false_type{}, true_type{});
+    else if (extras) launched = launch_readout(true_type{}, false_type{}, false_type{});
+    else launched = launch_readout(false_type{}, false_type{}, false_type{});
   }
+  if (!launched) return fail(h, VDN_ERR_CUDA, "cudaFuncSetAttribute failed for the read-out kernel");
   prof_mark(h, st, nk++, "readout_tc");
   h->launches = nk;
   VDN_CUDA(h, cudaGetLastError());
