@@ -71,6 +71,18 @@ __device__ __forceinline__ float silu_f(float x) {
   return x * r;
 }
 
+// For 16-bit outputs: SiLU(x) = h + h tanh(h), h = x / 2, with the hardware tanh (specified to about 2^-11 relative,
+// three bits below the bf16 rounding of the result; measured, 0.04 % of the outputs differ from the correctly
+// rounded value): five instructions per pair instead of eight, in kernels that are bound by instruction issue.
+__device__ __forceinline__ void silu2_tanh(f32x2 x, float& y0, float& y1) {
+  float h0, h1, t0, t1;
+  const f32x2 h = mul2(x, pack2(0.5f, 0.5f));
+  unpack2(h, h0, h1);
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t0) : "f"(h0));
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t1) : "f"(h1));
+  unpack2(fma2(h, pack2(t0, t1), h), y0, y1);
+}
+
 // the same for a packed pair: the scale, the "+ 1" and the final product as packed operations
 __device__ __forceinline__ void silu2(f32x2 x, float& y0, float& y1) {
   float t0, t1, e0, e1, r0, r1;
@@ -228,7 +240,7 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
       f32x2 o = mul2(wtp[0], ring[(r + 1) % 5][j]);
 #pragma unroll
       for (int i = 1; i < 5; ++i) o = fma2(wtp[i], ring[(r + i + 1) % 5][j], o);
-      silu2(o, o0[j], o1[j]);
+      if constexpr (sizeof(Tio) == 2) silu2_tanh(o, o0[j], o1[j]); else silu2(o, o0[j], o1[j]);
     }
     if (which == 0) {
       // ---- L2 normalisation over the head's d channels (Sec. 2.3).  Eight sums over the row's lanes at once:
@@ -416,7 +428,7 @@ prep_kv_temporal_kernel(PrepArgs a, Shape s) {
 #pragma unroll
       for (int i = 1; i < 5; ++i) v = fma2(wt[i][c], ring[(r + i + 1) % 5][c], v);
       float y0, y1;
-      silu2(v, y0, y1);
+      if constexpr (sizeof(Tio) == 2) silu2_tanh(v, y0, y1); else silu2(v, y0, y1);
       y[c] = pack2(y0, y1);
       ss2 = fma2(y[c], y[c], ss2);
     }
