@@ -128,6 +128,10 @@ def test_768p_queries_normalised_by_the_readout_full_size():
     torch.cuda.synchronize()
     assert vda.status() == binding.VDN_OK
     assert vda.uses_tensor_cores()
+    again = vda.forward(q_raw, x["k"], x["v"], x["beta"], x["gate"], q_l2_eps=1e-6)
+    torch.cuda.synchronize()
+    assert torch.equal(out, again)          # the norms travel between warps through shared memory: no race
+    del again
     for (b, h) in sampled_pairs(w, 2):
         q, k, v, beta, gate = inputs.head_slice(x, b, h)
         qn = po.l2_normalise(q_raw[b, :, :, h, :].double().cpu().numpy(), 1e-6)
