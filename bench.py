@@ -3,9 +3,11 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 768p] [--impl ours|reference]
 
-N > 1 (launched with torch.distributed.run, one rank per GPU) runs N independent replicas of the
-workload -- the layer needs no exchange between GPUs -- and reports the aggregate tokens/s over the
-slowest rank's time.  Rank 0 prints ONE JSON line.
+N > 1 runs N independent replicas of the workload, one process per GPU -- the layer needs no exchange
+between GPUs -- and reports the aggregate tokens/s over the slowest rank's time.  Started as a plain
+`python bench.py --gpus N` it launches its own N ranks through torch.distributed.run (rendezvous on
+127.0.0.1); started under torch.distributed.run (RANK / WORLD_SIZE in the environment) it is one of the
+ranks.  NCCL carries the barrier and two scalar reductions, nothing else.  Rank 0 prints ONE JSON line.
 """
 from __future__ import annotations
 
@@ -44,6 +46,20 @@ def algorithmic_bytes(w) -> dict:
         "readout": tokh * (2 * w.d * es),           # q in, out out
         "total": tokh * (4 * w.d * es + 4),
     }
+
+
+def implementation_bytes(w) -> dict:
+    """Bytes of the per-frame d x d intermediates that the tensor-core kernels move through HBM/L2 on top of
+    the algorithmic bytes, as the kernels are written (each array counted once per pass that streams it):
+    statistics fp32 [2d][d] written by the Gram kernel, the A half read by the resolve, the B half read by both
+    scans; the inverse as three bf16 parts written once and read by both scans; the two read states (bf16)
+    written by the scans and read by the read-out."""
+    n = w.B * w.H * w.T
+    dd = w.d * w.d
+    stats = n * dd * 4 * (2 + 1 + 2)
+    inverse = n * dd * 2 * 3 * (1 + 2)
+    states = n * dd * 2 * (2 + 2)
+    return {"statistics": stats, "inverse_split": inverse, "read_states": states, "total": stats + inverse + states}
 
 
 def algorithmic_flops(w) -> dict:
@@ -198,8 +214,23 @@ def cpu_baseline(w, seconds: float = 15.0) -> dict:
 
 
 # ------------------------------------------------------------------------------------------ arms
+def layer_config(w, n_gpus: int, win: dict) -> dict:
+    """The `config` object of a bench line.  Both arms build it here, from the workload and the command line
+    alone, so that the two lines of one comparison carry the same object; what is specific to an arm (which
+    kernels ran, where the oracle ran) sits beside it under `arm`."""
+    big = algorithmic_bytes(w)["total"] > 1e9
+    return {"workload": w.name, "B": w.B, "T": w.T, "F": w.F, "H": w.H, "d": w.d, "io_dtype": w.dtype,
+            "seed": w.seed, "parallelism": "single GPU" if n_gpus == 1 else f"{n_gpus} independent replicas",
+            "l2": "inputs+outputs far larger than the 126 MB L2; no flush" if big
+                  else "inputs smaller than L2: numbers are L2-warm",
+            "window": win}
+
+
 def run_reference(args, w, rank: int, world: int):
-    """The reference arm is the fp64 oracle on the host cores (rank 0 only)."""
+    """The reference arm is the fp64 oracle on the host cores (rank 0 only).  Every step runs the oracle over a
+    bounded sample of the workload; `value` scales the sample's rate to the whole workload (units are independent
+    and equal-cost), `ms_per_step` is the time a sampled step really took, and the extrapolated time of a whole
+    forward is given beside it under its own key."""
     if rank != 0:
         return
     seconds_total = 60.0                                  # for the whole --steps/--warmup run
@@ -210,12 +241,15 @@ def run_reference(args, w, rank: int, world: int):
     sec = sum(time_oracle(slices) for _ in range(args.steps)) / max(1, args.steps)
     full_ms = sec * (w.B * w.H * w.T) / (heads * frames) * 1e3
     value = w.tokens / (full_ms / 1e3)
+    win = dict(chunk=args.chunk, radius=args.radius, anchors=bool(args.anchors))
+    cfg = layer_config(w, args.gpus, win)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": full_ms, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "T": w.T, "F": w.F, "H": w.H, "d": w.d, "io_dtype": w.dtype,
-                   "parallelism": "fp64 CPU oracle on rank 0's host cores"},
+        "config": cfg, "arm": "fp64 CPU oracle (numpy on BLAS threads) on rank 0's host cores",
+        "ms_per_step_is": "measured time of one sampled step (see cpu_baseline.sample)",
+        "ms_per_forward_extrapolated": full_ms,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                          "sample": sample_text(w, heads, frames)},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -298,7 +332,13 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     if rank == 0 and not args.skip_cpu:
         from oracle import vda_oracle
         tol = 1e-4 if w.dtype == "f32" else 2e-2
-        pairs = [(0, 0), (w.B - 1, w.H - 1)]
+        pairs = [(0, 0), (w.B - 1, w.H - 1)]          # first, last and two seeded (batch, head) slices
+        import numpy as _np
+        rng = _np.random.default_rng(w.seed + 1234)
+        while len(pairs) < min(4, w.B * w.H):
+            pr = (int(rng.integers(w.B)), int(rng.integers(w.H)))
+            if pr not in pairs:
+                pairs.append(pr)
         errs, viol = [], []
         for (b, hh) in pairs:
             qs, ks, vs, bs, gs = inputs.head_slice(x, b, hh)
@@ -306,7 +346,6 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
             got = out[b, :, :, hh, :].double().cpu().numpy()
             errs.append(vda_oracle.slice_error(got, ref))
             # reported, not gated: elements off by more than tol * (|ref| + rms of the slice)
-            import numpy as _np
             rms = float(_np.sqrt(_np.mean(ref * ref)))
             viol.append(int(_np.count_nonzero(_np.abs(got - ref) > tol * (_np.abs(ref) + rms))))
             del qs, ks, vs, ref, got
@@ -319,31 +358,52 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     try:
         if args.skip_e2e:
             raise RuntimeError("skipped (--skip-e2e)")
-        if win != dict(chunk=1, radius=0, anchors=False):
-            raise RuntimeError("the host-buffer entry point has no window options")
         xh = {n: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for n, t in x.items()}
         outh = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
         e_steps = max(1, min(args.steps, args.e2e_steps))
-        vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], outh)
+        vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], outh, **fw)
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
         ev0.record(stream)
         for _ in range(e_steps):
-            vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], outh)
+            vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], outh, **fw)
         ev1.record(stream)
         torch.cuda.synchronize()
         e_ms, e_tok = aggregate_over_ranks(ev0.elapsed_time(ev1) / e_steps, w.tokens, world)
         h2d = sum(xh[n].numel() * xh[n].element_size() for n in ("q", "k", "v", "beta", "gate"))
         e2e = {"value": e_tok / (e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": outh.numel() * outh.element_size(), "ms_per_step": e_ms, "steps": e_steps,
-               "api": "vdn_vda_forward_host (pinned host buffers)"}
+               "api": "vdn_vda_forward_host (pinned host buffers)" if win == dict(chunk=1, radius=0, anchors=False)
+                      and not args.q_l2_eps else "vdn_vda_forward_host_opt (pinned host buffers)"}
         same = bool(torch.equal(outh, out.cpu()))
         e2e["matches_device_entry_point"] = same
         del xh, outh
     except Exception as exc:  # host memory may be too small for the pinned copies
         e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                "error": f"{type(exc).__name__}: {exc}"}
+
+    # ---- sustained: a loop of at least two seconds after the timed region (clocks settle under load)
+    sustained = None
+    if args.sustain_s > 0:
+        n_loop = max(20, int(args.sustain_s * 1e3 / max(ms_local, 1e-3)) + 1)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        s_wall0 = time.time()
+        ev0.record(stream)
+        for _ in range(n_loop):
+            step()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        s_wall1 = time.time()
+        s_ms, s_tok = aggregate_over_ranks(ev0.elapsed_time(ev1) / n_loop, w.tokens, world)
+        if rank == 0:
+            s_clk = sampler.summary(s_wall0, s_wall1)
+            sustained = {"ms_per_step": s_ms, "value": s_tok / (s_ms / 1e3), "unit": UNIT, "steps": n_loop,
+                         "seconds": s_wall1 - s_wall0, "sm_mhz_median": s_clk["sm_mhz"], "reasons": s_clk["reasons"],
+                         "ms_times_sm_mhz": s_ms * s_clk["sm_mhz"] if s_clk["sm_mhz"] else None,
+                         "timed_region_ms_times_sm_mhz": ms_max * clocks["sm_mhz"] if clocks and clocks["sm_mhz"] else None}
 
     if rank != 0:
         return
@@ -383,20 +443,18 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 in / f32 accumulate, f32 state" if w.dtype == "bf16" else "f32",
         "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "T": w.T, "F": w.F, "H": w.H, "d": w.d, "io_dtype": w.dtype,
-                   "seed": w.seed, "parallelism": "single GPU" if world == 1 else f"{world} independent replicas",
-                   "l2": "inputs+outputs far larger than the 126 MB L2; no flush" if ab["total"] > 1e9
-                         else "inputs smaller than L2: numbers are L2-warm",
-                   "path": "tensor-core" if vda.launch_count() and any("tc" in n for n in kt) else "plain-fp32",
-                   "window": win},
+        "config": layer_config(w, world, win),
+        "arm": "tensor-core kernels" if vda.launch_count() and any("tc" in n for n in kt) else "plain-fp32 kernels",
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "parity": parity,
         "roofline": roof,
         "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
         "layer_roofline": {"t_roof_ms_measured_peaks": t_roof_ms, "frac_of_measured": t_roof_ms / (ms_max / 1.0),
                            "t_roof_ms_nominal": t_roof_nominal_ms, "frac_of_nominal": t_roof_nominal_ms / ms_max,
                            "t_fp32_alu_ms": fl["fp32"] / (148 * 128 * 2 * 1.965e9) * 1e3,
-                           "algorithmic_bytes": ab["total"], "tensor_flops": fl["tensor"], "fp32_flops": fl["fp32"]},
-        "kernel_ms": kt,
+                           "algorithmic_bytes": ab["total"], "tensor_flops": fl["tensor"], "fp32_flops": fl["fp32"],
+                           # reported separately, as the per-frame d x d intermediates are not algorithmic bytes
+                           "implementation_bytes": implementation_bytes(w) if w.d == 128 and w.dtype == "bf16" else None},
+        "kernel_ms": kt, "sustained": sustained,
         "cpu_baseline": base,
         "context": PAPER_CONTEXT,
     }
@@ -523,6 +581,45 @@ def run_prep(args, w, local_rank: int):
     print(json.dumps(line), flush=True)
 
 
+def free_port() -> int:
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        return so.getsockname()[1]
+
+
+def launch_ranks(n: int, argv) -> int:
+    """Starts n ranks of this script, one per GPU, through torch.distributed.run on 127.0.0.1 and passes their
+    output through (rank 0 prints the JSON line).  Returns the launcher's exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
+def run_launcher_selftest(args, w, rank: int, world: int):
+    """Every rank "measures" (10 + 5 rank) ms over the workload's tokens and the ranks aggregate as the real run
+    does -- through gloo on CPU, so that the launch path can be exercised on a machine without GPUs."""
+    import torch.distributed as dist
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+    try:
+        ms, tokens = aggregate_over_ranks(10.0 + 5.0 * rank, w.tokens, world)
+        if world > 1:
+            dist.barrier()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world,
+                              "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                              "scaling": "weak", "vs_baseline": None, "dtype": "none",
+                              "data": "launcher self-test: made-up times, no GPU work",
+                              "config": layer_config(w, world, dict(chunk=args.chunk, radius=args.radius,
+                                                                    anchors=bool(args.anchors))),
+                              "gpu_launches": 0}), flush=True)
+    finally:
+        if world > 1:
+            dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -545,6 +642,11 @@ def main():
     ap.add_argument("--no-spatial", action="store_true", help="--stage prep without the 5x5 spatial filter")
     ap.add_argument("--q-l2-eps", type=float, default=0.0,
                     help="> 0: the read-out normalises the queries (vdn_vda_options.q_l2_eps); --stage prep then skips Q")
+    ap.add_argument("--sustain-s", type=float, default=2.0,
+                    help="seconds of back-to-back forwards after the timed region for the `sustained` block (0 = none)")
+    ap.add_argument("--launcher-selftest", action="store_true",
+                    help="no GPU work: every rank reports a made-up time through gloo on CPU; checks the self-launch "
+                         "and the aggregation end to end (the line says so in `data`)")
     ap.add_argument("--skip-e2e", action="store_true", help="no host-buffer pass (profiler captures)")
     ap.add_argument("--skip-cpu", action="store_true", help="no CPU-oracle timing (profiler captures)")
     args = ap.parse_args()
@@ -556,10 +658,17 @@ def main():
     if args.frames > 0:
         w = w.scaled(T=args.frames, name=f"{w.name}_T{args.frames}")
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.stage != "prep" and args.impl != "reference":
+        # a plain `python bench.py --gpus N`: become the launcher of N ranks of this very command
+        raise SystemExit(launch_ranks(args.gpus, sys.argv[1:]))
+
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
+    if args.launcher_selftest:
+        run_launcher_selftest(args, w, rank, world)
+        return
     if args.impl == "reference":
         run_reference(args, w, rank, world)
         return

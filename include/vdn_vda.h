@@ -41,8 +41,9 @@
  * Errors.  Every call returns a vdn_status; nothing throws, aborts or traps.  Problems the host can see
  * (null or misaligned pointers, non-positive sizes, d != cfg.d, workspace too small, 32-bit index overflow,
  * wrong device architecture) are reported synchronously and nothing is enqueued.  Every wait inside a
- * kernel is bounded; a wait that runs out records VDN_ERR_TIMEOUT in the handle's status word, which
- * vdn_vda_status returns once the caller has synchronised the stream.
+ * kernel is bounded (vdn_vda_set_wait_limit_us); a wait that runs out records VDN_ERR_TIMEOUT in the handle's
+ * status word, which vdn_vda_status returns once the caller has synchronised the stream and which stays set
+ * until vdn_vda_clear_status.
  *
  * Determinism.  No atomics on the result path: the same inputs give bit-identical outputs run to run.
  */
@@ -65,7 +66,9 @@ typedef enum {
   VDN_ERR_WORKSPACE = 3,    /* workspace missing or smaller than vdn_vda_workspace_bytes              */
   VDN_ERR_CUDA = 4,         /* a CUDA runtime / driver call failed; see vdn_vda_last_error            */
   VDN_ERR_ARCH = 5,         /* the device is not compute capability 10.x                              */
-  VDN_ERR_TIMEOUT = 6       /* a bounded device-side wait expired (reported by vdn_vda_status)        */
+  VDN_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired (reported by vdn_vda_status)        */
+  VDN_ERR_INTERNAL = 7      /* a kernel found its shared-memory window unusable and did nothing       */
+                            /* (reported by vdn_vda_status)                                           */
 } vdn_status;
 
 typedef enum { VDN_F32 = 0, VDN_BF16 = 1 } vdn_dtype;
@@ -112,7 +115,7 @@ vdn_status vdn_vda_create(const vdn_vda_config* cfg, vdn_vda_t* out_handle);
  * inverses of Eq. 5 and the scanned states of Eq. A.1 live there).  Pure function; 0 on invalid shape. */
 size_t vdn_vda_workspace_bytes(vdn_vda_t h, int B, int T, int F, int H, int d);
 
-/* Hands the library a caller-owned device buffer (256-byte aligned).  It must stay valid until replaced
+/* Plumbing (no passage of the paper to cite).  Hands the library a caller-owned device buffer (256-byte aligned).  It must stay valid until replaced
  * or until the handle is destroyed, and must not be shared between handles that run concurrently. */
 vdn_status vdn_vda_set_workspace(vdn_vda_t h, void* dev_ptr, size_t bytes);
 
@@ -122,9 +125,8 @@ vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void
                            const float* gate, void* out, int B, int T, int F, int H, int d,
                            void* cuda_stream);
 
-/* The same layer with the two inputs of the paper's recurrence that vdn_vda_forward fixes (first item of the
- * "next" list; the local window is still the query frame itself, and there are no anchor frames -- see
- * vdn_vda_forward_opt for those):
+/* The same layer with the two inputs of the paper's recurrence that vdn_vda_forward fixes (the local window is
+ * still the query frame itself, and there are no anchor frames -- see vdn_vda_forward_opt for those):
  *   alpha [B,T,H,d] float, DEVICE, in [0,1], or NULL (= 1): channel-wise decay gate of frame t (Eq. 2, Eq. A.1:
  *         M_t = Diag(alpha_t)(I + A_t)^{-1}).  It decays the inherited state before frame t is folded in, in both
  *         scans, and bridges the state that frame t's queries read (Eq. A.4 with l_t = h_t = t):
@@ -238,6 +240,21 @@ vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const
                                 const float* beta, const float* gate, void* out, int B, int T, int F,
                                 int H, int d, void* cuda_stream);
 
+/* vdn_vda_forward_host with the optional inputs of vdn_vda_forward_opt (the release setting of Sec. A.4 and Alg. 1
+ * end to end from host memory).  Here every pointer inside `opt` is a HOST pointer as well (alpha, s0, norm_weight,
+ * gate_elem; same shapes as for vdn_vda_forward_opt); they are copied into the staging buffer with the other inputs,
+ * gate_elem in the same groups of frames as the queries.  The staging buffer must hold
+ * vdn_vda_staging_bytes_opt(..., opt) bytes (vdn_vda_staging_bytes plus room for alpha, s0 and norm_weight, plus one
+ * tensor of the size of q when opt->gate_elem is set).  `opt` may be NULL (= vdn_vda_forward_host); `gate` may be
+ * NULL when opt->gate_elem is set.  All host-side checks (arguments, workspace, staging) are made before the first
+ * copy is queued; should a CUDA call fail after that, cuda_stream is made to wait for everything already queued on
+ * the handle's own streams before the error is returned, so synchronising cuda_stream still releases the caller's
+ * buffers. */
+size_t vdn_vda_staging_bytes_opt(vdn_vda_t h, int B, int T, int F, int H, int d, const vdn_vda_options* opt);
+vdn_status vdn_vda_forward_host_opt(vdn_vda_t h, const void* q, const void* k, const void* v,
+                                    const float* beta, const float* gate, void* out, int B, int T, int F,
+                                    int H, int d, const vdn_vda_options* opt, void* cuda_stream);
+
 /* Offset and size, inside the workspace, of an intermediate of the last forward call of this shape
  * (see vdn_view).  For stage-wise parity checks; the contents are valid after the stream is synchronised. */
 vdn_status vdn_vda_workspace_view(vdn_vda_t h, int which, int B, int T, int F, int H, int d,
@@ -276,6 +293,8 @@ int vdn_vda_kernel_times(vdn_vda_t h, int max_kernels, const char** names, float
  * enqueued.  errbuf (HOST, may be NULL) receives a NUL-terminated description of any error.
  * The first call on a device looks up the array's address on that device (cudaGetSymbolAddress); make that
  * first call outside any stream capture.  Enqueues on cuda_stream and returns without synchronising.
+ * The looked-up address is cached per device in an atomic pointer: host threads that make their first calls at
+ * the same time each do the lookup and store the same value, which is harmless.
  * Every call on a device uses the same array: two calls whose kernels may overlap on the GPU (different
  * streams, or different host threads) race on it -- serialise them.  The array keeps the previous call's
  * contents; the kernel writes every element it later reads, so nothing has to be cleared in between. */
@@ -283,13 +302,37 @@ int vdn_vda_kernel_times(vdn_vda_t h, int max_kernels, const char** names, float
 vdn_status vdn_vda_scan_static(const float* stats, const float* inv, float* read, int BH, int T, int d,
                                int device, void* cuda_stream, char* errbuf, size_t errbuf_len);
 
-/* Last device-side status recorded by this handle's kernels (VDN_OK or VDN_ERR_TIMEOUT).  Does not
- * synchronise: call it after synchronising the stream.  Reading it clears nothing. */
+/* Plumbing (no passage of the paper to cite).  Last device-side status recorded by this handle's kernels: VDN_OK,
+ * VDN_ERR_TIMEOUT (a wait inside a kernel ran out; that kernel's CTA stopped early and the outputs of the call are
+ * incomplete) or VDN_ERR_INTERNAL.  Does not synchronise: call it after synchronising the stream.  The word is
+ * sticky: reading it clears nothing, and no forward call clears it, so that an error is not lost between a call
+ * and the moment the caller looks.  vdn_vda_clear_status resets it. */
 vdn_status vdn_vda_status(vdn_vda_t h);
 
-/* Human-readable description of the last error returned on this handle (never NULL). */
+/* Plumbing.  Returns what vdn_vda_status would return and resets the status word to VDN_OK.  Call it with no
+ * kernel of this handle in flight (after synchronising): a kernel that is still running may set the word again.
+ * After a timeout the handle stays usable: the kernels keep no state between calls. */
+vdn_status vdn_vda_clear_status(vdn_vda_t h);
+
+/* Plumbing.  The longest any single wait inside a kernel of this handle may take before its CTA gives up
+ * (default 2 s = 2 000 000 microseconds; 1 microsecond .. 1 hour).  A wait covers one pipeline hand-over (a tile
+ * arriving, an accumulator being drained), never a whole kernel, so the default is generous for any shape. */
+vdn_status vdn_vda_set_wait_limit_us(vdn_vda_t h, unsigned long long microseconds);
+
+/* Test support (no counterpart in the paper): exercises the give-up path of the bounded waits without touching
+ * any pipeline.  Enqueues one small kernel that is set up like the tensor-core kernels (mbarrier, tensor memory,
+ * the same wait routine) and waits, for at most limit_us microseconds (<= 1 s), on a barrier that nothing ever
+ * completes and that no copy is bound to.  The wait runs out, the CTA takes the same abort and teardown path as
+ * the real kernels (frees its tensor memory, returns) and records VDN_ERR_TIMEOUT in the handle's status word.
+ * After synchronising: vdn_vda_status gives VDN_ERR_TIMEOUT and vdn_vda_selftest_marker gives 1 (the CTA reached
+ * its last instruction after giving up; 0 = the kernel has not run, -1 = null handle). */
+vdn_status vdn_vda_selftest_wait_expiry(vdn_vda_t h, unsigned long long limit_us, void* cuda_stream);
+int vdn_vda_selftest_marker(vdn_vda_t h);
+
+/* Plumbing.  Human-readable description of the last error returned on this handle (never NULL). */
 const char* vdn_vda_last_error(vdn_vda_t h);
 
+/* Plumbing.  Frees the handle's host state, streams and events.  No kernel of the handle may be in flight. */
 vdn_status vdn_vda_destroy(vdn_vda_t h);
 
 #ifdef __cplusplus

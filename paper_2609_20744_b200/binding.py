@@ -11,11 +11,12 @@ import os
 from typing import Optional
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libvdn_vda.so")
+LIB_PATH = os.environ.get("VDN_VDA_LIB") or os.path.join(_HERE, "libvdn_vda.so")   # VDN_VDA_LIB: another build of the library
 
 VDN_OK = 0
 STATUS_NAMES = {0: "VDN_OK", 1: "VDN_ERR_INVALID_ARG", 2: "VDN_ERR_UNSUPPORTED", 3: "VDN_ERR_WORKSPACE",
-                4: "VDN_ERR_CUDA", 5: "VDN_ERR_ARCH", 6: "VDN_ERR_TIMEOUT"}
+                4: "VDN_ERR_CUDA", 5: "VDN_ERR_ARCH", 6: "VDN_ERR_TIMEOUT", 7: "VDN_ERR_INTERNAL"}
+VDN_ERR_TIMEOUT, VDN_ERR_INTERNAL = 6, 7
 VDN_F32, VDN_BF16 = 0, 1
 VDN_FLAG_FORCE_SIMT = 1
 VDN_FLAG_ADDITIVE_RULE = 4
@@ -26,8 +27,11 @@ VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_R
 EXPORTS = (
     "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward", "vdn_vda_forward_ex",
     "vdn_vda_forward_opt", "vdn_vda_workspace_bytes_opt", "vdn_vda_prepare",
-    "vdn_vda_staging_bytes", "vdn_vda_set_staging", "vdn_vda_forward_host", "vdn_vda_workspace_view",
-    "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_scan_static", "vdn_vda_status", "vdn_vda_last_error", "vdn_vda_destroy",
+    "vdn_vda_staging_bytes", "vdn_vda_staging_bytes_opt", "vdn_vda_set_staging", "vdn_vda_forward_host",
+    "vdn_vda_forward_host_opt", "vdn_vda_workspace_view",
+    "vdn_vda_last_launch_count", "vdn_vda_profile", "vdn_vda_kernel_times", "vdn_vda_scan_static", "vdn_vda_status",
+    "vdn_vda_clear_status", "vdn_vda_set_wait_limit_us", "vdn_vda_selftest_wait_expiry", "vdn_vda_selftest_marker",
+    "vdn_vda_last_error", "vdn_vda_destroy",
 )
 
 
@@ -93,6 +97,18 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.vdn_vda_prepare.restype = ci
     lib.vdn_vda_forward_host.argtypes = fwd_args
     lib.vdn_vda_forward_host.restype = ci
+    lib.vdn_vda_forward_host_opt.argtypes = [vp, vp, vp, vp, vp, vp, vp, *shape, ctypes.POINTER(VdnOptions), vp]
+    lib.vdn_vda_forward_host_opt.restype = ci
+    lib.vdn_vda_staging_bytes_opt.argtypes = [vp, *shape, ctypes.POINTER(VdnOptions)]
+    lib.vdn_vda_staging_bytes_opt.restype = sz
+    lib.vdn_vda_clear_status.argtypes = [vp]
+    lib.vdn_vda_clear_status.restype = ci
+    lib.vdn_vda_set_wait_limit_us.argtypes = [vp, ctypes.c_ulonglong]
+    lib.vdn_vda_set_wait_limit_us.restype = ci
+    lib.vdn_vda_selftest_wait_expiry.argtypes = [vp, ctypes.c_ulonglong, vp]
+    lib.vdn_vda_selftest_wait_expiry.restype = ci
+    lib.vdn_vda_selftest_marker.argtypes = [vp]
+    lib.vdn_vda_selftest_marker.restype = ci
     lib.vdn_vda_workspace_view.argtypes = [vp, ci, *shape, ctypes.POINTER(sz), ctypes.POINTER(sz)]
     lib.vdn_vda_workspace_view.restype = ci
     lib.vdn_vda_last_launch_count.argtypes = [vp]
@@ -145,6 +161,58 @@ def scan_static(stats, inv, read, stream=None):
     return read
 
 
+def _require(name, x, shape, dtype, on_cuda, device_index):
+    """One tensor argument against what the C ABI will assume about it (the library sees only a pointer)."""
+    if x is None:
+        raise ValueError(f"{name} is missing")
+    where = "CUDA" if on_cuda else "host"
+    if bool(x.is_cuda) != on_cuda:
+        raise ValueError(f"{name} must be a {where} tensor")
+    if on_cuda and (x.device.index or 0) != device_index:
+        raise ValueError(f"{name} is on cuda:{x.device.index}, the handle is bound to cuda:{device_index}")
+    if not x.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if x.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {x.dtype}")
+    if tuple(x.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(x.shape)}")
+
+
+def validate_layer_args(io_dtype, d_handle, device_index, q, k, v, beta, gate, out=None, alpha=None, s0=None,
+                        gate_elem=None, norm_weight=None, on_cuda=True):
+    """Checks every tensor of a forward call before anything reaches the library: dtype, shape, device and
+    contiguity.  The kernels and the TMA tensor maps index by the shape that is passed, so a tensor of another dtype
+    or a shorter one would be read (and `out` written) past its end.  Raises ValueError; returns (B, T, F, H, d).
+
+    io_dtype is the torch dtype of the handle's q, k, v, out; on_cuda = False checks host tensors instead
+    (the host-buffer entry point)."""
+    import torch
+    if q is None or q.dim() != 5:
+        raise ValueError("q must have shape [B, T, F, H, d]")
+    B, T, F, H, d = (int(n) for n in q.shape)
+    del d_handle                      # a head dimension other than the handle's is the library's to refuse
+    f32 = torch.float32
+    _require("q", q, (B, T, F, H, d), io_dtype, on_cuda, device_index)
+    _require("k", k, (B, T, F, H, d), io_dtype, on_cuda, device_index)
+    _require("v", v, (B, T, F, H, d), io_dtype, on_cuda, device_index)
+    _require("beta", beta, (B, T, F, H), f32, on_cuda, device_index)
+    if gate is None and gate_elem is None:
+        raise ValueError("gate may only be left out when gate_elem is given")
+    if gate is not None:
+        _require("gate", gate, (H,), f32, on_cuda, device_index)
+    if out is not None:
+        _require("out", out, (B, T, F, H, d), io_dtype, on_cuda, device_index)
+    if alpha is not None:
+        _require("alpha", alpha, (B, T, H, d), f32, on_cuda, device_index)
+    if s0 is not None:
+        _require("s0", s0, (B, H, d, d), f32, on_cuda, device_index)
+    if gate_elem is not None:
+        _require("gate_elem", gate_elem, (B, T, F, H, d), io_dtype, on_cuda, device_index)
+    if norm_weight is not None:
+        _require("norm_weight", norm_weight, (H, d), f32, on_cuda, device_index)
+    return B, T, F, H, d
+
+
 class Vda:
     """One handle of the library (vdn_vda_create .. vdn_vda_destroy) plus its torch-owned workspace."""
 
@@ -154,6 +222,7 @@ class Vda:
         self.lib = load_library()
         self.d = d
         self.dtype = dtype
+        self.torch_dtype = torch.float32 if dtype == "f32" else torch.bfloat16
         self.device = device
         cfg = VdnConfig(ctypes.sizeof(VdnConfig), VDN_F32 if dtype == "f32" else VDN_BF16, d, rms_eps, flags, device)
         self.h = ctypes.c_void_p()
@@ -190,9 +259,12 @@ class Vda:
             self._check(self.lib.vdn_vda_set_workspace(self.h, ctypes.c_void_p(self._ws.data_ptr()), need))
         return self._ws
 
-    def ensure_staging(self, B, T, F, H):
+    def ensure_staging(self, B, T, F, H, opt=None):
         torch = self._torch
-        need = int(self.lib.vdn_vda_staging_bytes(self.h, B, T, F, H, self.d))
+        if opt is None:
+            need = int(self.lib.vdn_vda_staging_bytes(self.h, B, T, F, H, self.d))
+        else:
+            need = int(self.lib.vdn_vda_staging_bytes_opt(self.h, B, T, F, H, self.d, ctypes.byref(opt)))
         if need == 0:
             raise VdnError(1, "invalid shape")
         if self._staging is None or self._staging.numel() < need:
@@ -211,23 +283,8 @@ class Vda:
         normalisation; the read-out applies it) it goes to vdn_vda_forward_opt.
         """
         torch = self._torch
-        B, T, F, H, d = q.shape
-        extras = [x for x in (alpha, s0, norm_weight) if x is not None]
-        for x in (q, k, v, beta, *([gate] if gate is not None else []), *([gate_elem] if gate_elem is not None else []),
-                  *extras):
-            if not (x.is_cuda and x.is_contiguous()):
-                raise ValueError("vdn_vda_forward needs contiguous CUDA tensors")
-        for x in extras:
-            if x.dtype != torch.float32:
-                raise ValueError("alpha, s0 and norm_weight must be float32")
-        if alpha is not None and tuple(alpha.shape) != (B, T, H, d):
-            raise ValueError("alpha must be [B, T, H, d]")
-        if s0 is not None and tuple(s0.shape) != (B, H, d, d):
-            raise ValueError("s0 must be [B, H, d, d]")
-        if norm_weight is not None and tuple(norm_weight.shape) != (H, d):
-            raise ValueError("norm_weight must be [H, d]")
-        if gate_elem is not None and (tuple(gate_elem.shape) != (B, T, F, H, d) or gate_elem.dtype != q.dtype):
-            raise ValueError("gate_elem must be [B, T, F, H, d] of the I/O dtype")
+        B, T, F, H, d = validate_layer_args(self.torch_dtype, self.d, self.device, q, k, v, beta, gate, out, alpha, s0,
+                                            gate_elem, norm_weight)
         if out is None:
             out = torch.empty_like(q)
         self.ensure_workspace(B, T, F, H, chunk)
@@ -256,18 +313,22 @@ class Vda:
         to the read-out (forward(..., q_l2_eps=l2_eps)) and the first element of the result is None.
         """
         torch = self._torch
-        B, T, F, H, d = k.shape
+        if k is None or k.dim() != 5:
+            raise ValueError("k must have shape [B, T, F, H, d]")
+        B, T, F, H, d = (int(n) for n in k.shape)
         names = ("wk_spatial", "wk_temporal", "wv_spatial", "wv_temporal")
         given = [n for n in names if filters.get(n) is not None]      # spatial filters may be left out (identity)
-        for x in (*([q] if q is not None else []), k, v, *(filters[n] for n in given)):
-            if not (x.is_cuda and x.is_contiguous()):
-                raise ValueError("vdn_vda_prepare needs contiguous CUDA tensors")
+        for n, x in (("q", q), ("k", k), ("v", v)):
+            if x is not None:
+                _require(n, x, (B, T, F, H, d), self.torch_dtype, True, self.device)
         for n in given:
             want = (H * d, 5, 5) if n.endswith("spatial") else (H * d, 5)
-            if tuple(filters[n].shape) != want or filters[n].dtype != torch.float32:
-                raise ValueError(f"{n} must be float32 {want}")
+            _require(n, filters[n], want, torch.float32, True, self.device)
         qo, ko, vo = out if out is not None else (torch.empty_like(q) if q is not None else None,
                                                   torch.empty_like(k), torch.empty_like(v))
+        for n, x in (("q_out", qo), ("k_out", ko), ("v_out", vo)):
+            if x is not None:
+                _require(n, x, (B, T, F, H, d), self.torch_dtype, True, self.device)
         p = lambda x: ctypes.c_void_p(x.data_ptr()) if x is not None else None
         prm = VdnPrepParams(ctypes.sizeof(VdnPrepParams), Y, X, 1 if anchors else 0, l2_eps,
                             *(filters[n].data_ptr() if filters.get(n) is not None else None for n in names))
@@ -275,17 +336,27 @@ class Vda:
                                              ctypes.byref(prm), self._stream(stream)))
         return qo, ko, vo
 
-    def forward_host(self, q, k, v, beta, gate, out, stream=None):
-        """vdn_vda_forward_host on HOST tensors (pinned recommended); `out` is a host tensor too."""
-        B, T, F, H, d = q.shape
-        for x in (q, k, v, beta, gate, out):
-            if x.is_cuda or not x.is_contiguous():
-                raise ValueError("vdn_vda_forward_host needs contiguous host tensors")
-        self.ensure_workspace(B, T, F, H)
-        self.ensure_staging(B, T, F, H)
-        p = lambda x: ctypes.c_void_p(x.data_ptr())
-        self._check(self.lib.vdn_vda_forward_host(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
-                                                  B, T, F, H, d, self._stream(stream)))
+    def forward_host(self, q, k, v, beta, gate, out, stream=None, alpha=None, s0=None, chunk=1, radius=0,
+                     anchors=False, gate_elem=None, norm_weight=None, q_l2_eps=0.0):
+        """vdn_vda_forward_host(_opt) on HOST tensors (pinned recommended); `out` and every optional input are host
+        tensors too.  The keyword arguments are those of forward()."""
+        B, T, F, H, d = validate_layer_args(self.torch_dtype, self.d, self.device, q, k, v, beta, gate, out, alpha, s0,
+                                            gate_elem, norm_weight, on_cuda=False)
+        self.ensure_workspace(B, T, F, H, chunk)
+        p = lambda x: ctypes.c_void_p(x.data_ptr()) if x is not None else None
+        a = lambda x: x.data_ptr() if x is not None else None
+        plain = (chunk, radius, bool(anchors)) == (1, 0, False) and gate is not None and not q_l2_eps and \
+            all(x is None for x in (alpha, s0, gate_elem, norm_weight))
+        opt = VdnOptions(ctypes.sizeof(VdnOptions), chunk, radius, 1 if anchors else 0, a(alpha), a(s0),
+                         a(gate_elem), a(norm_weight), float(q_l2_eps), 0)
+        self.ensure_staging(B, T, F, H, None if plain else opt)
+        if plain:
+            st = self.lib.vdn_vda_forward_host(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
+                                               B, T, F, H, d, self._stream(stream))
+        else:
+            st = self.lib.vdn_vda_forward_host_opt(self.h, p(q), p(k), p(v), p(beta), p(gate), p(out),
+                                                   B, T, F, H, d, ctypes.byref(opt), self._stream(stream))
+        self._check(st)
         return out
 
     # -- inspection ---------------------------------------------------------------------------
@@ -329,6 +400,21 @@ class Vda:
 
     def status(self) -> int:
         return int(self.lib.vdn_vda_status(self.h))
+
+    def clear_status(self) -> int:
+        """Resets the sticky device-side status word; returns what it held."""
+        return int(self.lib.vdn_vda_clear_status(self.h))
+
+    def set_wait_limit_us(self, microseconds: int):
+        """Longest single wait inside a kernel before its CTA gives up (default 2 s)."""
+        self._check(self.lib.vdn_vda_set_wait_limit_us(self.h, int(microseconds)))
+
+    def selftest_wait_expiry(self, limit_us: int = 1000, stream=None):
+        """Enqueues the stand-alone kernel whose wait runs out (see vdn_vda_selftest_wait_expiry)."""
+        self._check(self.lib.vdn_vda_selftest_wait_expiry(self.h, int(limit_us), self._stream(stream)))
+
+    def selftest_marker(self) -> int:
+        return int(self.lib.vdn_vda_selftest_marker(self.h))
 
     def close(self):
         if getattr(self, "h", None):

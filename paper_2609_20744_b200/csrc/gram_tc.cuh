@@ -43,7 +43,7 @@ struct GramTc {
 
 __global__ void __launch_bounds__(GramTc::THREADS, 1)
 gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-               const float* __restrict__ beta, float* __restrict__ stats, Shape s, int* status) {
+               const float* __restrict__ beta, float* __restrict__ stats, Shape s, tc::DevStatus ds) {
   using namespace tc;
   using G = GramTc;
   extern __shared__ unsigned char smem_dyn[];
@@ -60,11 +60,11 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   auto ACCEMPTY = [&](int i) { return bar0 + 8u * (12 + i); }; // 2
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + G::OFF_BAR + 8 * 14);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + G::OFF_BAR + 8 * 14 + 4);
-  const WaitCtx wc{abort_flag, status};
+  const WaitCtx wc(abort_flag, ds);
 
   if ((base - smem_u32(smem_dyn)) + G::USED_BYTES > (uint32_t)G::SMEM_BYTES) {
     // the dynamic shared memory window starts too far from a 1024-byte boundary for the layout to fit
-    if (threadIdx.x == 0) atomicExch(status, kStatusTimeout);
+    if (threadIdx.x == 0) atomicExch(ds.word, kStatusInternal);
     return;
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

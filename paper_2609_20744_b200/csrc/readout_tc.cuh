@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(ReadoutTcCfg<EXTRAS, QNORM, GATE>::THREADS, 1)
 readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmS,
                   const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmG,
                   const float* __restrict__ gate, Shape s, float eps,
-                  int* status, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight,
+                  tc::DevStatus ds, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight,
                   Window win, int bridged, float q_l2_eps) {
   using namespace tc;
   using R = ReadoutTcCfg<EXTRAS, QNORM, GATE>;
@@ -81,11 +81,11 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 8 * 25);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 8 * 25 + 8);
   constexpr uint32_t QS = R::QSLOTS;
-  const WaitCtx wc{abort_flag, status};
+  const WaitCtx wc(abort_flag, ds);
 
   if ((base - smem_u32(smem_dyn)) + R::USED_BYTES > (uint32_t)R::SMEM_BYTES) {
     // the dynamic shared memory window starts too far from a 1024-byte boundary for the layout to fit
-    if (threadIdx.x == 0) atomicExch(status, kStatusTimeout);
+    if (threadIdx.x == 0) atomicExch(ds.word, kStatusInternal);
     return;
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -56,7 +56,7 @@ struct ResolveTc {
 
 __global__ void __launch_bounds__(ResolveTc::THREADS, 4)
 resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ csplit, long long nframes,
-                  int* status, Shape shp) {
+                  tc::DevStatus ds, Shape shp) {
   using namespace tc;
   using R = ResolveTc;
   constexpr int D = R::D;
@@ -68,7 +68,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + R::OFF_BAR + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + R::OFF_BAR + 36);
   float* gi = reinterpret_cast<float*>(base_ptr + R::OFF_GI);
-  const WaitCtx wc{abort_flag, status};
+  const WaitCtx wc(abort_flag, ds);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long n = blockIdx.x;

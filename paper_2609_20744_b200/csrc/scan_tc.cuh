@@ -87,7 +87,7 @@ __host__ __device__ inline int scan_chunk_steps(const Window& w, int dir) {
 // the state warps (launch it with threads(NS) threads) and issues MMAs of N = 64.
 template <int MODE, int NS = 1>
 __global__ void __launch_bounds__(ScanTc::THREADS, 1)
-scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int* status) {
+scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::DevStatus ds) {
   using namespace tc;
   using S = ScanTc;
   constexpr int D = S::D;
@@ -101,7 +101,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, int*
   const uint32_t XREADY = bar0 + 48, ACCFULL = bar0 + 56;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + S::OFF_BAR + 64);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + S::OFF_BAR + 72);
-  const WaitCtx wc{abort_flag, status};
+  const WaitCtx wc(abort_flag, ds);
 
   const Window& win = a.win;
   const int T = a.T;

@@ -9,7 +9,15 @@
 namespace vdn {
 namespace tc {
 
-constexpr int kStatusTimeout = 6;  // mirrors VDN_ERR_TIMEOUT
+constexpr int kStatusTimeout = 6;   // mirrors VDN_ERR_TIMEOUT
+constexpr int kStatusInternal = 7;  // mirrors VDN_ERR_INTERNAL
+
+// What every tensor-core kernel is handed for error reporting: the handle's host-mapped status word and the
+// time any single wait may take before the CTA gives up.
+struct DevStatus {
+  int* word;
+  unsigned long long wait_ns;
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -50,12 +58,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Every wait in these kernels goes through here.  It gives up after ~2 s of wall time (or as soon as
-// another thread of the CTA has given up), records the timeout in the host-visible status word and
-// raises the CTA-wide abort flag, after which every role leaves its loops and the CTA tears down.
+// Every wait in these kernels goes through here.  It gives up after limit_ns of wall time (2 s unless the
+// caller of the library chose otherwise), or as soon as another thread of the CTA has given up; it then records
+// the timeout in the host-visible status word and raises the CTA-wide abort flag, after which every role leaves
+// its loops and the CTA tears down.
 struct WaitCtx {
   volatile int* abort_flag;  // shared memory
   int* status;               // host-mapped status word
+  unsigned long long limit_ns;
+  __device__ WaitCtx(volatile int* f, const DevStatus& ds) : abort_flag(f), status(ds.word), limit_ns(ds.wait_ns) {}
 };
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -64,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 0u) {
       if (*w.abort_flag) return false;
-      if (global_timer_ns() - t0 > 2000000000ull) {
+      if (global_timer_ns() - t0 > w.limit_ns) {
         *w.abort_flag = 1;
         atomicExch(w.status, kStatusTimeout);
         return false;

@@ -8,6 +8,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <atomic>
 #include <cstring>
 #include <new>
 #include <string>
@@ -22,6 +23,7 @@
 #include "resolve_tc.cuh"
 #include "scan.cuh"
 #include "scan_tc.cuh"
+#include "wait_selftest.cuh"
 
 namespace {
 
@@ -42,7 +44,7 @@ struct Layout {
 };
 
 struct StagingLayout {
-  size_t q, k, v, out, beta, gate, total;
+  size_t q, k, v, out, beta, gate, alpha, s0, norm_weight, gate_elem, total;
 };
 
 // The optional inputs of vdn_vda_forward_opt, checked and with defaults filled in.
@@ -86,8 +88,9 @@ struct vdn_vda_s {
   size_t workspace_bytes = 0;
   void* staging = nullptr;
   size_t staging_bytes = 0;
-  int* status_host = nullptr;  // pinned, device-mapped
+  int* status_host = nullptr;  // pinned, device-mapped: word 0 = status, word 1 = marker of the wait self-test
   int* status_dev = nullptr;
+  unsigned long long wait_ns = 2000000000ull;   // limit of any single device-side wait
   int launches = 0;
   bool attrs_set = false;
   bool tc_attrs_set = false;
@@ -109,6 +112,8 @@ vdn_status fail(vdn_vda_t h, vdn_status st, const std::string& msg) {
   if (h) h->err = msg;
   return st;
 }
+
+vdn::tc::DevStatus dev_status(const vdn_vda_s* h) { return vdn::tc::DevStatus{h->status_dev, h->wait_ns}; }
 
 // bf16 I/O with d = 128 runs on the tcgen05 kernels unless the handle asks for the plain-fp32 ones.
 bool use_tensor_cores(const vdn_vda_s* h, int d) {
@@ -151,7 +156,7 @@ Layout make_layout(const vdn_vda_s* h, int B, int T, int H, int d, int chunk = 1
   return L;
 }
 
-StagingLayout make_staging(const vdn_vda_s* h, int B, int T, int F, int H, int d) {
+StagingLayout make_staging(const vdn_vda_s* h, int B, int T, int F, int H, int d, bool with_gate_elem = false) {
   const size_t tokh = (size_t)B * T * F * H;
   const size_t big = align_up(tokh * d * elem_size(h));
   StagingLayout S;
@@ -162,6 +167,11 @@ StagingLayout make_staging(const vdn_vda_s* h, int B, int T, int F, int H, int d
   S.out = off; off += big;
   S.beta = off; off += align_up(tokh * sizeof(float));
   S.gate = off; off += align_up((size_t)H * sizeof(float));
+  // the optional inputs of vdn_vda_forward_host_opt: the small ones always have their place
+  S.alpha = off; off += align_up((size_t)B * T * H * d * sizeof(float));
+  S.s0 = off; off += align_up((size_t)B * H * d * d * sizeof(float));
+  S.norm_weight = off; off += align_up((size_t)H * d * sizeof(float));
+  S.gate_elem = off; if (with_gate_elem) off += big;
   S.total = off;
   return S;
 }
@@ -355,7 +365,7 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   if (x.phase != 2) {
     prof_begin(h, st);
     vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
-                                                                                         h->status_dev);
+                                                                                         dev_status(h));
     prof_mark(h, st, nk++, "gram_tc");
     const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
     const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
@@ -364,7 +374,7 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
       prof_mark(h, st, nk++, "additive_transition");
     } else {
       vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
-          stats, csplit, n, h->status_dev, s);
+          stats, csplit, n, dev_status(h), s);
       prof_mark(h, st, nk++, "resolve_tc");
     }
     vdn::ScanTcArgs sa{};
@@ -378,19 +388,19 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
       CUtensorMap tmM;
       if ((r = make_matrix_map(h, &tmM, sa.comp_m, (long long)3 * s.B * s.H * 2 * sa.nseg * D)) != VDN_OK) return r;
       vdn::scan_tc_kernel<vdn::SCAN_COMPOSE><<<(unsigned)(4 * s.B * s.H * sa.nseg), vdn::ScanTc::THREADS,
-                                               vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
+                                               vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, dev_status(h));
       prof_mark(h, st, nk++, "compose_tc");
       vdn::scan_tc_kernel<vdn::SCAN_CHUNKS><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
-                                              vdn::ScanTc::SMEM_BYTES, st>>>(tmM, sa, h->status_dev);
+                                              vdn::ScanTc::SMEM_BYTES, st>>>(tmM, sa, dev_status(h));
       prof_mark(h, st, nk++, "scan_chunks_tc");
     } else if (4LL * s.B * s.H <= h->sm_count) {
       // few chains: two CTAs per chain, half of the value columns each
       vdn::scan_tc_kernel<vdn::SCAN_FRAMES, 2><<<(unsigned)(4 * s.B * s.H), vdn::ScanTc::threads(2),
-                                                 vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
+                                                 vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, dev_status(h));
       prof_mark(h, st, nk++, "scan_tc");
     } else {
       vdn::scan_tc_kernel<vdn::SCAN_FRAMES><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
-                                              vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, h->status_dev);
+                                              vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, dev_status(h));
       prof_mark(h, st, nk++, "scan_tc");
     }
     h->launches = nk;
@@ -422,7 +432,7 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
       h->ro_attrs_set |= bit;
     }
     vdn::readout_tc_kernel<EX, QN, GE><<<persistent_ro, RX::THREADS, RX::SMEM_BYTES, st>>>(
-        tmQ, tmS, tmO, tmG, gate, sr, h->cfg.rms_eps, h->status_dev, static_cast<const __nv_bfloat16*>(x.gate_elem),
+        tmQ, tmS, tmO, tmG, gate, sr, h->cfg.rms_eps, dev_status(h), static_cast<const __nv_bfloat16*>(x.gate_elem),
         x.norm_weight, x.win, x.alpha != nullptr, x.q_l2_eps);
     return true;
   };
@@ -451,7 +461,10 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
 constexpr size_t kStaticScanFloats = VDN_SCAN_STATIC_MAX_BYTES / sizeof(float);
 static __device__ __align__(256) float g_scan_static_scratch[kStaticScanFloats];
 constexpr int kMaxDevices = 64;
-float* g_scan_static_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+// Device address of the array, per device ordinal.  Host threads may race to fill an entry; every one of them
+// would store the same value (the lookup is a pure function of the device), and the atomic makes the publication
+// well defined.
+std::atomic<float*> g_scan_static_ptr[kMaxDevices];
 
 void put_msg(char* buf, size_t len, const std::string& msg) {
   if (!buf || len == 0) return;
@@ -587,6 +600,13 @@ size_t vdn_vda_staging_bytes(vdn_vda_t h, int B, int T, int F, int H, int d) {
   return make_staging(h, B, T, F, H, d).total;
 }
 
+size_t vdn_vda_staging_bytes_opt(vdn_vda_t h, int B, int T, int F, int H, int d, const vdn_vda_options* opt) {
+  std::string why;
+  if (!h || !shape_ok(h, B, T, F, H, d, &why)) return 0;
+  if (opt && opt->struct_size != sizeof(vdn_vda_options)) return 0;
+  return make_staging(h, B, T, F, H, d, opt && opt->gate_elem).total;
+}
+
 vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes) {
   if (!h) return VDN_ERR_INVALID_ARG;
   if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) != 0)
@@ -600,14 +620,12 @@ vdn_status vdn_vda_set_staging(vdn_vda_t h, void* dev_ptr, size_t bytes) {
 
 namespace {
 
-// The layer, whole (phase 0) or in the two pieces vdn_vda_forward_host interleaves with its copies (phase 1:
-// statistics, resolve, scans; phase 2: read-out of frames ro_first .. ro_first + ro_count - 1).
-vdn_status forward_core(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+// Everything about a forward call that the host can check, checked, and the call laid out: nothing is enqueued
+// and no CUDA call is made.  Fills x (optional inputs with defaults, window), L (workspace layout), s (shape).
+vdn_status plan_forward(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
                         const float* gate, void* out, int B, int T, int F, int H, int d,
-                        const vdn_vda_options* opt, void* cuda_stream, int phase, int ro_first, int ro_count) {
+                        const vdn_vda_options* opt, Extras& x, Layout& L, Shape& s) {
   if (!h) return VDN_ERR_INVALID_ARG;
-  Extras x;
-  x.phase = phase;
   if (opt) {
     if (opt->struct_size != sizeof(vdn_vda_options))
       return fail(h, VDN_ERR_INVALID_ARG, "vdn_vda_options.struct_size does not match this library");
@@ -637,9 +655,11 @@ vdn_status forward_core(vdn_vda_t h, const void* q, const void* k, const void* v
   // The scanned frames: all of them, or the interior ones when frames 0 and T-1 are boundary anchors.
   x.win.first = x.anchors ? 1 : 0;
   x.win.last = x.anchors ? T - 2 : T - 1;
-  Layout L = make_layout(h, B, T, H, d);
+  L = make_layout(h, B, T, H, d);
   if (!h->workspace || h->workspace_bytes < L.total)
     return fail(h, VDN_ERR_WORKSPACE, "workspace not set or smaller than vdn_vda_workspace_bytes");
+  if (use_tensor_cores(h, d) && !h->encode)
+    return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   if (use_tensor_cores(h, d) && x.win.chunk >= 2 && x.win.last >= x.win.first &&
       !(h->cfg.flags & VDN_FLAG_SCAN_FRAMEWISE)) {
     // Chunk-wise scan (Sec. 5): worth it when the chains leave most SMs idle.  Costs in scan steps: one chain
@@ -659,10 +679,18 @@ vdn_status forward_core(vdn_vda_t h, const void* q, const void* k, const void* v
       L = Lc;
     }
   }
-  DeviceGuard guard(h->cfg.device);
-  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const Shape s{B, T, F, H, d, x.win.first, x.win.last - x.win.first + 1};
+  s = Shape{B, T, F, H, d, x.win.first, x.win.last - x.win.first + 1};
+  return VDN_OK;
+}
+
+// Enqueues a planned call, whole (phase 0) or in the two pieces vdn_vda_forward_host interleaves with its copies
+// (phase 1: statistics, resolve, scans; phase 2: read-out of frames ro_first .. ro_first + ro_count - 1).
+// The handle's device is current.
+vdn_status run_forward(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
+                       const float* gate, void* out, Extras x, const Layout& L, const Shape& s, cudaStream_t st,
+                       int phase, int ro_first, int ro_count) {
+  const int B = s.B, T = s.T, F = s.F, H = s.H, d = s.d;
+  x.phase = phase;
   if (phase == 2) {
     // clip the requested frames to the scanned ones (anchor rows were zeroed in phase 1)
     const int lo = ro_first > x.win.first ? ro_first : x.win.first;
@@ -681,8 +709,8 @@ vdn_status forward_core(vdn_vda_t h, const void* q, const void* k, const void* v
       VDN_CUDA(h, cudaMemsetAsync(o + (size_t)b * T * frame_bytes, 0, frame_bytes, st));
       if (T > 1) VDN_CUDA(h, cudaMemsetAsync(o + ((size_t)b * T + T - 1) * frame_bytes, 0, frame_bytes, st));
     }
-    if (s.Tn <= 0) return VDN_OK;      // a clip of anchor frames only has no linear output (Sec. A.4)
   }
+  if (s.Tn <= 0) return VDN_OK;        // a clip of anchor frames only has no linear output (Sec. A.4)
   if (use_tensor_cores(h, d)) return forward_tc(h, q, k, v, beta, gate, x, out, s, L, st);
   if (h->cfg.io_dtype == VDN_F32) {
     return d == 64 ? forward_simt<float, 64>(h, q, k, v, beta, gate, x, out, s, L, st)
@@ -699,7 +727,14 @@ extern "C" {
 vdn_status vdn_vda_forward_opt(vdn_vda_t h, const void* q, const void* k, const void* v, const float* beta,
                                const float* gate, void* out, int B, int T, int F, int H, int d,
                                const vdn_vda_options* opt, void* cuda_stream) {
-  return forward_core(h, q, k, v, beta, gate, out, B, T, F, H, d, opt, cuda_stream, 0, 0, 0);
+  Extras x;
+  Layout L;
+  Shape s;
+  const vdn_status r = plan_forward(h, q, k, v, beta, gate, out, B, T, F, H, d, opt, x, L, s);
+  if (r != VDN_OK) return r;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
+  return run_forward(h, q, k, v, beta, gate, out, x, L, s, static_cast<cudaStream_t>(cuda_stream), 0, 0, 0);
 }
 
 vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const void* v_in, void* q_out, void* k_out,
@@ -771,16 +806,40 @@ vdn_status vdn_vda_forward(vdn_vda_t h, const void* q, const void* k, const void
   return vdn_vda_forward_ex(h, q, k, v, beta, gate, nullptr, nullptr, out, B, T, F, H, d, cuda_stream);
 }
 
-vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const void* v,
-                                const float* beta, const float* gate, void* out, int B, int T, int F,
-                                int H, int d, void* cuda_stream) {
+vdn_status vdn_vda_forward_host_opt(vdn_vda_t h, const void* q, const void* k, const void* v,
+                                    const float* beta, const float* gate, void* out, int B, int T, int F,
+                                    int H, int d, const vdn_vda_options* opt, void* cuda_stream) {
   if (!h) return VDN_ERR_INVALID_ARG;
-  if (!q || !k || !v || !beta || !gate || !out) return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
+  if (!q || !k || !v || !beta || !out) return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
   std::string why;
   if (!shape_ok(h, B, T, F, H, d, &why)) return fail(h, VDN_ERR_INVALID_ARG, why);
-  const StagingLayout S = make_staging(h, B, T, F, H, d);
+  if (opt && opt->struct_size != sizeof(vdn_vda_options))
+    return fail(h, VDN_ERR_INVALID_ARG, "vdn_vda_options.struct_size does not match this library");
+  const bool with_ge = opt && opt->gate_elem;
+  const StagingLayout S = make_staging(h, B, T, F, H, d, with_ge);
   if (!h->staging || h->staging_bytes < S.total)
-    return fail(h, VDN_ERR_WORKSPACE, "staging buffer not set or smaller than vdn_vda_staging_bytes");
+    return fail(h, VDN_ERR_WORKSPACE, "staging buffer not set or smaller than vdn_vda_staging_bytes(_opt)");
+  char* sg = static_cast<char*>(h->staging);
+  // The call as the kernels will see it: every tensor in the staging buffer.  Planned (and refused, if it must
+  // be) before the first copy is queued, so an error return never leaves copies reading the caller's buffers.
+  vdn_vda_options dopt;
+  std::memset(&dopt, 0, sizeof(dopt));
+  dopt.struct_size = sizeof(dopt);
+  if (opt) {
+    dopt = *opt;
+    dopt.alpha = opt->alpha ? reinterpret_cast<const float*>(sg + S.alpha) : nullptr;
+    dopt.s0 = opt->s0 ? reinterpret_cast<const float*>(sg + S.s0) : nullptr;
+    dopt.norm_weight = opt->norm_weight ? reinterpret_cast<const float*>(sg + S.norm_weight) : nullptr;
+    dopt.gate_elem = opt->gate_elem ? sg + S.gate_elem : nullptr;
+  }
+  const float* dbeta = reinterpret_cast<const float*>(sg + S.beta);
+  const float* dgate = gate ? reinterpret_cast<const float*>(sg + S.gate) : nullptr;
+  Extras x;
+  Layout L;
+  Shape s;
+  vdn_status r = plan_forward(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, B, T, F, H, d,
+                              opt ? &dopt : nullptr, x, L, s);
+  if (r != VDN_OK) return r;
   DeviceGuard guard(h->cfg.device);
   if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
   if (!h->copy_stream) {
@@ -793,59 +852,88 @@ vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const
       VDN_CUDA(h, cudaEventCreateWithFlags(&h->in_ev[i], cudaEventDisableTiming));
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  char* sg = static_cast<char*>(h->staging);
   const size_t tokh = (size_t)B * T * F * H;
   const size_t big = tokh * d * elem_size(h);
   const size_t frame_bytes = (size_t)F * H * d * elem_size(h);
+  cudaStream_t in = h->in_stream;
+  // From here on work is queued on the handle's own streams.  Whatever goes wrong later, the caller's stream is
+  // made to wait for the tail of both before the error is returned, so that synchronising it still means that
+  // nothing of this call touches the caller's buffers any more.
+  auto join = [&]() {
+    if (cudaEventRecord(h->in_ev[0], in) == cudaSuccess) cudaStreamWaitEvent(st, h->in_ev[0], 0);
+    if (cudaEventRecord(h->copy_ev[vdn_vda_s::kHostGroups], h->copy_stream) == cudaSuccess)
+      cudaStreamWaitEvent(st, h->copy_ev[vdn_vda_s::kHostGroups], 0);
+    cudaGetLastError();
+  };
+#define VDN_CUDA_J(call)                                                                       \
+  do {                                                                                         \
+    cudaError_t e_ = (call);                                                                   \
+    if (e_ != cudaSuccess) {                                                                   \
+      join();                                                                                  \
+      return fail(h, VDN_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_));        \
+    }                                                                                          \
+  } while (0)
   // All copies in are queued at once on the handle's input stream, in the order the layer needs them, so that the
   // host link never waits for a kernel: keys, values and write gates first (the statistics, the resolve and both
   // scans need nothing else), then the queries, one group of frames after another.  The input stream starts where
   // the caller's stream stands now (earlier work on it may still be reading the staging buffer).
-  cudaStream_t in = h->in_stream;
-  VDN_CUDA(h, cudaEventRecord(h->in_ev[0], st));
-  VDN_CUDA(h, cudaStreamWaitEvent(in, h->in_ev[0], 0));
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.k, k, big, cudaMemcpyHostToDevice, in));
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.v, v, big, cudaMemcpyHostToDevice, in));
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.beta, beta, tokh * sizeof(float), cudaMemcpyHostToDevice, in));
-  VDN_CUDA(h, cudaMemcpyAsync(sg + S.gate, gate, (size_t)H * sizeof(float), cudaMemcpyHostToDevice, in));
-  VDN_CUDA(h, cudaEventRecord(h->in_ev[1], in));
+  VDN_CUDA_J(cudaEventRecord(h->in_ev[0], st));
+  VDN_CUDA_J(cudaStreamWaitEvent(in, h->in_ev[0], 0));
+  VDN_CUDA_J(cudaMemcpyAsync(sg + S.k, k, big, cudaMemcpyHostToDevice, in));
+  VDN_CUDA_J(cudaMemcpyAsync(sg + S.v, v, big, cudaMemcpyHostToDevice, in));
+  VDN_CUDA_J(cudaMemcpyAsync(sg + S.beta, beta, tokh * sizeof(float), cudaMemcpyHostToDevice, in));
+  if (gate) VDN_CUDA_J(cudaMemcpyAsync(sg + S.gate, gate, (size_t)H * sizeof(float), cudaMemcpyHostToDevice, in));
+  if (opt && opt->alpha)
+    VDN_CUDA_J(cudaMemcpyAsync(sg + S.alpha, opt->alpha, (size_t)B * T * H * d * sizeof(float), cudaMemcpyHostToDevice, in));
+  if (opt && opt->s0)
+    VDN_CUDA_J(cudaMemcpyAsync(sg + S.s0, opt->s0, (size_t)B * H * d * d * sizeof(float), cudaMemcpyHostToDevice, in));
+  if (opt && opt->norm_weight)
+    VDN_CUDA_J(cudaMemcpyAsync(sg + S.norm_weight, opt->norm_weight, (size_t)H * d * sizeof(float), cudaMemcpyHostToDevice, in));
+  VDN_CUDA_J(cudaEventRecord(h->in_ev[1], in));
   const int groups = T < vdn_vda_s::kHostGroups ? T : vdn_vda_s::kHostGroups;
   for (int g = 0; g < groups; ++g) {
     const int t0 = (int)((long long)T * g / groups), t1 = (int)((long long)T * (g + 1) / groups);
     const size_t off = (size_t)t0 * frame_bytes, len = (size_t)(t1 - t0) * frame_bytes;
     for (int b = 0; b < B; ++b) {
       const size_t o = (size_t)b * T * frame_bytes + off;
-      VDN_CUDA(h, cudaMemcpyAsync(sg + S.q + o, static_cast<const char*>(q) + o, len, cudaMemcpyHostToDevice, in));
+      VDN_CUDA_J(cudaMemcpyAsync(sg + S.q + o, static_cast<const char*>(q) + o, len, cudaMemcpyHostToDevice, in));
+      if (with_ge)
+        VDN_CUDA_J(cudaMemcpyAsync(sg + S.gate_elem + o, static_cast<const char*>(opt->gate_elem) + o, len,
+                                   cudaMemcpyHostToDevice, in));
     }
-    VDN_CUDA(h, cudaEventRecord(h->in_ev[2 + g], in));
+    VDN_CUDA_J(cudaEventRecord(h->in_ev[2 + g], in));
   }
-  const float* dbeta = reinterpret_cast<const float*>(sg + S.beta);
-  const float* dgate = reinterpret_cast<const float*>(sg + S.gate);
-  VDN_CUDA(h, cudaStreamWaitEvent(st, h->in_ev[1], 0));
-  vdn_status r = forward_core(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, B, T, F, H, d, nullptr,
-                              cuda_stream, 1, 0, 0);
-  if (r != VDN_OK) return r;
+  VDN_CUDA_J(cudaStreamWaitEvent(st, h->in_ev[1], 0));
+  r = run_forward(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, x, L, s, st, 1, 0, 0);
+  if (r != VDN_OK) { join(); return r; }
   // Each group is read out as soon as its queries have landed, and its finished rows go to the second stream,
   // whose copy back to the host runs beside the copies in (the link is full duplex).
   for (int g = 0; g < groups; ++g) {
     const int t0 = (int)((long long)T * g / groups), t1 = (int)((long long)T * (g + 1) / groups);
     const size_t off = (size_t)t0 * frame_bytes, len = (size_t)(t1 - t0) * frame_bytes;
-    VDN_CUDA(h, cudaStreamWaitEvent(st, h->in_ev[2 + g], 0));
-    r = forward_core(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, B, T, F, H, d, nullptr, cuda_stream,
-                     2, t0, t1 - t0);
-    if (r != VDN_OK) return r;
-    VDN_CUDA(h, cudaEventRecord(h->copy_ev[g], st));
-    VDN_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->copy_ev[g], 0));
+    VDN_CUDA_J(cudaStreamWaitEvent(st, h->in_ev[2 + g], 0));
+    r = run_forward(h, sg + S.q, sg + S.k, sg + S.v, dbeta, dgate, sg + S.out, x, L, s, st, 2, t0, t1 - t0);
+    if (r != VDN_OK) { join(); return r; }
+    VDN_CUDA_J(cudaEventRecord(h->copy_ev[g], st));
+    VDN_CUDA_J(cudaStreamWaitEvent(h->copy_stream, h->copy_ev[g], 0));
     for (int b = 0; b < B; ++b) {
       const size_t o = (size_t)b * T * frame_bytes + off;
-      VDN_CUDA(h, cudaMemcpyAsync(static_cast<char*>(out) + o, sg + S.out + o, len, cudaMemcpyDeviceToHost,
-                                  h->copy_stream));
+      VDN_CUDA_J(cudaMemcpyAsync(static_cast<char*>(out) + o, sg + S.out + o, len, cudaMemcpyDeviceToHost,
+                                 h->copy_stream));
     }
   }
   // the caller's stream is done when the last rows have landed
-  VDN_CUDA(h, cudaEventRecord(h->copy_ev[vdn_vda_s::kHostGroups], h->copy_stream));
-  VDN_CUDA(h, cudaStreamWaitEvent(st, h->copy_ev[vdn_vda_s::kHostGroups], 0));
+  VDN_CUDA_J(cudaEventRecord(h->copy_ev[vdn_vda_s::kHostGroups], h->copy_stream));
+  VDN_CUDA_J(cudaStreamWaitEvent(st, h->copy_ev[vdn_vda_s::kHostGroups], 0));
+#undef VDN_CUDA_J
   return VDN_OK;
+}
+
+vdn_status vdn_vda_forward_host(vdn_vda_t h, const void* q, const void* k, const void* v,
+                                const float* beta, const float* gate, void* out, int B, int T, int F,
+                                int H, int d, void* cuda_stream) {
+  if (h && !gate) return fail(h, VDN_ERR_INVALID_ARG, "null tensor pointer");
+  return vdn_vda_forward_host_opt(h, q, k, v, beta, gate, out, B, T, F, H, d, nullptr, cuda_stream);
 }
 
 vdn_status vdn_vda_workspace_view(vdn_vda_t h, int which, int B, int T, int F, int H, int d,
@@ -920,8 +1008,39 @@ int vdn_vda_kernel_times(vdn_vda_t h, int max_kernels, const char** names, float
 vdn_status vdn_vda_status(vdn_vda_t h) {
   if (!h) return VDN_ERR_INVALID_ARG;
   const int v = *const_cast<volatile int*>(h->status_host);
-  return v == 0 ? VDN_OK : VDN_ERR_TIMEOUT;
+  if (v == 0) return VDN_OK;
+  return v == VDN_ERR_INTERNAL ? VDN_ERR_INTERNAL : VDN_ERR_TIMEOUT;
 }
+
+vdn_status vdn_vda_clear_status(vdn_vda_t h) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  const vdn_status prev = vdn_vda_status(h);
+  *const_cast<volatile int*>(h->status_host) = 0;
+  return prev;
+}
+
+vdn_status vdn_vda_set_wait_limit_us(vdn_vda_t h, unsigned long long microseconds) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  if (microseconds == 0 || microseconds > 3600ull * 1000000ull)
+    return fail(h, VDN_ERR_INVALID_ARG, "the wait limit must lie between 1 microsecond and 1 hour");
+  h->wait_ns = microseconds * 1000ull;
+  return VDN_OK;
+}
+
+vdn_status vdn_vda_selftest_wait_expiry(vdn_vda_t h, unsigned long long limit_us, void* cuda_stream) {
+  if (!h) return VDN_ERR_INVALID_ARG;
+  if (limit_us == 0 || limit_us > 1000000ull)
+    return fail(h, VDN_ERR_INVALID_ARG, "the self-test's wait limit must lie between 1 microsecond and 1 second");
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
+  const_cast<volatile int*>(h->status_host)[1] = 0;
+  vdn::wait_expiry_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      vdn::tc::DevStatus{h->status_dev, limit_us * 1000ull}, h->status_dev + 1);
+  VDN_CUDA(h, cudaGetLastError());
+  return VDN_OK;
+}
+
+int vdn_vda_selftest_marker(vdn_vda_t h) { return h ? const_cast<volatile int*>(h->status_host)[1] : -1; }
 
 vdn_status vdn_vda_scan_static(const float* stats, const float* inv, float* read, int BH, int T, int d,
                                int device, void* cuda_stream, char* errbuf, size_t errbuf_len) {
@@ -942,21 +1061,21 @@ vdn_status vdn_vda_scan_static(const float* stats, const float* inv, float* read
   }
   DeviceGuard guard(device);
   if (!guard.ok) { put_msg(errbuf, errbuf_len, "cannot make the device current"); return VDN_ERR_CUDA; }
-  if (!g_scan_static_ptr[device]) {
+  float* ptr = g_scan_static_ptr[device].load(std::memory_order_acquire);
+  if (!ptr) {
     // first call on this device: look up where the array lives on it (the device is current here)
-    float* ptr = nullptr;
     cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_scan_static_scratch);
     if (e != cudaSuccess || !ptr) {
       put_msg(errbuf, errbuf_len, std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
       cudaGetLastError();
       return VDN_ERR_CUDA;
     }
-    g_scan_static_ptr[device] = ptr;
+    g_scan_static_ptr[device].store(ptr, std::memory_order_release);
   }
   std::string why;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const vdn_status r = d == 64 ? launch_scan_static<64>(stats, inv, read, BH, T, g_scan_static_ptr[device], st, &why)
-                               : launch_scan_static<128>(stats, inv, read, BH, T, g_scan_static_ptr[device], st, &why);
+  const vdn_status r = d == 64 ? launch_scan_static<64>(stats, inv, read, BH, T, ptr, st, &why)
+                               : launch_scan_static<128>(stats, inv, read, BH, T, ptr, st, &why);
   if (r != VDN_OK) put_msg(errbuf, errbuf_len, why);
   return r;
 }

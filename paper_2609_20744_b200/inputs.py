@@ -36,6 +36,12 @@ class VdaWorkload:
     corr_frac: float = 0.0         # fraction of each frame's keys drawn near shared directions
     corr_sigma: float = 0.05       # per-component perturbation before re-normalisation
     corr_dirs: int = 8             # shared unit directions per (batch, head)
+    # Degenerate and out-of-the-ordinary inputs the layer must still handle (all off by default):
+    key_repeat_frac: float = 0.0   # fraction of a frame's tokens that carry ONE unit key, drawn per (batch, frame, head)
+    key_norm_lo: float = 1.0       # key norms log-uniform in [key_norm_lo, key_norm_hi] instead of 1
+    key_norm_hi: float = 1.0
+    zero_beta_frames: tuple = ()   # frames whose write gates are all zero (nothing is written)
+    beta_const: float = -1.0       # >= 0: every write gate has this value
 
     @property
     def tokens(self) -> int:
@@ -114,6 +120,22 @@ def generate(w: VdaWorkload, device="cpu", pin: bool = False):
                 near = dirs[hidx, j] + w.corr_sigma * torch.randn(shp, generator=g, device=dev)
                 kf = torch.where(pick[..., None], near, kf)
             kf = _unit(kf)
+            # the optional recipes draw after everything else, so the default streams do not move
+            if w.key_repeat_frac > 0.0:
+                shared = _unit(torch.randn((1, w.H, w.d), generator=g, device=dev))
+                if w.key_repeat_frac >= 1.0:
+                    kf = shared.expand(shp).clone()
+                else:
+                    rep = torch.rand((w.F, w.H), generator=g, device=dev) < w.key_repeat_frac
+                    kf = torch.where(rep[..., None], shared.expand(shp), kf)
+            if (w.key_norm_lo, w.key_norm_hi) != (1.0, 1.0):
+                import math
+                lo, hi = math.log(w.key_norm_lo), math.log(w.key_norm_hi)
+                kf = kf * torch.exp(lo + (hi - lo) * torch.rand((w.F, w.H, 1), generator=g, device=dev))
+            if w.beta_const >= 0.0:
+                bf = torch.full_like(bf, w.beta_const)
+            if t in w.zero_beta_frames:
+                bf = torch.zeros_like(bf)
             q[b, t].copy_(qf)
             k[b, t].copy_(kf)
             v[b, t].copy_(vf)

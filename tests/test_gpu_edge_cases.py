@@ -1,0 +1,154 @@
+"""The method's degenerate and ill-conditioned cases on the GPU, through the C ABI, against the fp64 checker.
+
+  * repeated keys (Sec. A.3, Eq. A.3): every token of a frame -- or nine in ten -- carries the same unit key, so
+    lambda_max(A_t) reaches sum(beta) (hundreds at F = 300, about two thousand at F = 4080) and I + A_t is as
+    ill-conditioned as the method allows for unit keys;
+  * write gates that are all zero (A_t = B_t = 0: Eq. 5 passes the decayed state through), for one frame and for
+    the whole clip;
+  * keys that are not unit-norm (Proposition 1 needs only beta >= 0): norms spread over [0.25, 4] with most keys
+    near two shared directions, lambda_max in the thousands.
+
+Tolerances are the ones of every other parity test (2e-2 for bf16 I/O, 1e-4 for f32 I/O, oracle.slice_error); none
+is loosened here.  What the cases below establish is the range of inputs in which each mode holds its tolerance
+(measured on B200; the same table is in the library header):
+
+  * f32 I/O forms (I + A_t)^{-1} explicitly in fp32, as the paper's kernel does.  An explicit fp32 inverse is
+    good to about eps * lambda_max relative to the largest entry of the state.  When *every* key of a frame is the
+    same vector and the values are random, the state itself is small (the values average out), and 1e-4 holds
+    only up to lambda_max of about 60; with nine keys in ten identical it holds up to about two thousand.
+  * bf16 I/O through the plain-fp32 kernels (VDN_FLAG_FORCE_SIMT) takes the 16-bit inputs as exact and holds 2e-2
+    in every case here, up to lambda_max beyond 1e5.
+  * bf16 I/O through the tensor-core kernels rounds each token's weighted key beta_u k_u to bf16 for the
+    contraction (a relative 2^-9 per element, different from token to token).  The update of Eq. 5 damps what a
+    frame writes along its repeated key direction by 1 / (1 + lambda_max), but not the rounding residue, which
+    lies off that direction: the error relative to the result grows with the share of identical keys and with
+    lambda_max.  2e-2 holds with nine keys in ten identical up to lambda_max of about two thousand (the most that
+    unit keys can give at F = 4080), and for key norms spread over [0.25, 4] around shared directions; it does not
+    hold for frames in which 99 % or more of the keys are bit-identical (measured 3e-2 .. 8e-2 at 99 %, worse at
+    100 %) nor for lambda_max far beyond 1e4.  Those cases are checked through the plain-fp32 kernels.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import vda_oracle as orc
+from paper_2609_20744_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+SIMT = binding.VDN_FLAG_FORCE_SIMT
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    binding.load_library()
+
+
+def run_case(w, flags=0, alpha=None, s0=None):
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
+    out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], alpha=alpha, s0=s0)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    worst, lam = 0.0, 0.0
+    for b in range(w.B):
+        for h in range(w.H):
+            q, k, v, beta, gate = inputs.head_slice(x, b, h)
+            a = None if alpha is None else alpha[b, :, h].double().cpu().numpy()
+            s = None if s0 is None else s0[b, h].double().cpu().numpy()
+            ref = orc.vda_slice(q, k, v, beta, gate, 1e-6, alpha=a, s0=s, want=("A",))
+            lam = max(lam, max(float(np.linalg.eigvalsh(m)[-1]) for m in ref["A"]))
+            got = out[b, :, :, h, :].double().cpu().numpy()
+            assert np.isfinite(got).all()
+            worst = max(worst, orc.slice_error(got, ref["out"]))
+    return worst, lam, out, x
+
+
+MODES = [("bf16", 128, 0), ("bf16", 128, SIMT), ("f32", 128, 0), ("f32", 64, 0)]
+
+
+# ------------------------------------------------------------------------------ repeated keys (Eq. A.3)
+@pytest.mark.parametrize("dtype,d,flags", MODES)
+@pytest.mark.parametrize("F,frac", [(300, 1.0), (300, 0.9), (4080, 0.9), (4080, 1.0), (32, 1.0)])
+def test_repeated_keys(dtype, d, flags, F, frac):
+    if dtype == "f32" and (F, frac) in ((300, 1.0), (4080, 1.0), (4080, 0.9)):
+        pytest.skip("outside the range in which an explicit fp32 inverse holds 1e-4 (see the module docstring)")
+    if dtype == "bf16" and flags == 0 and frac == 1.0:
+        pytest.skip("bit-identical keys throughout a frame: outside the tensor-core kernels' range (module docstring)")
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=1, H=2, T=5, F=F, key_repeat_frac=frac, seed=21)
+    err, lam, _, _ = run_case(w, flags)
+    assert lam > 0.4 * 0.9 * F * min(frac, 1.0) * 0.5          # the recipe did produce a dominant eigenvalue ~ sum(beta)
+    assert err <= TOL[dtype], f"lambda_max {lam:.0f}: error {err:.3e}"
+
+
+@pytest.mark.parametrize("dtype,d,flags,beta0", [("bf16", 128, 0, 0.5), ("bf16", 128, SIMT, 0.3), ("f32", 64, 0, 0.3)])
+def test_repeated_keys_closed_form_holds_on_the_gpu(dtype, d, flags, beta0):
+    # Eq. A.3 itself, read off the GPU's stored forward state: with one key k repeated F times and a common write
+    # gate beta, S_t k = S_bar k / (1 + F beta) + F beta / (1 + F beta) * mean(v).  First frame, zero initial state.
+    # (Tensor-core kernels: with a power of two for beta the weighted key beta k is exact in bf16, which keeps this
+    # case inside their range; see the module docstring.)
+    F = 300
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=1, H=1, T=3, F=F, key_repeat_frac=1.0, beta_const=beta0, seed=5)
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
+    vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
+    torch.cuda.synchronize()
+    if vda.uses_tensor_cores():
+        p0 = vda.view(binding.VIEW_READ_FWD, w.B, w.T, w.F, w.H)[0, 0, 1].double().cpu().numpy()   # slot 1 = P_0, [d_v][d_k]
+    else:
+        p0 = vda.view(binding.VIEW_FWD, w.B, w.T, w.F, w.H)[0, 0, 0].double().cpu().numpy().T       # P_0 transposed
+    k0 = x["k"][0, 0, 0, 0].double().cpu().numpy()
+    vbar = x["v"][0, 0, :, 0].double().mean(0).cpu().numpy()
+    kk = float(k0 @ k0)                                           # a 16-bit key is unit only to 2^-9
+    b0 = float(x["beta"][0, 0, 0, 0])
+    want = F * b0 / (1.0 + F * b0 * kk) * vbar * kk
+    got = p0 @ k0
+    tol = 2e-2 if vda.uses_tensor_cores() else 1e-3               # bf16 storage of the state / fp32 throughout
+    assert np.max(np.abs(got - want)) <= tol * np.max(np.abs(want))
+
+
+# ------------------------------------------------------------------------------ all-zero write gates (A_t = 0)
+@pytest.mark.parametrize("dtype,d,flags", MODES)
+@pytest.mark.parametrize("which", ["one_frame", "whole_clip"])
+def test_zero_write_gates_pass_the_state_through(dtype, d, flags, which):
+    T = 6
+    frames = (2,) if which == "one_frame" else tuple(range(T))
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=1, H=2, T=T, F=150, zero_beta_frames=frames, seed=31)
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    err, _, out, x = run_case(w, flags, alpha=alpha, s0=s0)
+    assert err <= TOL[dtype], f"error {err:.3e}"
+    if which == "whole_clip":
+        # without a text state nothing is ever written: the output is exactly zero
+        vda = binding.Vda(w.d, w.dtype, flags=flags)
+        out0 = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
+        torch.cuda.synchronize()
+        assert torch.count_nonzero(out0) == 0
+
+
+# ------------------------------------------------------------------------------ keys that are not unit-norm
+@pytest.mark.parametrize("dtype,d,flags", MODES)
+def test_key_norms_spread_over_a_decade_with_shared_directions(dtype, d, flags):
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=1, H=2, T=4, F=4096, corr_frac=0.9, corr_dirs=2,
+                           key_norm_lo=0.25, key_norm_hi=4.0, seed=22)
+    err, lam, _, _ = run_case(w, flags)
+    assert 1e3 <= lam <= 1e4
+    assert err <= TOL[dtype], f"lambda_max {lam:.0f}: error {err:.3e}"
+
+
+# ------------------------------------------------------------------------------ the supported range, pinned
+@pytest.mark.parametrize("F,scale,dtype,flags,lam_min", [
+    (4080, 1.0, "bf16", 0, 1.5e3), (4080, 8.0, "bf16", SIMT, 1e5),
+    (300, 2.0, "f32", 0, 400.0),
+])
+def test_error_growth_with_conditioning(F, scale, dtype, flags, lam_min):
+    # Points near the ends of the ranges the header states, nine keys in ten identical, norms scaled up.
+    # bf16 I/O: the tensor-core kernels hold 2e-2 at the largest lambda_max unit keys can give (about 1850 here);
+    # the plain-fp32 kernels for any key norm -- lambda_max beyond 1e5 here.
+    # f32 I/O: the explicit fp32 inverse holds 1e-4 up to lambda_max of about two thousand for this recipe (measured
+    # 7e-5 .. 9e-5 there); the point checked here, lambda_max of about 500, has a margin of five.
+    w = inputs.TINY.scaled(dtype=dtype, d=128, B=1, H=2, T=4, F=F, key_repeat_frac=0.9, key_norm_lo=scale,
+                           key_norm_hi=scale, seed=23)
+    err, lam, _, _ = run_case(w, flags)
+    assert lam > lam_min
+    assert err <= TOL[dtype], f"{dtype} flags={flags} lambda_max {lam:.3g}: {err:.3e}"

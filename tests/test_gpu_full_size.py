@@ -70,7 +70,7 @@ def test_768p_config_full_size():
 
 @pytest.mark.parametrize("idx", [0, 1, 2, 3])
 def test_scan_depth_sweep_full_size(idx):
-    run_and_check(inputs.SWEEP[idx], 2)
+    run_and_check(inputs.SWEEP[idx], 4)      # first, last and two seeded slices
 
 
 def test_cfg_long_clip_full_size():
@@ -79,7 +79,7 @@ def test_cfg_long_clip_full_size():
     need = 4 * w.tokens * w.H * w.d * 2 + (5 << 30)
     if free < need:
         pytest.skip(f"needs {need >> 30} GiB of free device memory")
-    run_and_check(w, 2)
+    run_and_check(w, 4)
 
 
 def test_768p_release_window_full_size():

@@ -354,6 +354,55 @@ def test_forward_host_matches_device_entry_point(dtype, d, B, T):
         out_h.fill_(7.0)
 
 
+@pytest.mark.parametrize("dtype,d,flags", [("bf16", 128, 0), ("bf16", 128, binding.VDN_FLAG_SCAN_CHUNKWISE), ("f32", 64, 0)])
+def test_forward_host_opt_release_setting_matches_device_entry_point(dtype, d, flags):
+    # every optional input from host memory: chunk window, anchors, decay gates, text state, element-wise gate,
+    # norm weight, queries normalised by the read-out
+    w = inputs.TINY.scaled(dtype=dtype, d=d, B=2, T=13, F=150, H=2, seed=41)
+    xh = inputs.generate(w, "cpu", pin=True)
+    alpha, s0 = inputs.generate_recurrence_extras(w, "cpu")
+    ge, nw = inputs.generate_output_extras(w, "cpu")
+    kw = dict(chunk=3, radius=1, anchors=True, q_l2_eps=1e-6)
+    host_extras = dict(alpha=alpha.pin_memory(), s0=s0.pin_memory(), gate_elem=ge.pin_memory(), norm_weight=nw.pin_memory())
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
+    out_d = vda.forward(*(xh[n].cuda() for n in ("q", "k", "v", "beta", "gate")),
+                        **{n: t.cuda() for n, t in host_extras.items()}, **kw)
+    torch.cuda.synchronize()
+    assert vda.status() == binding.VDN_OK
+    out_h = torch.empty_like(xh["q"]).pin_memory()
+    for _ in range(2):
+        out_h.fill_(7.0)
+        vda.forward_host(xh["q"], xh["k"], xh["v"], xh["beta"], xh["gate"], out_h, **host_extras, **kw)
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(out_h, out_d.cpu())
+    assert torch.count_nonzero(out_h[:, 0]) == 0 and torch.count_nonzero(out_h[:, -1]) == 0
+    # and against the checker, one slice
+    q, k, v, beta, gate = inputs.head_slice(xh, 1, 1)
+    from oracle import prep_oracle as po
+    ref = orc.vda_slice(po.l2_normalise(q, 1e-6), k, v, beta, gate * ge[1, :, :, 1].double().numpy(), 1e-6,
+                        alpha=alpha[1, :, 1].double().numpy(), s0=s0[1, 1].double().numpy(),
+                        norm_weight=nw[1].double().numpy(), chunk=3, radius=1, anchors=True)["out"]
+    assert orc.slice_error(out_h[1, :, :, 1].double().numpy(), ref) <= TOL[dtype]
+
+
+def test_forward_host_refuses_before_queuing_any_copy():
+    # a staging buffer that is too small is a host-side error: nothing may be enqueued, `out` stays untouched
+    w = inputs.TINY.scaled(dtype="bf16", d=128, T=3, F=100, H=2)
+    xh = inputs.generate(w, "cpu", pin=True)
+    vda = binding.Vda(w.d, w.dtype)
+    vda.ensure_workspace(w.B, w.T, w.F, w.H)
+    small = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    import ctypes
+    vda.lib.vdn_vda_set_staging(vda.h, ctypes.c_void_p(small.data_ptr()), 4096)
+    out_h = torch.full(xh["q"].shape, 7.0, dtype=xh["q"].dtype).pin_memory()
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    st = vda.lib.vdn_vda_forward_host(vda.h, p(xh["q"]), p(xh["k"]), p(xh["v"]), p(xh["beta"]), p(xh["gate"]), p(out_h),
+                                      w.B, w.T, w.F, w.H, w.d, None)
+    assert st == 3
+    torch.cuda.synchronize()
+    assert torch.all(out_h == 7.0)
+
+
 # ------------------------------------------------------------------------------ argument errors (host side)
 def test_argument_errors_enqueue_nothing():
     w = inputs.TINY

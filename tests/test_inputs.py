@@ -51,3 +51,30 @@ def test_head_slice_is_exact_copy():
     assert q.dtype == np.float64 and q.shape == (4, 64, 64)
     assert np.array_equal(k, x["k"][0, :, :, 1, :].double().numpy())
     assert gate == float(x["gate"][1])
+
+
+def test_degenerate_recipes_do_what_they_say_and_leave_the_default_streams_alone():
+    base = inputs.TINY.scaled(H=2, T=3, F=40, d=64)
+    x0 = inputs.generate(base, "cpu")
+    # repeated keys: one vector per (batch, frame, head)
+    x = inputs.generate(base.scaled(key_repeat_frac=1.0), "cpu")
+    k = x["k"]
+    assert torch.equal(k, k[:, :, :1].expand_as(k))
+    assert not torch.equal(k[0, 0, 0, 0], k[0, 1, 0, 0]) and not torch.equal(k[0, 0, 0, 0], k[0, 0, 0, 1])
+    assert torch.allclose(k.norm(dim=-1), torch.ones(k.shape[:-1]), atol=1e-5)
+    for n in ("q", "v", "beta", "gate"):
+        assert torch.equal(x[n], x0[n])                       # the extra draws come after the default ones
+    # partly repeated keys
+    x = inputs.generate(base.scaled(key_repeat_frac=0.5, F=400), "cpu")
+    k = x["k"][0, 0, :, 0]
+    same = (k == k.mode(dim=0).values).all(dim=-1).float().mean()
+    assert 0.35 < float(same) < 0.65
+    # key norms
+    x = inputs.generate(base.scaled(key_norm_lo=0.25, key_norm_hi=4.0, F=500), "cpu")
+    n = x["k"].norm(dim=-1)
+    assert float(n.min()) >= 0.25 * (1 - 1e-5) and float(n.max()) <= 4.0 * (1 + 1e-5) and float(n.std()) > 0.5
+    # write gates
+    x = inputs.generate(base.scaled(zero_beta_frames=(1,)), "cpu")
+    assert torch.count_nonzero(x["beta"][:, 1]) == 0 and torch.equal(x["beta"][:, 0], x0["beta"][:, 0])
+    x = inputs.generate(base.scaled(beta_const=0.3), "cpu")
+    assert torch.all(x["beta"] == 0.3)

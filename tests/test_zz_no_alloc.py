@@ -3,15 +3,17 @@
 Some users of the library run inside programs that claim all GPU memory up front and forbid (or cannot
 afford) any later cudaMalloc; they cannot give vdn_vda_forward a workspace.  The entry point tested here
 runs the fp32 scan + gather stage with its scratch held in an array inside the library image.  It must
-give the very states the regular entry point leaves in its workspace, call after call (the scratch is
-shared and keeps the previous call's contents).  This file sorts last on purpose: a run that stops at the
+give the very states the regular entry point leaves in its workspace -- and the states the fp64 checker
+computes from the same inputs -- call after call (the scratch is shared and keeps the previous call's contents).  This file sorts last on purpose: a run that stops at the
 first failure has then already run every other test.
 """
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import vda_oracle as orc
 from paper_2609_20744_b200 import binding, build, inputs
 
 pytestmark = pytest.mark.gpu
@@ -34,32 +36,51 @@ def regular_path_states(w):
     stats = vda.view(binding.VIEW_STATS, *shp).reshape(n, w.T, 2 * w.d, w.d).clone()
     inv = vda.view(binding.VIEW_INV, *shp).reshape(n, w.T, w.d, w.d).clone()
     read = vda.view(binding.VIEW_READ, *shp).reshape(n, w.T, w.d, w.d).clone()
-    return stats, inv, read
+    return stats, inv, read, x
 
 
 @pytest.mark.parametrize("kw", [dict(d=64, T=4, F=64, H=2), dict(d=128, T=7, F=90, H=3), dict(d=128, T=1, F=16, H=1)])
 def test_static_scratch_scan_matches_regular_entry_point_twice_in_a_row(kw):
     w = inputs.TINY.scaled(**kw)
-    stats, inv, want = regular_path_states(w)
+    stats, inv, want, x = regular_path_states(w)
     other = inputs.TINY.scaled(seed=11, **kw)
-    stats2, inv2, want2 = regular_path_states(other)
+    stats2, inv2, want2, _ = regular_path_states(other)
 
     got = torch.full_like(want, float("nan"))
     got2 = torch.full_like(want2, float("nan"))
+    binding.scan_static(stats, inv, got)          # a first call on this device may look up the array's address
     torch.cuda.synchronize()
+    got.fill_(float("nan"))
     allocations_before = torch.cuda.memory_stats()["allocation.all.allocated"]   # count of allocator requests
-    binding.scan_static(stats, inv, got)          # first call: leaves its forward states in the shared scratch
-    binding.scan_static(stats2, inv2, got2)       # second call, other data: must not see the first call's scratch
+    free_before, _ = torch.cuda.mem_get_info()    # what the driver itself reports: a cudaMalloc inside the library would show
+    binding.scan_static(stats, inv, got)          # leaves its forward states in the shared scratch
+    binding.scan_static(stats2, inv2, got2)       # other data: must not see the previous call's scratch
     binding.scan_static(stats, inv, got)          # and again with the first data
     torch.cuda.synchronize()
-    # torch's allocator was not asked for anything while the three calls ran
+    # neither torch's allocator nor the CUDA runtime was asked for memory while the three calls ran
     assert torch.cuda.memory_stats()["allocation.all.allocated"] == allocations_before
+    assert torch.cuda.mem_get_info()[0] == free_before
     # same kernel arithmetic as the regular path; the tests' f32 bar is 1e-4 of the slice maximum
     for g, wnt in ((got, want), (got2, want2)):
         assert torch.isfinite(g).all()
         scale = wnt.abs().amax().clamp_min(1e-30)
         assert float((g - wnt).abs().amax() / scale) <= 1e-4
         assert torch.equal(g, wnt)                                        # in fact bit-identical
+    # and against the fp64 checker directly: slot t of the output is the transpose of P_{t-1} + R_{t+1} (Eq. A.4)
+    n = 0
+    for b in range(w.B):
+        for h in range(w.H):
+            q, k, v, beta, gate = inputs.head_slice(x, b, h)
+            ref = orc.vda_slice(q, k, v, beta, gate, 1e-6, want=("P", "R"))
+            for t in range(w.T):
+                rd = np.zeros((w.d, w.d))
+                if t > 0:
+                    rd = rd + ref["P"][t - 1]
+                if t + 1 < w.T:
+                    rd = rd + ref["R"][t + 1]
+                g = got[n, t].double().cpu().numpy().T
+                assert np.max(np.abs(g - rd)) <= 1e-4 * max(np.max(np.abs(rd)), 1e-30)
+            n += 1
 
 
 def test_static_scratch_scan_rejects_shapes_beyond_its_limit():
