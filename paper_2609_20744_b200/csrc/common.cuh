@@ -9,11 +9,15 @@ namespace vdn {
 // Problem shape in the library's naming: T latent frames of F tokens, H heads, d = d_k = d_v.
 // t0 / Tn: the frames the linear branch works on, t0 .. t0+Tn-1 (all T frames, or the interior frames when the
 // first and the last frame are boundary anchors, Sec. A.4).  Workspace indices always count all T frames.
+// bh0 / bhn: the (batch, head) pairs a persistent kernel works on, pair index b*H + h in bh0 .. bh0+bhn-1 (bhn = 0: all
+// of them).  The read-out of a layer with more scan chains than SMs is launched in two parts.
 struct Shape {
   int B, T, F, H, d;
   int t0, Tn;
-  __host__ __device__ long long frames() const { return (long long)B * H * T; }       // (b,h,t) triples
-  __host__ __device__ long long work_items() const { return (long long)B * H * Tn; }  // ... that are worked on
+  int bh0 = 0, bhn = 0;
+  __host__ __device__ int pairs() const { return bhn > 0 ? bhn : B * H; }
+  __host__ __device__ long long frames() const { return (long long)B * H * T; }          // (b,h,t) triples
+  __host__ __device__ long long work_items() const { return (long long)pairs() * Tn; }   // ... that are worked on
 };
 
 // Local window of a query frame in temporal chunks (Sec. 2.1), clipped to the scanned frames first..last
@@ -45,16 +49,17 @@ __device__ __forceinline__ void split_frame(const Shape& s, long long n, int& b,
   b = (int)(bh / s.H);
 }
 
-// Work order of the persistent tensor-core kernels: work item w (of s.work_items()) -> (b, t, h) with the head fastest, so
-// that CTAs running side by side stream the same token rows (a token's H heads are contiguous in memory:
-// neighbouring 256-byte pieces of one DRAM page, and shared 32-byte sectors of beta).  Returns the frame
+// Work order of the persistent tensor-core kernels: work item w (of s.work_items()) -> (b, h, t) with the (batch,
+// head) pair fastest, so that CTAs running side by side stream the same token rows (a token's H heads are contiguous
+// in memory: neighbouring 256-byte pieces of one DRAM page, and shared 32-byte sectors of beta).  Returns the frame
 // index n = (b*H + h)*T + t that addresses the workspace.
 __device__ __forceinline__ long long split_work(const Shape& s, long long w, int& b, int& h, int& t) {
-  h = (int)(w % s.H);
-  long long bt = w / s.H;
-  t = s.t0 + (int)(bt % s.Tn);
-  b = (int)(bt / s.Tn);
-  return ((long long)b * s.H + h) * s.T + t;
+  const int np = s.pairs();
+  const int pair = s.bh0 + (int)(w % np);
+  t = s.t0 + (int)(w / np);
+  h = pair % s.H;
+  b = pair / s.H;
+  return (long long)pair * s.T + t;
 }
 
 __device__ __forceinline__ float to_float(float x) { return x; }

@@ -24,20 +24,26 @@
 
 namespace vdn {
 
-template <bool EXTRAS, bool QNORM = false, bool GATE = false>
+// SHORT: the layout for short frames (few token tiles per frame).  There a frame's two states are as many bytes as
+// its queries, and with one state buffer the producer could fetch the next frame's states only after the last MMA
+// of this frame had retired: their latency was exposed once per frame.  SHORT keeps two state buffers and pays for
+// them with one Q stage and one staging tile.
+template <bool EXTRAS, bool QNORM = false, bool GATE = false, bool SHORT = false>
 struct ReadoutTcCfg {
   static_assert(EXTRAS || !GATE, "the element-wise gate is one of the optional factors");
+  static_assert(!(SHORT && GATE), "the gate path keeps its three staging tiles");
   static constexpr int D = 128;
   static constexpr int TILE = 128;
   // GATE: gate tiles arrive by TMA in the output staging tiles, two tiles ahead; a third staging tile takes the
   // place of a Q stage (with 3 Q stages, 2 staging tiles and a one-tile lookahead the gate path takes 2.47 ms
   // instead of 1.76 ms on the 768p clip; without a gate the third Q stage is worth more: 1.24 against 1.37 ms)
-  static constexpr int QSTAGES = GATE ? 2 : 3;
-  static constexpr int NOUT = GATE ? 3 : 2;
+  static constexpr int QSTAGES = (GATE || SHORT) ? 2 : 3;
+  static constexpr int NOUT = GATE ? 3 : (SHORT ? 1 : 2);
+  static constexpr int STSTAGES = SHORT ? 2 : 1;
   static constexpr int BOX_BYTES = 128 * 128;          // 128 rows x 128 B
   static constexpr int TILE_BYTES = 2 * BOX_BYTES;     // 32 KB: state, Q tile or output tile
   static constexpr int OFF_STATE = 0;
-  static constexpr int OFF_Q = 2 * TILE_BYTES;
+  static constexpr int OFF_Q = STSTAGES * 2 * TILE_BYTES;
   static constexpr int OFF_OUT = OFF_Q + QSTAGES * TILE_BYTES;
   static constexpr int OFF_NW = OFF_OUT + NOUT * TILE_BYTES;   // norm weights of the current head, 128 floats
   // QNORM: 1/|q| of the tokens of QSLOTS tiles, 128 floats each.  (Four slots instead of two for the variant with
@@ -51,20 +57,21 @@ struct ReadoutTcCfg {
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one SM");
 };
 using ReadoutTc = ReadoutTcCfg<false>;
+constexpr int kReadoutShortTiles = 4;     // frames of at most this many 128-token tiles take the SHORT layout
 
 // EXTRAS = true adds the optional factors of Eq. 1c to the epilogue: a per-channel norm scale norm_weight [H,d]
 // (kept in shared memory per frame; may be null), a per-head gate that may be null (read as 1) and, with GATE, an
 // element-wise (content-dependent) gate gate_elem [B,T,F,H,d] bf16 (tensor map tmG; its tiles arrive by TMA in the
 // very staging tile the output is then written to, two tiles ahead).  The plain instantiation carries none of that.
-template <bool EXTRAS, bool QNORM = false, bool GATE = false>
-__global__ void __launch_bounds__(ReadoutTcCfg<EXTRAS, QNORM, GATE>::THREADS, 1)
+template <bool EXTRAS, bool QNORM = false, bool GATE = false, bool SHORT = false>
+__global__ void __launch_bounds__(ReadoutTcCfg<EXTRAS, QNORM, GATE, SHORT>::THREADS, 1)
 readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmS,
                   const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmG,
                   const float* __restrict__ gate, Shape s, float eps,
                   tc::DevStatus ds, const __nv_bfloat16* __restrict__ gate_elem, const float* __restrict__ norm_weight,
                   Window win, int bridged, float q_l2_eps) {
   using namespace tc;
-  using R = ReadoutTcCfg<EXTRAS, QNORM, GATE>;
+  using R = ReadoutTcCfg<EXTRAS, QNORM, GATE, SHORT>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -123,18 +130,19 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
         int b, h, t;
         const long long n = split_work(s, item, b, h, t);
-        if (!mbar_wait(STEMPTY(0), (si & 1) ^ 1, wc)) { ok = false; break; }
-        mbar_arrive_expect_tx(STFULL(0), 2 * R::TILE_BYTES);
-        const uint32_t sdst = base + R::OFF_STATE;
+        const int sb = si % R::STSTAGES;
+        if (!mbar_wait(STEMPTY(sb), ((si / R::STSTAGES) & 1) ^ 1, wc)) { ok = false; break; }
+        mbar_arrive_expect_tx(STFULL(sb), 2 * R::TILE_BYTES);
+        const uint32_t sdst = base + R::OFF_STATE + sb * 2 * R::TILE_BYTES;
         // Slot of the forward state in rows [nf*128, +128), of the reverse state in rows [nrev*128, +128).  With
         // decay gates every frame has its own (bridged) pair; without, the frames of a window share the states
         // stored at the window's ends (slot l_t of the forward scan, slot h_t of the reverse scan; Eq. A.4).
         const long long nf = bridged ? n : n - t + win.lo(t);
         const long long nrev = s.frames() + (bridged ? n : n - t + win.hi(t));
-        tma_load_2d(sdst, &tmS, STFULL(0), 0, (int)(nf * R::D));
-        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(nf * R::D));
-        tma_load_2d(sdst + 2 * R::BOX_BYTES, &tmS, STFULL(0), 0, (int)(nrev * R::D));
-        tma_load_2d(sdst + 3 * R::BOX_BYTES, &tmS, STFULL(0), 64, (int)(nrev * R::D));
+        tma_load_2d(sdst, &tmS, STFULL(sb), 0, (int)(nf * R::D));
+        tma_load_2d(sdst + R::BOX_BYTES, &tmS, STFULL(sb), 64, (int)(nf * R::D));
+        tma_load_2d(sdst + 2 * R::BOX_BYTES, &tmS, STFULL(sb), 0, (int)(nrev * R::D));
+        tma_load_2d(sdst + 3 * R::BOX_BYTES, &tmS, STFULL(sb), 64, (int)(nrev * R::D));
         for (int tile = 0; tile < ntiles; ++tile, ++qi) {
           const int st = qi % R::QSTAGES;
           if (!mbar_wait(QEMPTY(st), ((qi / R::QSTAGES) & 1) ^ 1, wc)) { ok = false; break; }
@@ -156,8 +164,9 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       uint32_t qi = 0, si = 0;
       bool ok = true;
       for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
-        if (!mbar_wait(STFULL(0), si & 1, wc)) { ok = false; break; }
-        const uint32_t sbase = base + R::OFF_STATE;
+        const int sb = si % R::STSTAGES;
+        if (!mbar_wait(STFULL(sb), (si / R::STSTAGES) & 1, wc)) { ok = false; break; }
+        const uint32_t sbase = base + R::OFF_STATE + sb * 2 * R::TILE_BYTES;
         for (int tile = 0; tile < ntiles; ++tile, ++qi) {
           const int st = qi % R::QSTAGES;
           const int a = qi & 3;
@@ -179,7 +188,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           mma_commit(QEMPTY(st));
           mma_commit(ACCFULL(a));
         }
-        if (ok) mma_commit(STEMPTY(0));
+        if (ok) mma_commit(STEMPTY(sb));
       }
     }
   } else if (QNORM && warp >= 6) {

@@ -67,6 +67,7 @@ struct ScanTcArgs {
   const float* alpha;        // [B,T,H,d] or null
   const float* s0;           // [B,H,d_v,d_k] or null
   int T, H;
+  int bh0;                   // first (batch, head) pair of this launch (CTA x works on pair bh0 + x / (2 NS))
   float additive_bscale;     // > 0: the additive baseline, Z_t = C_t (alpha Z) + bscale B_t^T
   Window win;
   // chunk composites (SCAN_COMPOSE writes, SCAN_CHUNKS reads); position p of a chain's direction is the p-th chunk
@@ -124,7 +125,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
     f_hi = min(win.last, (kc + 1) * win.chunk - 1);
     nsteps = f_hi - f_lo + 1;
   } else {
-    bh = (blockIdx.x / NS) >> 1;
+    bh = a.bh0 + (int)((blockIdx.x / NS) >> 1);
     dir = (blockIdx.x / NS) & 1;
     // steps this chain runs: up to the last state that some frame reads (P_{l-1} of the last frame's window,
     // R_{h+1} of the first frame's)

@@ -9,6 +9,7 @@
 #include <cmath>
 #include <cstdio>
 #include <atomic>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -95,6 +96,12 @@ struct vdn_vda_s {
   bool attrs_set = false;
   bool tc_attrs_set = false;
   unsigned ro_attrs_set = 0;       // read-out instantiations whose shared-memory attribute has been set
+  int ro_short = 1;                // use the short-frame read-out layout where it applies (VDN_RO_SHORT=0 turns it off)
+  // More scan chains than SMs: the surplus chains run on a side stream beside the read-out of the others
+  // (stream and events made on first use; VDN_SCAN_SPLIT=0 turns it off)
+  int scan_split = 1;
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t side_ev[2] = {};
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;  // driver entry point, resolved at create
   // vdn_vda_forward_host: inputs arrive on one stream of the handle's own and results leave on another, in groups of
   // frames (streams and events made on first use)
@@ -361,7 +368,14 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
 
   const long long nwork = s.work_items();
   const unsigned persistent = (unsigned)(nwork < h->sm_count ? nwork : h->sm_count);
-  int nk = 0;
+  int nk = 0, nk_side = 0;
+  const int pairs_a = h->sm_count / 2;
+  const bool split_scan = x.phase == 0 && !x.composed && h->scan_split && 2LL * s.B * s.H > h->sm_count &&
+                          s.B * s.H < 2 * pairs_a;      // worth it while the surplus is less than a full wave
+  if (split_scan && !h->side_stream) {
+    VDN_CUDA(h, cudaStreamCreateWithFlags(&h->side_stream, cudaStreamNonBlocking));
+    for (cudaEvent_t& e : h->side_ev) VDN_CUDA(h, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  }
   if (x.phase != 2) {
     prof_begin(h, st);
     vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
@@ -398,6 +412,20 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
       vdn::scan_tc_kernel<vdn::SCAN_FRAMES, 2><<<(unsigned)(4 * s.B * s.H), vdn::ScanTc::threads(2),
                                                  vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, dev_status(h));
       prof_mark(h, st, nk++, "scan_tc");
+    } else if (split_scan) {
+      // More chains than SMs (one CTA per SM): a second wave would hold the whole GPU for a handful of chains.
+      // The first sm_count / 2 pairs are scanned here; the rest on the side stream once these are done, beside the
+      // read-out of the first part, which leaves SMs free (see below).
+      vdn::scan_tc_kernel<vdn::SCAN_FRAMES><<<(unsigned)(2 * pairs_a), vdn::ScanTc::THREADS,
+                                              vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, dev_status(h));
+      prof_mark(h, st, nk++, "scan_tc");
+      VDN_CUDA(h, cudaEventRecord(h->side_ev[0], st));
+      VDN_CUDA(h, cudaStreamWaitEvent(h->side_stream, h->side_ev[0], 0));
+      sa.bh0 = pairs_a;
+      vdn::scan_tc_kernel<vdn::SCAN_FRAMES><<<(unsigned)(2 * (s.B * s.H - pairs_a)), vdn::ScanTc::THREADS,
+                                              vdn::ScanTc::SMEM_BYTES, h->side_stream>>>(tmC, sa, dev_status(h));
+      VDN_CUDA(h, cudaEventRecord(h->side_ev[1], h->side_stream));
+      nk_side = 1;
     } else {
       vdn::scan_tc_kernel<vdn::SCAN_FRAMES><<<(unsigned)(2 * s.B * s.H), vdn::ScanTc::THREADS,
                                               vdn::ScanTc::SMEM_BYTES, st>>>(tmC, sa, dev_status(h));
@@ -413,44 +441,59 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   // (measured on three workloads: 124 CTAs beat 148 by 5 %; fewer interleaved read/write streams at the DRAM).
   // With the optional factors or the query norms it is paced by its epilogue warps and wants every SM (768p clip,
   // warm GPU, 124 -> 148 CTAs: queries normalised 1.36 -> 1.25 ms, gate + norm weight 2.09 -> 1.87 ms).
-  Shape sr = s;                                       // the frames to read out
-  if (x.phase == 2) { sr.t0 = x.ro_first; sr.Tn = x.ro_count; }
-  const long long nread = sr.work_items();
   const bool extras = x.gate_elem || x.norm_weight || !gate;
   const long long ro_target = (extras || x.q_l2_eps > 0.f) ? h->sm_count : ((long long)h->sm_count * 27 + 16) / 32;
-  const unsigned persistent_ro = (unsigned)(nread < ro_target ? nread : ro_target);
   CUtensorMap tmG = tmO;                                        // the gate tensor has the layout of the output
   if (x.gate_elem && (r = make_token_map(h, &tmG, x.gate_elem, s)) != VDN_OK) return r;
-  auto launch_readout = [&](auto ex, auto qn, auto ge) {
-    constexpr bool EX = decltype(ex)::value, QN = decltype(qn)::value, GE = decltype(ge)::value;
-    using RX = vdn::ReadoutTcCfg<EX, QN, GE>;
-    constexpr unsigned bit = 1u << ((EX ? 1 : 0) | (QN ? 2 : 0) | (GE ? 4 : 0));
+  // short frames (at most kReadoutShortTiles token tiles): the plain read-out with two state buffers
+  const bool short_frames = (s.F + 127) / 128 <= vdn::kReadoutShortTiles && h->ro_short != 0;
+  auto launch_readout = [&](const Shape& sr, auto ex, auto qn, auto ge, auto sh) {
+    constexpr bool EX = decltype(ex)::value, QN = decltype(qn)::value, GE = decltype(ge)::value, SH = decltype(sh)::value;
+    using RX = vdn::ReadoutTcCfg<EX, QN, GE, SH>;
+    constexpr unsigned bit = 1u << ((EX ? 1 : 0) | (QN ? 2 : 0) | (GE ? 4 : 0) | (SH ? 8 : 0));
     if (!(h->ro_attrs_set & bit)) {        // per handle, i.e. per device
-      if (cudaFuncSetAttribute(vdn::readout_tc_kernel<EX, QN, GE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      if (cudaFuncSetAttribute(vdn::readout_tc_kernel<EX, QN, GE, SH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                RX::SMEM_BYTES) != cudaSuccess)
         return false;
       h->ro_attrs_set |= bit;
     }
-    vdn::readout_tc_kernel<EX, QN, GE><<<persistent_ro, RX::THREADS, RX::SMEM_BYTES, st>>>(
+    const long long nread = sr.work_items();
+    const unsigned persistent_ro = (unsigned)(nread < ro_target ? nread : ro_target);
+    vdn::readout_tc_kernel<EX, QN, GE, SH><<<persistent_ro, RX::THREADS, RX::SMEM_BYTES, st>>>(
         tmQ, tmS, tmO, tmG, gate, sr, h->cfg.rms_eps, dev_status(h), static_cast<const __nv_bfloat16*>(x.gate_elem),
         x.norm_weight, x.win, x.alpha != nullptr, x.q_l2_eps);
     return true;
   };
   using std::true_type;
   using std::false_type;
+  auto readout = [&](const Shape& sr) {
+    if (x.q_l2_eps > 0.f) {
+      if (x.gate_elem) return launch_readout(sr, true_type{}, true_type{}, true_type{}, false_type{});
+      if (extras) return launch_readout(sr, true_type{}, true_type{}, false_type{}, false_type{});
+      return launch_readout(sr, false_type{}, true_type{}, false_type{}, false_type{});
+    }
+    if (x.gate_elem) return launch_readout(sr, true_type{}, false_type{}, true_type{}, false_type{});
+    if (extras) return launch_readout(sr, true_type{}, false_type{}, false_type{}, false_type{});
+    if (short_frames) return launch_readout(sr, false_type{}, false_type{}, false_type{}, true_type{});
+    return launch_readout(sr, false_type{}, false_type{}, false_type{}, false_type{});
+  };
+  Shape sr = s;                                       // the frames to read out
+  if (x.phase == 2) { sr.t0 = x.ro_first; sr.Tn = x.ro_count; }
   bool launched;
-  if (x.q_l2_eps > 0.f) {
-    if (x.gate_elem) launched = launch_readout(true_type{}, true_type{}, true_type{});
-    else if (extras) launched = launch_readout(true_type{}, true_type{}, false_type{});
-    else launched = launch_readout(false_type{}, true_type{}, false_type{});
+  if (split_scan) {
+    // the pairs whose chains are done; then, once the side stream's chains are done too, the others
+    sr.bh0 = 0; sr.bhn = pairs_a;
+    launched = readout(sr);
+    prof_mark(h, st, nk++, "readout_tc");
+    VDN_CUDA(h, cudaStreamWaitEvent(st, h->side_ev[1], 0));
+    sr.bh0 = pairs_a; sr.bhn = s.B * s.H - pairs_a;
+    launched = launched && readout(sr);
   } else {
-    if (x.gate_elem) launched = launch_readout(true_type{}, false_type{}, true_type{});
-    else if (extras) launched = launch_readout(true_type{}, false_type{}, false_type{});
-    else launched = launch_readout(false_type{}, false_type{}, false_type{});
+    launched = readout(sr);
   }
   if (!launched) return fail(h, VDN_ERR_CUDA, "cudaFuncSetAttribute failed for the read-out kernel");
-  prof_mark(h, st, nk++, "readout_tc");
-  h->launches = nk;
+  prof_mark(h, st, nk++, split_scan ? "readout_tc_rest" : "readout_tc");
+  h->launches = nk + nk_side;
   VDN_CUDA(h, cudaGetLastError());
   return VDN_OK;
 }
@@ -550,6 +593,8 @@ vdn_status vdn_vda_create(const vdn_vda_config* cfg, vdn_vda_t* out_handle) {
   h->cfg = *cfg;
   if (!(h->cfg.rms_eps > 0.f)) h->cfg.rms_eps = 1e-6f;
   h->sm_count = prop.multiProcessorCount;
+  if (const char* e = std::getenv("VDN_RO_SHORT")) h->ro_short = std::atoi(e);
+  if (const char* e = std::getenv("VDN_SCAN_SPLIT")) h->scan_split = std::atoi(e);
   DeviceGuard guard(cfg->device);
   if (!guard.ok || cudaHostAlloc(reinterpret_cast<void**>(&h->status_host), 64, cudaHostAllocMapped) != cudaSuccess ||
       cudaHostGetDevicePointer(reinterpret_cast<void**>(&h->status_dev), h->status_host, 0) != cudaSuccess) {
@@ -1092,6 +1137,11 @@ vdn_status vdn_vda_destroy(vdn_vda_t h) {
     for (cudaEvent_t e : h->in_ev)
       if (e) cudaEventDestroy(e);
     if (h->in_stream) cudaStreamDestroy(h->in_stream);
+  }
+  if (h->side_stream) {
+    for (cudaEvent_t e : h->side_ev)
+      if (e) cudaEventDestroy(e);
+    cudaStreamDestroy(h->side_stream);
   }
   if (h->status_host) cudaFreeHost(h->status_host);
   delete h;

@@ -168,6 +168,23 @@ def test_additive_rule_matches_oracle(dtype, d, flags, extras):
     assert not torch.allclose(out.float(), out2.float(), atol=1e-2)
 
 
+@pytest.mark.parametrize("B,H", [(1, 80), (2, 45)])
+def test_more_scan_chains_than_sms(B, H):
+    # 2 B H chains on 148 SMs: the surplus chains are scanned on the library's side stream beside the read-out of
+    # the first 74 (batch, head) pairs; pairs on both sides of the split, and the ends, against the checker
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=B, H=H, T=5, F=130, seed=61)
+    x = inputs.generate(w, "cuda")
+    vda, out = run_gpu(w, x)
+    assert vda.uses_tensor_cores()
+    pairs = [(0, 0), (B - 1, H - 1)] + [divmod(p, H) for p in (72, 73, 74, 75)]
+    check_heads(w, x, out, pairs, TOL["bf16"])
+    ms = out.float().pow(2).mean(dim=-1)                      # every pair was read out: rows have gate-sized rms
+    assert torch.allclose(ms, x["gate"].pow(2)[None, None, None, :].expand_as(ms), rtol=3e-2)
+    again = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
+    torch.cuda.synchronize()
+    assert torch.equal(again, out)
+
+
 def test_bf16_through_plain_fp32_kernels():
     w = inputs.TINY.scaled(dtype="bf16", d=128, T=4, F=200, H=2)
     x = inputs.generate(w, "cuda")
