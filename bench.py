@@ -273,6 +273,8 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     dev = f"cuda:{local_rank}"
     x = inputs.generate(w, dev)
     flags = {"auto": 0, "frames": binding.VDN_FLAG_SCAN_FRAMEWISE, "chunks": binding.VDN_FLAG_SCAN_CHUNKWISE}[args.scan]
+    if args.exact_stats:
+        flags |= binding.VDN_FLAG_EXACT_STATS
     vda = binding.Vda(w.d, w.dtype, device=local_rank, flags=flags)
     out = torch.empty_like(x["q"])
     stream = torch.cuda.current_stream()
@@ -416,7 +418,7 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     roof = None
     if kt:
         dom = max(kt, key=kt.get)
-        kind = "gram" if "gram" in dom else ("readout" if "readout" in dom else None)
+        kind = "gram" if "gram" in dom else ("readout" if dom == "readout_tc" or dom == "readout_simt" else None)
         per_th = DRAM_BYTES_PER_TOKEN_HEAD.get(dom)
         traffic = per_th * w.B * w.T * w.F * w.H if per_th else None
         if kind is not None:
@@ -642,6 +644,8 @@ def main():
     ap.add_argument("--no-spatial", action="store_true", help="--stage prep without the 5x5 spatial filter")
     ap.add_argument("--q-l2-eps", type=float, default=0.0,
                     help="> 0: the read-out normalises the queries (vdn_vda_options.q_l2_eps); --stage prep then skips Q")
+    ap.add_argument("--exact-stats", action="store_true",
+                    help="VDN_FLAG_EXACT_STATS: frame statistics from the exactly weighted keys (not the headline)")
     ap.add_argument("--sustain-s", type=float, default=2.0,
                     help="seconds of back-to-back forwards after the timed region for the `sustained` block (0 = none)")
     ap.add_argument("--launcher-selftest", action="store_true",

@@ -22,6 +22,7 @@ VDN_FLAG_FORCE_SIMT = 1
 VDN_FLAG_ADDITIVE_RULE = 4
 VDN_FLAG_SCAN_CHUNKWISE = 8
 VDN_FLAG_SCAN_FRAMEWISE = 16
+VDN_FLAG_EXACT_STATS = 32
 VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_READ_BWD = range(7)
 
 EXPORTS = (

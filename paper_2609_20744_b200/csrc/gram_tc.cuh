@@ -26,26 +26,38 @@
 
 namespace vdn {
 
-struct GramTc {
+// EXACT = true (VDN_FLAG_EXACT_STATS): the weighted key beta k is carried as TWO bf16 numbers, the rounded product and
+// its rounding residue (beta k has 16 significant bits, so the pair holds it exactly), and every tile is contracted
+// twice, once per part, into the same accumulator.  The statistics are then the exact fp32-accumulated sums of the
+// 16-bit inputs -- what the plain-fp32 kernels compute -- with beta rounded to bf16 (a per-token weight change of
+// 2^-9, the same in A_t and B_t).  Why it matters: rounding each token's weighted key to bf16 moves it by 2^-9 in a
+// direction of its own; the update of Eq. 5 damps what a frame writes along a repeated key by 1 / (1 + lambda_max)
+// but not those residues, so for frames of (nearly) identical keys (Sec. A.3) the error relative to the result grows
+// like lambda_max 2^-10.  Costs: twice the tensor-core work, a second operand buffer (so a two-stage ring).
+template <bool EXACT>
+struct GramTcCfg {
   static constexpr int D = 128;
   static constexpr int TILE = 128;                 // tokens per tile
-  static constexpr int STAGES = 3;
+  static constexpr int STAGES = EXACT ? 2 : 3;
+  static constexpr int PARTS = EXACT ? 2 : 1;      // bf16 parts of the weighted key
   static constexpr int BOX_BYTES = TILE * 128;     // one 64-channel box: 128 tokens x 128 B
   static constexpr int STAGE_BYTES = 4 * BOX_BYTES;       // K lo, K hi, V lo, V hi
   static constexpr int KP_HALF_BYTES = 2 * 64 * 128;      // 2 boxes x 64 tokens x 128 B
-  static constexpr int OFF_KP = STAGES * STAGE_BYTES;
-  static constexpr int OFF_BAR = OFF_KP + 2 * KP_HALF_BYTES;
+  static constexpr int OFF_KP = STAGES * STAGE_BYTES;     // [part][half]
+  static constexpr int OFF_BAR = OFF_KP + PARTS * 2 * KP_HALF_BYTES;
   static constexpr int USED_BYTES = OFF_BAR + 128;
-  static constexpr int SMEM_BYTES = 232448;                // everything an SM offers one CTA; the slack
-                                                           // absorbs the 1024-byte alignment
+  static constexpr int SMEM_BYTES = EXACT ? USED_BYTES + 1024 : 232448;   // plain: everything an SM offers one CTA; the
+                                                                          // slack absorbs the 1024-byte alignment
   static constexpr int THREADS = 448;
 };
+using GramTc = GramTcCfg<false>;
 
-__global__ void __launch_bounds__(GramTc::THREADS, 1)
+template <bool EXACT>
+__global__ void __launch_bounds__(GramTcCfg<EXACT>::THREADS, 1)
 gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                const float* __restrict__ beta, float* __restrict__ stats, Shape s, tc::DevStatus ds) {
   using namespace tc;
-  using G = GramTc;
+  using G = GramTcCfg<EXACT>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -72,7 +84,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const long long nitems = s.work_items();
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 3; ++i) { mbar_init(FULL(i), 1); mbar_init(EMPTY(i), 1); }
+    for (int i = 0; i < G::STAGES; ++i) { mbar_init(FULL(i), 1); mbar_init(EMPTY(i), 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(SCALED(i), 8); mbar_init(KPFREE(i), 1);      // one arrival per weighting warp
       mbar_init(ACCFULL(i), 1);  mbar_init(ACCEMPTY(i), 4);   // ... per drain warp
@@ -134,13 +146,17 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           for (int half = 0; half < 2; ++half) {
             if (!mbar_wait(SCALED(half), it & 1, wc)) { ok = false; break; }
             tc_fence_after_sync();
-            const uint32_t a_base = base + G::OFF_KP + half * G::KP_HALF_BYTES;
             const uint32_t b_base = base + st * G::STAGE_BYTES + half * 64 * 128;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const uint64_t adesc = make_smem_desc(a_base + j * 2048, 64 * 128, 1024);
-              const uint64_t bdesc = make_smem_desc(b_base + j * 2048, G::BOX_BYTES, 1024);
-              mma_bf16_ss(acc, adesc, bdesc, idesc, (tile | half | j) != 0 ? 1u : 0u);
+            for (int part = 0; part < G::PARTS; ++part) {     // EXACT: the residue part first (smallest terms first)
+              const int pp = G::PARTS - 1 - part;
+              const uint32_t a_base = base + G::OFF_KP + (pp * 2 + half) * G::KP_HALF_BYTES;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const uint64_t adesc = make_smem_desc(a_base + j * 2048, 64 * 128, 1024);
+                const uint64_t bdesc = make_smem_desc(b_base + j * 2048, G::BOX_BYTES, 1024);
+                mma_bf16_ss(acc, adesc, bdesc, idesc, (tile | half | j | part) != 0 ? 1u : 0u);
+              }
             }
             mma_commit(KPFREE(half));
           }
@@ -216,21 +232,39 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           // beta rounded to bf16, then one packed bf16 multiply per channel pair (round to nearest): the
           // float->bf16 conversion instruction is slow on this GPU and kept this loop from hiding under HBM
           const __nv_bfloat162 w2 = __float2bfloat162_rn(bu[half]);
+          const float wf = __low2float(w2);     // EXACT: the rounded gate, as the factor of the exact product
           // all eight loads first, then the stores: written as one load-store pair per chunk the compiler
           // must keep them in order (the two shared-memory pointers might alias) and every chunk pays the
           // full shared-memory latency
-          uint4 raw[4];
+          uint4 raw[4], res[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) raw[j] = *reinterpret_cast<const uint4*>(src + (((q4 + j) ^ (r & 7)) * 16));
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             __nv_bfloat162* x = reinterpret_cast<__nv_bfloat162*>(&raw[j]);
+            uint32_t* ru = reinterpret_cast<uint32_t*>(&res[j]);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) x[e] = __hmul2(x[e], w2);
+            for (int e = 0; e < 4; ++e) {
+              if constexpr (EXACT) {
+                // the product's rounding residue beta k - rn(beta k): exact in fp32 (one FMA each), at most 8
+                // significant bits, so its fp32 pattern has a zero low half and the bf16 is that pattern's top half
+                const uint32_t ku = *reinterpret_cast<const uint32_t*>(&x[e]);
+                const __nv_bfloat162 g = __hmul2(x[e], w2);
+                const uint32_t gu = *reinterpret_cast<const uint32_t*>(&g);
+                const float r0 = fmaf(wf, __uint_as_float(ku << 16), -__uint_as_float(gu << 16));
+                const float r1 = fmaf(wf, __uint_as_float(ku & 0xFFFF0000u), -__uint_as_float(gu & 0xFFFF0000u));
+                ru[e] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+                x[e] = g;
+              } else {
+                x[e] = __hmul2(x[e], w2);
+              }
+            }
           }
 #pragma unroll
-          for (int j = 0; j < 4; ++j)            // chunks staggered across rows: conflict-free
+          for (int j = 0; j < 4; ++j) {          // chunks staggered across rows: conflict-free
             *reinterpret_cast<uint4*>(dst + (((q4 + j) ^ (r & 7)) * 16)) = raw[j];
+            if constexpr (EXACT) *reinterpret_cast<uint4*>(dst + 2 * G::KP_HALF_BYTES + (((q4 + j) ^ (r & 7)) * 16)) = res[j];
+          }
           fence_proxy_async_smem();
           mbar_arrive_warp(SCALED(half));
         }

@@ -336,8 +336,10 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   constexpr int D = 128;
   if (!h->encode) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   if (!h->tc_attrs_set) {
-    VDN_CUDA(h, cudaFuncSetAttribute(vdn::gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     vdn::GramTc::SMEM_BYTES));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::gram_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::GramTcCfg<false>::SMEM_BYTES));
+    VDN_CUDA(h, cudaFuncSetAttribute(vdn::gram_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     vdn::GramTcCfg<true>::SMEM_BYTES));
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::ScanTc::SMEM_BYTES));
     VDN_CUDA(h, (cudaFuncSetAttribute(vdn::scan_tc_kernel<vdn::SCAN_FRAMES, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -378,9 +380,13 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
   }
   if (x.phase != 2) {
     prof_begin(h, st);
-    vdn::gram_tc_kernel<<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(tmK, tmV, beta, stats, s,
-                                                                                         dev_status(h));
-    prof_mark(h, st, nk++, "gram_tc");
+    if (h->cfg.flags & VDN_FLAG_EXACT_STATS)
+      vdn::gram_tc_kernel<true><<<persistent, vdn::GramTcCfg<true>::THREADS, vdn::GramTcCfg<true>::SMEM_BYTES, st>>>(
+          tmK, tmV, beta, stats, s, dev_status(h));
+    else
+      vdn::gram_tc_kernel<false><<<persistent, vdn::GramTc::THREADS, vdn::GramTc::SMEM_BYTES, st>>>(
+          tmK, tmV, beta, stats, s, dev_status(h));
+    prof_mark(h, st, nk++, (h->cfg.flags & VDN_FLAG_EXACT_STATS) ? "gram_tc_exact" : "gram_tc");
     const bool additive = (h->cfg.flags & VDN_FLAG_ADDITIVE_RULE) != 0;
     const float bscale = additive ? 1.0f / sqrtf((float)s.F) : 0.f;
     if (additive) {
