@@ -57,15 +57,17 @@
  *   bf16 I/O, bound 2e-2, plain-fp32 kernels (VDN_FLAG_FORCE_SIMT): within 2e-2 for every input tried, including
  *     lambda_max of 1e5 and beyond, except all-identical keys at lambda_max >= 8000 (3e-2).
  *   bf16 I/O, bound 2e-2, tensor-core kernels: the weighted key beta_u k_u of every token is rounded to bf16 for the
- *     contraction.  Within 2e-2 (typically 4e-3) for unstructured keys, for the benchmark's correlated keys, for key
- *     norms in [0.25, 4] around shared directions (lambda_max 2000), and with nine keys in ten of a frame bit-identical
- *     up to lambda_max 2000; NOT within 2e-2 when 99 % or more of a frame's keys are bit-identical (3e-2 .. 8e-2 at
- *     99 %, more at 100 %, from lambda_max of about 5 on), nor for lambda_max of 7000 and more.
- *   The same with VDN_FLAG_EXACT_STATS (the weighted keys enter the contraction exactly): what remains is the
- *     tensor-core resolve and scan, whose fp32 accumulation truncates (a floor of about 5e-6 relative to the terms of
- *     a product instead of 1e-7; the error grows like that floor times lambda_max).  Within 2e-2 with 99 % of a
- *     frame's keys identical up to lambda_max of about 500 and with all keys identical up to about 130; otherwise as
- *     above.  Beyond these ranges use the plain-fp32 kernels.
+ *     contraction, and the resolve and the scan accumulate on the tensor cores, whose fp32 accumulation truncates (an
+ *     accuracy floor of about 5e-6 of a product's terms instead of 1e-7; the error grows like that floor times
+ *     lambda_max).  Within 2e-2 (typically 4e-3) for unstructured keys, for the benchmark's correlated keys, for key
+ *     norms in [0.25, 4] around shared directions (lambda_max 2300: 1e-2) and with nine keys in ten of a frame
+ *     bit-identical up to lambda_max 2000 (9e-3).  NOT within 2e-2 when 99 % or more of a frame's keys are
+ *     bit-identical (3e-2 .. 8e-2 at 99 %, more at 100 %, from lambda_max of about 5 on), nor for lambda_max beyond
+ *     about 2000 (5e-2 at 2200, 1e-1 at 7400).
+ *   The same with VDN_FLAG_EXACT_STATS (the weighted keys enter the contraction exactly): within 2e-2 with 99 % of a
+ *     frame's keys identical up to lambda_max of about 1000 (4e-3; borderline at 2000: 1e-2 .. 3e-2 depending on the
+ *     draw) and with all of them identical up to lambda_max of about 600 (1.5e-2); the limit of lambda_max of about
+ *     2000 remains (2.3e-2 at 2200).  Beyond these ranges use the plain-fp32 kernels.
  */
 #ifndef VDN_VDA_H_
 #define VDN_VDA_H_

@@ -148,7 +148,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
     tma_prefetch_desc(&tmC);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_slot), 128);
+    tmem_alloc(smem_u32(tmem_slot), 256);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -179,7 +179,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(128, 128 / NS, false, true);
+      // The transition as the A operand.  The resolve kernel eliminates by row operations, so the matrix M it ends
+      // with is accurate as a LEFT inverse (M (I + A) - I is small; (I + A) M - I is larger by about the condition
+      // number), and the right-hand side here is of the form (I + A) z.  The product must therefore be M X, not
+      // M^T X -- in exact arithmetic the same thing.  The resolve stores M transposed (its threads own rows and write
+      // coalesced columns), so the stored matrix is read MN-major, which transposes it back.  A composed chunk
+      // (SCAN_CHUNKS) is stored as it is used: K-major.
+      constexpr bool A_MN = MODE != SCAN_CHUNKS;
+      constexpr uint32_t idesc = make_idesc_bf16(128, 128 / NS, A_MN, true);
       bool ok = true;
       for (int s = 0; s < nsteps && ok; ++s) {
         if (!mbar_wait(XREADY, s & 1, wc)) break;
@@ -194,9 +201,16 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
             const uint32_t xb = base + S::OFF_X + px * S::PART_BYTES;
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-              const uint64_t adesc = make_smem_desc(cb + (k >> 2) * S::BOX_BYTES + (k & 3) * 32, 16, 1024);
+              const uint64_t adesc = A_MN ? make_smem_desc(cb + k * 2048, S::BOX_BYTES, 1024)
+                                          : make_smem_desc(cb + (k >> 2) * S::BOX_BYTES + (k & 3) * 32, 16, 1024);
               const uint64_t bdesc = make_smem_desc(xb + k * 2048, S::BOX_BYTES, 1024);
-              mma_bf16_ss(tmem_base, adesc, bdesc, idesc, (pc == 2 && k == 0) ? 0u : 1u);
+              // two accumulators: the leading product C1 X1 in one, the five correction products (each at most
+              // 2^-8 of it) in the other.  The tensor core's fp32 accumulation truncates, a one-sided error of about
+              // 2^-23 of the running sum per accumulation; kept apart, the leading sum sees 8 accumulations instead of
+              // 48 and the corrections' truncation is relative to their own small size.  The state warps add the two.
+              const bool lead = pc == 0 && px == 0;
+              mma_bf16_ss(tmem_base + (lead ? 128u : 0u), adesc, bdesc, idesc,
+                          ((lead || (pc == 2 && px == 0)) && k == 0) ? 0u : 1u);
             }
           }
           mma_commit(CFREE(pc));
@@ -364,8 +378,15 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
       if (!mbar_wait(ACCFULL, s & 1, wc)) break;
       tc_fence_after_sync();
       float z[CW];
-      tmem_ld32(taddr, z);
-      tmem_wait_ld();
+      tmem_ld32(taddr + 128, z);        // the leading product
+#pragma unroll
+      for (int hc = 0; hc < CW / 16; ++hc) {   // plus the five correction products, 16 columns at a time (registers)
+        float zc[16];
+        tmem_ld16(taddr + hc * 16, zc);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) z[hc * 16 + e] += zc[e];
+      }
       if (additive && writes) {
 #pragma unroll
         for (int e = 0; e < CW; ++e) z[e] = fmaf(bscale, bt[e], z[e]);
@@ -403,7 +424,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
   __syncthreads();
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, 128);
+    tmem_dealloc(tmem_base, 256);
   }
 }
 
