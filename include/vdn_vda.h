@@ -57,9 +57,9 @@
  *   bf16 I/O, bound 2e-2, plain-fp32 kernels (VDN_FLAG_FORCE_SIMT): within 2e-2 for every input tried, including
  *     lambda_max of 1e5 and beyond, except all-identical keys at lambda_max >= 8000 (3e-2).
  *   bf16 I/O, bound 2e-2, tensor-core kernels: the weighted key beta_u k_u of every token is rounded to bf16 for the
- *     contraction, and the resolve and the scan accumulate on the tensor cores, whose fp32 accumulation truncates (an
- *     accuracy floor of about 5e-6 of a product's terms instead of 1e-7; the error grows like that floor times
- *     lambda_max).  Within 2e-2 (typically 4e-3) for unstructured keys, for the benchmark's correlated keys, for key
+ *     contraction, and the inverse comes from the tensor-core resolve, which reaches about 5e-6 of the inverse's
+ *     largest entry where the plain-fp32 resolve reaches 1e-6 (measured against an fp64 inverse of the same matrix);
+ *     the error of the layer grows like that figure times lambda_max.  Within 2e-2 (typically 4e-3) for unstructured keys, for the benchmark's correlated keys, for key
  *     norms in [0.25, 4] around shared directions (lambda_max 2300: 1e-2) and with nine keys in ten of a frame
  *     bit-identical up to lambda_max 2000 (9e-3).  NOT within 2e-2 when 99 % or more of a frame's keys are
  *     bit-identical (3e-2 .. 8e-2 at 99 %, more at 100 %, from lambda_max of about 5 on), nor for lambda_max beyond

@@ -148,7 +148,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
     tma_prefetch_desc(&tmC);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_slot), 256);
+    tmem_alloc(smem_u32(tmem_slot), 128);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -204,13 +204,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
               const uint64_t adesc = A_MN ? make_smem_desc(cb + k * 2048, S::BOX_BYTES, 1024)
                                           : make_smem_desc(cb + (k >> 2) * S::BOX_BYTES + (k & 3) * 32, 16, 1024);
               const uint64_t bdesc = make_smem_desc(xb + k * 2048, S::BOX_BYTES, 1024);
-              // two accumulators: the leading product C1 X1 in one, the five correction products (each at most
-              // 2^-8 of it) in the other.  The tensor core's fp32 accumulation truncates, a one-sided error of about
-              // 2^-23 of the running sum per accumulation; kept apart, the leading sum sees 8 accumulations instead of
-              // 48 and the corrections' truncation is relative to their own small size.  The state warps add the two.
-              const bool lead = pc == 0 && px == 0;
-              mma_bf16_ss(tmem_base + (lead ? 128u : 0u), adesc, bdesc, idesc,
-                          ((lead || (pc == 2 && px == 0)) && k == 0) ? 0u : 1u);
+              mma_bf16_ss(tmem_base, adesc, bdesc, idesc, (pc == 2 && k == 0) ? 0u : 1u);
             }
           }
           mma_commit(CFREE(pc));
@@ -378,15 +372,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
       if (!mbar_wait(ACCFULL, s & 1, wc)) break;
       tc_fence_after_sync();
       float z[CW];
-      tmem_ld32(taddr + 128, z);        // the leading product
-#pragma unroll
-      for (int hc = 0; hc < CW / 16; ++hc) {   // plus the five correction products, 16 columns at a time (registers)
-        float zc[16];
-        tmem_ld16(taddr + hc * 16, zc);
-        tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 16; ++e) z[hc * 16 + e] += zc[e];
-      }
+      tmem_ld32(taddr, z);
+      tmem_wait_ld();
       if (additive && writes) {
 #pragma unroll
         for (int e = 0; e < CW; ++e) z[e] = fmaf(bscale, bt[e], z[e]);
@@ -424,7 +411,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
   __syncthreads();
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, 256);
+    tmem_dealloc(tmem_base, 128);
   }
 }
 

@@ -29,10 +29,10 @@ is loosened here.  What the cases below establish is the range of inputs in whic
   * the same kernels with VDN_FLAG_EXACT_STATS contract the exactly weighted keys (two bf16 parts).  2e-2 then holds
     with 99 % identical keys up to lambda_max of about one thousand (at two thousand it is borderline: 1e-2 .. 3e-2
     depending on the draw) and with all keys identical up to about 600.
-  * either way the tensor-core resolve and scan set a limit of their own: their fp32 accumulation truncates, which
-    leaves a floor of about 5e-6 relative to a product's terms instead of 1e-7, and the error grows like that floor
-    times lambda_max: 2e-2 is left at lambda_max of a little over two thousand.  Beyond, the plain-fp32 kernels are
-    the ones to use.
+  * either way the tensor-core resolve sets a limit of its own: its inverse is good to about 5e-6 of the largest
+    entry (the plain-fp32 resolve: 1e-6; both measured against an fp64 inverse of the same matrix), and the error
+    of the layer grows like that figure times lambda_max: 2e-2 is left at lambda_max of a little over two thousand.
+    Beyond, the plain-fp32 kernels are the ones to use.
 """
 import numpy as np
 import pytest
