@@ -547,8 +547,9 @@ def run_prep(args, w, local_rank: int):
         roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peaks['source']}",
                 "kernel_ms": kt[dom], "algorithmic_bytes_per_launch": kb}
-    if dom == "prep_kv":
-        achieved = flops / (kt[dom] / 1e3) / 1e12
+    if dom == "prep_spatial":
+        sp_flops = 2 * elems * 2 * 25                # K and V: 25 fused multiply-adds per element
+        achieved = sp_flops / (kt[dom] / 1e3) / 1e12
         roof = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
                 "frac": achieved / alu_peak, "traffic": None,
                 "peak_source": f"{prop.multi_processor_count} SMs x 128 fp32 lanes x 2 x 1.965 GHz",

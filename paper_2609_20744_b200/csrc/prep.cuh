@@ -1,20 +1,16 @@
 // Feature preparation in front of the recurrence (Sec. 2.3; "VDA-Prep", Sec. 5):
 //     K, V : depthwise 5 x 5 spatial filter and five-tap temporal filter (one pair per channel, taps centred,
 //            zero padding), then SiLU;      K, Q : L2 normalisation over the d channels of a (token, head).
-// One pass over K and V: every input element is read once from HBM (its halo re-reads hit L2), nothing
-// intermediate is written.
 //
-// prep_kv_kernel: one CTA per (head, spatial tile of ROWS x 8 tokens, batch, tensor) walks the frames in order.
-// A thread owns two neighbouring channels of the head (the two lanes of every packed fp32 FMA) and one tile row of
-// 8 tokens.  Per frame: the tile and its 2-token halo arrive in shared memory (cp.async, double buffered); the
-// thread slides along its row, five inputs per column, scattering each column into the (up to) five outputs it
-// touches, so an input is read from shared memory once per output row, not once per tap; the spatial result
-// enters a five-frame ring in registers, from which the temporal filter produces the frame two steps back;
-// SiLU; for K the sum of squares over the head's channels (warp shuffles, plus one shared-memory exchange when
-// the head spans two warps); store.  30 fused multiply-adds per element: this kernel is bound by the fp32 pipe.
-//
-// prep_kv_temporal_kernel: the same without the spatial filter (a streaming kernel, bound by HBM).
+// prep_spatial_kernel: the 5 x 5 spatial filter, 25 fused multiply-adds per element: bound by the fp32 pipe.
+// prep_kv_temporal_kernel: the temporal filter, SiLU and the norm of K, one read and one write per element: bound
+//     by HBM.  Run in place on the spatial kernel's result, or alone when no spatial filters are passed (the
+//     operation of the paper's VDA-Prep).
 // prep_q_kernel: L2 normalisation of Q; bound by HBM.
+//
+// A single kernel that did all of it in one pass over K and V (tile + halo in shared memory, the spatial results of
+// five frames in a register ring) was the first version: 242 registers, one CTA of eight warps per SM, 8.9 ms on
+// the 768p shape where the two kernels take 4.9 + 2.3 ms.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -94,17 +90,6 @@ __device__ __forceinline__ void silu2(f32x2 x, float& y0, float& y1) {
   unpack2(mul2(x, pack2(r0, r1)), y0, y1);
 }
 
-struct PrepKv {
-  static constexpr int TX = 8;          // tile columns = tokens per thread
-  static constexpr int HALO = 2;
-  static constexpr int THREADS = 256;
-  __host__ __device__ static constexpr int rows(int D) { return THREADS / (D / 2); }            // tile rows
-  __host__ __device__ static constexpr int tile_tokens(int D) { return (rows(D) + 2 * HALO) * (TX + 2 * HALO); }
-  // two tiles (the asynchronous copies' double buffer) and the exchange area of the norm
-  static constexpr size_t RED_BYTES = 1024;
-  static constexpr size_t smem_bytes(int D, int es) { return (size_t)2 * tile_tokens(D) * D * es + RED_BYTES; }
-};
-
 struct PrepArgs {
   const void* in[2];          // k, v   [B,T,F,H,d]
   void* out[2];
@@ -114,56 +99,66 @@ struct PrepArgs {
   float l2_eps;
 };
 
+// The spatial filter alone: out[t, y, x, c] = sum_{i,j} ws[c, i, j] in[t, y+i-2, x+j-2, c]  (the first half of the
+// preparation; prep_kv_temporal_kernel, run in place on the result, is the second).  Splitting the fused kernel in
+// two costs one more round trip of K and V through HBM (the temporal half streams at copy speed) and, for 16-bit
+// I/O, one rounding of the intermediate to the I/O type; it frees the 80 registers of the fused kernel's five-frame
+// ring, which held it to one CTA of eight warps per SM, its fp32 pipe idle through every barrier and every
+// temporal / SiLU / norm phase.
+//
+// One CTA per (head, 8 x 8 token tile, batch, tensor) walks the frames; the tile and its 2-token halo arrive by
+// cp.async, double buffered.  A thread owns two neighbouring channels (the lanes of the packed fp32 FMA) and two
+// tile rows of eight tokens: six input rows per column feed ten tap rows, 400 packed FMAs for 72 shared-memory
+// reads.  Two CTAs per SM.
+struct PrepSpatial {
+  static constexpr int TX = 8, RPT = 2, HALO = 2;            // columns and rows per thread
+  static constexpr int THREADS = 256;
+  __host__ __device__ static constexpr int rows(int D) { return RPT * THREADS / (D / 2); }      // tile rows
+  __host__ __device__ static constexpr int tile_tokens(int D) { return (rows(D) + 2 * HALO) * (TX + 2 * HALO); }
+  static constexpr size_t smem_bytes(int D, int es) { return (size_t)2 * tile_tokens(D) * D * es; }
+};
+
 template <typename Tio, int D>
-__global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a, Shape s) {
-  using P = PrepKv;
+__global__ void __launch_bounds__(PrepSpatial::THREADS, sizeof(Tio) == 2 ? 2 : 1) prep_spatial_kernel(PrepArgs a, Shape s) {
+  using P = PrepSpatial;
   constexpr int ROWS = P::rows(D);
-  constexpr int TX = P::TX, HALO = P::HALO;
+  constexpr int TX = P::TX, HALO = P::HALO, RPT = P::RPT;
   constexpr int SW = TX + 2 * HALO, SH = ROWS + 2 * HALO;       // tile with halo
-  constexpr int GT = D / 2;                                      // threads per tile row (one head's channel pairs)
-  constexpr int NW = GT / 32;                                    // warps per tile row
-  static_assert(TX == 8, "the norm's reduction is written for eight tokens per thread");
+  constexpr int GT = D / 2;                                      // threads per row pair (one head's channel pairs)
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Tio* tile = reinterpret_cast<Tio*>(smem_raw);                  // [2][SH][SW][D]
-  float* red = reinterpret_cast<float*>(smem_raw + (size_t)2 * SH * SW * D * sizeof(Tio));     // [2][ROWS][NW][TX]
 
   const int h = blockIdx.x;
   const int tiles_x = (a.X + TX - 1) / TX;
   const int x0 = (blockIdx.y % tiles_x) * TX, y0 = (blockIdx.y / tiles_x) * ROWS;
-  const int which = blockIdx.z & 1;                              // 0 = K (normalised), 1 = V
+  const int which = blockIdx.z & 1;                              // 0 = K, 1 = V
   const int b = blockIdx.z >> 1;
   const Tio* __restrict__ src = static_cast<const Tio*>(which == 0 ? a.in[0] : a.in[1]);
   Tio* __restrict__ dst = static_cast<Tio*>(which == 0 ? a.out[0] : a.out[1]);
 
-  const int tid = threadIdx.x, lane = tid & 31;
-  const int g = tid / GT;                   // tile row of this thread
+  const int tid = threadIdx.x;
+  const int g = tid / GT;                   // row pair of this thread: tile rows 2g, 2g+1
   const int cp = tid % GT;                  // channel pair within the head
-  const int ch = h * D + 2 * cp;            // first of this thread's two channels, [H*d] index
+  const int ch = h * D + 2 * cp;
 
-  // this thread's filters, both channels packed: 25 spatial + 5 temporal taps
-  f32x2 wsp[5][5], wtp[5];
+  f32x2 wsp[5][5];
   {
     const float* w0 = (which == 0 ? a.ws[0] : a.ws[1]) + (size_t)ch * 25;
 #pragma unroll
     for (int i = 0; i < 5; ++i)
 #pragma unroll
       for (int j = 0; j < 5; ++j) wsp[i][j] = pack2(__ldg(w0 + i * 5 + j), __ldg(w0 + 25 + i * 5 + j));
-    const float* t0 = (which == 0 ? a.wt[0] : a.wt[1]) + (size_t)ch * 5;
-#pragma unroll
-    for (int i = 0; i < 5; ++i) wtp[i] = pack2(__ldg(t0 + i), __ldg(t0 + 5 + i));
   }
 
   const int first = s.t0, last = s.t0 + s.Tn - 1;
   const size_t frame_elems = (size_t)s.F * s.H * D;
-  // this thread's first output element: token (y0 + g, x0) of the first scanned frame, its channel pair
-  Tio* pdst = dst + token_offset(s, b, first, min(y0 + g, a.Y - 1) * a.X + x0, h) + 2 * cp;
-  const bool row_ok = y0 + g < a.Y;
+  const int yr = y0 + RPT * g;              // first of this thread's two output rows
+  Tio* pdst = dst + token_offset(s, b, first, min(yr, a.Y - 1) * a.X + x0, h) + 2 * cp;
 
-  // Frame t's tile (with halo) -> raw buffer t & 1; tokens outside the frame are zeros.  A thread copies the same
-  // 16-byte pieces of every frame, so their offsets inside a frame are worked out once (-1: outside the frame).
-  constexpr int CHUNKS = D * (int)sizeof(Tio) / 16;              // 16-byte pieces per token
+  // 16-byte pieces of the tile this thread copies, the same for every frame (-1: outside the frame -> zeros)
+  constexpr int CHUNKS = D * (int)sizeof(Tio) / 16;
   constexpr int NPIECE = (SH * SW * CHUNKS + P::THREADS - 1) / P::THREADS;
-  int goff[NPIECE];                                              // byte offset inside the frame, or -1
+  int goff[NPIECE];
 #pragma unroll
   for (int i = 0; i < NPIECE; ++i) {
     const int e = tid + i * P::THREADS;
@@ -188,128 +183,48 @@ __global__ void __launch_bounds__(PrepKv::THREADS, 1) prep_kv_kernel(PrepArgs a,
     cp_async_commit();
   };
 
-  f32x2 ring[5][TX];                        // spatial results of the last five frames (slot = step % 5)
+  stage(first);
+#pragma unroll 1
+  for (int t = first; t <= last; ++t) {
+    if (t + 1 <= last) { stage(t + 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+    __syncthreads();                        // frame t's tile is complete
+    const Tio* base = tile + (size_t)(t & 1) * SH * SW * D + (size_t)(RPT * g) * SW * D + 2 * cp;
+    f32x2 acc[RPT][TX];
 #pragma unroll
-  for (int i = 0; i < 5; ++i)
+    for (int r = 0; r < RPT; ++r)
 #pragma unroll
-    for (int j = 0; j < TX; ++j) ring[i][j] = 0ull;
-
-  int par = 0;                              // which half of the norm's exchange area this step uses
-
-  // One step: spatial filter of frame t = first + step into ring slot r, then the temporal filter, SiLU, norm and
-  // store of frame t - 2.  EDGE = false is the steady state, where all the frames involved exist.
-  auto one_step = [&](auto rc, auto ec, int step) {
-    constexpr int r = decltype(rc)::value;
-    constexpr bool EDGE = decltype(ec)::value;
-    const int t = first + step;             // input frame of this step; the output frame is t - 2
-    if (!EDGE || t <= last) {
-      if (!EDGE || t + 1 <= last) { stage(t + 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
-      __syncthreads();                      // frame t's tile is complete
-      // (Widening a 16-bit tile to fp32 once per frame, so that the loop below reads ready pairs, was slower:
-      // 12.8 ms instead of 10.4 ms on the 768p clip; the shared-memory port is the scarcer resource here.)
-      const Tio* base = tile + (size_t)(t & 1) * SH * SW * D + (size_t)g * SW * D + 2 * cp;
-      // ---- spatial filter of frame t for this thread's row: slide over the SW input columns
-      f32x2 (&acc)[TX] = ring[r];           // the spatial result accumulates straight into this step's ring slot
+      for (int j = 0; j < TX; ++j) acc[r][j] = 0ull;
 #pragma unroll
-      for (int j = 0; j < TX; ++j) acc[j] = 0ull;
+    for (int xi = 0; xi < SW; ++xi) {       // input column xi sits at x0 - 2 + xi
+      f32x2 in[4 + RPT];
 #pragma unroll
-      for (int xi = 0; xi < SW; ++xi) {     // input column xi sits at x0 - 2 + xi
-        f32x2 in[5];
+      for (int i = 0; i < 4 + RPT; ++i) in[i] = load_pair(base + ((size_t)i * SW + xi) * D);
 #pragma unroll
-        for (int i = 0; i < 5; ++i) in[i] = load_pair(base + ((size_t)i * SW + xi) * D);
+      for (int i = 0; i < 5; ++i) {
 #pragma unroll
-        for (int i = 0; i < 5; ++i) {       // neighbouring instructions update different accumulators
+        for (int j = 0; j < 5; ++j) {       // tap column j: output column xo = xi - j
+          const int xo = xi - j;
+          if (xo < 0 || xo >= TX) continue;
 #pragma unroll
-          for (int j = 0; j < 5; ++j) {     // tap column j: output column xo = xi - j
-            const int xo = xi - j;
-            if (xo < 0 || xo >= TX) continue;
-            acc[xo] = fma2(wsp[i][j], in[i], acc[xo]);
+          for (int r = 0; r < RPT; ++r) acc[r][xo] = fma2(wsp[i][j], in[i + r], acc[r][xo]);
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < RPT; ++r) {
+      if (yr + r < a.Y) {
+#pragma unroll
+        for (int j = 0; j < TX; ++j) {
+          if (x0 + j < a.X) {
+            float o0, o1;
+            unpack2(acc[r][j], o0, o1);
+            store_pair(pdst + ((size_t)r * a.X + j) * (s.H * D), o0, o1);
           }
         }
       }
-      __syncthreads();                      // the buffer is overwritten by the copy issued at the start of the next step
-    } else {
-#pragma unroll
-      for (int j = 0; j < TX; ++j) ring[r][j] = 0ull;
-    }
-    // ---- temporal filter: output frame to = t - 2 = sum_i wt[i] S[to + i - 2]; S[to + i - 2] sits in slot (r + i + 1) % 5
-    if (EDGE && step < HALO) return;
-    float o0[TX], o1[TX];
-#pragma unroll
-    for (int j = 0; j < TX; ++j) {
-      f32x2 o = mul2(wtp[0], ring[(r + 1) % 5][j]);
-#pragma unroll
-      for (int i = 1; i < 5; ++i) o = fma2(wtp[i], ring[(r + i + 1) % 5][j], o);
-      if constexpr (sizeof(Tio) == 2) silu2_tanh(o, o0[j], o1[j]); else silu2(o, o0[j], o1[j]);
-    }
-    if (which == 0) {
-      // ---- L2 normalisation over the head's d channels (Sec. 2.3).  Eight sums over the row's lanes at once:
-      // each exchange halves the number of tokens a lane still carries, so a warp needs 9 shuffles instead of 40;
-      // the totals go through shared memory to every thread of the row.
-      float v4[4], v2[2], v1;
-      const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float lo = fmaf(o0[j], o0[j], o1[j] * o1[j]), hi = fmaf(o0[j + 4], o0[j + 4], o1[j + 4] * o1[j + 4]);
-        v4[j] = (b16 ? hi : lo) + __shfl_xor_sync(0xffffffffu, b16 ? lo : hi, 16);
-      }
-#pragma unroll
-      for (int j = 0; j < 2; ++j) v2[j] = (b8 ? v4[j + 2] : v4[j]) + __shfl_xor_sync(0xffffffffu, b8 ? v4[j] : v4[j + 2], 8);
-      v1 = (b4 ? v2[1] : v2[0]) + __shfl_xor_sync(0xffffffffu, b4 ? v2[0] : v2[1], 4);
-      v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
-      v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-      // this lane now holds the warp's sum for token 4 [lane & 16] + 2 [lane & 8] + [lane & 4]
-      float* mine = red + ((par * ROWS + g) * NW) * TX;
-      if ((lane & 3) == 0) mine[((tid >> 5) % NW) * TX + (b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)] = v1;
-      if constexpr (NW == 1) __syncwarp();
-      else asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(GT) : "memory");
-      float ss[TX];
-      {
-        const float4 x0 = *reinterpret_cast<const float4*>(mine), x1 = *reinterpret_cast<const float4*>(mine + 4);
-        ss[0] = x0.x; ss[1] = x0.y; ss[2] = x0.z; ss[3] = x0.w; ss[4] = x1.x; ss[5] = x1.y; ss[6] = x1.z; ss[7] = x1.w;
-      }
-#pragma unroll
-      for (int w = 1; w < NW; ++w) {
-        const float4 x0 = *reinterpret_cast<const float4*>(mine + w * TX), x1 = *reinterpret_cast<const float4*>(mine + w * TX + 4);
-        ss[0] += x0.x; ss[1] += x0.y; ss[2] += x0.z; ss[3] += x0.w; ss[4] += x1.x; ss[5] += x1.y; ss[6] += x1.z; ss[7] += x1.w;
-      }
-      par ^= 1;                             // the next step writes the other half: no second barrier (the block-wide
-                                            // barriers of the steps in between order the reuse)
-#pragma unroll
-      for (int j = 0; j < TX; ++j) {
-        float sc;
-        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(sc) : "f"(ss[j] + a.l2_eps));
-        o0[j] *= sc;
-        o1[j] *= sc;
-      }
-    }
-    if (row_ok) {
-#pragma unroll
-      for (int j = 0; j < TX; ++j)
-        if (x0 + j < a.X) store_pair(pdst + (size_t)j * (s.H * D), o0[j], o1[j]);
     }
     pdst += frame_elems;
-  };
-
-  using std::integral_constant;
-  const int nsteps = s.Tn + HALO;           // two extra steps flush the last two output frames
-  stage(first);
-#pragma unroll 1
-  for (int sb = 0; sb < nsteps; sb += 5) {
-    // ring slot r = step % 5 is static: sb is a multiple of five
-    if (sb >= 5 && sb + 4 + 1 <= s.Tn - 1) {
-      one_step(integral_constant<int, 0>{}, integral_constant<bool, false>{}, sb);
-      one_step(integral_constant<int, 1>{}, integral_constant<bool, false>{}, sb + 1);
-      one_step(integral_constant<int, 2>{}, integral_constant<bool, false>{}, sb + 2);
-      one_step(integral_constant<int, 3>{}, integral_constant<bool, false>{}, sb + 3);
-      one_step(integral_constant<int, 4>{}, integral_constant<bool, false>{}, sb + 4);
-    } else {
-      if (sb + 0 < nsteps) one_step(integral_constant<int, 0>{}, integral_constant<bool, true>{}, sb);
-      if (sb + 1 < nsteps) one_step(integral_constant<int, 1>{}, integral_constant<bool, true>{}, sb + 1);
-      if (sb + 2 < nsteps) one_step(integral_constant<int, 2>{}, integral_constant<bool, true>{}, sb + 2);
-      if (sb + 3 < nsteps) one_step(integral_constant<int, 3>{}, integral_constant<bool, true>{}, sb + 3);
-      if (sb + 4 < nsteps) one_step(integral_constant<int, 4>{}, integral_constant<bool, true>{}, sb + 4);
-    }
+    __syncthreads();                        // the buffer is overwritten by the copy issued at the start of the next step
   }
 }
 

@@ -537,41 +537,45 @@ vdn_status launch_scan_static(const float* stats, const float* inv, float* read,
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Feature preparation: two launches (K and V in one, Q in the other).
+// Feature preparation: the spatial filter of K and V (when filters are passed), their temporal half in place, Q.
 template <typename Tio, int D>
 vdn_status launch_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const void* v_in, void* q_out, void* k_out,
                           void* v_out, const Shape& s, const vdn_vda_prep_params& p, cudaStream_t st) {
-  using P = vdn::PrepKv;
-  const size_t smem = P::smem_bytes(D, (int)sizeof(Tio));
-  VDN_CUDA(h, cudaFuncSetAttribute(vdn::prep_kv_kernel<Tio, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   vdn::PrepArgs a;
   a.in[0] = k_in; a.in[1] = v_in; a.out[0] = k_out; a.out[1] = v_out;
   a.ws[0] = p.wk_spatial; a.ws[1] = p.wv_spatial; a.wt[0] = p.wk_temporal; a.wt[1] = p.wv_temporal;
   a.Y = p.Y; a.X = p.X;
   a.l2_eps = p.l2_eps > 0.f ? p.l2_eps : 1e-6f;
-  const int tiles = ((p.X + P::TX - 1) / P::TX) * ((p.Y + P::rows(D) - 1) / P::rows(D));
   prof_begin(h, st);
-  if (p.wk_spatial) {
-    vdn::prep_kv_kernel<Tio, D><<<dim3((unsigned)s.H, (unsigned)tiles, (unsigned)(2 * s.B)), P::THREADS, smem, st>>>(a, s);
-    prof_mark(h, st, 0, "prep_kv");
-  } else {
+  int nk = 0;
+  {
+    if (p.wk_spatial) {
+      // spatial filter into the outputs, then the temporal half in place on them
+      using P = vdn::PrepSpatial;
+      const size_t smem = P::smem_bytes(D, (int)sizeof(Tio));
+      VDN_CUDA(h, cudaFuncSetAttribute(vdn::prep_spatial_kernel<Tio, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      const int tiles = ((p.X + P::TX - 1) / P::TX) * ((p.Y + P::rows(D) - 1) / P::rows(D));
+      vdn::prep_spatial_kernel<Tio, D><<<dim3((unsigned)s.H, (unsigned)tiles, (unsigned)(2 * s.B)), P::THREADS, smem, st>>>(a, s);
+      prof_mark(h, st, nk++, "prep_spatial");
+      a.in[0] = k_out; a.in[1] = v_out;
+    }
     VDN_CUDA(h, cudaFuncSetAttribute(vdn::prep_kv_temporal_kernel<Tio, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      vdn::PrepKvTemporal::SMEM_BYTES));
     const long long threads = (long long)s.F * s.H * (D * (int)sizeof(Tio) / 16);
     constexpr int NT = vdn::PrepKvTemporal::THREADS;
     vdn::prep_kv_temporal_kernel<Tio, D><<<dim3((unsigned)((threads + NT - 1) / NT), (unsigned)(2 * s.B)), NT,
                                            vdn::PrepKvTemporal::SMEM_BYTES, st>>>(a, s);
-    prof_mark(h, st, 0, "prep_kv_temporal");
+    prof_mark(h, st, nk++, "prep_kv_temporal");
   }
-  h->launches = 1;
+  h->launches = nk;
   if (!q_in) { VDN_CUDA(h, cudaGetLastError()); return VDN_OK; }   // the queries are normalised by the read-out
   const long long rows = (long long)s.B * s.Tn * s.F * s.H;
   const long long per_cta = 8LL * (32 / (D * (int)sizeof(Tio) / 16)) * 4;       // rows one CTA covers per trip
   const long long want = (rows + per_cta - 1) / per_cta;
   const unsigned grid = (unsigned)(want < (long long)h->sm_count * 8 ? want : (long long)h->sm_count * 8);
   vdn::prep_q_kernel<Tio, D><<<grid, 256, 0, st>>>(static_cast<const Tio*>(q_in), static_cast<Tio*>(q_out), s, a.l2_eps);
-  prof_mark(h, st, 1, "prep_q");
-  h->launches = 2;
+  prof_mark(h, st, nk++, "prep_q");
+  h->launches = nk;
   VDN_CUDA(h, cudaGetLastError());
   return VDN_OK;
 }
@@ -811,7 +815,7 @@ vdn_status vdn_vda_prepare(vdn_vda_t h, const void* q_in, const void* k_in, cons
     return fail(h, VDN_ERR_INVALID_ARG, "Y * X must equal F");
   if ((long long)F * H * d * (long long)elem_size(h) > 0x7fffffffLL)
     return fail(h, VDN_ERR_UNSUPPORTED, "one frame of a tensor must stay below 2 GiB");
-  if (H > 65535 || 2LL * B > 65535 || ((long long)(p->X + 7) / 8) * ((p->Y + 3) / 4) > 65535)
+  if (H > 65535 || 2LL * B > 65535 || ((long long)(p->X + 7) / 8) * ((p->Y + 7) / 8) > 65535)
     return fail(h, VDN_ERR_UNSUPPORTED, "grid too large for the preparation kernel");
   DeviceGuard guard(h->cfg.device);
   if (!guard.ok) return fail(h, VDN_ERR_CUDA, "cannot make the handle's device current");
