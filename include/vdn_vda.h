@@ -35,8 +35,11 @@
  * Asynchrony.  vdn_vda_forward validates its arguments on the host, enqueues its kernels on `cuda_stream`
  * (a cudaStream_t passed as void*, NULL = the legacy default stream) and returns without synchronising.
  * One handle (one workspace) must not be used from two streams at the same time.  The device entry points
- * (forward, forward_ex, forward_opt, prepare) enqueue only kernels and memsets, so after one ordinary call of
- * the same kind (which sets kernel attributes) they may be recorded in a CUDA stream capture and replayed.
+ * (forward, forward_ex, forward_opt, prepare) enqueue only kernels, memsets and event waits, so after one ordinary
+ * call of the same kind (which sets kernel attributes and creates what the handle needs) they may be recorded in a
+ * CUDA stream capture and replayed.  When a layer has more scan chains (2 B H) than the GPU has SMs, part of the scan
+ * runs on a stream owned by the handle, forked from and joined back into cuda_stream by events inside the call:
+ * synchronising cuda_stream still covers everything.
  *
  * Errors.  Every call returns a vdn_status; nothing throws, aborts or traps.  Problems the host can see
  * (null or misaligned pointers, non-positive sizes, d != cfg.d, workspace too small, 32-bit index overflow,

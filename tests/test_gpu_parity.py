@@ -326,6 +326,28 @@ def test_forward_can_be_captured_in_a_cuda_graph():
     assert torch.equal(out, eager2) and not torch.equal(out, eager)
 
 
+def test_split_scan_can_be_captured_in_a_cuda_graph():
+    # more chains than SMs: the forward forks to the handle's side stream and joins again; captured, the fork becomes
+    # two branches of the graph.  After one eager call (which creates the side stream and its events).
+    w = inputs.TINY.scaled(dtype="bf16", d=128, B=1, H=80, T=4, F=130, seed=62)
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype)
+    eager = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"]).clone()
+    torch.cuda.synchronize()
+    out = torch.empty_like(x["q"])
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], out=out, stream=side)
+    for _ in range(2):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert vda.status() == binding.VDN_OK
+        assert torch.equal(out, eager)
+
+
 def test_token_permutation_within_frames_permutes_rows_only():
     w = inputs.TINY.scaled(d=128, T=3, F=96, H=2)
     x = inputs.generate(w, "cuda")
