@@ -275,6 +275,8 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
     flags = {"auto": 0, "frames": binding.VDN_FLAG_SCAN_FRAMEWISE, "chunks": binding.VDN_FLAG_SCAN_CHUNKWISE}[args.scan]
     if args.exact_stats:
         flags |= binding.VDN_FLAG_EXACT_STATS
+    if args.fp32_resolve:
+        flags |= binding.VDN_FLAG_FP32_RESOLVE
     vda = binding.Vda(w.d, w.dtype, device=local_rank, flags=flags)
     out = torch.empty_like(x["q"])
     stream = torch.cuda.current_stream()
@@ -647,6 +649,8 @@ def main():
                     help="> 0: the read-out normalises the queries (vdn_vda_options.q_l2_eps); --stage prep then skips Q")
     ap.add_argument("--exact-stats", action="store_true",
                     help="VDN_FLAG_EXACT_STATS: frame statistics from the exactly weighted keys (not the headline)")
+    ap.add_argument("--fp32-resolve", action="store_true",
+                    help="VDN_FLAG_FP32_RESOLVE: the inverse from the plain-fp32 Gauss-Jordan kernel (not the headline)")
     ap.add_argument("--sustain-s", type=float, default=2.0,
                     help="seconds of back-to-back forwards after the timed region for the `sustained` block (0 = none)")
     ap.add_argument("--launcher-selftest", action="store_true",

@@ -59,18 +59,22 @@
  *     60, 4e-4 at 150, 1e-2 at 2000.
  *   bf16 I/O, bound 2e-2, plain-fp32 kernels (VDN_FLAG_FORCE_SIMT): within 2e-2 for every input tried, including
  *     lambda_max of 1e5 and beyond, except all-identical keys at lambda_max >= 8000 (3e-2).
- *   bf16 I/O, bound 2e-2, tensor-core kernels: the weighted key beta_u k_u of every token is rounded to bf16 for the
- *     contraction, and the inverse comes from the tensor-core resolve, which reaches about 5e-6 of the inverse's
- *     largest entry where the plain-fp32 resolve reaches 1e-6 (measured against an fp64 inverse of the same matrix);
- *     the error of the layer grows like that figure times lambda_max.  Within 2e-2 (typically 4e-3) for unstructured keys, for the benchmark's correlated keys, for key
- *     norms in [0.25, 4] around shared directions (lambda_max 2300: 1e-2) and with nine keys in ten of a frame
- *     bit-identical up to lambda_max 2000 (9e-3).  NOT within 2e-2 when 99 % or more of a frame's keys are
- *     bit-identical (3e-2 .. 8e-2 at 99 %, more at 100 %, from lambda_max of about 5 on), nor for lambda_max beyond
- *     about 2000 (5e-2 at 2200, 1e-1 at 7400).
- *   The same with VDN_FLAG_EXACT_STATS (the weighted keys enter the contraction exactly): within 2e-2 with 99 % of a
- *     frame's keys identical up to lambda_max of about 1000 (4e-3; borderline at 2000: 1e-2 .. 3e-2 depending on the
- *     draw) and with all of them identical up to lambda_max of about 600 (1.5e-2); the limit of lambda_max of about
- *     2000 remains (2.3e-2 at 2200).  Beyond these ranges use the plain-fp32 kernels.
+ *   bf16 I/O, bound 2e-2, tensor-core kernels.  Two things set their range.  (1) The weighted key beta_u k_u of every
+ *     token is rounded to bf16 for the contraction, a 2^-9 move in a direction of its own; Eq. 5 damps what a frame
+ *     writes along a repeated key by 1 / (1 + lambda_max) but not those residues.  (2) The tensor-core resolve takes the
+ *     pivot rows from the matrix's own columns (it keeps the matrix symmetric only up to rounding) and reaches about
+ *     5e-6 of the inverse's largest entry where the plain-fp32 resolve reaches 1e-6; the error of the layer grows like
+ *     that figure times lambda_max.  As they come: within 2e-2 (typically 4e-3) for unstructured keys, for the
+ *     benchmark's correlated keys, for key norms in [0.25, 4] around shared directions (lambda_max 2300: 1e-2) and with
+ *     nine keys in ten of a frame bit-identical up to lambda_max 2000 (9e-3).  NOT within 2e-2 when 99 % or more of a
+ *     frame's keys are bit-identical (3e-2 .. 8e-2 at 99 %, more at 100 %, from lambda_max of about 5 on), nor for
+ *     lambda_max beyond about 2000 (5e-2 at 2200, 1e-1 at 7400).
+ *   VDN_FLAG_EXACT_STATS removes (1): within 2e-2 with 99 % of a frame's keys identical up to lambda_max of about 1000
+ *     and with all of them identical up to about 600.  VDN_FLAG_FP32_RESOLVE removes (2): within 2e-2 (5e-3 .. 1e-2)
+ *     for partly repeated or correlated keys of any norm tried (lambda_max up to 1e8) at F = 4080.  Both together
+ *     bring the tensor-core kernels to the figures of the plain-fp32 kernels (3e-3 .. 4e-3 up to lambda_max 1e8;
+ *     all-identical keys 1e-2 up to lambda_max 1e4) at 3.9 ms instead of 3.0 ms per forward on the 768p benchmark
+ *     shape (the plain-fp32 kernels: 49 ms).
  */
 #ifndef VDN_VDA_H_
 #define VDN_VDA_H_
@@ -112,6 +116,9 @@ typedef enum { VDN_F32 = 0, VDN_BF16 = 1 } vdn_dtype;
                                    /* weighted keys beta k (two bf16 parts) instead of their bf16 rounding: twice the  */
                                    /* tensor-core work in the statistics kernel, for frames whose keys (nearly) all    */
                                    /* coincide (Sec. A.3); see "Accuracy" above                                        */
+#define VDN_FLAG_FP32_RESOLVE 64u   /* tensor-core kernels: form (I + A_t)^{-1} with the plain-fp32 Gauss-Jordan kernel  */
+                                   /* (accurate to 1e-6 of its largest entry where the tensor-core resolve reaches      */
+                                   /* 5e-6) for frames with lambda_max in the thousands; see "Accuracy" above           */
 
 typedef struct {
   uint32_t struct_size; /* sizeof(vdn_vda_config), checked                                            */
@@ -133,7 +140,11 @@ typedef enum {
   /* tensor-core kernels (bf16 I/O, d = 128) */
   VDN_VIEW_INV_SPLIT = 4, /* bf16 [B,H,T,3,d,d]: C_t as C1 + C2 + C3 (bf16 parts of the fp32 inverse)         */
   VDN_VIEW_READ_FWD = 5,  /* bf16 [B,H,T,d_v,d_k]: slot t = P_{t-1} (zero for t = 0)                  (A.4)  */
-  VDN_VIEW_READ_BWD = 6   /* bf16 [B,H,T,d_v,d_k]: slot t = R_{t+1} (zero for t = T-1)                (A.4)  */
+  VDN_VIEW_READ_BWD = 6,  /* bf16 [B,H,T,d_v,d_k]: slot t = R_{t+1} (zero for t = T-1)                (A.4)  */
+  /* ... after a forward call that scanned chunk-wise (Sec. 5): the composites S_out = S_in M + J of the chunks each  */
+  /* direction folds, position p = the p-th chunk in that direction's order; n = number of chunks (size / per-chunk)  */
+  VDN_VIEW_COMP_M = 7,    /* bf16 [B*H,2,n,3,d,d]: M as three bf16 parts, stored as the scan multiplies: Z <- M Z  */
+  VDN_VIEW_COMP_J = 8     /* float [B*H,2,n,d_v,d_k]: J                                                             */
 } vdn_view;
 
 /* Sec. 3 (the layer as a whole).  Creates a handle bound to cfg->device.  Allocates host memory only

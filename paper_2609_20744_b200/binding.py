@@ -23,7 +23,8 @@ VDN_FLAG_ADDITIVE_RULE = 4
 VDN_FLAG_SCAN_CHUNKWISE = 8
 VDN_FLAG_SCAN_FRAMEWISE = 16
 VDN_FLAG_EXACT_STATS = 32
-VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_READ_BWD = range(7)
+VDN_FLAG_FP32_RESOLVE = 64
+VIEW_STATS, VIEW_INV, VIEW_FWD, VIEW_READ, VIEW_INV_SPLIT, VIEW_READ_FWD, VIEW_READ_BWD, VIEW_COMP_M, VIEW_COMP_J = range(9)
 
 EXPORTS = (
     "vdn_vda_create", "vdn_vda_workspace_bytes", "vdn_vda_set_workspace", "vdn_vda_forward", "vdn_vda_forward_ex",
@@ -375,6 +376,10 @@ class Vda:
             return raw.view(torch.bfloat16).view(B, H, T, 3, d, d)
         if which in (VIEW_READ_FWD, VIEW_READ_BWD):
             return raw.view(torch.bfloat16).view(B, H, T, d, d)
+        if which == VIEW_COMP_M:
+            return raw.view(torch.bfloat16).view(B * H, 2, -1, 3, d, d)
+        if which == VIEW_COMP_J:
+            return raw.view(torch.float32).view(B * H, 2, -1, d, d)
         return raw.view(torch.float32).view(B, H, T, d, d)
 
     def uses_tensor_cores(self) -> bool:

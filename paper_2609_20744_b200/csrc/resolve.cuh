@@ -141,7 +141,9 @@ __global__ void __launch_bounds__(256, 2) resolve_kernel(const float* __restrict
 #pragma unroll
     for (int c = 0; c < R; ++c) {
       const int i = ty + 16 * r, j = tx + 16 * c;
-      m[r][c] = __ldg(A + (size_t)i * D + j) + (i == j ? 1.0f : 0.0f);
+      // the symmetric part: the tensor-core statistics are symmetric only up to the bf16 rounding of one factor
+      // (the plain-fp32 ones to the last bit or two), and the symmetric part is what Eq. 3b means
+      m[r][c] = 0.5f * (__ldg(A + (size_t)i * D + j) + __ldg(A + (size_t)j * D + i)) + (i == j ? 1.0f : 0.0f);
     }
 
   gauss_jordan_tiles<D>(m, rowbuf, colbuf, tx, ty, [] { __syncthreads(); });

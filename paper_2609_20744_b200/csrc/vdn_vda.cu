@@ -93,6 +93,9 @@ struct vdn_vda_s {
   int* status_dev = nullptr;
   unsigned long long wait_ns = 2000000000ull;   // limit of any single device-side wait
   int launches = 0;
+  // where the last chunk-wise scan left its composites (views VDN_VIEW_COMP_M / _J); nseg = 0: it did not run
+  size_t last_comp_m = 0, last_comp_j = 0;
+  int last_nseg = 0;
   bool attrs_set = false;
   bool tc_attrs_set = false;
   unsigned ro_attrs_set = 0;       // read-out instantiations whose shared-memory attribute has been set
@@ -392,6 +395,10 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
     if (additive) {
       vdn::additive_transition_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n, 1.0f / (float)s.F, s);
       prof_mark(h, st, nk++, "additive_transition");
+    } else if (h->cfg.flags & VDN_FLAG_FP32_RESOLVE) {
+      // the plain-fp32 Gauss-Jordan (true pivot rows and columns), writing the three bf16 parts the scan reads
+      vdn::resolve_kernel<D><<<(unsigned)n, 256, 0, st>>>(stats, nullptr, csplit, n, s);
+      prof_mark(h, st, nk++, "resolve");
     } else {
       vdn::resolve_tc_kernel<<<(unsigned)n, vdn::ResolveTc::THREADS, vdn::ResolveTc::SMEM_BYTES, st>>>(
           stats, csplit, n, dev_status(h), s);
@@ -405,6 +412,7 @@ vdn_status forward_tc(vdn_vda_t h, const void* q, const void* k, const void* v, 
       sa.nseg = x.win.last / x.win.chunk - x.win.first / x.win.chunk + 1;
       sa.comp_m = reinterpret_cast<__nv_bfloat16*>(ws + L.comp_m);
       sa.comp_j = reinterpret_cast<float*>(ws + L.comp_j);
+      h->last_comp_m = L.comp_m; h->last_comp_j = L.comp_j; h->last_nseg = sa.nseg;
       CUtensorMap tmM;
       if ((r = make_matrix_map(h, &tmM, sa.comp_m, (long long)3 * s.B * s.H * 2 * sa.nseg * D)) != VDN_OK) return r;
       vdn::scan_tc_kernel<vdn::SCAN_COMPOSE><<<(unsigned)(4 * s.B * s.H * sa.nseg), vdn::ScanTc::THREADS,
@@ -755,6 +763,7 @@ vdn_status run_forward(vdn_vda_t h, const void* q, const void* k, const void* v,
     x.ro_count = hi - lo + 1;
   } else {
     h->launches = 0;
+    h->last_nseg = 0;
   }
   if (x.anchors && phase != 2) {
     // Alg. 1 step 7: anchor rows of the linear output are zero (frames 0 and T-1 of every clip)
@@ -1016,6 +1025,12 @@ vdn_status vdn_vda_workspace_view(vdn_vda_t h, int which, int B, int T, int F, i
     case VDN_VIEW_READ_BWD:
       if (!tcp) return fail(h, VDN_ERR_UNSUPPORTED, "the plain-fp32 kernels store the summed read state (VDN_VIEW_READ)");
       *offset_bytes = which == VDN_VIEW_READ_FWD ? L.fwd : L.read; *size_bytes = L.state_bytes; break;
+    case VDN_VIEW_COMP_M:
+    case VDN_VIEW_COMP_J:
+      if (!tcp || h->last_nseg == 0) return fail(h, VDN_ERR_UNSUPPORTED, "the last forward call did not scan chunk-wise");
+      *offset_bytes = which == VDN_VIEW_COMP_M ? h->last_comp_m : h->last_comp_j;
+      *size_bytes = (size_t)B * H * 2 * h->last_nseg * dd * (which == VDN_VIEW_COMP_M ? 3 * 2 : sizeof(float));
+      break;
     default: return fail(h, VDN_ERR_INVALID_ARG, "unknown view");
   }
   return VDN_OK;
