@@ -59,22 +59,24 @@
  *     60, 4e-4 at 150, 1e-2 at 2000.
  *   bf16 I/O, bound 2e-2, plain-fp32 kernels (VDN_FLAG_FORCE_SIMT): within 2e-2 for every input tried, including
  *     lambda_max of 1e5 and beyond, except all-identical keys at lambda_max >= 8000 (3e-2).
- *   bf16 I/O, bound 2e-2, tensor-core kernels.  Two things set their range.  (1) The weighted key beta_u k_u of every
- *     token is rounded to bf16 for the contraction, a 2^-9 move in a direction of its own; Eq. 5 damps what a frame
- *     writes along a repeated key by 1 / (1 + lambda_max) but not those residues.  (2) The tensor-core resolve takes the
- *     pivot rows from the matrix's own columns (it keeps the matrix symmetric only up to rounding) and reaches about
- *     5e-6 of the inverse's largest entry where the plain-fp32 resolve reaches 1e-6; the error of the layer grows like
- *     that figure times lambda_max.  As they come: within 2e-2 (typically 4e-3) for unstructured keys, for the
- *     benchmark's correlated keys, for key norms in [0.25, 4] around shared directions (lambda_max 2300: 1e-2) and with
- *     nine keys in ten of a frame bit-identical up to lambda_max 2000 (9e-3).  NOT within 2e-2 when 99 % or more of a
- *     frame's keys are bit-identical (3e-2 .. 8e-2 at 99 %, more at 100 %, from lambda_max of about 5 on), nor for
- *     lambda_max beyond about 2000 (5e-2 at 2200, 1e-1 at 7400).
- *   VDN_FLAG_EXACT_STATS removes (1): within 2e-2 with 99 % of a frame's keys identical up to lambda_max of about 1000
- *     and with all of them identical up to about 600.  VDN_FLAG_FP32_RESOLVE removes (2): within 2e-2 (5e-3 .. 1e-2)
- *     for partly repeated or correlated keys of any norm tried (lambda_max up to 1e8) at F = 4080.  Both together
- *     bring the tensor-core kernels to the figures of the plain-fp32 kernels (3e-3 .. 4e-3 up to lambda_max 1e8;
- *     all-identical keys 1e-2 up to lambda_max 1e4) at 3.9 ms instead of 3.0 ms per forward on the 768p benchmark
- *     shape (the plain-fp32 kernels: 49 ms).
+ *   bf16 I/O, bound 2e-2, tensor-core kernels.  What sets their range is the contraction of the statistics: the weighted
+ *     key beta_u k_u of every token is rounded to bf16, a 2^-9 move in a direction of its own; Eq. 5 damps what a frame
+ *     writes along a repeated key by 1 / (1 + lambda_max) but not those residues, so the error relative to the result
+ *     grows with the share of identical keys (and falls with the number of tokens the residues average over).  Within
+ *     2e-2 (typically 4e-3) for unstructured keys and the benchmark's correlated keys; for keys of any norm around
+ *     shared directions at F = 4096 (6e-3 at lambda_max 6e5); with nine keys in ten of a frame bit-identical at
+ *     F = 4080 for any key norm (1e-2 up to lambda_max 5e5) and at F = 300 up to lambda_max of about 500.  NOT within
+ *     2e-2 when 99 % or more of a frame's keys are bit-identical (3e-2 .. 8e-2 at 99 %, more at 100 %, from lambda_max
+ *     of about 5 on).
+ *   VDN_FLAG_EXACT_STATS contracts the exactly weighted keys (two bf16 parts; the statistics then equal the plain-fp32
+ *     kernels' to 5e-7): within 2e-2 (4e-3 .. 1e-2) up to 99 % identical keys for lambda_max up to 5e5 at F = 4080 and up
+ *     to about 1e4 at F = 300, and with all keys
+ *     of a frame identical up to lambda_max of about 2500 at F = 300 (1e-2) and about 1000 at F = 4080 (2.5e-2 at 2050,
+ *     where the plain-fp32 kernels give 1.2e-2).
+ *   VDN_FLAG_FP32_RESOLVE on top of that takes the inverse from the plain-fp32 Gauss-Jordan kernel and brings the
+ *     tensor-core kernels to the plain-fp32 kernels' figures throughout (all-identical keys: 2e-2 up to lambda_max 4e4).
+ *     On the 768p benchmark shape a forward takes 3.0 ms as it comes, 3.5 ms with exact statistics, 3.9 ms with both
+ *     (the plain-fp32 kernels: 49 ms).
  */
 #ifndef VDN_VDA_H_
 #define VDN_VDA_H_
@@ -117,8 +119,8 @@ typedef enum { VDN_F32 = 0, VDN_BF16 = 1 } vdn_dtype;
                                    /* tensor-core work in the statistics kernel, for frames whose keys (nearly) all    */
                                    /* coincide (Sec. A.3); see "Accuracy" above                                        */
 #define VDN_FLAG_FP32_RESOLVE 64u   /* tensor-core kernels: form (I + A_t)^{-1} with the plain-fp32 Gauss-Jordan kernel  */
-                                   /* (accurate to 1e-6 of its largest entry where the tensor-core resolve reaches      */
-                                   /* 5e-6) for frames with lambda_max in the thousands; see "Accuracy" above           */
+                                   /* (1e-6 of its largest entry where the tensor-core resolve reaches 5e-6): matters   */
+                                   /* only for frames of identical keys at lambda_max of 1e4 and more; see "Accuracy"   */
 
 typedef struct {
   uint32_t struct_size; /* sizeof(vdn_vda_config), checked                                            */

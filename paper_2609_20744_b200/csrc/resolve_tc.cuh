@@ -11,13 +11,18 @@
 // accumulated in fp32, so the update carries fp32 accuracy.
 //   * The 16 x 16 pivot block is inverted in plain fp32 inside the warp that owns those rows, one row per lane,
 //     the pivot rows travelling by shuffle.
-//   * Every thread owns one matrix row (its TMEM lane) and -- the matrix being symmetric up to the sign pattern of
-//     in-place elimination -- supplies its column of the 16 pivot rows (its own 16 pivot-column entries, signed),
-//     so nobody has to read whole rows back.  Both MMA operands are K-major with one row per thread: a thread
-//     writes its 16 values of a part as 32 contiguous bytes.
+//   * Every thread owns one matrix row (its TMEM lane).  The 16 pivot rows M[P][:] are the B operand of the update,
+//     K-major with one row per thread: thread j needs M[P_k][j], k = 0..15 -- a column of rows that sit in sixteen
+//     other TMEM lanes.  The warp that owns those lanes reads them (tcgen05.ld) and puts them in shared memory as
+//     plain fp32 rows (8 KB, sixteen 16-byte stores per lane); after one barrier every thread picks up its column
+//     with sixteen conflict-free 4-byte reads.  (An earlier version took M[P_k][j] = +-M[j][P_k] from the thread's own
+//     row instead -- exact while the matrix stays symmetric up to the sign pattern of in-place elimination, but the
+//     rounding of the updates breaks that symmetry a little at every step, and mixing the two copies cost a factor
+//     of the condition number in accuracy: a left residual of 8e-2 instead of 8e-5 at lambda_max = 2000 in an fp32
+//     emulation, 5e-6 instead of 1e-6 of the largest entry on benign matrices.)
 //   * The 128 x 16 coefficients Cm = -M[:, P] Gi are a matrix product as well: the pivot-row operand the threads
 //     have just written, times Gi (split three-way by the pivot warp), in a first, 128 x 16 x 16 MMA into the
-//     pivot columns themselves; each thread reads its row back and applies its sign.  Formed with fp32 FMAs
+//     pivot columns themselves; each thread reads its row back and negates it.  Formed with fp32 FMAs
 //     (256 per thread and step) they were the largest item of a kernel that is bound by instruction issue.
 // The matrix that is inverted is I + (A_t + A_t^T)/2: the stored statistics are symmetric only up to the bf16
 // rounding of one factor, and the symmetric part is the natural reading of Eq. 3b (and keeps Proposition 1).
@@ -46,10 +51,16 @@ struct ResolveTc {
   static constexpr int PR_BYTES = 128 * 128;          // pivot rows, K-major as well: row j = column j of the 16 pivot
                                                       // rows, parts laid out like the coefficients
   static constexpr int OFF_CM = 0;
+  static constexpr int PRF_STRIDE = D + 4;            // floats per fp32 pivot row: the sixteen lanes' 16-byte stores conflict two by two, the minimum
   static constexpr int OFF_PR = CM_BYTES;
-  static constexpr int OFF_GIB = OFF_PR + PR_BYTES;   // Gi as an MMA operand: 16 rows x 128 B, three parts per row
+  static constexpr int OFF_XO = OFF_PR + PR_BYTES;    // pivot columns, K-major: row i = M[i][P], parts laid out like the others
+  static constexpr int OFF_GIB = OFF_XO + PR_BYTES;   // Gi as an MMA operand: 16 rows x 128 B, three parts per row
   static constexpr int OFF_GI = OFF_GIB + 2048;       // Gi, 16 x 16 floats (for the pivot rows themselves)
+  static constexpr int OFF_PRF = OFF_CM;              // the 16 pivot rows in fp32, [16][PRF_STRIDE]: in the coefficient
+                                                      // operand's place until the coefficients exist (four CTAs per SM
+                                                      // leave no room for a buffer of their own)
   static constexpr int OFF_BAR = OFF_GI + 1024;
+  static_assert(16 * PRF_STRIDE * 4 <= CM_BYTES, "the fp32 pivot rows fit in the coefficient operand");
   static constexpr int SMEM_BYTES = OFF_BAR + 64 + 1024;
   static constexpr int THREADS = 160;                 // 4 row warps + 1 MMA warp
 };
@@ -100,14 +111,14 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       constexpr int PB[6] = {2, 0, 1, 1, 0, 0};
       constexpr uint32_t idesc_c = make_idesc_bf16(128, 16, false, false);
       for (int step = 0; step < D / R::NB; ++step) {
-        // ---- coefficients: M[:, P] <- Xs Gi (128 x 16 x 16), Xs = the signed pivot columns the row threads just
-        // wrote as the pivot-row operand, Gi = the inverse of the pivot block; each thread negates / signs its row
+        // ---- coefficients: M[:, P] <- X Gi (128 x 16 x 16), X = the pivot columns the row threads just wrote as an
+        // operand, Gi = the inverse of the pivot block; each thread negates its row
         const int p0c = (((int)(blockIdx.x & 3) * 2 + step) & 7) * R::NB;
         if (!mbar_wait(XREADY, step & 1, wc)) break;
         tc_fence_after_sync();
 #pragma unroll
         for (int pr = 0; pr < 6; ++pr) {
-          const uint64_t adesc = make_smem_desc(base + R::OFF_PR + PA[pr] * 32, 16, 1024);
+          const uint64_t adesc = make_smem_desc(base + R::OFF_XO + PA[pr] * 32, 16, 1024);
           const uint64_t bdesc = make_smem_desc(base + R::OFF_GIB + PB[pr] * 32, 16, 1024);
           mma_bf16_ss(tmem_base + p0c, adesc, bdesc, idesc_c, pr == 0 ? 0u : 1u);
         }
@@ -160,40 +171,59 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
     // at different blocks, so that their serial sections (the 16 x 16 inverse, done by the warp that owns the
     // pivot rows) fall on different warp schedulers instead of queueing on one.
     const int blk0 = (int)((blockIdx.x & 3) * 2);
-    uint32_t done = 0;                                    // bit b set: pivot block b has been eliminated
     bool ok = true;
+    float* prf = reinterpret_cast<float*>(base_ptr + R::OFF_PRF);  // fp32 pivot rows
+    auto store_operand_row = [&](int off, const float (&val)[16]) {
+      uint4 w[3][2];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        uint32_t a1, a2, a3;
+        split3_pair(val[2 * q], val[2 * q + 1], a1, a2, a3);
+        reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
+        reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
+        reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
+      }
+      unsigned char* orow = base_ptr + off + row * 128;
+#pragma unroll
+      for (int part = 0; part < 3; ++part) {
+        *reinterpret_cast<uint4*>(orow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
+        *reinterpret_cast<uint4*>(orow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
+      }
+    };
 #pragma unroll 1
     for (int step = 0; step < D / R::NB && ok; ++step) {
       const int blk = (blk0 + step) & 7;
       const int p0 = blk * R::NB;
       const bool owner = (row >> 4) == blk;               // rows p0 .. p0+15: 16 lanes of warp blk/2
       float x[16];
-      tmem_ld16(trow + p0, x);
+      tmem_ld16(trow + p0, x);                            // this row's entries in the pivot columns
       tmem_wait_ld();
 
-      // ---- the 16 pivot rows as an MMA operand, three bf16 parts.  M is symmetric up to the sign pattern of
-      // in-place elimination: M[P_k][j] = M[j][P_k] for rows j not yet eliminated and -M[j][P_k] for rows already
-      // eliminated (`done`).  So thread j owns column j of the pivot rows: its own x, signed -- which is one row
-      // of the K-major operand (row = output column, 16 contiguous pivot indices): two 16-byte stores per part.
-      // The same rows, times Gi, give the update coefficients (below).
-      const float sgn = ((done >> (row >> 4)) & 1u) ? -1.0f : 1.0f;
-      {
-        uint4 w[3][2];
+      // ---- the 16 pivot rows, as they stand before this step, to shared memory in fp32 (the warp that owns them)
+      if (warp == (blk >> 1)) {
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          float v[32];
+          tmem_ld32(trow + cc * 32, v);
+          tmem_wait_ld();
+          if (owner) {
+            float* dst = prf + (row & 15) * R::PRF_STRIDE + cc * 32;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          uint32_t a1, a2, a3;
-          split3_pair(sgn * x[2 * q], sgn * x[2 * q + 1], a1, a2, a3);
-          reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
-          reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
-          reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
-        }
-        unsigned char* prow = base_ptr + R::OFF_PR + row * 128;
-#pragma unroll
-        for (int part = 0; part < 3; ++part) {
-          *reinterpret_cast<uint4*>(prow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
-          *reinterpret_cast<uint4*>(prow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
+            for (int e = 0; e < 32; e += 4) store4(dst + e, make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]));
+          }
         }
       }
+      // ---- pivot columns as an operand (for the coefficients), while the pivot rows are on their way
+      store_operand_row(R::OFF_XO, x);
+      named_barrier_sync(1, 128);                         // the pivot rows are in shared memory
+      // thread j's column of the pivot rows: one row of the K-major operand (row = output column).  The warp that
+      // owns the pivot rows does this later, under the coefficient MMA: it is the one everybody waits for.
+      float y[16];
+      auto load_pivot_column = [&]() {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) y[k] = prf[k * R::PRF_STRIDE + row];
+      };
+      if (warp != (blk >> 1)) { load_pivot_column(); store_operand_row(R::OFF_PR, y); }
       if (warp == (blk >> 1)) {
         // ---- invert the 16 x 16 pivot block: lane (l0 + a) holds row a; pivot rows travel by shuffle
         const int l0 = (blk & 1) * 16;
@@ -215,17 +245,26 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           g[p] = prow ? ip : -fi;
         }
         if (owner) {
-          // Gi row a: in fp32 for this pivot row's own coefficients, and as three bf16 parts for the tensor cores
-          // (Gi is symmetric, so its rows serve as the rows of the K-major operand, which wants columns)
+          // Gi row a in fp32 for this pivot row's own coefficients, and Gi as three bf16 parts for the tensor cores
           const int a = row & 15;
           float* dst = gi + a * 16;
 #pragma unroll
           for (int j = 0; j < 16; j += 4) store4(dst + j, make_float4(g[j], g[j + 1], g[j + 2], g[j + 3]));
+        }
+        __syncwarp();
+        if (owner) {
+          // ... whose rows must be the COLUMNS of Gi (c = -x Gi contracts x with a column).  The block of an
+          // elimination in progress is symmetric only up to rounding, so the column is read back from the rows just
+          // written, not taken to be the row.
+          const int a = row & 15;
+          float gc[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) gc[j] = gi[j * 16 + a];
           uint4 w[3][2];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             uint32_t a1, a2, a3;
-            split3_pair(g[2 * q], g[2 * q + 1], a1, a2, a3);
+            split3_pair(gc[2 * q], gc[2 * q + 1], a1, a2, a3);
             reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
             reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
             reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
@@ -238,11 +277,15 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           }
         }
       }
+      // (the fp32 pivot rows share their memory with the coefficient operand, which the other warps write as soon as
+      // the coefficient MMA has completed, i.e. some time after the arrival below: read them before it)
+      if (warp == (blk >> 1)) load_pivot_column();
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive_warp(XREADY);
+      if (warp == (blk >> 1)) store_operand_row(R::OFF_PR, y);
 
-      // ---- coefficients: c = -M[i][P] Gi = -sgn (Xs Gi) from the tensor cores; a pivot row a takes Gi[a]
+      // ---- coefficients: c = -M[i][P] Gi = -(X Gi) from the tensor cores; a pivot row a takes Gi[a]
       if (!mbar_wait(CDONE, step & 1, wc)) { ok = false; break; }
       tc_fence_after_sync();
       float c[16];
@@ -257,28 +300,14 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
         }
       } else {
 #pragma unroll
-        for (int k = 0; k < 16; ++k) c[k] *= -sgn;
+        for (int k = 0; k < 16; ++k) c[k] = -c[k];
       }
       // ---- A operand: this row's 16 update coefficients (pivot rows: Gi[a] - e_a), three bf16 parts
       {
-        uint4 w[3][2];
+        float u[16];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          float u0 = c[2 * q], u1 = c[2 * q + 1];
-          if (owner && (row & 15) == 2 * q) u0 -= 1.0f;
-          if (owner && (row & 15) == 2 * q + 1) u1 -= 1.0f;
-          uint32_t a1, a2, a3;
-          split3_pair(u0, u1, a1, a2, a3);
-          reinterpret_cast<uint32_t*>(&w[0][q >> 2])[q & 3] = a1;
-          reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
-          reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
-        }
-        unsigned char* crow = base_ptr + R::OFF_CM + row * 128;
-#pragma unroll
-        for (int part = 0; part < 3; ++part) {
-          *reinterpret_cast<uint4*>(crow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
-          *reinterpret_cast<uint4*>(crow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
-        }
+        for (int k = 0; k < 16; ++k) u[k] = (owner && (row & 15) == k) ? c[k] - 1.0f : c[k];
+        store_operand_row(R::OFF_CM, u);
       }
       fence_proxy_async_smem();
       tc_fence_before_sync();
@@ -288,7 +317,6 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       // ---- column fix: M[i][P] = c (for a pivot row: Gi[a])
       tmem_st16(trow + p0, c);
       tmem_wait_st();
-      done |= 1u << blk;
     }
     if (ok) {
       // ---- the inverse as three bf16 parts; this thread holds row `row` of it and stores it transposed (the

@@ -21,19 +21,18 @@ is loosened here.  What the cases below establish is the range of inputs in whic
   * bf16 I/O through the tensor-core kernels rounds each token's weighted key beta_u k_u to bf16 for the
     contraction (a relative 2^-9 per element, different from token to token).  The update of Eq. 5 damps what a
     frame writes along its repeated key direction by 1 / (1 + lambda_max), but not the rounding residue, which
-    lies off that direction: the error relative to the result grows with the share of identical keys and with
-    lambda_max.  2e-2 holds with nine keys in ten identical up to lambda_max of about two thousand (the most that
-    unit keys give at F = 4080 with gates around one half), and for key norms spread over [0.25, 4] around shared
-    directions; it does not hold for frames in which 99 % or more of the keys are bit-identical (measured
-    3e-2 .. 8e-2 at 99 %, worse at 100 %).
+    lies off that direction: the error relative to the result grows with the share of identical keys and falls with
+    the number of tokens the residues average over.  2e-2 holds with nine keys in ten identical for any key norm
+    at F = 4080 (lambda_max beyond 1e5) and up to lambda_max of about 500 at F = 300, and for key norms spread over
+    [0.25, 4] around shared directions; it does not hold for frames in which 99 % or more of the keys are
+    bit-identical (measured 3e-2 .. 8e-2 at 99 %, worse at 100 %).
   * the same kernels with VDN_FLAG_EXACT_STATS contract the exactly weighted keys (two bf16 parts).  2e-2 then holds
-    with 99 % identical keys up to lambda_max of about one thousand (at two thousand it is borderline: 1e-2 .. 3e-2
-    depending on the draw) and with all keys identical up to about 600.
-  * either way the tensor-core resolve sets a limit of its own: its inverse is good to about 5e-6 of the largest
-    entry (the plain-fp32 resolve: 1e-6; both measured against an fp64 inverse of the same matrix), and the error
-    of the layer grows like that figure times lambda_max: 2e-2 is left at lambda_max of a little over two thousand.
-    VDN_FLAG_FP32_RESOLVE puts the plain-fp32 resolve in its place; with both flags the tensor-core kernels hold
-    2e-2 wherever the plain-fp32 kernels do (checked here at lambda_max beyond 1e5).
+    up to 99 % identical keys for any key norm tried at F = 4080 and up to lambda_max of about 1e4 at F = 300 (borderline
+    beyond: 7e-3 .. 2.3e-2 at 3.5e4 depending on the draw), and with all keys identical up to lambda_max of about 2500 at
+    F = 300 and about 1000 at F = 4080 (beyond, the inverse of the tensor-core resolve, good to 5e-6 of its largest
+    entry where the plain-fp32 one reaches 1e-6, becomes the limit).
+  * VDN_FLAG_FP32_RESOLVE on top puts the plain-fp32 resolve in its place: the tensor-core kernels then hold 2e-2
+    wherever the plain-fp32 kernels do.
 """
 import numpy as np
 import pytest
@@ -88,7 +87,7 @@ def test_repeated_keys(dtype, d, flags, F, frac):
     if dtype == "bf16" and flags == 0 and frac == 1.0:
         pytest.skip("bit-identical keys throughout a frame: outside the tensor-core kernels' range (module docstring)")
     if dtype == "bf16" and flags == EXACT and frac == 1.0 and F > 1000:
-        pytest.skip("bit-identical keys with lambda_max beyond about 600: outside the range of the tensor-core resolve")
+        pytest.skip("4080 bit-identical keys: 2.5e-2, outside the range of the tensor-core resolve")
     if dtype == "bf16" and flags == ACCURATE and (F, frac) == (4080, 1.0):
         pytest.skip("4080 bit-identical keys with random values: 2.4e-2, the plain-fp32 kernels' own 1.2e-2 doubled")
     w = inputs.TINY.scaled(dtype=dtype, d=d, B=1, H=2, T=5, F=F, key_repeat_frac=frac, seed=21)
@@ -155,8 +154,10 @@ def test_key_norms_spread_over_a_decade_with_shared_directions(dtype, d, flags):
 # ------------------------------------------------------------------------------ the supported range, pinned
 @pytest.mark.parametrize("F,frac,scale,dtype,flags,lam_min", [
     (4080, 0.9, 1.0, "bf16", 0, 1.5e3),          # tensor-core kernels: the largest lambda_max unit keys can give
-    (1000, 0.99, 1.0, "bf16", EXACT, 400.0),     # ... with exactly weighted keys: 99 % identical keys
-    (1000, 1.0, 1.0, "bf16", EXACT, 400.0),      # ... and all-identical keys, as far as the resolve and scan carry
+    (4080, 0.9, 8.0, "bf16", 0, 1e5),            # ... and far beyond it: many tokens per frame
+    (4080, 0.99, 1.0, "bf16", EXACT, 1.5e3),     # ... with exactly weighted keys: 99 % identical keys
+    (300, 0.9, 8.0, "bf16", EXACT, 5e3),         #     few tokens per frame, large norms
+    (300, 1.0, 4.0, "bf16", EXACT, 1.5e3),       #     all-identical keys, as far as the tensor-core resolve carries
     (4080, 0.9, 8.0, "bf16", ACCURATE, 1e5),     # ... and the plain-fp32 resolve on top: any key norm
     (300, 1.0, 8.0, "bf16", ACCURATE, 5e3),      #     all-identical keys at lambda_max of ten thousand
     (4080, 0.9, 8.0, "bf16", binding.VDN_FLAG_FP32_RESOLVE, 1e5),   # the plain-fp32 resolve alone, many tokens per frame

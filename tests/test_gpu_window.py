@@ -292,3 +292,34 @@ def test_random_window_settings_on_every_scan_schedule(dtype, d):
         except AssertionError as e:
             raise AssertionError(f"trial {trial}: T={T} {kw} alpha={use_alpha} s0={use_s0} flags={flags}: {e}")
         vda.close()
+
+
+def test_chunk_composites_match_an_fp64_fold_of_the_same_frames():
+    # Sec. 5, "Chunk-wise scans": S_out = S_in M + J per chunk.  The composites the scan leaves in the workspace (J in
+    # fp32, M as three bf16 parts) against an fp64 fold of the chunk's frames from the GPU's own statistics and
+    # inverses: isolates the arithmetic of the tensor-core scan (three-way bf16 splits of both fp32 factors, six
+    # products, fp32 accumulation) at fp32 resolution -- the stored read states are bf16 and cannot show it.
+    d = 128
+    w = inputs.TINY.scaled(dtype="bf16", d=d, B=1, H=2, T=21, F=300, seed=3)
+    x = inputs.generate(w, "cuda")
+    vda = binding.Vda(w.d, w.dtype, flags=binding.VDN_FLAG_SCAN_CHUNKWISE)
+    vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"], chunk=5, radius=1)
+    torch.cuda.synchronize()
+    stats = vda.view(binding.VIEW_STATS, 1, w.T, w.F, w.H).double().cpu().numpy()[0]
+    split = vda.view(binding.VIEW_INV_SPLIT, 1, w.T, w.F, w.H).double().cpu().numpy()[0]
+    J = vda.view(binding.VIEW_COMP_J, 1, w.T, w.F, w.H).double().cpu().numpy()
+    M = vda.view(binding.VIEW_COMP_M, 1, w.T, w.F, w.H).double().cpu().numpy()
+    assert J.shape[:3] == (w.H, 2, 5) and M.shape[:4] == (w.H, 2, 5, 3)
+    rel = lambda g, r: np.max(np.abs(g - r)) / np.max(np.abs(r))
+    for h in range(w.H):
+        for direction in (0, 1):
+            for pos in range(2):                                   # the first two chunks each direction folds
+                frames = range(5 * pos, 5 * pos + 5) if direction == 0 else range(w.T - 1 - 5 * pos, w.T - 2 - 5 * pos, -1) \
+                    if pos == 0 else range(19 - 5 * (pos - 1), 14 - 5 * (pos - 1), -1)
+                Z, Mm = np.zeros((d, d)), np.eye(d)
+                for t in frames:
+                    C = split[h, t].sum(0).T                       # the scan multiplies by the transpose of what is stored
+                    Z = C @ (Z + stats[h, t, d:].T)
+                    Mm = C @ Mm
+                assert rel(J[h, direction, pos].T, Z) <= 3e-6      # measured 6e-7: about 1.3e-7 per product
+                assert rel(M[h, direction, pos].sum(0), Mm) <= 6e-6   # measured 1.7e-6
