@@ -67,9 +67,12 @@
  *     shared directions at F = 4096 (6e-3 at lambda_max 6e5); with nine keys in ten of a frame bit-identical at
  *     F = 4080 for any key norm (1e-2 up to lambda_max 5e5) and at F = 300 up to lambda_max of about 500.  NOT within
  *     2e-2 when 99 % or more of a frame's keys are bit-identical (3e-2 .. 8e-2 at 99 %, more at 100 %, from lambda_max
- *     of about 5 on).
+ *     of about 5 on), nor when all keys of a frame lie within a few degrees of one direction: unit keys drawn as one
+ *     direction plus N(0, s^2) per component give 6e-3 at s = 0.05, 1e-2 at 0.02, 1.7e-2 at 0.01 (a cone of about six
+ *     degrees), 3.5e-2 at 0.005, 8e-2 at 0.002 -- the rounding of the weighted keys (4e-3) must stay small against
+ *     the keys' own spread.
  *   VDN_FLAG_EXACT_STATS contracts the exactly weighted keys (two bf16 parts; the statistics then equal the plain-fp32
- *     kernels' to 5e-7): within 2e-2 (4e-3 .. 1e-2) up to 99 % identical keys for lambda_max up to 5e5 at F = 4080 and up
+ *     kernels' to 5e-7): 4e-3 for keys within any cone (s = 0.002 .. 0.05 above); within 2e-2 (4e-3 .. 1e-2) up to 99 % identical keys for lambda_max up to 5e5 at F = 4080 and up
  *     to about 1e4 at F = 300, and with all keys
  *     of a frame identical up to lambda_max of about 2500 at F = 300 (1e-2) and about 1000 at F = 4080 (2.5e-2 at 2050,
  *     where the plain-fp32 kernels give 1.2e-2).
