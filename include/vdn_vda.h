@@ -153,7 +153,10 @@ typedef enum {
 } vdn_view;
 
 /* Sec. 3 (the layer as a whole).  Creates a handle bound to cfg->device.  Allocates host memory only
- * (one pinned, device-mapped status word).  Returns VDN_ERR_ARCH when the device is not sm_100. */
+ * (one pinned, device-mapped status word).  Returns VDN_ERR_ARCH when the device is not sm_100.
+ * Two environment variables are read here, for measurements only: VDN_SCAN_SPLIT=0 keeps all scan chains in one
+ * launch even when there are more of them than SMs, VDN_RO_SHORT=0 keeps the read-out's long-frame layout for short
+ * frames; both default to 1. */
 vdn_status vdn_vda_create(const vdn_vda_config* cfg, vdn_vda_t* out_handle);
 
 /* Bytes of device workspace a forward call of this shape needs (per-frame statistics of Eq. 3b, the
