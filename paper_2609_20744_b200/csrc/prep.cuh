@@ -10,13 +10,14 @@
 //
 // A single kernel that did all of it in one pass over K and V (tile + halo in shared memory, the spatial results of
 // five frames in a register ring) was the first version: 242 registers, one CTA of eight warps per SM, 8.9 ms on
-// the 768p shape where the two kernels take 4.9 + 2.3 ms.
+// the 768p shape where the two kernels take 4.4 + 2.3 ms.
 #pragma once
 #include <cuda_bf16.h>
 
 #include <type_traits>
 
 #include "common.cuh"
+#include "tc_common.cuh"
 
 namespace vdn {
 
@@ -106,40 +107,62 @@ struct PrepArgs {
 // ring, which held it to one CTA of eight warps per SM, its fp32 pipe idle through every barrier and every
 // temporal / SiLU / norm phase.
 //
-// One CTA per (head, 8 x 8 token tile, batch, tensor) walks the frames; the tile and its 2-token halo arrive by
-// cp.async, double buffered.  A thread owns two neighbouring channels (the lanes of the packed fp32 FMA) and two
-// tile rows of eight tokens: six input rows per column feed ten tap rows, 400 packed FMAs for 72 shared-memory
-// reads.  Two CTAs per SM.
+// One CTA per (head, 8 x 8 token tile, batch, tensor) walks the frames.  The tile and its 2-token halo arrive by TMA,
+// double buffered: the tensor is mapped as (channel, head, x, y, frame) so that one box is the halo tile of one head,
+// and whatever hangs over the frame's edge (negative x or y included) is zero-filled by the copy engine -- one
+// instruction of one thread per frame, where sixteen-byte asynchronous copies with their bounds checks cost 131 of
+// the kernel's 900 instructions per warp and tile.  A thread owns two neighbouring channels (the lanes of the packed
+// fp32 FMA) and two tile rows of eight tokens: six input rows per column feed ten tap rows, 400 packed FMAs for 72
+// shared-memory reads.  Two CTAs per SM.  The wait for a tile is bounded like every other.
 struct PrepSpatial {
   static constexpr int TX = 8, RPT = 2, HALO = 2;            // columns and rows per thread
   static constexpr int THREADS = 256;
   __host__ __device__ static constexpr int rows(int D) { return RPT * THREADS / (D / 2); }      // tile rows
   __host__ __device__ static constexpr int tile_tokens(int D) { return (rows(D) + 2 * HALO) * (TX + 2 * HALO); }
-  static constexpr size_t smem_bytes(int D, int es) { return (size_t)2 * tile_tokens(D) * D * es; }
+  // two tiles, the barriers, and slack for the 128-byte alignment of the tiles
+  static constexpr size_t smem_bytes(int D, int es) { return (size_t)2 * tile_tokens(D) * D * es + 64 + 128; }
 };
 
 template <typename Tio, int D>
-__global__ void __launch_bounds__(PrepSpatial::THREADS, sizeof(Tio) == 2 ? 2 : 1) prep_spatial_kernel(PrepArgs a, Shape s) {
+__global__ void __launch_bounds__(PrepSpatial::THREADS, sizeof(Tio) == 2 ? 2 : 1)
+prep_spatial_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, PrepArgs a, Shape s,
+                    tc::DevStatus ds) {
+  using namespace tc;
   using P = PrepSpatial;
   constexpr int ROWS = P::rows(D);
   constexpr int TX = P::TX, HALO = P::HALO, RPT = P::RPT;
   constexpr int SW = TX + 2 * HALO, SH = ROWS + 2 * HALO;       // tile with halo
   constexpr int GT = D / 2;                                      // threads per row pair (one head's channel pairs)
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  Tio* tile = reinterpret_cast<Tio*>(smem_raw);                  // [2][SH][SW][D]
+  constexpr uint32_t TILE_BYTES = (uint32_t)(SH * SW * D * sizeof(Tio));
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 127u) & ~127u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  const Tio* tile = reinterpret_cast<const Tio*>(base_ptr);      // [2][SH][SW][D]
+  const uint32_t bar0 = base + 2 * TILE_BYTES;                   // FULL[2]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + 2 * TILE_BYTES + 16);
+  const WaitCtx wc(abort_flag, ds);
 
   const int h = blockIdx.x;
   const int tiles_x = (a.X + TX - 1) / TX;
   const int x0 = (blockIdx.y % tiles_x) * TX, y0 = (blockIdx.y / tiles_x) * ROWS;
   const int which = blockIdx.z & 1;                              // 0 = K, 1 = V
   const int b = blockIdx.z >> 1;
-  const Tio* __restrict__ src = static_cast<const Tio*>(which == 0 ? a.in[0] : a.in[1]);
+  const CUtensorMap* tm = which == 0 ? &tmK : &tmV;
   Tio* __restrict__ dst = static_cast<Tio*>(which == 0 ? a.out[0] : a.out[1]);
 
   const int tid = threadIdx.x;
   const int g = tid / GT;                   // row pair of this thread: tile rows 2g, 2g+1
   const int cp = tid % GT;                  // channel pair within the head
   const int ch = h * D + 2 * cp;
+
+  if (tid == 0) {
+    mbar_init(bar0, 1);
+    mbar_init(bar0 + 8, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(tm);
+  }
+  __syncthreads();
 
   f32x2 wsp[5][5];
   {
@@ -155,40 +178,20 @@ __global__ void __launch_bounds__(PrepSpatial::THREADS, sizeof(Tio) == 2 ? 2 : 1
   const int yr = y0 + RPT * g;              // first of this thread's two output rows
   Tio* pdst = dst + token_offset(s, b, first, min(yr, a.Y - 1) * a.X + x0, h) + 2 * cp;
 
-  // 16-byte pieces of the tile this thread copies, the same for every frame (-1: outside the frame -> zeros)
-  constexpr int CHUNKS = D * (int)sizeof(Tio) / 16;
-  constexpr int NPIECE = (SH * SW * CHUNKS + P::THREADS - 1) / P::THREADS;
-  int goff[NPIECE];
-#pragma unroll
-  for (int i = 0; i < NPIECE; ++i) {
-    const int e = tid + i * P::THREADS;
-    const int c = e % CHUNKS, tok = e / CHUNKS;
-    const int yy = y0 - HALO + tok / SW, xx = x0 - HALO + tok % SW;
-    const bool in = e < SH * SW * CHUNKS && yy >= 0 && yy < a.Y && xx >= 0 && xx < a.X;
-    goff[i] = in ? (int)((((size_t)(yy * a.X + xx) * s.H + h) * D) * sizeof(Tio)) + c * 16 : -1;
-  }
-  const size_t frame_bytes = frame_elems * sizeof(Tio);
-  const unsigned char* src_b = reinterpret_cast<const unsigned char*>(src) + (size_t)b * s.T * frame_bytes;
+  // frame t's halo tile -> buffer t & 1 (one thread; the engine zero-fills what lies outside the frame)
   auto stage = [&](int t) {
-    unsigned char* buf = reinterpret_cast<unsigned char*>(tile) + (size_t)(t & 1) * SH * SW * D * sizeof(Tio);
-    const unsigned char* fr = src_b + (size_t)t * frame_bytes;
-#pragma unroll
-    for (int i = 0; i < NPIECE; ++i) {
-      const int e = tid + i * P::THREADS;
-      if (e < SH * SW * CHUNKS) {
-        if (goff[i] >= 0) cp_async16(buf + (size_t)e * 16, fr + goff[i]);
-        else *reinterpret_cast<uint4*>(buf + (size_t)e * 16) = make_uint4(0u, 0u, 0u, 0u);
-      }
-    }
-    cp_async_commit();
+    const uint32_t bar = bar0 + 8u * (t & 1);
+    mbar_arrive_expect_tx(bar, TILE_BYTES);
+    tma_load_5d(base + (uint32_t)(t & 1) * TILE_BYTES, tm, bar, 0, h, x0 - HALO, y0 - HALO, b * s.T + t);
   };
 
-  stage(first);
+  if (tid == 0) stage(first);
 #pragma unroll 1
   for (int t = first; t <= last; ++t) {
-    if (t + 1 <= last) { stage(t + 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
-    __syncthreads();                        // frame t's tile is complete
-    const Tio* base = tile + (size_t)(t & 1) * SH * SW * D + (size_t)(RPT * g) * SW * D + 2 * cp;
+    // the other buffer was last read for frame t - 1; every thread passed the barrier that closed that frame
+    if (tid == 0 && t + 1 <= last) stage(t + 1);
+    if (!mbar_wait(bar0 + 8u * (t & 1), ((t - first) >> 1) & 1, wc)) break;        // frame t's tile has landed
+    const Tio* tbase = tile + (size_t)(t & 1) * SH * SW * D + (size_t)(RPT * g) * SW * D + 2 * cp;
     f32x2 acc[RPT][TX];
 #pragma unroll
     for (int r = 0; r < RPT; ++r)
@@ -198,7 +201,7 @@ __global__ void __launch_bounds__(PrepSpatial::THREADS, sizeof(Tio) == 2 ? 2 : 1
     for (int xi = 0; xi < SW; ++xi) {       // input column xi sits at x0 - 2 + xi
       f32x2 in[4 + RPT];
 #pragma unroll
-      for (int i = 0; i < 4 + RPT; ++i) in[i] = load_pair(base + ((size_t)i * SW + xi) * D);
+      for (int i = 0; i < 4 + RPT; ++i) in[i] = load_pair(tbase + ((size_t)i * SW + xi) * D);
 #pragma unroll
       for (int i = 0; i < 5; ++i) {
 #pragma unroll
@@ -224,7 +227,12 @@ __global__ void __launch_bounds__(PrepSpatial::THREADS, sizeof(Tio) == 2 ? 2 : 1
       }
     }
     pdst += frame_elems;
-    __syncthreads();                        // the buffer is overwritten by the copy issued at the start of the next step
+    __syncthreads();                        // this frame's buffer may be overwritten by the copy issued two frames on
+  }
+  if (tid == 0 && *abort_flag) {
+    // a wait gave up: give the copy that may still be in flight a bounded chance to land before the CTA retires
+    for (int i = 0; i < 2; ++i)
+      for (int spin = 0; spin < 4096 && !mbar_try_wait(bar0 + 8u * i, 0) && !mbar_try_wait(bar0 + 8u * i, 1); ++spin) {}
   }
 }
 

@@ -560,10 +560,32 @@ vdn_status launch_prepare(vdn_vda_t h, const void* q_in, const void* k_in, const
     if (p.wk_spatial) {
       // spatial filter into the outputs, then the temporal half in place on them
       using P = vdn::PrepSpatial;
+      if (!h->encode) return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
       const size_t smem = P::smem_bytes(D, (int)sizeof(Tio));
       VDN_CUDA(h, cudaFuncSetAttribute(vdn::prep_spatial_kernel<Tio, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      // [B,T,F,H,d] with F = Y * X as a 5-D map (d, H, X, Y, B*T): one box = the halo tile of one head in one frame
+      CUtensorMap tmk, tmv;
+      {
+        const cuuint64_t es = sizeof(Tio);
+        const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)s.H, (cuuint64_t)p.X, (cuuint64_t)p.Y, (cuuint64_t)s.B * s.T};
+        const cuuint64_t strides[4] = {D * es, (cuuint64_t)s.H * D * es, (cuuint64_t)p.X * s.H * D * es,
+                                       (cuuint64_t)s.F * s.H * D * es};
+        const cuuint32_t box[5] = {(cuuint32_t)D, 1, (cuuint32_t)(P::TX + 2 * P::HALO), (cuuint32_t)(P::rows(D) + 2 * P::HALO), 1};
+        const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        const CUtensorMapDataType dt = sizeof(Tio) == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+        const void* srcs[2] = {k_in, v_in};
+        CUtensorMap* maps[2] = {&tmk, &tmv};
+        for (int i = 0; i < 2; ++i) {
+          CUresult cr = h->encode(maps[i], dt, 5, const_cast<void*>(srcs[i]), dims, strides, box, estr,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+          if (cr != CUDA_SUCCESS)
+            return fail(h, VDN_ERR_CUDA, "cuTensorMapEncodeTiled (preparation input) failed: " + std::to_string((int)cr));
+        }
+      }
       const int tiles = ((p.X + P::TX - 1) / P::TX) * ((p.Y + P::rows(D) - 1) / P::rows(D));
-      vdn::prep_spatial_kernel<Tio, D><<<dim3((unsigned)s.H, (unsigned)tiles, (unsigned)(2 * s.B)), P::THREADS, smem, st>>>(a, s);
+      vdn::prep_spatial_kernel<Tio, D><<<dim3((unsigned)s.H, (unsigned)tiles, (unsigned)(2 * s.B)), P::THREADS, smem, st>>>(
+          tmk, tmv, a, s, dev_status(h));
       prof_mark(h, st, nk++, "prep_spatial");
       a.in[0] = k_out; a.in[1] = v_out;
     }
