@@ -10,7 +10,7 @@
 //
 // A single kernel that did all of it in one pass over K and V (tile + halo in shared memory, the spatial results of
 // five frames in a register ring) was the first version: 242 registers, one CTA of eight warps per SM, 8.9 ms on
-// the 768p shape where the two kernels take 4.4 + 2.3 ms.
+// the 768p shape where the two kernels take 4.2 + 2.3 ms.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -107,15 +107,15 @@ struct PrepArgs {
 // ring, which held it to one CTA of eight warps per SM, its fp32 pipe idle through every barrier and every
 // temporal / SiLU / norm phase.
 //
-// One CTA per (head, 8 x 8 token tile, batch, tensor) walks the frames.  The tile and its 2-token halo arrive by TMA,
+// One CTA per (head, 12 x 8 token tile, batch, tensor) walks the frames.  The tile and its 2-token halo arrive by TMA,
 // double buffered: the tensor is mapped as (channel, head, x, y, frame) so that one box is the halo tile of one head,
 // and whatever hangs over the frame's edge (negative x or y included) is zero-filled by the copy engine -- one
 // instruction of one thread per frame, where sixteen-byte asynchronous copies with their bounds checks cost 131 of
 // the kernel's 900 instructions per warp and tile.  A thread owns two neighbouring channels (the lanes of the packed
-// fp32 FMA) and two tile rows of eight tokens: six input rows per column feed ten tap rows, 400 packed FMAs for 72
-// shared-memory reads.  Two CTAs per SM.  The wait for a tile is bounded like every other.
+// fp32 FMA) and three tile rows of eight tokens: seven input rows per column feed fifteen tap rows, 600 packed FMAs
+// for 84 shared-memory reads (with two rows: 400 for 72, and 4.44 ms instead of 4.22 ms on the 768p shape).  Two CTAs per SM.  The wait for a tile is bounded like every other.
 struct PrepSpatial {
-  static constexpr int TX = 8, RPT = 2, HALO = 2;            // columns and rows per thread
+  static constexpr int TX = 8, RPT = 3, HALO = 2;            // columns and rows per thread
   static constexpr int THREADS = 256;
   __host__ __device__ static constexpr int rows(int D) { return RPT * THREADS / (D / 2); }      // tile rows
   __host__ __device__ static constexpr int tile_tokens(int D) { return (rows(D) + 2 * HALO) * (TX + 2 * HALO); }
@@ -151,7 +151,7 @@ prep_spatial_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   Tio* __restrict__ dst = static_cast<Tio*>(which == 0 ? a.out[0] : a.out[1]);
 
   const int tid = threadIdx.x;
-  const int g = tid / GT;                   // row pair of this thread: tile rows 2g, 2g+1
+  const int g = tid / GT;                   // row group of this thread: tile rows RPT g .. RPT g + RPT - 1
   const int cp = tid % GT;                  // channel pair within the head
   const int ch = h * D + 2 * cp;
 
@@ -175,7 +175,7 @@ prep_spatial_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
   const int first = s.t0, last = s.t0 + s.Tn - 1;
   const size_t frame_elems = (size_t)s.F * s.H * D;
-  const int yr = y0 + RPT * g;              // first of this thread's two output rows
+  const int yr = y0 + RPT * g;              // first of this thread's output rows
   Tio* pdst = dst + token_offset(s, b, first, min(yr, a.Y - 1) * a.X + x0, h) + 2 * cp;
 
   // frame t's halo tile -> buffer t & 1 (one thread; the engine zero-fills what lies outside the frame)
