@@ -429,15 +429,27 @@ def run_ours(args, w, rank: int, local_rank: int, world: int):
                     "frac": achieved / peaks["hbm_gbs"], "traffic": traffic, "peak_source": f"of {peaks['source']}",
                     "kernel_ms": kt[dom], "algorithmic_bytes_per_launch": ab[kind]}
         else:
-            # fp32 ALU-bound stage (resolve / scan): peak = SMs x 128 lanes x 2 flop x max SM clock
-            import torch as _t
-            prop = _t.cuda.get_device_properties(local_rank)
-            peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+            # resolve / scan: 2 d^3 (Gauss-Jordan) resp. 2 x 2 d^3 (two directions) fp32-equivalent flops per frame
             work = (2 if "resolve" in dom else 4) * w.B * w.H * w.T * w.d ** 3
-            achieved = work / (kt[dom] / 1e3) / 1e12
-            roof = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                    "frac": achieved / peak, "traffic": None, "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
-                    "kernel_ms": kt[dom]}
+            if dom.endswith("_tc"):
+                # on the tensor cores every fp32 product is six bf16 partial products (three-way splits of both
+                # factors): the fraction is of the bf16 tensor peak, counting those; a chain of T dependent
+                # frame steps per (batch, head, direction) bounds the scan long before the peak does
+                achieved = 6 * work / (kt[dom] / 1e3) / 1e12
+                roof = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["bf16_tflops"],
+                        "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                        "peak_source": f"of {peaks['source']} (bf16 burst); six bf16 partial products per fp32 product",
+                        "kernel_ms": kt[dom], "fp32_equivalent_tflops": work / (kt[dom] / 1e3) / 1e12}
+            else:
+                # plain fp32 kernels: peak = SMs x 128 lanes x 2 flop x max SM clock
+                import torch as _t
+                prop = _t.cuda.get_device_properties(local_rank)
+                peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+                achieved = work / (kt[dom] / 1e3) / 1e12
+                roof = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                        "frac": achieved / peak, "traffic": None,
+                        "peak_source": f"{prop.multi_processor_count} SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                        "kernel_ms": kt[dom]}
     t_roof_ms = max(ab["total"] / (peaks["hbm_gbs"] * 1e9), fl["tensor"] / (peaks["bf16_tflops_sustained"] * 1e12)) * 1e3
     t_roof_nominal_ms = max(ab["total"] / 8e12, fl["tensor"] / 2.25e15) * 1e3
 

@@ -17,13 +17,22 @@
 //     plain fp32 rows (8 KB, sixteen 16-byte stores per lane); after one barrier every thread picks up its column
 //     with sixteen conflict-free 4-byte reads.  (An earlier version took M[P_k][j] = +-M[j][P_k] from the thread's own
 //     row instead -- exact while the matrix stays symmetric up to the sign pattern of in-place elimination, but the
-//     rounding of the updates breaks that symmetry a little at every step, and mixing the two copies cost a factor
-//     of the condition number in accuracy: a left residual of 8e-2 instead of 8e-5 at lambda_max = 2000 in an fp32
-//     emulation, 5e-6 instead of 1e-6 of the largest entry on benign matrices.)
-//   * The 128 x 16 coefficients Cm = -M[:, P] Gi are a matrix product as well: the pivot-row operand the threads
-//     have just written, times Gi (split three-way by the pivot warp), in a first, 128 x 16 x 16 MMA into the
-//     pivot columns themselves; each thread reads its row back and negates it.  Formed with fp32 FMAs
-//     (256 per thread and step) they were the largest item of a kernel that is bound by instruction issue.
+//     rounding of the updates breaks that symmetry a little at every step, and pivot rows taken from the columns cost
+//     a factor of the condition number in accuracy: a left residual of 8e-2 instead of 8e-5 at lambda_max = 2000 in
+//     an fp32 emulation, 5e-6 instead of 1e-6 of the largest entry on benign matrices.)
+//   * The 128 x 16 coefficients Cm = -M[:, P] Gi are a matrix product as well, in a first, 128 x 16 x 16 MMA into the
+//     pivot columns themselves; each thread reads its row back and fixes the sign.  Its A operand is the pivot-row
+//     operand just written: row i of it is M[P][i], which equals M[i][P] up to the sign pattern (minus for a row
+//     whose block has been a pivot block already, plus otherwise) and up to rounding.  This direction of the
+//     substitution is harmless -- the update stays an exact row operation with the true pivot rows, only its
+//     coefficients are perturbed at rounding level (same fp32 emulation: left residual 1.1e-4 against 0.8e-4 with
+//     the true columns at lambda_max = 2000) -- and it saves forming a second operand per step.  Formed with fp32
+//     FMAs (256 per thread and step) the coefficients were the largest item of a kernel that is bound by
+//     instruction issue.
+//   * The operand rows of the 16 pivot rows themselves are never needed: as A rows they produce the pivot rows'
+//     coefficients, which are replaced by Gi; as B rows they produce the update of the pivot columns, which the
+//     column fix overwrites.  The warp that owns the pivot rows therefore writes no operand at all, and the sixteen
+//     other rows of that warp are written by half of a neighbouring warp while the pivot block is being inverted.
 // The matrix that is inverted is I + (A_t + A_t^T)/2: the stored statistics are symmetric only up to the bf16
 // rounding of one factor, and the symmetric part is the natural reading of Eq. 3b (and keeps Proposition 1).
 // The inverse is written as three bf16 parts C1 + C2 + C3 for the tensor-core scan.
@@ -53,8 +62,7 @@ struct ResolveTc {
   static constexpr int OFF_CM = 0;
   static constexpr int PRF_STRIDE = D + 4;            // floats per fp32 pivot row: the sixteen lanes' 16-byte stores conflict two by two, the minimum
   static constexpr int OFF_PR = CM_BYTES;
-  static constexpr int OFF_XO = OFF_PR + PR_BYTES;    // pivot columns, K-major: row i = M[i][P], parts laid out like the others
-  static constexpr int OFF_GIB = OFF_XO + PR_BYTES;   // Gi as an MMA operand: 16 rows x 128 B, three parts per row
+  static constexpr int OFF_GIB = OFF_PR + PR_BYTES;   // Gi as an MMA operand: 16 rows x 128 B, three parts per row
   static constexpr int OFF_GI = OFF_GIB + 2048;       // Gi, 16 x 16 floats (for the pivot rows themselves)
   static constexpr int OFF_PRF = OFF_CM;              // the 16 pivot rows in fp32, [16][PRF_STRIDE]: in the coefficient
                                                       // operand's place until the coefficients exist (four CTAs per SM
@@ -111,14 +119,14 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       constexpr int PB[6] = {2, 0, 1, 1, 0, 0};
       constexpr uint32_t idesc_c = make_idesc_bf16(128, 16, false, false);
       for (int step = 0; step < D / R::NB; ++step) {
-        // ---- coefficients: M[:, P] <- X Gi (128 x 16 x 16), X = the pivot columns the row threads just wrote as an
-        // operand, Gi = the inverse of the pivot block; each thread negates its row
+        // ---- coefficients: M[:, P] <- Y Gi (128 x 16 x 16), Y = the pivot-row operand the row threads just wrote
+        // (row i = M[P][i] = +-M[i][P]), Gi = the inverse of the pivot block; each thread fixes the sign of its row
         const int p0c = (((int)(blockIdx.x & 3) * 2 + step) & 7) * R::NB;
         if (!mbar_wait(XREADY, step & 1, wc)) break;
         tc_fence_after_sync();
 #pragma unroll
         for (int pr = 0; pr < 6; ++pr) {
-          const uint64_t adesc = make_smem_desc(base + R::OFF_XO + PA[pr] * 32, 16, 1024);
+          const uint64_t adesc = make_smem_desc(base + R::OFF_PR + PA[pr] * 32, 16, 1024);
           const uint64_t bdesc = make_smem_desc(base + R::OFF_GIB + PB[pr] * 32, 16, 1024);
           mma_bf16_ss(tmem_base + p0c, adesc, bdesc, idesc_c, pr == 0 ? 0u : 1u);
         }
@@ -140,8 +148,8 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
     const int row = warp * 32 + lane;
     const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
     // M = I + (A_t + A_t^T)/2 into TMEM.  The stored block is K^T (beta K) with one factor rounded to bf16,
-    // symmetric only up to that rounding; its symmetric part is what gets inverted, and exact symmetry is
-    // what lets every thread supply its share of the pivot rows below.  Column `row` is read with
+    // symmetric only up to that rounding; its symmetric part is what gets inverted (the coefficients below
+    // rely on the symmetry).  Column `row` is read with
     // consecutive lanes on consecutive addresses, row `row` as 16-byte pieces (mostly L1/L2 hits).
     {
       const float* col = stats + (size_t)n * (2 * D * D) + row;
@@ -173,7 +181,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
     const int blk0 = (int)((blockIdx.x & 3) * 2);
     bool ok = true;
     float* prf = reinterpret_cast<float*>(base_ptr + R::OFF_PRF);  // fp32 pivot rows
-    auto store_operand_row = [&](int off, const float (&val)[16]) {
+    auto store_operand_row = [&](int off, int r, const float (&val)[16]) {
       uint4 w[3][2];
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
@@ -183,24 +191,31 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
         reinterpret_cast<uint32_t*>(&w[1][q >> 2])[q & 3] = a2;
         reinterpret_cast<uint32_t*>(&w[2][q >> 2])[q & 3] = a3;
       }
-      unsigned char* orow = base_ptr + off + row * 128;
+      unsigned char* orow = base_ptr + off + r * 128;
 #pragma unroll
       for (int part = 0; part < 3; ++part) {
-        *reinterpret_cast<uint4*>(orow + (((2 * part) ^ (row & 7)) * 16)) = w[part][0];
-        *reinterpret_cast<uint4*>(orow + (((2 * part + 1) ^ (row & 7)) * 16)) = w[part][1];
+        *reinterpret_cast<uint4*>(orow + (((2 * part) ^ (r & 7)) * 16)) = w[part][0];
+        *reinterpret_cast<uint4*>(orow + (((2 * part + 1) ^ (r & 7)) * 16)) = w[part][1];
       }
     };
+    // The pivot-row operand's rows that belong to the pivot rows themselves are never needed (see below); they are
+    // zero from the start rather than whatever the memory held.
+    {
+      uint4* z = reinterpret_cast<uint4*>(base_ptr + R::OFF_PR + row * 128);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) z[e] = make_uint4(0u, 0u, 0u, 0u);
+    }
 #pragma unroll 1
     for (int step = 0; step < D / R::NB && ok; ++step) {
       const int blk = (blk0 + step) & 7;
       const int p0 = blk * R::NB;
       const bool owner = (row >> 4) == blk;               // rows p0 .. p0+15: 16 lanes of warp blk/2
+      const bool eliminated = (((row >> 4) - blk0) & 7) < step;   // this row's block was a pivot block already
       float x[16];
-      tmem_ld16(trow + p0, x);                            // this row's entries in the pivot columns
-      tmem_wait_ld();
 
       // ---- the 16 pivot rows, as they stand before this step, to shared memory in fp32 (the warp that owns them)
       if (warp == (blk >> 1)) {
+        tmem_ld16(trow + p0, x);                          // the pivot block itself: this row's entries in the pivot columns
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
           float v[32];
@@ -213,17 +228,21 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           }
         }
       }
-      // ---- pivot columns as an operand (for the coefficients), while the pivot rows are on their way
-      store_operand_row(R::OFF_XO, x);
       named_barrier_sync(1, 128);                         // the pivot rows are in shared memory
       // thread j's column of the pivot rows: one row of the K-major operand (row = output column).  The warp that
       // owns the pivot rows does this later, under the coefficient MMA: it is the one everybody waits for.
       float y[16];
-      auto load_pivot_column = [&]() {
+      auto load_pivot_column = [&](int r) {
 #pragma unroll
-        for (int k = 0; k < 16; ++k) y[k] = prf[k * R::PRF_STRIDE + row];
+        for (int k = 0; k < 16; ++k) y[k] = prf[k * R::PRF_STRIDE + r];
       };
-      if (warp != (blk >> 1)) { load_pivot_column(); store_operand_row(R::OFF_PR, y); }
+      if (warp != (blk >> 1)) { load_pivot_column(row); store_operand_row(R::OFF_PR, row, y); }
+      if (warp == (((blk >> 1) + 1) & 3) && lane < 16) {
+        // the sixteen rows that share a warp with the pivot rows: that warp is busy with the pivot block
+        const int hrow = (blk ^ 1) * 16 + lane;
+        load_pivot_column(hrow);
+        store_operand_row(R::OFF_PR, hrow, y);
+      }
       if (warp == (blk >> 1)) {
         // ---- invert the 16 x 16 pivot block: lane (l0 + a) holds row a; pivot rows travel by shuffle
         const int l0 = (blk & 1) * 16;
@@ -277,15 +296,13 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           }
         }
       }
-      // (the fp32 pivot rows share their memory with the coefficient operand, which the other warps write as soon as
-      // the coefficient MMA has completed, i.e. some time after the arrival below: read them before it)
-      if (warp == (blk >> 1)) load_pivot_column();
+      // (the fp32 pivot rows share their memory with the coefficient operand, which the warps write once the
+      // coefficient MMA has completed, i.e. after all four arrivals below: every read of them comes before)
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive_warp(XREADY);
-      if (warp == (blk >> 1)) store_operand_row(R::OFF_PR, y);
 
-      // ---- coefficients: c = -M[i][P] Gi = -(X Gi) from the tensor cores; a pivot row a takes Gi[a]
+      // ---- coefficients: c = -M[i][P] Gi = -+(Y Gi) from the tensor cores; a pivot row a takes Gi[a]
       if (!mbar_wait(CDONE, step & 1, wc)) { ok = false; break; }
       tc_fence_after_sync();
       float c[16];
@@ -300,14 +317,14 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
         }
       } else {
 #pragma unroll
-        for (int k = 0; k < 16; ++k) c[k] = -c[k];
+        for (int k = 0; k < 16; ++k) c[k] = eliminated ? c[k] : -c[k];
       }
       // ---- A operand: this row's 16 update coefficients (pivot rows: Gi[a] - e_a), three bf16 parts
       {
         float u[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) u[k] = (owner && (row & 15) == k) ? c[k] - 1.0f : c[k];
-        store_operand_row(R::OFF_CM, u);
+        store_operand_row(R::OFF_CM, row, u);
       }
       fence_proxy_async_smem();
       tc_fence_before_sync();
