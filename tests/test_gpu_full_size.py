@@ -34,9 +34,9 @@ def sampled_pairs(w, count):
     return pairs[:count]
 
 
-def run_and_check(w, nheads):
+def run_and_check(w, nheads, flags=0):
     x = inputs.generate(w, "cuda")
-    vda = binding.Vda(w.d, w.dtype)
+    vda = binding.Vda(w.d, w.dtype, flags=flags)
     assert vda.uses_tensor_cores()
     out = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
     torch.cuda.synchronize()
@@ -66,6 +66,15 @@ def run_and_check(w, nheads):
 
 def test_768p_config_full_size():
     run_and_check(inputs.CLIP_768P, 4)       # first, last and two seeded (batch, head) slices
+
+
+@pytest.mark.parametrize("flags", [binding.VDN_FLAG_EXACT_STATS,
+                                   binding.VDN_FLAG_EXACT_STATS | binding.VDN_FLAG_FP32_RESOLVE])
+def test_768p_config_full_size_accuracy_options(flags):
+    # the statistics from exact weighted keys, and with the plain-fp32 inverse behind them: other kernels in the same
+    # launch configuration; the error is the default path's less the share of the bf16-rounded weighted keys
+    worst = run_and_check(inputs.CLIP_768P, 2, flags=flags)
+    assert worst <= 6e-3, f"flags={flags}: {worst:.3e}"
 
 
 @pytest.mark.parametrize("idx", [0, 1, 2, 3])
