@@ -70,7 +70,11 @@
  *     of about 5 on), nor when all keys of a frame lie within a few degrees of one direction: unit keys drawn as one
  *     direction plus N(0, s^2) per component give 6e-3 at s = 0.05, 1e-2 at 0.02, 1.7e-2 at 0.01 (a cone of about six
  *     degrees), 3.5e-2 at 0.005, 8e-2 at 0.002 -- the rounding of the weighted keys (4e-3) must stay small against
- *     the keys' own spread.
+ *     the keys' own spread.  The states a frame reads (P_{t-1}, R_{t+1}) reach the read-out as bf16 as well: a row
+ *     whose read-out nearly cancels, |S q| << |S| |q|, keeps that much less of it, and the RMSNorm rescales what is
+ *     left.  States of thousands of tokens have full rank and no query is orthogonal to them; with ONE token per
+ *     frame and one frame left to read, a query at |cos| = 2e-4 to that frame's key gave 1e-1 (plain-fp32 kernels,
+ *     whose states stay fp32: 4e-3).
  *   VDN_FLAG_EXACT_STATS contracts the exactly weighted keys (two bf16 parts; the statistics then equal the plain-fp32
  *     kernels' to 5e-7): 4e-3 for keys within any cone (s = 0.002 .. 0.05 above); within 2e-2 (4e-3 .. 1e-2) up to 99 % identical keys for lambda_max up to 5e5 at F = 4080 and up
  *     to about 1e4 at F = 300, and with all keys
