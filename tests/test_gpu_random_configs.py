@@ -1,5 +1,6 @@
 """Parity on seeded random configurations: shapes that straddle the 128-token tile and the SM count, with a random
-choice of kernel path, window, anchors, decay gates, text state, element-wise gate, norm weight and rule.
+choice of kernel path, window, anchors, decay gates, text state, element-wise gate, norm weight, rule, value scale
+and gate sign.
 
 The hand-picked cases of test_gpu_parity.py and test_gpu_window.py name the edges one at a time; this file draws
 combinations of them.  The draws are fixed by the case number, so a failure names a reproducible configuration.
@@ -64,6 +65,8 @@ def draw(case):
         cfg["flags"] = (cfg["flags"] & binding.VDN_FLAG_FORCE_SIMT) | binding.VDN_FLAG_ADDITIVE_RULE
     cfg["sched"] = int(rng.choice([0, binding.VDN_FLAG_SCAN_CHUNKWISE, binding.VDN_FLAG_SCAN_FRAMEWISE]))
     cfg["via_host"] = bool(rng.random() < 0.25)        # through the host-buffer entry point (pinned memory)
+    cfg["v_scale_log2"] = int(rng.choice([0, 0, -10, 10]))   # values far from unit scale (exact in bf16): the RMSNorm's
+    cfg["negative_gates"] = bool(rng.random() < 0.25)        # epsilon against small read-outs; gates of either sign
     return cfg
 
 
@@ -73,6 +76,10 @@ def test_random_configuration_matches_oracle(case):
     w = inputs.TINY.scaled(dtype=c["dtype"], d=c["d"], B=c["B"], H=c["H"], T=c["T"], F=c["F"], seed=9000 + case)
     x = inputs.generate(w, "cuda")
     alpha, s0 = inputs.generate_recurrence_extras(w, "cuda")
+    x["v"] = x["v"] * (2.0 ** c["v_scale_log2"])
+    s0 = s0 * (2.0 ** c["v_scale_log2"])
+    if c["negative_gates"]:
+        x["gate"] = x["gate"] * (1.0 - 2.0 * (torch.arange(w.H, device="cuda") % 2)).to(x["gate"].dtype)
     gen = torch.Generator(device="cpu").manual_seed(9100 + case)
     io = torch.bfloat16 if c["dtype"] == "bf16" else torch.float32
     ge = nw = None
