@@ -297,6 +297,40 @@ def test_run_to_run_bitwise_determinism_and_canaries():
     assert torch.all(buf[:pad] == 7.0) and torch.all(buf[pad + n:] == 7.0)
 
 
+def test_one_handle_across_shapes_and_two_handles_on_two_streams():
+    # a handle carries no shape: calls of different shapes in turn give what a fresh handle gives, bit for bit; and
+    # two handles (each with its own workspace) run side by side on two streams without touching each other
+    shapes = [dict(T=4, F=333, H=3), dict(T=7, F=128, H=1, B=2), dict(T=2, F=1000, H=5), dict(T=4, F=333, H=3)]
+    ws = [inputs.TINY.scaled(dtype="bf16", d=128, seed=300 + i, **kw) for i, kw in enumerate(shapes)]
+    xs = [inputs.generate(w, "cuda") for w in ws]
+    fresh = []
+    for w, x in zip(ws, xs):
+        v = binding.Vda(w.d, w.dtype)
+        fresh.append(v.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"]).clone())
+        torch.cuda.synchronize()
+        v.close()
+    vda = binding.Vda(128, "bf16")
+    for w, x, want in zip(ws, xs, fresh):
+        got = vda.forward(x["q"], x["k"], x["v"], x["beta"], x["gate"])
+        torch.cuda.synchronize()
+        assert torch.equal(got, want), f"shape {w.T}x{w.F}x{w.H} after another shape on the same handle"
+    a, b = binding.Vda(128, "bf16"), binding.Vda(128, "bf16")
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs_a, outs_b = [], []
+    for _ in range(3):
+        with torch.cuda.stream(sa):
+            outs_a.append(a.forward(xs[0]["q"], xs[0]["k"], xs[0]["v"], xs[0]["beta"], xs[0]["gate"]).clone())
+        with torch.cuda.stream(sb):
+            outs_b.append(b.forward(xs[2]["q"], xs[2]["k"], xs[2]["v"], xs[2]["beta"], xs[2]["gate"]).clone())
+    torch.cuda.synchronize()
+    assert a.status() == binding.VDN_OK and b.status() == binding.VDN_OK
+    for o in outs_a:
+        assert torch.equal(o, fresh[0])
+    for o in outs_b:
+        assert torch.equal(o, fresh[2])
+
+
 def test_forward_can_be_captured_in_a_cuda_graph():
     # the layer only enqueues kernels and memsets on the caller's stream (tensor maps travel as kernel parameters):
     # after one eager call (which sets the kernels' attributes) it can be captured and replayed; replays are
