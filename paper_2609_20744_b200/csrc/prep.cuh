@@ -190,44 +190,49 @@ prep_spatial_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   for (int t = first; t <= last; ++t) {
     // the other buffer was last read for frame t - 1; every thread passed the barrier that closed that frame
     if (tid == 0 && t + 1 <= last) stage(t + 1);
-    if (!mbar_wait(bar0 + 8u * (t & 1), ((t - first) >> 1) & 1, wc)) break;        // frame t's tile has landed
-    const Tio* tbase = tile + (size_t)(t & 1) * SH * SW * D + (size_t)(RPT * g) * SW * D + 2 * cp;
-    f32x2 acc[RPT][TX];
+    // frame t's tile has landed -- or the wait ran out: such a thread skips the frame and says so at the barrier
+    // that closes it, where all leave together (a lone `break` would leave the others standing at that barrier)
+    const bool landed = mbar_wait(bar0 + 8u * (t & 1), ((t - first) >> 1) & 1, wc);
+    if (landed) {
+      const Tio* tbase = tile + (size_t)(t & 1) * SH * SW * D + (size_t)(RPT * g) * SW * D + 2 * cp;
+      f32x2 acc[RPT][TX];
 #pragma unroll
-    for (int r = 0; r < RPT; ++r)
+      for (int r = 0; r < RPT; ++r)
 #pragma unroll
-      for (int j = 0; j < TX; ++j) acc[r][j] = 0ull;
+        for (int j = 0; j < TX; ++j) acc[r][j] = 0ull;
 #pragma unroll
-    for (int xi = 0; xi < SW; ++xi) {       // input column xi sits at x0 - 2 + xi
-      f32x2 in[4 + RPT];
+      for (int xi = 0; xi < SW; ++xi) {       // input column xi sits at x0 - 2 + xi
+        f32x2 in[4 + RPT];
 #pragma unroll
-      for (int i = 0; i < 4 + RPT; ++i) in[i] = load_pair(tbase + ((size_t)i * SW + xi) * D);
+        for (int i = 0; i < 4 + RPT; ++i) in[i] = load_pair(tbase + ((size_t)i * SW + xi) * D);
 #pragma unroll
-      for (int i = 0; i < 5; ++i) {
+        for (int i = 0; i < 5; ++i) {
 #pragma unroll
-        for (int j = 0; j < 5; ++j) {       // tap column j: output column xo = xi - j
-          const int xo = xi - j;
-          if (xo < 0 || xo >= TX) continue;
+          for (int j = 0; j < 5; ++j) {       // tap column j: output column xo = xi - j
+            const int xo = xi - j;
+            if (xo < 0 || xo >= TX) continue;
 #pragma unroll
-          for (int r = 0; r < RPT; ++r) acc[r][xo] = fma2(wsp[i][j], in[i + r], acc[r][xo]);
+            for (int r = 0; r < RPT; ++r) acc[r][xo] = fma2(wsp[i][j], in[i + r], acc[r][xo]);
+          }
         }
       }
-    }
 #pragma unroll
-    for (int r = 0; r < RPT; ++r) {
-      if (yr + r < a.Y) {
+      for (int r = 0; r < RPT; ++r) {
+        if (yr + r < a.Y) {
 #pragma unroll
-        for (int j = 0; j < TX; ++j) {
-          if (x0 + j < a.X) {
-            float o0, o1;
-            unpack2(acc[r][j], o0, o1);
-            store_pair(pdst + ((size_t)r * a.X + j) * (s.H * D), o0, o1);
+          for (int j = 0; j < TX; ++j) {
+            if (x0 + j < a.X) {
+              float o0, o1;
+              unpack2(acc[r][j], o0, o1);
+              store_pair(pdst + ((size_t)r * a.X + j) * (s.H * D), o0, o1);
+            }
           }
         }
       }
     }
     pdst += frame_elems;
-    __syncthreads();                        // this frame's buffer may be overwritten by the copy issued two frames on
+    // this frame's buffer may be overwritten by the copy issued two frames on
+    if (__syncthreads_or(landed ? 0 : 1)) break;
   }
   if (tid == 0 && *abort_flag) {
     // a wait gave up: give the copy that may still be in flight a bounded chance to land before the CTA retires

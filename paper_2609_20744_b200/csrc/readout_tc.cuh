@@ -251,6 +251,13 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     bool ok = true;
     constexpr bool use_ge = GATE;            // (gate_elem itself is read through its tensor map)
     float* nws = reinterpret_cast<float*>(base_ptr + R::OFF_NW);
+    // A warp whose wait ran out does not just leave: the other three, whose wait may have been satisfied a moment
+    // earlier, would stand at their next block barrier for ever.  It goes to that barrier -- between two barriers
+    // every wait of a tile has the same next one: 1 without a gate tile, else 2 -- says so there, and all leave.
+    auto give_up = [&]() {
+      named_barrier_or(use_ge ? 2 : 1, 128, true);
+      ok = false;
+    };
     // EXTRAS: the gate tile of tile number q (counted over this CTA's tiles) is copied into staging tile q % NOUT,
     // where the output of that tile is then written; issued by one thread, two tiles ahead
     auto issue_gate = [&](uint32_t q, long long gitem, int gtile) {
@@ -276,15 +283,15 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // this head's norm weights into shared memory (all epilogue threads are past the previous frame's reads:
         // they met at the barrier before its last store)
         nws[et] = __ldg(norm_weight + (size_t)h * R::D + et);
-        named_barrier_sync(1, 128);
+        if (named_barrier_or(1, 128, false)) { ok = false; break; }
       }
       for (int tile = 0; tile < ntiles; ++tile, ++qi) {
         const int a = qi & 3;
-        if (!mbar_wait(ACCFULL(a), (qi >> 2) & 1, wc)) { ok = false; break; }
+        if (!mbar_wait(ACCFULL(a), (qi >> 2) & 1, wc)) { give_up(); break; }
         tc_fence_after_sync();
         float qrs = 1.0f;
         if constexpr (QNORM) {
-          if (!mbar_wait(QNFULL(qi % QS), (qi / QS) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait(QNFULL(qi % QS), (qi / QS) & 1, wc)) { give_up(); break; }
           qrs = reinterpret_cast<const float*>(base_ptr + R::OFF_QN)[(qi % QS) * 128 + row];
         }
         const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + a * 128;
@@ -314,10 +321,10 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (use_ge) {
           // the gate tile sits in the staging tile (its copy was issued after the store that last used the tile
           // had been read)
-          if (!mbar_wait(GFULL(ob), (qi / R::NOUT) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait(GFULL(ob), (qi / R::NOUT) & 1, wc)) { give_up(); break; }
         } else {
           if (et == 0) tma_store_wait_read<R::NOUT - 1>();   // the store that last used this staging tile has read it
-          named_barrier_sync(1, 128);
+          if (named_barrier_or(1, 128, false)) { ok = false; break; }
         }
         unsigned char* orow = base_ptr + R::OFF_OUT + ob * R::TILE_BYTES + row * 128;
 #pragma unroll
@@ -358,7 +365,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           }
         }
         fence_proxy_async_smem();
-        named_barrier_sync(2, 128);
+        if (named_barrier_or(2, 128, false)) { ok = false; break; }
         if (et == 0) {
           const uint32_t src = base + R::OFF_OUT + ob * R::TILE_BYTES;
           tma_store_5d(&tmO, src, 0, h, tile * R::TILE, t, b);

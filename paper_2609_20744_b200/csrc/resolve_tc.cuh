@@ -206,7 +206,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       for (int e = 0; e < 8; ++e) z[e] = make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll 1
-    for (int step = 0; step < D / R::NB && ok; ++step) {
+    for (int step = 0; step < D / R::NB; ++step) {
       const int blk = (blk0 + step) & 7;
       const int p0 = blk * R::NB;
       const bool owner = (row >> 4) == blk;               // rows p0 .. p0+15: 16 lanes of warp blk/2
@@ -228,7 +228,9 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
           }
         }
       }
-      named_barrier_sync(1, 128);                         // the pivot rows are in shared memory
+      // the pivot rows are in shared memory -- or a wait of the step before ran out somewhere: a thread that gave up
+      // comes here all the same (`continue` below, not `break`), so that nobody is left standing at this barrier
+      if (named_barrier_or(1, 128, !ok)) { ok = false; break; }
       // thread j's column of the pivot rows: one row of the K-major operand (row = output column).  The warp that
       // owns the pivot rows does this later, under the coefficient MMA: it is the one everybody waits for.
       float y[16];
@@ -303,7 +305,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       mbar_arrive_warp(XREADY);
 
       // ---- coefficients: c = -M[i][P] Gi = -+(Y Gi) from the tensor cores; a pivot row a takes Gi[a]
-      if (!mbar_wait(CDONE, step & 1, wc)) { ok = false; break; }
+      if (!mbar_wait(CDONE, step & 1, wc)) { ok = false; continue; }
       tc_fence_after_sync();
       float c[16];
       tmem_ld16(trow + p0, c);
@@ -329,7 +331,7 @@ resolve_tc_kernel(const float* __restrict__ stats, __nv_bfloat16* __restrict__ c
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive_warp(OPREADY);
-      if (!mbar_wait(MMADONE, step & 1, wc)) { ok = false; break; }
+      if (!mbar_wait(MMADONE, step & 1, wc)) { ok = false; continue; }
       tc_fence_after_sync();
       // ---- column fix: M[i][P] = c (for a pivot row: Gi[a])
       tmem_st16(trow + p0, c);

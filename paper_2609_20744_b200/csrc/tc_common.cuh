@@ -253,5 +253,21 @@ __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// A block-level barrier that also tells every participant whether any of them has given up on a wait.  A thread whose
+// wait ran out does not leave at once -- the others, whose wait may have been satisfied a moment earlier, would then
+// stand at their next bar.sync for ever -- but comes to that barrier with `gave_up` set, and all leave together.
+__device__ __forceinline__ bool named_barrier_or(int id, int nthreads, bool gave_up) {
+  uint32_t any;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(any)
+      : "r"(id), "r"(nthreads), "r"(gave_up ? 1u : 0u)
+      : "memory");
+  return any != 0;
+}
+
 }  // namespace tc
 }  // namespace vdn
