@@ -376,8 +376,10 @@ vdn_status vdn_vda_set_wait_limit_us(vdn_vda_t h, unsigned long long microsecond
  * the same wait routine) and waits, for at most limit_us microseconds (<= 1 s), on a barrier that nothing ever
  * completes and that no copy is bound to.  The wait runs out, the CTA takes the same abort and teardown path as
  * the real kernels (frees its tensor memory, returns) and records VDN_ERR_TIMEOUT in the handle's status word.
- * After synchronising: vdn_vda_status gives VDN_ERR_TIMEOUT and vdn_vda_selftest_marker gives 1 (the CTA reached
- * its last instruction after giving up; 0 = the kernel has not run, -1 = null handle). */
+ * After synchronising: vdn_vda_status gives VDN_ERR_TIMEOUT and vdn_vda_selftest_marker gives 3 (bit 0: the CTA
+ * reached its last instruction after giving up; bit 1: its other warp, which had waited for nothing, learned of the
+ * timeout at the block-level barrier the two share, the way threads of the real kernels leave together; 0 = the
+ * kernel has not run, -1 = null handle). */
 vdn_status vdn_vda_selftest_wait_expiry(vdn_vda_t h, unsigned long long limit_us, void* cuda_stream);
 int vdn_vda_selftest_marker(vdn_vda_t h);
 
