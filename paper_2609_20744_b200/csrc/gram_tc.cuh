@@ -124,9 +124,8 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         }
       }
       if (!ok) {
-        // give copies that are already in flight a bounded chance to land before the CTA retires
-        for (int st = 0; st < G::STAGES; ++st)
-          for (int spin = 0; spin < 4096 && !mbar_try_wait(FULL(st), 0) && !mbar_try_wait(FULL(st), 1); ++spin) {}
+        // give copies that are already in flight (`it` were issued) a bounded chance to land before the CTA retires
+        mbar_drain_ring(FULL(0), G::STAGES, it);
       }
     }
   } else if (warp == 1) {

@@ -179,7 +179,9 @@ prep_spatial_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   Tio* pdst = dst + token_offset(s, b, first, min(yr, a.Y - 1) * a.X + x0, h) + 2 * cp;
 
   // frame t's halo tile -> buffer t & 1 (one thread; the engine zero-fills what lies outside the frame)
+  int last_staged = first - 1;
   auto stage = [&](int t) {
+    last_staged = t;
     const uint32_t bar = bar0 + 8u * (t & 1);
     mbar_arrive_expect_tx(bar, TILE_BYTES);
     tma_load_5d(base + (uint32_t)(t & 1) * TILE_BYTES, tm, bar, 0, h, x0 - HALO, y0 - HALO, b * s.T + t);
@@ -235,9 +237,8 @@ prep_spatial_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (__syncthreads_or(landed ? 0 : 1)) break;
   }
   if (tid == 0 && *abort_flag) {
-    // a wait gave up: give the copy that may still be in flight a bounded chance to land before the CTA retires
-    for (int i = 0; i < 2; ++i)
-      for (int spin = 0; spin < 4096 && !mbar_try_wait(bar0 + 8u * i, 0) && !mbar_try_wait(bar0 + 8u * i, 1); ++spin) {}
+    // a wait gave up: give the copies that may still be in flight a bounded chance to land before the CTA retires
+    for (int tt = max(first, last_staged - 1); tt <= last_staged; ++tt) mbar_drain(bar0 + 8u * (tt & 1), ((tt - first) >> 1) & 1);
   }
 }
 

@@ -125,13 +125,14 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t qi = 0, si = 0;
+      uint32_t qi = 0, si = 0, states_issued = 0;
       bool ok = true;
       for (long long item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++si) {
         int b, h, t;
         const long long n = split_work(s, item, b, h, t);
         const int sb = si % R::STSTAGES;
         if (!mbar_wait(STEMPTY(sb), ((si / R::STSTAGES) & 1) ^ 1, wc)) { ok = false; break; }
+        states_issued = si + 1;
         mbar_arrive_expect_tx(STFULL(sb), 2 * R::TILE_BYTES);
         const uint32_t sdst = base + R::OFF_STATE + sb * 2 * R::TILE_BYTES;
         // Slot of the forward state in rows [nf*128, +128), of the reverse state in rows [nrev*128, +128).  With
@@ -153,8 +154,10 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
       }
       if (!ok) {
-        for (int st = 0; st < R::QSTAGES; ++st)
-          for (int spin = 0; spin < 4096 && !mbar_try_wait(QFULL(st), 0) && !mbar_try_wait(QFULL(st), 1); ++spin) {}
+        // give the copies already in flight (qi query tiles, states_issued pairs of states) a bounded chance to land
+        // before the CTA retires
+        mbar_drain_ring(QFULL(0), R::QSTAGES, qi);
+        mbar_drain_ring(STFULL(0), R::STSTAGES, states_issued);
       }
     }
   } else if (warp == 1) {
@@ -260,6 +263,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     };
     // EXTRAS: the gate tile of tile number q (counted over this CTA's tiles) is copied into staging tile q % NOUT,
     // where the output of that tile is then written; issued by one thread, two tiles ahead
+    uint32_t gates_issued = 0;
     auto issue_gate = [&](uint32_t q, long long gitem, int gtile) {
       while (gtile >= ntiles) { gtile -= ntiles; gitem += gridDim.x; }
       if (gitem >= nitems) return;
@@ -267,6 +271,7 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       split_work(s, gitem, gb, gh, gt);
       const int ob = q % R::NOUT;
       const uint32_t dstg = base + R::OFF_OUT + ob * R::TILE_BYTES;
+      gates_issued = q + 1;
       mbar_arrive_expect_tx(GFULL(ob), R::TILE_BYTES);
       tma_load_5d(dstg, &tmG, GFULL(ob), 0, gh, gtile * R::TILE, gt, gb);
       tma_load_5d(dstg + R::BOX_BYTES, &tmG, GFULL(ob), 64, gh, gtile * R::TILE, gt, gb);
@@ -380,7 +385,11 @@ readout_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
       }
     }
-    if (et == 0) tma_store_wait_all<0>();
+    if (et == 0) {
+      tma_store_wait_all<0>();
+      // a wait gave up: the gate tiles already on their way get a bounded chance to land before the CTA retires
+      if (use_ge && !ok) mbar_drain_ring(GFULL(0), R::NOUT, gates_issued);
+    }
   }
 
   // ------------------------------------------------------------------ teardown

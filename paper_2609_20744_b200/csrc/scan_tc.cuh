@@ -163,17 +163,25 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tmC, const ScanTcArgs a, tc::
     // of this step's MMA time plus the state warps' turn to arrive.
     if (lane == 0) {
       bool ok = true;
+      uint32_t issued[3] = {0u, 0u, 0u};
       for (int s = 0; s < nsteps && ok; ++s) {
         const long long n = item_of(s);
 #pragma unroll
         for (int p = 2; p >= 0; --p) {
           if (!mbar_wait(CFREE(p), (s & 1) ^ 1, wc)) { ok = false; break; }
+          issued[p] = (uint32_t)s + 1u;
           mbar_arrive_expect_tx(CFULL(p), S::PART_BYTES);
           const uint32_t dst = base + S::OFF_C + p * S::PART_BYTES;
           const int row = (int)((n * 3 + p) * D);
           tma_load_2d(dst, &tmC, CFULL(p), 0, row);
           tma_load_2d(dst + S::BOX_BYTES, &tmC, CFULL(p), 64, row);
         }
+      }
+      if (!ok) {
+        // give the copies already in flight a bounded chance to land before the CTA retires
+#pragma unroll
+        for (int p = 0; p < 3; ++p)
+          if (issued[p]) mbar_drain(CFULL(p), (issued[p] - 1u) & 1u);
       }
     }
   } else if (warp == 1) {

@@ -84,6 +84,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
   }
 }
 
+// After a wait gave up: the copy last issued on `bar` completes the phase of parity `parity`; give it a bounded
+// chance to land before the CTA retires and its shared memory goes to another CTA.  (Asking for either parity would
+// return at once: the phase before the current one always counts as complete.)
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  for (int spin = 0; spin < 4096 && !mbar_try_wait(bar, parity); ++spin) {}
+}
+// ... for a ring of `stages` barriers (`first` + 8 * stage) on which `issued` copies went out round-robin, copy j on
+// stage j % stages completing that stage's phase j / stages
+__device__ __forceinline__ void mbar_drain_ring(uint32_t first, uint32_t stages, uint32_t issued) {
+  for (uint32_t st = 0; st < stages && st < issued; ++st) {
+    const uint32_t j = ((issued - 1 - st) / stages) * stages + st;      // the last copy issued on this stage
+    mbar_drain(first + 8u * st, (j / stages) & 1u);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------- proxies
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
