@@ -33,7 +33,7 @@ PAPER_CONTEXT = ("paper (context only, whole pipeline on 8xB200): 6.70 s DiT den
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per token-head from the ncu captures summarised
 # under profiles/ (a 20-frame case of the 768p recipe; traffic grows in proportion to the token-heads a launch
 # processes, so it is scaled to the benchmarked workload by that count).
-DRAM_BYTES_PER_TOKEN_HEAD = {"gram_tc": 547.7, "readout_tc": 514.6}
+DRAM_BYTES_PER_TOKEN_HEAD = {"gram_tc": 547.5, "readout_tc": 514.4}
 
 
 # ------------------------------------------------------------------------------------------ helpers
